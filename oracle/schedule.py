@@ -1,0 +1,173 @@
+"""Sample-size schedule, round step sizes and the simulated-time event schedule.
+
+TEST INFRASTRUCTURE (see the package header).  Integer arithmetic only, apart
+from the step size.
+
+Follows the paper as below.
+* Section 5 "Objective function" / Appendix Table 2: s_i = a * i^p + b with
+  p = 1; the experiments give every node its own sequence s_{i,c} = a*i + b
+  (Appendix A.2), which is the reading used here.
+* Section 4.1: the step size is constant inside a round and diminishes as
+  eta_0 / (1 + beta * sqrt(t)), t = iterations done before the round (here:
+  the client's own count).
+* Algorithm 3: a round ends (the event triggers) when the local counter h
+  reaches s_{i,c}; the node then sends (c, U_i, i).  Receive applies
+  w -= eta_k * U and bumps H_v.  Synchronize(H, d, i) blocks while
+  max_e (i - H_e) > d.  Because H only grows and i is fixed within a round, the
+  check can only block before the round's first iteration, so it is evaluated
+  at round start.
+* Section 3.3.2 / Section 5 "System delay": a random compute delay per SGD
+  iteration and a random network delay per transmitted update sum.
+Client-server form of Section 1: the server applies update sums in arrival
+order; a client pulls the server's model when its round starts.
+
+Conventions the paper leaves open (fixed for this build):
+* time is integer ticks, 2^20 per unit; ties are ordered by
+  (tick, APPLY before START, client, round);
+* H_c counts the updates of client c the server has applied (Algorithm 3 bumps
+  H_v once per message whatever its round), the maximum runs over e != c, and
+  a lone client never waits;
+* stragglers are the last n_stragglers client ids; their compute-delay draws
+  are scaled by a Q16 fixed-point factor.
+"""
+import heapq
+import math
+import struct
+
+from . import rng
+
+APPLY, START = 0, 1
+NEVER_WAIT = 0xFFFFFFFF
+EVENT_STRUCT = struct.Struct("<4Q8I")   # layout of the library's event record
+
+
+def sample_size(a: int, b: int, i: int) -> int:
+    return a * i + b
+
+
+def samples_before(a: int, b: int, base: int, i: int) -> int:
+    """Samples a client has consumed before round i (rounds base .. i-1)."""
+    return sum(sample_size(a, b, j) for j in range(base, i))
+
+
+def rounds_needed(K: int, a: int, b: int, base: int) -> int:
+    """Smallest T with s_base + ... + s_{base+T-1} >= K (Section 4.1: K = sum s_j)."""
+    total, T = 0, 0
+    while total < K:
+        total += sample_size(a, b, base + T)
+        T += 1
+    return T
+
+
+def round_step_size(lr: float, beta: float, t: int) -> float:
+    return lr / (1.0 + beta * math.sqrt(t))
+
+
+def new_state(cfg):
+    return dict(clock=0, H=[0] * cfg["n_clients"], rounds_done=0)
+
+
+def _delay(cfg, which, r):
+    if cfg["delay_dist"] == 0:
+        return rng.exp_ticks(r, rng.to_ticks(cfg[which + "_delay_mean"]))
+    return rng.uniform_ticks(r, rng.to_ticks(cfg[which + "_delay_lo"]),
+                             rng.to_ticks(cfg[which + "_delay_hi"]))
+
+
+def simulate(cfg, n_rounds, state=None):
+    """Run the event schedule for n_rounds more rounds per client, to quiescence.
+
+    Returns (events ordered by seq, summary, state_after).
+    """
+    n = cfg["n_clients"]
+    a, b, base, B = cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["batch"]
+    d = cfg["max_lag_d"]
+    seed = cfg["seed"]
+    st = new_state(cfg) if state is None else state
+    H = list(st["H"])
+    t0 = st["clock"]
+    first = base + st["rounds_done"]
+    last = first + n_rounds
+    straggler_q16 = rng.to_q16(cfg["straggler_factor"])
+
+    key_c = [rng.stream_key(seed, rng.STREAM_COMPUTE, c) for c in range(n)]
+    key_n = [rng.stream_key(seed, rng.STREAM_NETWORK, c) for c in range(n)]
+    ready = [t0] * n
+    blocked = {}
+    heap = [(t0, START, c, first) for c in range(n)] if n_rounds > 0 else []
+    heapq.heapify(heap)
+    events = []
+    by_task = {}
+    seq = 0
+
+    def min_other(c):
+        if n == 1:
+            return None
+        m = min(H)
+        if H[c] != m or H.count(m) > 1:
+            return m
+        return min(H[e] for e in range(n) if e != c)
+
+    def lag_of(c, i):
+        m = min_other(c)
+        return 0 if m is None else max(0, (i - base) - m)
+
+    while heap:
+        t, kind, c, i = heapq.heappop(heap)
+        if kind == APPLY:
+            H[c] += 1
+            by_task[(c, i)]["seq"] = seq
+            seq += 1
+            for bc in sorted(blocked):
+                if d == NEVER_WAIT or lag_of(bc, blocked[bc]) <= d:
+                    heapq.heappush(heap, (t, START, bc, blocked.pop(bc)))
+            continue
+        lag = lag_of(c, i)
+        if d != NEVER_WAIT and lag > d:
+            blocked[c] = i
+            continue
+        s = sample_size(a, b, i)
+        if s % B:
+            raise ValueError("batch must divide every s_i")
+        steps = s // B
+        it0 = samples_before(a, b, base, i) // B
+        straggler = c >= n - cfg["n_stragglers"]
+        busy = 0
+        for j in range(steps):
+            dt = _delay(cfg, "compute", rng.draw(key_c[c], it0 + j))
+            if straggler:
+                dt = max(1, (dt * straggler_q16) >> 16)
+            busy += dt
+        t_trigger = t + busy
+        t_apply = t_trigger + _delay(cfg, "network", rng.draw(key_n[c], i))
+        by_task[(c, i)] = ev = dict(t_start=t, t_trigger=t_trigger, t_apply=t_apply,
+                                    wait_ticks=t - ready[c], client=c, round=i, samples=s,
+                                    steps=steps, seq=None, seen=seq, lag=lag)
+        events.append(ev)
+        heapq.heappush(heap, (t_apply, APPLY, c, i))
+        ready[c] = t_trigger
+        if i + 1 < last:
+            heapq.heappush(heap, (t_trigger, START, c, i + 1))
+
+    assert not blocked and all(e["seq"] is not None for e in events)
+    events.sort(key=lambda e: e["seq"])
+    samples_total = sum(e["samples"] for e in events)
+    s_first = sample_size(a, b, base)
+    per_client = samples_total // n if n else 0
+    summary = dict(
+        messages_up=len(events), model_pulls=len(events), samples_total=samples_total,
+        messages_if_per_sample=samples_total // B,
+        messages_if_constant_b=(n * -(-per_client // s_first)) if s_first else 0,
+        t_end_ticks=max((e["t_apply"] for e in events), default=t0))
+    after = dict(clock=summary["t_end_ticks"], H=H, rounds_done=st["rounds_done"] + n_rounds)
+    return events, summary, after
+
+
+def pack_events(events) -> bytes:
+    """The event log as the library lays it out (64 bytes per record)."""
+    out = bytearray()
+    for e in events:
+        out += EVENT_STRUCT.pack(e["t_start"], e["t_trigger"], e["t_apply"], e["wait_ticks"],
+                                 e["client"], e["round"], e["samples"], e["steps"],
+                                 e["seq"], e["seen"], e["lag"], 0)
+    return bytes(out)

@@ -1,0 +1,84 @@
+"""The whole hot path, sequentially: every client's local-SGD rounds and the
+server's ordered aggregation.
+
+TEST INFRASTRUCTURE (see the package header).  fp64 throughout.
+
+Algorithm 3, MainComputeNode: a round sets h = 0, U_i = 0 and repeats s_{i,c}
+times: sample xi from D_c; g = grad f(w_c, xi); w_c -= eta_i * g; U_i += g;
+then sends (c, U_i, i).  Receive: w -= eta_k * U.  Section 1 (client-server
+form): the server aggregates the received update sums into a global model that
+clients pick up.  Reading used here: a message takes effect at the receiver's
+next round start, so a client starts round i from the server's model at that
+time minus its own update sums that are still in flight (they are already in
+its local model through line "w_c -= eta_i g").
+"""
+import numpy as np
+
+from . import models, rng, schedule
+
+
+def f32(v) -> float:
+    """The library's config carries lr, lr_beta and l2 as fp32; use those values."""
+    return float(np.float32(v))
+
+
+def step_size(cfg, i):
+    a, b, base, B = cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["batch"]
+    t = schedule.samples_before(a, b, base, i) // B
+    return schedule.round_step_size(f32(cfg["lr"]), f32(cfg["lr_beta"]), t)
+
+
+def task_indices(cfg, c, i, n_c):
+    """Sample indices of round-task (c, i), shape [steps, B] (with replacement,
+    keyed by the client's running sample counter)."""
+    a, b, base, B = cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["batch"]
+    k0 = schedule.samples_before(a, b, base, i)
+    s = schedule.sample_size(a, b, i)
+    key = rng.stream_key(cfg["seed"], rng.STREAM_SAMPLE, c)
+    idx = [rng.sample_index(rng.draw(key, k0 + k), n_c) for k in range(s)]
+    return np.asarray(idx, dtype=np.int64).reshape(s // B, B)
+
+
+def run_task(cfg, client_data, c, i, w_start):
+    """One round of client c from model w_start: returns (U_i, w_end)."""
+    X, y = client_data
+    dims, l2, prec = cfg["dims"], f32(cfg["l2"]), cfg["precision"]
+    eta = step_size(cfg, i)
+    w = np.array(w_start, dtype=np.float64)
+    U = np.zeros_like(w)
+    for idx in task_indices(cfg, c, i, len(y)):
+        _, g = models.loss_and_grad(w, X[idx], y[idx], dims, l2, prec)
+        w -= eta * g
+        U += g
+    return U, w
+
+
+def run(cfg, data, w0, n_rounds=None, keep=False):
+    """All clients, n_rounds rounds each, to quiescence.
+
+    Returns dict(events, summary, w, U (by seq), w_start (by seq, if keep)).
+    """
+    n_rounds = cfg["n_rounds"] if n_rounds is None else n_rounds
+    events, summary, _ = schedule.simulate(cfg, n_rounds)
+    order = sorted([(e["t_apply"], schedule.APPLY, e["client"], e["round"], e) for e in events] +
+                   [(e["t_start"], schedule.START, e["client"], e["round"], e) for e in events],
+                   key=lambda r: r[:4])
+    w_g = np.array(w0, dtype=np.float64)
+    U_by_seq = [None] * len(events)
+    w_start_by_seq = [None] * len(events)
+    in_flight = {c: [] for c in range(cfg["n_clients"])}
+    for _, kind, c, i, e in order:
+        if kind == schedule.START:
+            w_start = w_g.copy()
+            for f in in_flight[c]:
+                w_start -= step_size(cfg, f["round"]) * U_by_seq[f["seq"]]
+            U, _ = run_task(cfg, data[c], c, i, w_start)
+            U_by_seq[e["seq"]] = U
+            if keep:
+                w_start_by_seq[e["seq"]] = w_start
+            in_flight[c].append(e)
+        else:
+            w_g -= step_size(cfg, i) * U_by_seq[e["seq"]]
+            in_flight[c].remove(e)
+    assert all(not v for v in in_flight.values())
+    return dict(events=events, summary=summary, w=w_g, U=U_by_seq, w_start=w_start_by_seq)

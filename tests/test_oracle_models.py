@@ -1,0 +1,102 @@
+"""Pins for the checker's losses and gradients (CPU only)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import models
+from paper_2112_13935_b200 import workloads
+
+
+def _rand_problem(dims, B, seed):
+    g = np.random.default_rng(seed)
+    P = workloads.n_params(dims)
+    w = g.normal(0, 0.3, size=P)
+    X = g.uniform(0, 1, size=(B, dims[0]))
+    y = g.integers(0, dims[-1], size=B)
+    return w, X, y
+
+
+@pytest.mark.parametrize("dims,B", [([7, 10], 1), ([7, 10], 5), ([9, 6, 10], 4), ([8, 7, 5, 10], 3)])
+@pytest.mark.parametrize("l2", [0.0, 0.05])
+def test_gradient_matches_central_differences(dims, B, l2):
+    w, X, y = _rand_problem(dims, B, 11)
+    _, g = models.loss_and_grad(w, X, y, dims, l2)
+    h = 1e-6
+    for j in np.random.default_rng(3).choice(w.size, size=min(60, w.size), replace=False):
+        e = np.zeros_like(w)
+        e[j] = h
+        fp, _ = models.loss_and_grad(w + e, X, y, dims, l2)
+        fm, _ = models.loss_and_grad(w - e, X, y, dims, l2)
+        assert abs((fp - fm) / (2 * h) - g[j]) < 1e-7, j
+
+
+def test_softmax_regression_gradient_at_zero_by_hand():
+    # w = 0: p = 1/10 for every class, so dW = x (p - onehot)^T and db = p - onehot.
+    dims = [4, 10]
+    x = np.array([[0.5, 0.0, 1.0, 0.25]])
+    loss, g = models.loss_and_grad(np.zeros(50), x, np.array([3]), dims)
+    delta = np.full(10, 0.1)
+    delta[3] -= 1.0
+    assert np.isclose(loss, np.log(10.0))
+    np.testing.assert_allclose(g[:40].reshape(4, 10), np.outer(x[0], delta), atol=1e-15)
+    np.testing.assert_allclose(g[40:], delta, atol=1e-15)
+
+
+def test_matches_torch_autograd_mlp():
+    # a library's reverse-mode derivative of the same loss, written independently
+    dims, B = [12, 8, 6, 10], 5
+    w, X, y = _rand_problem(dims, B, 4)
+    _, g = models.loss_and_grad(w, X, y, dims, 0.01)
+    wt = torch.tensor(w, dtype=torch.float64, requires_grad=True)
+    a, o, reg = torch.tensor(X), 0, 0.0
+    for l in range(3):
+        i, j = dims[l], dims[l + 1]
+        W = wt[o:o + i * j].reshape(i, j)
+        b = wt[o + i * j:o + i * j + j]
+        o += i * j + j
+        reg = reg + 0.5 * 0.01 * (W * W).sum()
+        a = a @ W + b
+        if l < 2:
+            a = torch.relu(a)
+    loss = torch.nn.functional.cross_entropy(a, torch.tensor(y)) + reg
+    loss.backward()
+    np.testing.assert_allclose(g, wt.grad.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_softmax_rows_sum_to_one_and_survive_large_logits():
+    Z = np.array([[1000.0, 999.0, -1000.0], [0.0, 0.0, 0.0]])
+    P = models.softmax_rows(Z)
+    np.testing.assert_allclose(P.sum(axis=1), 1.0, atol=1e-15)
+    assert np.isclose(P[0, 0], 1 / (1 + np.exp(-1.0)))
+
+
+def test_bf16_rounding_matches_a_library_conversion():
+    g = np.random.default_rng(0)
+    v = np.concatenate([g.normal(0, 1, 5000), g.uniform(0, 1, 5000), [0.0, 1.0, -1.0, 0.1, 3.0e-5]])
+    v32 = v.astype(np.float32)
+    want = torch.tensor(v32).to(torch.bfloat16).to(torch.float64).numpy()
+    got = models.round_bf16(v32.astype(np.float64))
+    np.testing.assert_array_equal(got, want)
+    # ties go to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert models.round_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert models.round_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+
+
+def test_bf16_path_uses_rounded_operands():
+    dims, B = [6, 5, 10], 4
+    w, X, y = _rand_problem(dims, B, 9)
+    l0, g0 = models.loss_and_grad(w, X, y, dims, 0.0, precision=0)
+    l1, g1 = models.loss_and_grad(w, X, y, dims, 0.0, precision=1)
+    assert 0 < abs(l1 - l0) < 2e-2 and 0 < np.abs(g1 - g0).max() < 5e-2
+    # rounding the inputs beforehand changes nothing: they are rounded at the same points
+    wq = w.copy()
+    l2_, g2 = models.loss_and_grad(wq, models.round_bf16(X), y, dims, 0.0, precision=1)
+    assert l2_ == l1 and np.array_equal(g1, g2)
+
+
+def test_full_loss_is_the_mean_over_all_clients():
+    dims = [5, 10]
+    w, X, y = _rand_problem(dims, 12, 2)
+    data = [(X[:5], y[:5]), (X[5:], y[5:])]
+    want, _ = models.loss_and_grad(w, X, y, dims, 0.3)
+    assert np.isclose(models.full_loss(w, data, dims, 0.3, chunk=4), want, rtol=1e-13)
