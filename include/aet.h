@@ -1,0 +1,199 @@
+/*
+ * aet.h - C ABI of the AET-SGD hot-path library for NVIDIA B200 (sm_100a).
+ *
+ * AET-SGD (asynchronous event-triggered SGD, arXiv 2112.13935): every client
+ * runs local-SGD rounds whose length grows linearly, s_i = a*i + b (Section 5,
+ * "Objective function"; Appendix Table 2), accumulates the update sum U_i of
+ * the round's gradients and sends (c, U_i, i) when the round's last sample is
+ * done - that is the event trigger (Algorithm 3, MainComputeNode).  A server
+ * applies w -= eta_k * U in arrival order (Algorithm 3, Receive; Section 1,
+ * client-server form) and clients pick the refreshed model up at their next
+ * round start, subject to the delay checkpoint Synchronize(H, d, i).  Compute
+ * and network delays are simulated (Section 3.3.2, Section 5 "System delay")
+ * with a seeded integer clock, so the asynchronous interleaving is reproducible.
+ *
+ * All clients run concurrently on one GPU.  Every call returns an aet_status;
+ * nothing throws, aborts or traps.  Out-parameters are untouched on error.
+ * Unless a parameter says otherwise, "device pointer" means memory of the
+ * current CUDA device and "host pointer" ordinary (pageable or pinned) memory.
+ *
+ * Parameter-vector layout (models, update sums): layers in order, each W_l
+ * row-major [in, out] followed by b_l [out]; fp32.
+ */
+#ifndef AET_H_
+#define AET_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct aet_handle aet_handle; /* opaque; owned by the library */
+
+typedef enum {
+  AET_OK = 0,
+  AET_ERR_ARG = 1,     /* null / out-of-range argument                      */
+  AET_ERR_CONFIG = 2,  /* configuration the library cannot run               */
+  AET_ERR_STATE = 3,   /* call out of order, or device bookkeeping mismatch  */
+  AET_ERR_NOMEM = 4,   /* host or device allocation failed                   */
+  AET_ERR_CUDA = 5,    /* a CUDA runtime call failed (see aet_last_error)    */
+  AET_ERR_TIMEOUT = 6, /* a bounded device-side wait gave up                 */
+  AET_ERR_NUMERIC = 7  /* non-finite value met in a model or update sum      */
+} aet_status;
+
+#define AET_MAX_LAYERS 7
+#define AET_NEVER_WAIT 0xFFFFFFFFu /* max_lag_d: the checkpoint never blocks */
+#define AET_TICKS_PER_UNIT (1u << 20)
+
+/* Run configuration.  Plain data; struct_size = sizeof(aet_config). */
+typedef struct {
+  uint32_t struct_size;
+  uint32_t n_clients;
+  uint32_t model;      /* 0 = softmax regression, 1 = ReLU MLP (Eq. 1: f(w; xi)) */
+  uint32_t n_layers;   /* weight layers = entries of dims - 1                     */
+  uint32_t dims[8];    /* {784,10}, {784,128,10}, {3072,256,128,10}               */
+  uint32_t precision;  /* 0 = fp32; 1 = bf16 operands, fp32 accumulate and master */
+  uint32_t batch;      /* samples per SGD iteration; must divide every s_i        */
+  uint32_t sched_a, sched_b; /* s_i = a*i + b (Section 5; Table 2)                */
+  uint32_t round_base; /* index of a client's first round                         */
+  uint32_t max_lag_d;  /* threshold d of Synchronize (Algorithm 3)                */
+  float lr, lr_beta;   /* eta_i = lr / (1 + lr_beta * sqrt(t)) (Section 5)        */
+  float l2;            /* lambda of (lambda/2)|W|^2 on weight matrices            */
+  uint32_t delay_dist; /* 0 = exponential(mean), 1 = uniform[lo, hi]              */
+  uint64_t seed;
+  double compute_delay_mean, network_delay_mean; /* time units, dist 0           */
+  double compute_delay_lo, compute_delay_hi;     /* time units, dist 1           */
+  double network_delay_lo, network_delay_hi;
+  double straggler_factor; /* scales the compute delay of the stragglers          */
+  uint32_t n_stragglers;   /* the last n_stragglers client ids                    */
+  uint32_t flags;          /* reserved, 0                                          */
+} aet_config;
+
+/* One round-task = one message (c, U_i, i) of Algorithm 3.  64 bytes.
+ * Times are integer ticks (2^20 per time unit). */
+typedef struct {
+  uint64_t t_start;    /* round began (after any checkpoint wait)                  */
+  uint64_t t_trigger;  /* h reached s_{i,c}: the update sum was sent               */
+  uint64_t t_apply;    /* the server applied it                                     */
+  uint64_t wait_ticks; /* time spent blocked in Synchronize before t_start         */
+  uint32_t client, round;
+  uint32_t samples;    /* s_{i,c}                                                   */
+  uint32_t steps;      /* SGD iterations = samples / batch                          */
+  uint32_t seq;        /* position in the server's apply order                      */
+  uint32_t seen;       /* updates already in the server model the round started from */
+  uint32_t lag;        /* max(0, rounds done - min over other clients of H) at start */
+  uint32_t pad;
+} aet_event;
+
+typedef struct {
+  uint64_t messages_up;            /* update sums sent = events                    */
+  uint64_t model_pulls;            /* round starts                                  */
+  uint64_t samples_total;
+  uint64_t messages_if_per_sample; /* one message per SGD iteration instead         */
+  uint64_t messages_if_constant_b; /* constant round size s = first round's size    */
+  uint64_t t_end_ticks;            /* simulated time of the last apply              */
+} aet_summary;
+
+/* Counters of the most recent aet_run_rounds (device times only when kernel
+ * timing is on).  kernel ids: 0 local-SGD, 1 ordered aggregation. */
+typedef struct {
+  uint64_t waves;              /* groups of independent round-tasks launched        */
+  uint64_t launches[4];        /* kernel launches per kernel id                     */
+  double kernel_ms[4];         /* summed device time per kernel id                  */
+  double plan_ms;              /* host time spent on schedule + launch plan         */
+} aet_stats;
+
+/* Create a run.  Allocates the global model (zeros) and per-client state on the
+ * current CUDA device.  Errors: AET_ERR_ARG (null, bad struct_size),
+ * AET_ERR_CONFIG (unsupported model/dims/batch), AET_ERR_CUDA, AET_ERR_NOMEM. */
+aet_status aet_create(const aet_config* cfg, aet_handle** out);
+
+/* Free everything the handle owns (synchronises the device first). */
+aet_status aet_destroy(aet_handle* h);
+
+/* Back to the state right after aet_create + aet_set_global_model + data load:
+ * global model = the last model set (zeros if none), no rounds done, clock 0,
+ * empty log.  Client data and cached schedules are kept. */
+aet_status aet_reset(aet_handle* h, void* cuda_stream);
+
+/* Set the server's model w_0 (Algorithm 2: "Initialize global model").
+ * w0: host or device pointer, n_params floats in the layout above. */
+aet_status aet_set_global_model(aet_handle* h, const float* w0, size_t n_params,
+                                void* cuda_stream);
+
+/* Give client `client` its local data set D_c (Section 1).  x: host or device
+ * pointer, row-major [n, dims[0]] fp32; y: host or device pointer, [n] int32
+ * class ids in [0, dims[last]).  The library copies (precision 1: converts to
+ * bf16 once); the caller may free its buffers once `cuda_stream` has completed.
+ * Errors: AET_ERR_ARG (client out of range, n == 0, n < batch, null). */
+aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x,
+                                const int32_t* y, uint32_t n, void* cuda_stream);
+
+/* Run n_rounds more rounds of every client (Algorithm 3, MainComputeNode loop
+ * "for round i") with all update sums applied by the server (Receive), to
+ * quiescence.  Asynchronous on `cuda_stream`; host work = the integer schedule
+ * and the launch plan.  Errors: AET_ERR_STATE (a client has no data),
+ * AET_ERR_CONFIG (batch does not divide s_i), AET_ERR_CUDA, AET_ERR_NOMEM. */
+aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream);
+
+/* Copy the server's model out (host or device pointer, n_params floats).
+ * Synchronises `cuda_stream`. */
+aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params,
+                                void* cuda_stream);
+
+/* The event log of all rounds run so far, ordered by seq within each
+ * aet_run_rounds call, and its summary.  `out` is a host array of `capacity`
+ * records (may be null with capacity 0 to query *n_events).  Synchronises the
+ * last stream used and cross-checks the trigger/apply records the kernels
+ * wrote against the schedule (AET_ERR_STATE on a mismatch). */
+aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity,
+                             size_t* n_events, aet_summary* summary);
+
+/* Update sum number `seq` of the most recent aet_run_rounds (host or device
+ * pointer, n_params floats).  Synchronises `cuda_stream`. */
+aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params,
+                              void* cuda_stream);
+
+/* Parity aid, not part of a run: one round-task (client, round) of Algorithm 3
+ * started from the caller's model w_in; writes the update sum U_i and the
+ * client's end-of-round model (either may be null).  Pointers: host or device,
+ * n_params floats each.  Uses the same sample indices the run would use.
+ * Leaves the handle's state unchanged.  Synchronises `cuda_stream`. */
+aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t round,
+                                      const float* w_in, float* U_out, float* w_out,
+                                      void* cuda_stream);
+
+/* Record CUDA events around every kernel of later runs (adds a little launch
+ * overhead) so that aet_get_stats can report device time per kernel. */
+aet_status aet_set_kernel_timing(aet_handle* h, int enable);
+aet_status aet_get_stats(aet_handle* h, aet_stats* out);
+
+size_t aet_n_params(const aet_handle* h);
+
+/* Text of the most recent error on this handle ("" if none); h may be null for
+ * the last aet_create failure of the calling thread. */
+const char* aet_last_error(const aet_handle* h);
+
+/* ---- host-only helpers (no GPU needed) -------------------------------- */
+
+/* The integer schedule alone: what aet_run_rounds(n_rounds) on a fresh handle
+ * would log.  Same record layout and ordering as aet_get_event_log. */
+aet_status aet_schedule_only(const aet_config* cfg, uint32_t n_rounds, aet_event* out,
+                             size_t capacity, size_t* n_events, aet_summary* summary);
+
+/* Draw number `counter` of stream (seed, stream, client); streams: 0 sample
+ * index, 1 compute delay, 2 network delay. */
+uint64_t aet_debug_draw(uint64_t seed, uint32_t stream, uint32_t client, uint64_t counter);
+/* Delay in ticks from a 64-bit draw: dist 0 -> exponential with mean p0 ticks,
+ * dist 1 -> uniform on [p0, p1] ticks. */
+uint64_t aet_debug_delay_ticks(uint32_t dist, uint64_t draw, uint64_t p0, uint64_t p1);
+/* Number of waves (groups of mutually independent round-tasks) the launch
+ * plan of a fresh run of n_rounds has; 0 on error. */
+uint32_t aet_debug_plan_waves(const aet_config* cfg, uint32_t n_rounds);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AET_H_ */

@@ -53,13 +53,15 @@ def run_task(cfg, client_data, c, i, w_start):
     return U, w
 
 
-def run(cfg, data, w0, n_rounds=None, keep=False):
+def run(cfg, data, w0, n_rounds=None, keep=False, state=None):
     """All clients, n_rounds rounds each, to quiescence.
 
-    Returns dict(events, summary, w, U (by seq), w_start (by seq, if keep)).
+    w0 is the server model the call starts from; state (from a previous call's
+    result) continues the simulated clock, histories and round counters.
+    Returns dict(events, summary, w, U (by seq), w_start (by seq, if keep), state).
     """
     n_rounds = cfg["n_rounds"] if n_rounds is None else n_rounds
-    events, summary, _ = schedule.simulate(cfg, n_rounds)
+    events, summary, state_after = schedule.simulate(cfg, n_rounds, state)
     order = sorted([(e["t_apply"], schedule.APPLY, e["client"], e["round"], e) for e in events] +
                    [(e["t_start"], schedule.START, e["client"], e["round"], e) for e in events],
                    key=lambda r: r[:4])
@@ -81,4 +83,5 @@ def run(cfg, data, w0, n_rounds=None, keep=False):
             w_g -= step_size(cfg, i) * U_by_seq[e["seq"]]
             in_flight[c].remove(e)
     assert all(not v for v in in_flight.values())
-    return dict(events=events, summary=summary, w=w_g, U=U_by_seq, w_start=w_start_by_seq)
+    return dict(events=events, summary=summary, w=w_g, U=U_by_seq, w_start=w_start_by_seq,
+                state=state_after)

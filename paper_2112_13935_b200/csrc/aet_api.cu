@@ -1,0 +1,572 @@
+// C ABI of the AET-SGD hot-path library: handle, device memory, and the run
+// loop that turns the integer schedule into waves of kernel launches.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <string.h>
+
+#include <chrono>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/aet.h"
+#include "aet_kernels.h"
+#include "aet_rng.h"
+#include "aet_schedule.h"
+
+using namespace aet;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+// Bump allocator over a few large device chunks: client data sets are many
+// small allocations of unknown count, and cudaMalloc per client is slow.
+struct Arena {
+  std::vector<void*> chunks;
+  char* cur = nullptr;
+  size_t left = 0;
+  static constexpr size_t kChunk = 256ull << 20;
+  void* alloc(size_t bytes) {
+    bytes = (bytes + 255) & ~(size_t)255;
+    if (bytes > left) {
+      size_t want = bytes > kChunk ? bytes : kChunk;
+      void* p = nullptr;
+      if (cudaMalloc(&p, want) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+      chunks.push_back(p);
+      cur = (char*)p;
+      left = want;
+    }
+    void* r = cur;
+    cur += bytes;
+    left -= bytes;
+    return r;
+  }
+  void release() {
+    for (void* p : chunks) cudaFree(p);
+    chunks.clear();
+    cur = nullptr;
+    left = 0;
+  }
+};
+
+template <class T>
+struct DevBuf {  // grow-only device array
+  T* p = nullptr;
+  size_t cap = 0;
+  bool reserve(size_t n) {
+    if (n <= cap) return true;
+    if (p) cudaFree(p);
+    p = nullptr;
+    cap = 0;
+    if (cudaMalloc((void**)&p, n * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+    cap = n;
+    return true;
+  }
+  void release() { if (p) cudaFree(p); p = nullptr; cap = 0; }
+};
+
+struct CachedPlan {
+  bool valid = false, uploaded = false;
+  uint32_t rounds_before = 0, n_rounds = 0;
+  SchedState before, after;
+  SchedResult sched;
+  Plan plan;
+};
+
+}  // namespace
+
+struct aet_handle {
+  aet_config cfg{};
+  uint32_t P = 0;
+  size_t stride = 0;
+  bool lr_fast = false;  // 784 -> 10, batch 1, fp32: the specialised kernel
+  MlpShape shape{};
+  std::string err;
+
+  SchedState st;
+  DelayCache delays;
+  CachedPlan cached;
+  std::vector<aet_event> log;
+  aet_summary total{};
+
+  Arena arena;
+  std::vector<ClientData> h_clients;
+  DevBuf<ClientData> d_clients;
+  DevBuf<uint64_t> d_keys;
+  DevBuf<uint32_t> d_H;
+  DevBuf<float> w_cur, w0, snaps, U, work, act, dbg;
+  DevBuf<TaskDesc> d_tasks;
+  DevBuf<InflightRef> d_inflight;
+  DevBuf<ApplyDesc> d_applies;
+  DevBuf<TriggerRec> d_trig;
+  DevBuf<ApplyRec> d_alog;
+  bool clients_dirty = true, have_w0 = false;
+
+  // most recent run, for the device-record cross-check and aet_get_update_sum
+  size_t last_first_event = 0, last_n_events = 0;
+  bool last_checked = true;
+  std::vector<uint32_t> last_H_before;
+  cudaStream_t last_stream = nullptr;
+
+  bool timing = false;
+  aet_stats stats{};
+  struct Timed { cudaEvent_t a, b; int id; };
+  std::vector<Timed> timed;
+  std::vector<cudaEvent_t> ev_pool;
+};
+
+namespace {
+
+aet_status fail(aet_handle* h, aet_status s, const std::string& msg) {
+  if (h) h->err = msg; else g_create_error = msg;
+  return s;
+}
+aet_status cuda_fail(aet_handle* h, cudaError_t e, const char* what) {
+  cudaGetLastError();
+  return fail(h, AET_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define AET_CUDA(h, call)                                         \
+  do {                                                            \
+    cudaError_t e_ = (call);                                      \
+    if (e_ != cudaSuccess) return cuda_fail(h, e_, #call);        \
+  } while (0)
+
+uint32_t count_params(const aet_config& c) {
+  uint64_t p = 0;
+  for (uint32_t l = 0; l < c.n_layers; ++l) p += (uint64_t)c.dims[l] * c.dims[l + 1] + c.dims[l + 1];
+  return p > 0xFFFFFFFFull ? 0 : (uint32_t)p;
+}
+
+cudaEvent_t get_event(aet_handle* h) {
+  if (!h->ev_pool.empty()) { cudaEvent_t e = h->ev_pool.back(); h->ev_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct KernelTimer {  // records a pair of events around a launch when timing is on
+  aet_handle* h; cudaStream_t s; int id; cudaEvent_t a = nullptr;
+  KernelTimer(aet_handle* h_, cudaStream_t s_, int id_) : h(h_), s(s_), id(id_) {
+    h->stats.launches[id] += 1;
+    if (h->timing) { a = get_event(h); cudaEventRecord(a, s); }
+  }
+  ~KernelTimer() {
+    if (h->timing) { cudaEvent_t b = get_event(h); cudaEventRecord(b, s); h->timed.push_back({a, b, id}); }
+  }
+};
+
+void collect_timings(aet_handle* h) {
+  for (auto& t : h->timed) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(t.b) == cudaSuccess && cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess)
+      h->stats.kernel_ms[t.id] += ms;
+    h->ev_pool.push_back(t.a);
+    h->ev_pool.push_back(t.b);
+  }
+  h->timed.clear();
+}
+
+aet_status upload_clients(aet_handle* h, cudaStream_t s) {
+  if (!h->clients_dirty) return AET_OK;
+  const uint32_t n = h->cfg.n_clients;
+  if (!h->d_clients.reserve(n) || !h->d_keys.reserve(n)) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  std::vector<uint64_t> keys(n);
+  for (uint32_t c = 0; c < n; ++c) keys[c] = stream_key(h->cfg.seed, kStreamSample, c);
+  AET_CUDA(h, cudaMemcpyAsync(h->d_clients.p, h->h_clients.data(), n * sizeof(ClientData), cudaMemcpyHostToDevice, s));
+  AET_CUDA(h, cudaMemcpyAsync(h->d_keys.p, keys.data(), n * sizeof(uint64_t), cudaMemcpyHostToDevice, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));  // the host vectors above go out of scope
+  h->clients_dirty = false;
+  return AET_OK;
+}
+
+aet_status launch_rounds(aet_handle* h, const RoundLaunch& r, cudaStream_t s) {
+  KernelTimer kt(h, s, 0);
+  cudaError_t e;
+  if (h->lr_fast) {
+    e = launch_lr_rounds(r, s);
+  } else {
+    MlpLaunch m;
+    m.r = r;
+    m.shape = h->shape;
+    m.work = h->work.p;
+    m.act = h->act.p;
+    m.act_stride = mlp_act_floats(h->shape);
+    e = launch_mlp_rounds(m, s);
+  }
+  if (e != cudaSuccess) return cuda_fail(h, e, "local-SGD kernel launch");
+  return AET_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+aet_status aet_create(const aet_config* cfg, aet_handle** out) {
+  if (!cfg || !out) return fail(nullptr, AET_ERR_ARG, "null argument");
+  std::string err;
+  if (cfg->struct_size != sizeof(aet_config)) return fail(nullptr, AET_ERR_ARG, "struct_size does not match sizeof(aet_config)");
+  if (!validate_config(*cfg, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+  const uint32_t P = count_params(*cfg);
+  if (!P) return fail(nullptr, AET_ERR_CONFIG, "model too large");
+  if (cfg->dims[cfg->n_layers] > 32) return fail(nullptr, AET_ERR_CONFIG, "at most 32 classes are supported");
+  int dev = 0;
+  cudaError_t ce = cudaGetDevice(&dev);
+  if (ce != cudaSuccess) { cudaGetLastError(); return fail(nullptr, AET_ERR_CUDA, std::string("no CUDA device: ") + cudaGetErrorString(ce)); }
+  aet_handle* h = new (std::nothrow) aet_handle();
+  if (!h) return fail(nullptr, AET_ERR_NOMEM, "out of host memory");
+  h->cfg = *cfg;
+  h->P = P;
+  h->stride = ((size_t)P + 31) & ~(size_t)31;
+  h->lr_fast = cfg->model == 0 && cfg->dims[0] == 784 && cfg->dims[1] == 10 && cfg->batch == 1 && cfg->precision == 0;
+  h->shape.n_layers = cfg->n_layers;
+  for (int i = 0; i < 8; ++i) h->shape.dims[i] = cfg->dims[i];
+  h->shape.batch = cfg->batch;
+  h->shape.precision = cfg->precision;
+  h->shape.cluster = mlp_pick_cluster(h->shape, cfg->n_clients);
+  if (!h->lr_fast) {
+    if (const char* why = mlp_check_shape(h->shape)) { delete h; return fail(nullptr, AET_ERR_CONFIG, why); }
+  }
+  h->h_clients.assign(cfg->n_clients, ClientData{nullptr, nullptr, 0, 0});
+  h->st.H.assign(cfg->n_clients, 0);
+  bool ok = h->w_cur.reserve(h->stride) && h->w0.reserve(h->stride) && h->d_H.reserve(cfg->n_clients);
+  if (ok && !h->lr_fast) ok = h->work.reserve((size_t)cfg->n_clients * h->stride);
+  if (!ok) { aet_destroy(h); return fail(nullptr, AET_ERR_NOMEM, "device allocation failed"); }
+  if (cudaMemset(h->w_cur.p, 0, h->stride * sizeof(float)) != cudaSuccess ||
+      cudaMemset(h->w0.p, 0, h->stride * sizeof(float)) != cudaSuccess ||
+      cudaMemset(h->d_H.p, 0, cfg->n_clients * sizeof(uint32_t)) != cudaSuccess) {
+    cudaError_t e = cudaGetLastError();
+    aet_destroy(h);
+    return fail(nullptr, AET_ERR_CUDA, std::string("cudaMemset: ") + cudaGetErrorString(e));
+  }
+  *out = h;
+  return AET_OK;
+}
+
+aet_status aet_destroy(aet_handle* h) {
+  if (!h) return AET_ERR_ARG;
+  cudaDeviceSynchronize();
+  collect_timings(h);
+  for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+  h->arena.release();
+  h->d_clients.release(); h->d_keys.release(); h->d_H.release();
+  h->w_cur.release(); h->w0.release(); h->snaps.release(); h->U.release();
+  h->work.release(); h->act.release(); h->dbg.release();
+  h->d_tasks.release(); h->d_inflight.release(); h->d_applies.release();
+  h->d_trig.release(); h->d_alog.release();
+  cudaGetLastError();
+  delete h;
+  return AET_OK;
+}
+
+aet_status aet_reset(aet_handle* h, void* cuda_stream) {
+  if (!h) return AET_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  AET_CUDA(h, cudaMemcpyAsync(h->w_cur.p, h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  AET_CUDA(h, cudaMemsetAsync(h->d_H.p, 0, h->cfg.n_clients * sizeof(uint32_t), s));
+  h->st = SchedState{};
+  h->st.H.assign(h->cfg.n_clients, 0);
+  h->log.clear();
+  h->total = aet_summary{};
+  h->last_n_events = 0;
+  h->last_checked = true;
+  h->last_stream = s;
+  return AET_OK;
+}
+
+aet_status aet_set_global_model(aet_handle* h, const float* w0, size_t n_params, void* cuda_stream) {
+  if (!h || !w0) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  AET_CUDA(h, cudaMemcpyAsync(h->w_cur.p, w0, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaMemcpyAsync(h->w0.p, h->w_cur.p, (size_t)h->P * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  h->have_w0 = true;
+  h->last_stream = s;
+  return AET_OK;
+}
+
+aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x, const int32_t* y,
+                                uint32_t n, void* cuda_stream) {
+  if (!h) return AET_ERR_ARG;
+  if (!x || !y) return fail(h, AET_ERR_ARG, "null data pointer");
+  if (client >= h->cfg.n_clients) return fail(h, AET_ERR_ARG, "client index out of range");
+  if (n == 0 || n < h->cfg.batch) return fail(h, AET_ERR_ARG, "a client needs at least max(1, batch) samples");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const size_t D = h->cfg.dims[0];
+  const size_t elems = (size_t)n * D;
+  const bool bf16 = h->cfg.precision == 1;
+  void* dx = h->arena.alloc(elems * (bf16 ? 2 : 4));
+  int32_t* dy = (int32_t*)h->arena.alloc((size_t)n * sizeof(int32_t));
+  if (!dx || !dy) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  if (!bf16) {
+    AET_CUDA(h, cudaMemcpyAsync(dx, x, elems * 4, cudaMemcpyDefault, s));
+  } else {
+    cudaPointerAttributes attr{};
+    cudaError_t pe = cudaPointerGetAttributes(&attr, x);
+    if (pe != cudaSuccess) cudaGetLastError();
+    const bool on_device = pe == cudaSuccess && (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged);
+    if (on_device) {
+      AET_CUDA(h, launch_to_bf16((const float*)x, dx, elems, s));
+    } else {
+      float* tmp = nullptr;
+      AET_CUDA(h, cudaMalloc((void**)&tmp, elems * 4));
+      cudaError_t e = cudaMemcpyAsync(tmp, x, elems * 4, cudaMemcpyHostToDevice, s);
+      if (e == cudaSuccess) e = launch_to_bf16(tmp, dx, elems, s);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+      cudaFree(tmp);
+      if (e != cudaSuccess) return cuda_fail(h, e, "bf16 conversion of client data");
+    }
+  }
+  AET_CUDA(h, cudaMemcpyAsync(dy, y, (size_t)n * sizeof(int32_t), cudaMemcpyDefault, s));
+  h->h_clients[client] = ClientData{dx, dy, n, 0};
+  h->clients_dirty = true;
+  h->last_stream = s;
+  return AET_OK;
+}
+
+aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
+  if (!h) return AET_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  for (uint32_t c = 0; c < h->cfg.n_clients; ++c)
+    if (!h->h_clients[c].x) return fail(h, AET_ERR_STATE, "client " + std::to_string(c) + " has no data");
+  if (n_rounds == 0) return AET_OK;
+  collect_timings(h);
+  h->stats = aet_stats{};
+
+  // ---- a0: integer schedule and launch plan (cached for repeated runs) ----
+  auto t0 = std::chrono::steady_clock::now();
+  CachedPlan& cp = h->cached;
+  if (!(cp.valid && cp.rounds_before == h->st.rounds_done && cp.n_rounds == n_rounds &&
+        cp.before.clock == h->st.clock && cp.before.H == h->st.H)) {
+    cp.valid = false;
+    cp.uploaded = false;
+    cp.before = h->st;
+    cp.rounds_before = h->st.rounds_done;
+    cp.n_rounds = n_rounds;
+    SchedState st = h->st;
+    std::string err;
+    if (!simulate(h->cfg, n_rounds, st, h->delays, cp.sched, err)) return fail(h, AET_ERR_CONFIG, err);
+    cp.after = st;
+    build_plan(h->cfg, cp.sched.events, cp.plan);
+    cp.valid = true;
+  }
+  const Plan& plan = cp.plan;
+  const size_t E = cp.sched.events.size();
+  h->stats.plan_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+
+  // ---- device buffers ----
+  aet_status st_up = upload_clients(h, s);
+  if (st_up != AET_OK) return st_up;
+  bool ok = h->snaps.reserve((size_t)plan.n_snap * h->stride) && h->U.reserve(E * h->stride) &&
+            h->d_tasks.reserve(E) && h->d_inflight.reserve(plan.inflight.size() + 1) &&
+            h->d_applies.reserve(E) && h->d_trig.reserve(E) && h->d_alog.reserve(E);
+  if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * mlp_act_floats(h->shape));
+  if (!ok) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  if (!cp.uploaded) {
+    AET_CUDA(h, cudaMemcpyAsync(h->d_tasks.p, plan.tasks.data(), E * sizeof(TaskDesc), cudaMemcpyHostToDevice, s));
+    if (!plan.inflight.empty())
+      AET_CUDA(h, cudaMemcpyAsync(h->d_inflight.p, plan.inflight.data(), plan.inflight.size() * sizeof(InflightRef), cudaMemcpyHostToDevice, s));
+    AET_CUDA(h, cudaMemcpyAsync(h->d_applies.p, plan.applies.data(), E * sizeof(ApplyDesc), cudaMemcpyHostToDevice, s));
+    AET_CUDA(h, cudaStreamSynchronize(s));
+    cp.uploaded = true;
+  }
+  AET_CUDA(h, cudaMemsetAsync(h->d_trig.p, 0, E * sizeof(TriggerRec), s));
+  // snapshot 0 = the server model as this call begins
+  AET_CUDA(h, cudaMemcpyAsync(h->snaps.p, h->w_cur.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
+
+  RoundLaunch r{};
+  r.tasks = h->d_tasks.p; r.inflight = h->d_inflight.p; r.clients = h->d_clients.p;
+  r.sample_keys = h->d_keys.p; r.snaps = h->snaps.p; r.U = h->U.p; r.w_end = nullptr;
+  r.trig = h->d_trig.p; r.stride = h->stride; r.l2 = h->cfg.l2;
+  ApplyLaunch a{};
+  a.applies = h->d_applies.p; a.U = h->U.p; a.snaps = h->snaps.p; a.w_cur = h->w_cur.p;
+  a.H = h->d_H.p; a.log = h->d_alog.p; a.stride = h->stride; a.n_params = h->P;
+
+  // ---- waves: a3/a4 local SGD of independent round-tasks, then a6 aggregation ----
+  const uint32_t n_waves = (uint32_t)plan.apply_upto.size();
+  uint32_t applied = 0;
+  for (uint32_t L = 0; L < n_waves; ++L) {
+    r.task_begin = plan.wave_off[L];
+    r.n_tasks = plan.wave_off[L + 1] - plan.wave_off[L];
+    aet_status rs = launch_rounds(h, r, s);
+    if (rs != AET_OK) return rs;
+    if (plan.apply_upto[L] > applied) {
+      a.lo = applied; a.hi = plan.apply_upto[L];
+      KernelTimer kt(h, s, 1);
+      cudaError_t e = launch_apply_updates(a, s);
+      if (e != cudaSuccess) return cuda_fail(h, e, "aggregation kernel launch");
+      applied = a.hi;
+    }
+  }
+  h->stats.waves = n_waves;
+
+  // ---- host bookkeeping ----
+  h->last_H_before = h->st.H;
+  h->last_first_event = h->log.size();
+  h->last_n_events = E;
+  h->last_checked = false;
+  h->last_stream = s;
+  h->log.insert(h->log.end(), cp.sched.events.begin(), cp.sched.events.end());
+  const aet_summary& q = cp.sched.summary;
+  h->total.messages_up += q.messages_up; h->total.model_pulls += q.model_pulls;
+  h->total.samples_total += q.samples_total; h->total.messages_if_per_sample += q.messages_if_per_sample;
+  h->total.messages_if_constant_b += q.messages_if_constant_b; h->total.t_end_ticks = q.t_end_ticks;
+  h->st = cp.after;
+  return AET_OK;
+}
+
+aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params, void* cuda_stream) {
+  if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  AET_CUDA(h, cudaMemcpyAsync(out, h->w_cur.p, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  return AET_OK;
+}
+
+aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params, void* cuda_stream) {
+  if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
+  if (seq >= h->last_n_events) return fail(h, AET_ERR_ARG, "seq is not an event of the most recent run");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  AET_CUDA(h, cudaMemcpyAsync(out, h->U.p + (size_t)seq * h->stride, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  return AET_OK;
+}
+
+aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity, size_t* n_events, aet_summary* summary) {
+  if (!h || !n_events) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (!h->last_checked && h->last_n_events) {
+    // Compare what the kernels recorded (trigger per round-task, apply order and
+    // history counts) with the schedule they were launched from.
+    const size_t E = h->last_n_events;
+    std::vector<TriggerRec> trig(E);
+    std::vector<ApplyRec> alog(E);
+    AET_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    AET_CUDA(h, cudaMemcpy(trig.data(), h->d_trig.p, E * sizeof(TriggerRec), cudaMemcpyDeviceToHost));
+    AET_CUDA(h, cudaMemcpy(alog.data(), h->d_alog.p, E * sizeof(ApplyRec), cudaMemcpyDeviceToHost));
+    std::vector<uint32_t> H = h->last_H_before;
+    for (size_t k = 0; k < E; ++k) {
+      const aet_event& e = h->log[h->last_first_event + k];
+      if (trig[k].flags != 1 || trig[k].client != e.client || trig[k].round != e.round || trig[k].samples_done != e.samples)
+        return fail(h, AET_ERR_STATE, "device trigger record " + std::to_string(k) + " does not match the schedule");
+      H[e.client] += 1;
+      if (alog[k].seq != k || alog[k].client != e.client || alog[k].round != e.round || alog[k].h_after != H[e.client])
+        return fail(h, AET_ERR_STATE, "device apply record " + std::to_string(k) + " does not match the schedule");
+    }
+    h->last_checked = true;
+  }
+  if (out) {
+    if (capacity < h->log.size()) return fail(h, AET_ERR_ARG, "capacity is smaller than the log");
+    memcpy(out, h->log.data(), h->log.size() * sizeof(aet_event));
+  }
+  *n_events = h->log.size();
+  if (summary) *summary = h->total;
+  return AET_OK;
+}
+
+aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t round, const float* w_in,
+                                      float* U_out, float* w_out, void* cuda_stream) {
+  if (!h || !w_in) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (client >= h->cfg.n_clients) return fail(h, AET_ERR_ARG, "client index out of range");
+  if (round < h->cfg.round_base) return fail(h, AET_ERR_ARG, "round is before round_base");
+  if (!h->h_clients[client].x) return fail(h, AET_ERR_STATE, "client has no data");
+  const uint32_t s_i = sample_size(h->cfg, round);
+  if (s_i == 0 || s_i % h->cfg.batch) return fail(h, AET_ERR_CONFIG, "batch must divide the round's sample count");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  aet_status up = upload_clients(h, s);
+  if (up != AET_OK) return up;
+  // private area: [snapshot | U | w_end | task | trigger record]
+  const size_t fl = 3 * h->stride + 64;
+  if (!h->dbg.reserve(fl)) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  if (!h->lr_fast && !h->act.reserve(mlp_act_floats(h->shape))) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  float* snap = h->dbg.p;
+  float* U = snap + h->stride;
+  float* wend = U + h->stride;
+  TaskDesc* dtask = (TaskDesc*)(wend + h->stride);
+  TriggerRec* dtrig = (TriggerRec*)((char*)dtask + sizeof(TaskDesc));
+  TaskDesc t{};
+  t.client = client; t.round = round; t.seq = 0; t.snap_slot = 0;
+  t.n_samples = s_i; t.steps = s_i / h->cfg.batch;
+  t.inflight_off = 0; t.inflight_cnt = 0;
+  t.sample_ctr0 = samples_before(h->cfg, round);
+  t.eta = (float)round_step_size(h->cfg, round);
+  AET_CUDA(h, cudaMemcpyAsync(snap, w_in, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaMemcpyAsync(dtask, &t, sizeof(t), cudaMemcpyHostToDevice, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  RoundLaunch r{};
+  r.tasks = dtask; r.inflight = nullptr; r.clients = h->d_clients.p; r.sample_keys = h->d_keys.p;
+  r.snaps = snap; r.U = U; r.w_end = wend; r.trig = dtrig; r.stride = h->stride;
+  r.task_begin = 0; r.n_tasks = 1; r.l2 = h->cfg.l2;
+  const aet_stats keep = h->stats;
+  const bool timing = h->timing;
+  h->timing = false;
+  aet_status rs = launch_rounds(h, r, s);
+  h->timing = timing;
+  h->stats = keep;
+  if (rs != AET_OK) return rs;
+  if (U_out) AET_CUDA(h, cudaMemcpyAsync(U_out, U, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  if (w_out) AET_CUDA(h, cudaMemcpyAsync(w_out, wend, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  return AET_OK;
+}
+
+aet_status aet_set_kernel_timing(aet_handle* h, int enable) {
+  if (!h) return AET_ERR_ARG;
+  h->timing = enable != 0;
+  return AET_OK;
+}
+
+aet_status aet_get_stats(aet_handle* h, aet_stats* out) {
+  if (!h || !out) return AET_ERR_ARG;
+  collect_timings(h);
+  *out = h->stats;
+  return AET_OK;
+}
+
+size_t aet_n_params(const aet_handle* h) { return h ? h->P : 0; }
+
+const char* aet_last_error(const aet_handle* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+aet_status aet_schedule_only(const aet_config* cfg, uint32_t n_rounds, aet_event* out, size_t capacity,
+                             size_t* n_events, aet_summary* summary) {
+  if (!cfg || !n_events) return fail(nullptr, AET_ERR_ARG, "null argument");
+  std::string err;
+  if (cfg->struct_size != sizeof(aet_config)) return fail(nullptr, AET_ERR_ARG, "struct_size does not match sizeof(aet_config)");
+  if (!validate_config(*cfg, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+  SchedState st;
+  DelayCache cache;
+  SchedResult res;
+  if (!simulate(*cfg, n_rounds, st, cache, res, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+  if (out) {
+    if (capacity < res.events.size()) return fail(nullptr, AET_ERR_ARG, "capacity is smaller than the log");
+    memcpy(out, res.events.data(), res.events.size() * sizeof(aet_event));
+  }
+  *n_events = res.events.size();
+  if (summary) *summary = res.summary;
+  return AET_OK;
+}
+
+uint64_t aet_debug_draw(uint64_t seed, uint32_t stream, uint32_t client, uint64_t counter) {
+  return draw(stream_key(seed, stream, client), counter);
+}
+
+uint64_t aet_debug_delay_ticks(uint32_t dist, uint64_t r, uint64_t p0, uint64_t p1) {
+  return dist == 0 ? exp_ticks(r, p0) : uniform_ticks(r, p0, p1);
+}
+
+uint32_t aet_debug_plan_waves(const aet_config* cfg, uint32_t n_rounds) {
+  if (!cfg || cfg->struct_size != sizeof(aet_config)) return 0;
+  std::string err;
+  if (!validate_config(*cfg, err)) return 0;
+  SchedState st;
+  DelayCache cache;
+  SchedResult res;
+  if (!simulate(*cfg, n_rounds, st, cache, res, err)) return 0;
+  Plan plan;
+  build_plan(*cfg, res.events, plan);
+  return (uint32_t)plan.apply_upto.size();
+}
+
+}  // extern "C"

@@ -1,0 +1,76 @@
+// Launch interfaces of the device kernels (plain structs, no library types).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "aet_schedule.h"
+
+namespace aet {
+
+// Device view of one client's local data set D_c.
+struct ClientData {
+  const void* x;     // [n, D] row-major; fp32, or bf16 when precision == 1
+  const int32_t* y;  // [n]
+  uint32_t n;
+  uint32_t pad;
+};
+
+// What a local-SGD kernel leaves behind when a round's last sample is done:
+// the device-side record of the event trigger (message (c, U_i, i)).
+struct TriggerRec { uint32_t client, round, samples_done, flags; };
+// What the aggregation kernel leaves behind per applied update.
+struct ApplyRec { uint32_t client, round, h_after, seq; };
+
+// Rows of the snapshot / update-sum / work arrays are `stride` floats apart
+// (n_params rounded up to a multiple of 32, so every row is 128-byte aligned).
+struct RoundLaunch {
+  const TaskDesc* tasks;         // device
+  const InflightRef* inflight;   // device
+  const ClientData* clients;     // device, [n_clients]
+  const uint64_t* sample_keys;   // device, [n_clients]
+  const float* snaps;            // [n_snap, stride] models rounds start from
+  float* U;                      // [n_events, stride] update sums, row = seq
+  float* w_end;                  // optional [n_events, stride] end-of-round models
+  TriggerRec* trig;              // [n_events], row = seq
+  size_t stride;
+  uint32_t task_begin, n_tasks;
+  float l2;
+};
+
+// Softmax regression 784 -> 10, batch 1: one CTA per round-task.
+cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s);
+
+struct MlpShape {
+  uint32_t n_layers, dims[8], batch, precision;
+  uint32_t cluster;              // CTAs per round-task
+};
+struct MlpLaunch {
+  RoundLaunch r;
+  MlpShape shape;
+  float* work;                   // [n_clients, stride] client's current model
+  float* act;                    // per-task activation scratch
+  size_t act_stride;             // floats per task
+};
+cudaError_t launch_mlp_rounds(const MlpLaunch& p, cudaStream_t s);
+size_t mlp_act_floats(const MlpShape& shape);
+uint32_t mlp_pick_cluster(const MlpShape& shape, uint32_t n_clients);
+const char* mlp_check_shape(const MlpShape& shape);  // null if the kernel can run it
+
+// Ordered aggregation: for seq in [lo, hi): w -= eta_seq * U[seq]; keep a copy
+// where a later round starts from it; bump H and log the apply.
+struct ApplyLaunch {
+  const ApplyDesc* applies;  // device, indexed by seq
+  const float* U;
+  float* snaps;
+  float* w_cur;              // server model [stride]
+  uint32_t* H;               // [n_clients]
+  ApplyRec* log;             // [n_events]
+  size_t stride;
+  uint32_t n_params, lo, hi;
+};
+cudaError_t launch_apply_updates(const ApplyLaunch& p, cudaStream_t s);
+
+// bf16 conversion of a client's rows at load time (precision 1).
+cudaError_t launch_to_bf16(const float* src, void* dst, size_t n, cudaStream_t s);
+
+}  // namespace aet

@@ -1,0 +1,302 @@
+// Integer discrete-event schedule of AET-SGD and the wave plan built from it.
+//
+// Algorithm 3 (MainComputeNode): round i of client c runs s_{i,c} = a*i + b
+// samples, then sends (c, U_i, i).  Section 3.3.2 / Section 5: every SGD
+// iteration takes a random compute delay and every message a random network
+// delay.  Receive bumps H_v per message; Synchronize(H, d, i) blocks a round
+// start while (rounds done - min over the others of H) > d.  Ties in simulated
+// time are broken by (tick, apply before start, client, round).
+#include "aet_schedule.h"
+
+#include <math.h>
+
+#include <algorithm>
+#include <queue>
+#include <thread>
+#include <tuple>
+
+#include "aet_rng.h"
+
+namespace aet {
+
+uint32_t sample_size(const aet_config& c, uint32_t round) { return c.sched_a * round + c.sched_b; }
+
+uint64_t samples_before(const aet_config& c, uint32_t round) {
+  // sum_{j=base}^{round-1} (a j + b)
+  uint64_t n = round - c.round_base;
+  uint64_t sum_j = n * (uint64_t)c.round_base + n * (n - 1) / 2;
+  return (uint64_t)c.sched_a * sum_j + (uint64_t)c.sched_b * n;
+}
+
+double round_step_size(const aet_config& c, uint32_t round) {
+  double t = (double)(samples_before(c, round) / c.batch);
+  return (double)c.lr / (1.0 + (double)c.lr_beta * sqrt(t));
+}
+
+static uint64_t to_ticks(double units) { return (uint64_t)floor(units * (double)AET_TICKS_PER_UNIT + 0.5); }
+
+bool validate_config(const aet_config& c, std::string& err) {
+  if (c.struct_size != sizeof(aet_config)) { err = "struct_size does not match this library's aet_config"; return false; }
+  if (c.n_clients == 0) { err = "n_clients must be at least 1"; return false; }
+  if (c.n_layers < 1 || c.n_layers > AET_MAX_LAYERS) { err = "n_layers out of range"; return false; }
+  for (uint32_t l = 0; l <= c.n_layers; ++l)
+    if (c.dims[l] == 0) { err = "a layer dimension is zero"; return false; }
+  if (c.model > 1 || (c.model == 0 && c.n_layers != 1)) { err = "model 0 has exactly one weight layer"; return false; }
+  if (c.precision > 1) { err = "precision must be 0 or 1"; return false; }
+  if (c.batch == 0) { err = "batch must be at least 1"; return false; }
+  if (c.delay_dist > 1) { err = "delay_dist must be 0 or 1"; return false; }
+  if (c.n_stragglers > c.n_clients) { err = "more stragglers than clients"; return false; }
+  if (!(c.lr > 0.f) || c.lr_beta < 0.f || c.l2 < 0.f) { err = "lr must be positive, lr_beta and l2 non-negative"; return false; }
+  if (c.delay_dist == 0 && (!(c.compute_delay_mean >= 0) || !(c.network_delay_mean >= 0))) { err = "negative delay mean"; return false; }
+  if (c.delay_dist == 1 && (c.compute_delay_hi < c.compute_delay_lo || c.network_delay_hi < c.network_delay_lo ||
+                            c.compute_delay_lo < 0 || c.network_delay_lo < 0)) { err = "uniform delay range is empty"; return false; }
+  if (!(c.straggler_factor >= 0) || c.straggler_factor > 65535.0) { err = "straggler_factor out of range"; return false; }
+  return true;
+}
+
+namespace {
+
+struct DelayModel {
+  uint32_t dist;
+  uint64_t c0, c1, n0, n1;  // dist 0: means; dist 1: lo / hi
+  uint64_t straggler_q16;
+  uint64_t compute(uint64_t r) const { return dist == 0 ? exp_ticks(r, c0) : uniform_ticks(r, c0, c1); }
+  uint64_t network(uint64_t r) const { return dist == 0 ? exp_ticks(r, n0) : uniform_ticks(r, n0, n1); }
+};
+
+DelayModel make_delay_model(const aet_config& c) {
+  DelayModel m;
+  m.dist = c.delay_dist;
+  if (c.delay_dist == 0) {
+    m.c0 = to_ticks(c.compute_delay_mean); m.c1 = 0;
+    m.n0 = to_ticks(c.network_delay_mean); m.n1 = 0;
+  } else {
+    m.c0 = to_ticks(c.compute_delay_lo); m.c1 = to_ticks(c.compute_delay_hi);
+    m.n0 = to_ticks(c.network_delay_lo); m.n1 = to_ticks(c.network_delay_hi);
+  }
+  m.straggler_q16 = (uint64_t)floor(c.straggler_factor * 65536.0 + 0.5);
+  return m;
+}
+
+// Fill cache.busy / cache.net for rounds [first, last) of every client.
+void fill_delays(const aet_config& c, uint32_t first, uint32_t last, DelayCache& cache) {
+  const uint32_t n = c.n_clients;
+  if (cache.busy.size() != n) { cache.busy.assign(n, {}); cache.net.assign(n, {}); }
+  const uint32_t need = last - c.round_base;
+  bool missing = false;
+  for (uint32_t cl = 0; cl < n; ++cl) missing |= cache.busy[cl].size() < need;
+  if (!missing) return;
+  const DelayModel dm = make_delay_model(c);
+  auto work = [&](uint32_t cl) {
+    const uint64_t kc = stream_key(c.seed, kStreamCompute, cl);
+    const uint64_t kn = stream_key(c.seed, kStreamNetwork, cl);
+    const bool straggler = cl >= n - c.n_stragglers;
+    std::vector<uint64_t>& busy = cache.busy[cl];
+    std::vector<uint64_t>& net = cache.net[cl];
+    for (uint32_t rel = (uint32_t)busy.size(); rel < need; ++rel) {
+      const uint32_t round = c.round_base + rel;
+      const uint64_t it0 = samples_before(c, round) / c.batch;
+      const uint32_t steps = sample_size(c, round) / c.batch;
+      uint64_t sum = 0;
+      for (uint32_t j = 0; j < steps; ++j) {
+        uint64_t dt = dm.compute(draw(kc, it0 + j));
+        if (straggler) { dt = (dt * dm.straggler_q16) >> 16; if (!dt) dt = 1; }
+        sum += dt;
+      }
+      busy.push_back(sum);
+      net.push_back(dm.network(draw(kn, round)));
+    }
+  };
+  unsigned hw = std::thread::hardware_concurrency();
+  unsigned nt = std::max(1u, std::min({hw ? hw : 1u, n, 32u}));
+  if (nt == 1) { for (uint32_t cl = 0; cl < n; ++cl) work(cl); return; }
+  std::vector<std::thread> pool;
+  for (unsigned t = 0; t < nt; ++t)
+    pool.emplace_back([&, t]() { for (uint32_t cl = t; cl < n; cl += nt) work(cl); });
+  for (auto& th : pool) th.join();
+}
+
+enum Kind : uint32_t { kApply = 0, kStart = 1 };
+struct QItem {
+  uint64_t t; uint32_t kind, client, round;
+  bool operator>(const QItem& o) const {
+    return std::tie(t, kind, client, round) > std::tie(o.t, o.kind, o.client, o.round);
+  }
+};
+
+}  // namespace
+
+bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache& cache,
+              SchedResult& out, std::string& err) {
+  const uint32_t n = c.n_clients;
+  if (st.H.size() != n) st.H.assign(n, 0);
+  const uint32_t first = c.round_base + st.rounds_done, last = first + n_rounds;
+  for (uint32_t r = first; r < last; ++r)
+    if (sample_size(c, r) == 0 || sample_size(c, r) % c.batch) {
+      err = "batch must divide every round's sample count, and rounds may not be empty";
+      return false;
+    }
+  fill_delays(c, first, last, cache);
+
+  out.events.clear();
+  out.events.reserve((size_t)n * n_rounds);
+  std::vector<uint32_t>& H = st.H;
+  std::vector<uint64_t> ready(n, st.clock);
+  std::vector<int64_t> blocked(n, -1);  // round a client is waiting to start, or -1
+  std::vector<uint32_t> ev_of((size_t)n * n_rounds);  // (client, round) -> index in out.events
+  std::priority_queue<QItem, std::vector<QItem>, std::greater<QItem>> q;
+  for (uint32_t cl = 0; cl < n && n_rounds; ++cl) q.push({st.clock, kStart, cl, first});
+  const bool never_wait = c.max_lag_d == AET_NEVER_WAIT;
+  uint32_t seq = 0, n_blocked = 0;
+
+  auto lag_of = [&](uint32_t cl, uint32_t round) -> uint32_t {
+    if (n == 1) return 0;
+    uint32_t m = UINT32_MAX;
+    for (uint32_t e = 0; e < n; ++e) if (e != cl && H[e] < m) m = H[e];
+    uint32_t rel = round - c.round_base;
+    return rel > m ? rel - m : 0;
+  };
+
+  while (!q.empty()) {
+    QItem it = q.top();
+    q.pop();
+    if (it.kind == kApply) {
+      H[it.client] += 1;
+      out.events[ev_of[(size_t)it.client * n_rounds + (it.round - first)]].seq = seq++;
+      if (n_blocked) {
+        // min and second min of H once, then an O(1) test per blocked client
+        uint32_t m1 = UINT32_MAX, m2 = UINT32_MAX, c1 = 0;
+        for (uint32_t e = 0; e < n; ++e) {
+          if (H[e] < m1) { m2 = m1; m1 = H[e]; c1 = 1; }
+          else if (H[e] == m1) { ++c1; }
+          else if (H[e] < m2) { m2 = H[e]; }
+        }
+        for (uint32_t b = 0; b < n; ++b) {
+          if (blocked[b] < 0) continue;
+          uint32_t mo = (H[b] == m1 && c1 == 1) ? m2 : m1;
+          uint32_t rel = (uint32_t)blocked[b] - c.round_base;
+          uint32_t lag = rel > mo ? rel - mo : 0;
+          if (never_wait || lag <= c.max_lag_d) {
+            q.push({it.t, kStart, b, (uint32_t)blocked[b]});
+            blocked[b] = -1;
+            --n_blocked;
+          }
+        }
+      }
+      continue;
+    }
+    const uint32_t cl = it.client, round = it.round;
+    const uint32_t lag = lag_of(cl, round);
+    if (!never_wait && lag > c.max_lag_d) { blocked[cl] = round; ++n_blocked; continue; }
+    aet_event e;
+    e.t_start = it.t;
+    e.t_trigger = it.t + cache.busy[cl][round - c.round_base];
+    e.t_apply = e.t_trigger + cache.net[cl][round - c.round_base];
+    e.wait_ticks = it.t - ready[cl];
+    e.client = cl; e.round = round;
+    e.samples = sample_size(c, round);
+    e.steps = e.samples / c.batch;
+    e.seq = 0; e.seen = seq; e.lag = lag; e.pad = 0;
+    ev_of[(size_t)cl * n_rounds + (round - first)] = (uint32_t)out.events.size();
+    out.events.push_back(e);
+    q.push({e.t_apply, kApply, cl, round});
+    ready[cl] = e.t_trigger;
+    if (round + 1 < last) q.push({e.t_trigger, kStart, cl, round + 1});
+  }
+  if (n_blocked || seq != out.events.size()) { err = "schedule did not reach quiescence"; return false; }
+  std::sort(out.events.begin(), out.events.end(),
+            [](const aet_event& a, const aet_event& b) { return a.seq < b.seq; });
+
+  aet_summary& s = out.summary;
+  s = aet_summary{};
+  s.messages_up = s.model_pulls = out.events.size();
+  for (const aet_event& e : out.events) s.samples_total += e.samples;
+  s.messages_if_per_sample = s.samples_total / c.batch;
+  const uint64_t s_first = sample_size(c, c.round_base);
+  const uint64_t per_client = n ? s.samples_total / n : 0;
+  s.messages_if_constant_b = s_first ? n * ((per_client + s_first - 1) / s_first) : 0;
+  s.t_end_ticks = out.events.empty() ? st.clock : out.events.back().t_apply;
+  st.clock = s.t_end_ticks;
+  st.rounds_done += n_rounds;
+  return true;
+}
+
+void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan& plan) {
+  const size_t E = events.size();
+  plan = Plan{};
+  plan.applies.resize(E);
+  // Level of a task = 1 + max(level of every update it starts from, level of
+  // the client's previous round).  Tasks of one level are mutually independent.
+  std::vector<uint32_t> order(E);
+  for (size_t k = 0; k < E; ++k) order[k] = (uint32_t)k;
+  std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+    return std::tie(events[a].t_start, events[a].client) < std::tie(events[b].t_start, events[b].client);
+  });
+  std::vector<uint32_t> level(E, 0), prev_level(c.n_clients, 0);
+  uint32_t pref = 0, pref_max = 0, n_waves = 0;
+  for (uint32_t k : order) {
+    const aet_event& e = events[k];
+    while (pref < e.seen) { pref_max = std::max(pref_max, level[pref]); ++pref; }
+    uint32_t lv = 1 + std::max(pref_max, prev_level[e.client]);
+    level[k] = lv;
+    prev_level[e.client] = lv;
+    n_waves = std::max(n_waves, lv);
+  }
+  // Snapshot slots: one per distinct `seen`; slot 0 is the model at call start.
+  std::vector<int32_t> slot_of(E + 1, -1);
+  slot_of[0] = 0;
+  plan.n_snap = 1;
+  for (const aet_event& e : events) if (slot_of[e.seen] < 0) slot_of[e.seen] = (int32_t)plan.n_snap++;
+  for (size_t k = 0; k < E; ++k) {
+    plan.applies[k].eta = (float)round_step_size(c, events[k].round);
+    plan.applies[k].snap_slot = slot_of[k + 1];
+    plan.applies[k].client = events[k].client;
+    plan.applies[k].round = events[k].round;
+  }
+  // Tasks grouped by wave, longest first.
+  std::vector<uint32_t> by_wave(E);
+  for (size_t k = 0; k < E; ++k) by_wave[k] = (uint32_t)k;
+  std::sort(by_wave.begin(), by_wave.end(), [&](uint32_t a, uint32_t b) {
+    if (level[a] != level[b]) return level[a] < level[b];
+    if (events[a].samples != events[b].samples) return events[a].samples > events[b].samples;
+    return a < b;
+  });
+  // seq of (client, round) for the in-flight lists
+  std::vector<std::vector<uint32_t>> mine(c.n_clients);
+  for (size_t k = 0; k < E; ++k) mine[events[k].client].push_back((uint32_t)k);
+  plan.tasks.reserve(E);
+  plan.wave_off.assign(n_waves + 1, 0);
+  plan.apply_upto.assign(n_waves, 0);
+  for (uint32_t k : by_wave) {
+    const aet_event& e = events[k];
+    TaskDesc t{};
+    t.client = e.client; t.round = e.round; t.seq = e.seq;
+    t.snap_slot = (uint32_t)slot_of[e.seen];
+    t.n_samples = e.samples; t.steps = e.steps;
+    t.sample_ctr0 = samples_before(c, e.round);
+    t.eta = (float)round_step_size(c, e.round);
+    t.inflight_off = (uint32_t)plan.inflight.size();
+    for (uint32_t j : mine[e.client])
+      if (events[j].round < e.round && events[j].seq >= e.seen)
+        plan.inflight.push_back({events[j].seq, (float)round_step_size(c, events[j].round)});
+    t.inflight_cnt = (uint32_t)plan.inflight.size() - t.inflight_off;
+    plan.wave_off[level[k]] += 1;  // size of wave level-1, shifted by one
+    plan.tasks.push_back(t);
+  }
+  // wave_off[L] holds the size of wave L-1; a running sum turns it into offsets.
+  for (uint32_t L = 1; L <= n_waves; ++L) plan.wave_off[L] += plan.wave_off[L - 1];
+  for (uint32_t L = 0; L < n_waves; ++L) {
+    plan.max_wave_tasks = std::max(plan.max_wave_tasks, plan.wave_off[L + 1] - plan.wave_off[L]);
+    // the next wave's tasks need every update with seq < their `seen`
+    uint32_t upto = 0;
+    if (L + 1 < n_waves) {
+      for (uint32_t k = plan.wave_off[L + 1]; k < plan.wave_off[L + 2]; ++k)
+        upto = std::max(upto, events[plan.tasks[k].seq].seen);
+    } else {
+      upto = (uint32_t)E;
+    }
+    plan.apply_upto[L] = std::max(upto, L ? plan.apply_upto[L - 1] : 0u);
+  }
+}
+
+}  // namespace aet

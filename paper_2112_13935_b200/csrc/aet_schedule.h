@@ -1,0 +1,68 @@
+// Host side of the hot path: the integer simulated-time schedule (which client
+// triggers when, in which order the server applies the update sums) and the
+// launch plan that groups independent round-tasks into waves.
+#pragma once
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/aet.h"
+
+namespace aet {
+
+// Simulated-time state carried from one aet_run_rounds call to the next.
+struct SchedState {
+  uint64_t clock = 0;
+  std::vector<uint32_t> H;  // updates of each client the server has applied
+  uint32_t rounds_done = 0;
+};
+
+// Sum of a round's per-iteration compute delays and its network delay depend
+// only on (client, round); cached so a repeated run does not redraw them.
+struct DelayCache {
+  std::vector<std::vector<uint64_t>> busy, net;  // [client][round - round_base]
+};
+
+struct SchedResult {
+  std::vector<aet_event> events;  // ordered by seq
+  aet_summary summary;
+};
+
+uint32_t sample_size(const aet_config& c, uint32_t round);
+uint64_t samples_before(const aet_config& c, uint32_t round);  // rounds round_base .. round-1
+double round_step_size(const aet_config& c, uint32_t round);
+
+// Returns false and fills err on an invalid configuration.
+bool validate_config(const aet_config& c, std::string& err);
+bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache& cache,
+              SchedResult& out, std::string& err);
+
+// ---- launch plan -------------------------------------------------------
+struct TaskDesc {          // one round-task, read by the local-SGD kernels
+  uint32_t client, round, seq;
+  uint32_t snap_slot;      // snapshot of the server model the round starts from
+  uint32_t n_samples, steps;
+  uint32_t inflight_off, inflight_cnt;  // own update sums not yet applied at start
+  uint64_t sample_ctr0;    // client's running sample counter at round start
+  float eta;               // round step size
+  uint32_t pad;
+};
+struct InflightRef { uint32_t seq; float eta; };
+struct ApplyDesc {         // one server update, in seq order
+  float eta;
+  int32_t snap_slot;       // where to keep the model after this update (-1: nowhere)
+  uint32_t client, round;
+};
+struct Plan {
+  std::vector<TaskDesc> tasks;       // sorted by wave, longest first inside a wave
+  std::vector<uint32_t> wave_off;    // tasks of wave L: [wave_off[L], wave_off[L+1])
+  std::vector<uint32_t> apply_upto;  // after wave L the server applies seq < apply_upto[L]
+  std::vector<InflightRef> inflight;
+  std::vector<ApplyDesc> applies;
+  uint32_t n_snap = 0;               // snapshot slots; slot 0 = model at call start
+  uint32_t max_wave_tasks = 0;
+};
+void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan& plan);
+
+}  // namespace aet

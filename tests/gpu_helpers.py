@@ -1,0 +1,56 @@
+"""Shared pieces of the GPU parity tests (every call goes through the C ABI)."""
+import numpy as np
+import torch
+
+from oracle import models, schedule, sim
+from paper_2112_13935_b200 import api, workloads
+
+U_TOL = 1e-5      # max_j |U_gpu - U_ref| / max_j |U_ref| per round-task (fp32 paths)
+LOSS_TOL = 1e-3   # |F(w_gpu) - F(w_ref)|, F evaluated by the checker in fp64
+
+
+def to_device(data):
+    return [(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()) for x, y in data]
+
+
+def make(cfg):
+    data = workloads.make_client_data(cfg)
+    w0 = workloads.make_start_model(cfg)
+    return data, w0
+
+
+def rel_err(got, want):
+    want = np.asarray(want, dtype=np.float64)
+    return float(np.abs(np.asarray(got, dtype=np.float64) - want).max() / max(np.abs(want).max(), 1e-300))
+
+
+def run_gpu(cfg, data, w0, n_rounds=None, want_U=True):
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        s.run(n_rounds)
+        blob, summary = s.log(raw=True)
+        w = s.model()
+        n = len(blob) // 64
+        U = [api.aet_get_update_sum(s.h, k) for k in range(n)] if want_U else None
+        stats = api.aet_get_stats(s.h)
+    return dict(blob=blob, summary=summary, w=w, U=U, stats=stats)
+
+
+def check_against_oracle(cfg, data, w0, gpu, ref, u_tol=U_TOL, loss_tol=LOSS_TOL):
+    assert gpu["blob"] == schedule.pack_events(ref["events"]), "event log differs"
+    assert gpu["summary"] == ref["summary"]
+    dims, l2, prec = cfg["dims"], sim.f32(cfg["l2"]), cfg["precision"]
+    f_gpu = models.full_loss(gpu["w"], data, dims, l2, prec)
+    f_ref = models.full_loss(ref["w"], data, dims, l2, prec)
+    assert abs(f_gpu - f_ref) <= loss_tol, (f_gpu, f_ref)
+    return f_gpu, f_ref
+
+
+def check_round_U(cfg, data, h, c, i, w_start, u_tol=U_TOL):
+    """Round-task (c, i) restarted on both sides from the same fp32 model."""
+    w32 = np.ascontiguousarray(w_start, dtype=np.float32)
+    U_gpu, w_gpu = api.aet_debug_run_client_round(h, c, i, w32)
+    U_ref, w_ref = sim.run_task(cfg, data[c], c, i, w32.astype(np.float64))
+    eu, ew = rel_err(U_gpu, U_ref), rel_err(w_gpu, w_ref)
+    assert eu <= u_tol, (c, i, eu)
+    assert ew <= u_tol, (c, i, ew)
+    return eu

@@ -1,0 +1,108 @@
+"""Host-side checks of the library that need no GPU: exported symbols, the
+integer generator and delay draws, and the schedule against the checker."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from oracle import rng, schedule
+from paper_2112_13935_b200 import _lib, api, build, workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "aet.h")).read()
+    declared = set(re.findall(r"\b(aet_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(_lib.PROTOTYPES), declared ^ set(_lib.PROTOTYPES)
+    lib = ctypes.CDLL(_lib.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_struct_sizes_match_the_header_layout():
+    assert ctypes.sizeof(_lib.AetEvent) == 64
+    assert ctypes.sizeof(_lib.AetSummary) == 48
+    cfg = api.make_config(workloads.get_config("cfg1"))
+    # the library rejects a config whose struct_size it does not recognise
+    ev, _ = api.aet_schedule_only(cfg, 1)
+    assert len(ev) == 4
+    cfg.struct_size += 4
+    with pytest.raises(api.AetError) as e:
+        api.aet_schedule_only(cfg, 1)
+    assert e.value.status == 1
+
+
+def test_generator_and_delay_draws_agree_with_the_checker():
+    for seed, st, c, k in [(0, 0, 0, 0), (0, 1, 3, 17), (12345, 2, 1023, 2 ** 40), (2 ** 63 + 5, 1, 7, 99)]:
+        r = api.aet_debug_draw(seed, st, c, k)
+        assert r == rng.draw(rng.stream_key(seed, st, c), k)
+        for mean in (1, 104858, 1 << 20, 100 << 20):
+            assert api.aet_debug_delay_ticks(0, r, mean) == rng.exp_ticks(r, mean)
+        assert api.aet_debug_delay_ticks(1, r, 1000, 5000) == rng.uniform_ticks(r, 1000, 5000)
+    for r in (0, 1, 2 ** 64 - 1, 2 ** 63):
+        assert api.aet_debug_delay_ticks(0, r, 1 << 20) == rng.exp_ticks(r, 1 << 20)
+
+
+def test_stored_generator_vectors():
+    # vectors written by tests/golden/make_golden.py from the checker alone
+    path = os.path.join(ROOT, "tests", "golden", "rng_vectors.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) >= 6
+    for seed, st, c, k, r, mean, ticks in rows:
+        got = api.aet_debug_draw(int(seed), int(st), int(c), int(k))
+        assert got == int(r, 16)
+        assert api.aet_debug_delay_ticks(0, got, int(mean)) == int(ticks)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4"])
+def test_schedule_is_bit_identical_to_the_checker(name):
+    cfg = workloads.get_config(name)
+    blob, summary = api.aet_schedule_only(cfg, cfg["n_rounds"], raw=True)
+    events, want, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    assert blob == schedule.pack_events(events)
+    assert summary == want
+
+
+@pytest.mark.parametrize("over", [
+    dict(max_lag_d=0), dict(max_lag_d=workloads.NEVER_WAIT), dict(n_clients=1),
+    dict(delay_dist=1), dict(n_stragglers=3, straggler_factor=37.5, max_lag_d=2),
+    dict(round_base=1, sched_b=0, lr_beta=0.01), dict(network_delay_mean=50.0, n_clients=9, max_lag_d=3),
+])
+def test_schedule_variants_match_the_checker(over):
+    cfg = workloads.get_config("cfg1", **over)
+    blob, summary = api.aet_schedule_only(cfg, 7, raw=True)
+    events, want, _ = schedule.simulate(cfg, 7)
+    assert blob == schedule.pack_events(events) and summary == want
+
+
+def test_schedule_rejects_bad_configs():
+    for over, status in [(dict(batch=3), 2), (dict(n_clients=0), 2), (dict(precision=5), 2),
+                         (dict(n_stragglers=9), 2), (dict(lr=0.0), 2), (dict(sched_b=0), 2)]:
+        with pytest.raises(api.AetError) as e:
+            api.aet_schedule_only(workloads.get_config("cfg1", **over), 3)
+        assert e.value.status == status, over
+
+
+def test_wave_plan_counts():
+    # one client: every round depends on the previous one
+    assert api.aet_debug_plan_waves(workloads.get_config("cfg1", n_clients=1), 5) == 5
+    # d = 0: rounds are lock-step, one wave per round
+    assert api.aet_debug_plan_waves(workloads.get_config("cfg1", max_lag_d=0), 5) == 5
+    w = api.aet_debug_plan_waves(workloads.get_config("cfg2"), 30)
+    assert 30 <= w <= 60
+
+
+def test_create_without_a_gpu_fails_cleanly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(api.AetError) as e:
+        api.aet_create(workloads.get_config("cfg1"))
+    assert e.value.status == 5

@@ -1,0 +1,163 @@
+"""GPU parity of the softmax-regression path against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import models, schedule, sim
+from paper_2112_13935_b200 import api, workloads
+from gpu_helpers import (LOSS_TOL, U_TOL, check_against_oracle, check_round_U, make, rel_err,
+                         run_gpu, to_device)
+
+pytestmark = pytest.mark.gpu
+
+
+def test_cfg1_every_round_U_from_the_checkers_start_model():
+    cfg = workloads.get_config("cfg1")
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        worst = max(check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
+                    for e in ref["events"])
+    assert worst <= U_TOL
+
+
+def test_cfg1_end_to_end():
+    cfg = workloads.get_config("cfg1")
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    for k, u in enumerate(gpu["U"]):
+        assert rel_err(u, ref["U"][k]) <= 1e-4, k     # start models differ by fp32 round-off here
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    assert gpu["stats"]["launches"][0] == gpu["stats"]["waves"] == api.aet_debug_plan_waves(cfg, 5)
+
+
+def test_cfg2_end_to_end_full_size():
+    cfg = workloads.get_config("cfg2")
+    data, w0 = make(cfg)
+    assert sorted(len(y) for _, y in data)[0] >= 8 and sum(len(y) for _, y in data) == 60000
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    f_gpu, f_ref = check_against_oracle(cfg, data, w0, gpu, ref)
+    assert f_ref < 0.5 * np.log(10.0)                  # it actually trained
+    # invariant at any size: w_g = w_0 - sum eta_k U_k over the GPU's own update sums
+    acc = w0.astype(np.float64)
+    for e in ref["events"]:
+        acc -= sim.step_size(cfg, e["round"]) * gpu["U"][e["seq"]].astype(np.float64)
+    assert np.abs(acc - gpu["w"]).max() <= 2e-6 * max(1.0, np.abs(acc).max())
+    # sampled round-tasks restarted from the checker's model
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for k in (0, 17, 200, 333, 479):
+            e = ref["events"][k]
+            check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][k])
+
+
+def test_cfg5_shape_64_clients_end_to_end():
+    cfg = workloads.get_config("cfg5", n_clients=64)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0)
+    gpu = run_gpu(cfg, data, w0, want_U=False)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 2e-5
+
+
+@pytest.mark.parametrize("over", [
+    dict(max_lag_d=0), dict(max_lag_d=workloads.NEVER_WAIT, network_delay_mean=20.0),
+    dict(n_clients=1), dict(lr_beta=0.05, l2=0.0), dict(delay_dist=1, n_stragglers=1, straggler_factor=30.0),
+    dict(sched_a=3, sched_b=1, n_rounds=7),   # ragged: rounds of 1, 4, 7, ... samples
+])
+def test_variants_end_to_end(over):
+    cfg = workloads.get_config("cfg1", data=dict(per_client=300), **over)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+
+
+def test_many_own_updates_in_flight():
+    # a slow network keeps several of a client's own sums in flight at round start
+    cfg = workloads.get_config("cfg1", n_clients=2, n_rounds=6, max_lag_d=workloads.NEVER_WAIT,
+                               network_delay_mean=500.0, data=dict(per_client=100))
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0)
+    assert max(e["round"] - sum(1 for f in ref["events"][:e["seen"]] if f["client"] == e["client"])
+               for e in ref["events"]) >= 3
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+
+
+def test_two_runs_are_bit_identical_and_reset_replays():
+    cfg = workloads.get_config("cfg1")
+    data, w0 = make(cfg)
+    a = run_gpu(cfg, data, w0)
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        s.run()
+        w1 = s.model().copy()
+        s.reset()
+        s.run()
+        w2 = s.model()
+        blob, _ = s.log(raw=True)
+    assert a["w"].tobytes() == w1.tobytes() == w2.tobytes()
+    assert blob == a["blob"]
+    assert all(u.tobytes() == v.tobytes() for u, v in zip(a["U"], run_gpu(cfg, data, w0)["U"]))
+
+
+def test_run_in_two_calls_matches_the_checker_continued():
+    cfg = workloads.get_config("cfg1")
+    data, w0 = make(cfg)
+    r1 = sim.run(cfg, data, w0, n_rounds=2)
+    r2 = sim.run(cfg, data, r1["w"], n_rounds=3, state=r1["state"])
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        s.run(2)
+        s.run(3)
+        blob, summary = s.log(raw=True)
+        w = s.model()
+    assert blob == schedule.pack_events(r1["events"]) + schedule.pack_events(r2["events"])
+    assert summary["samples_total"] == 600 and summary["t_end_ticks"] == r2["summary"]["t_end_ticks"]
+    assert np.abs(w - r2["w"]).max() <= 1e-5
+
+
+def test_host_buffers_are_accepted():
+    cfg = workloads.get_config("cfg1", n_rounds=2)
+    data, w0 = make(cfg)
+    gpu_dev = run_gpu(cfg, data, w0)
+    h = api.aet_create(cfg)
+    try:
+        api.aet_set_global_model(h, w0)
+        for c, (x, y) in enumerate(data):
+            api.aet_load_client_data(h, c, np.ascontiguousarray(x), np.ascontiguousarray(y))
+        api.aet_run_rounds(h, 2)
+        out = torch.empty(api.aet_n_params(h), dtype=torch.float32, device="cuda")
+        api.aet_get_global_model(h, out)
+        assert out.cpu().numpy().tobytes() == gpu_dev["w"].tobytes()
+    finally:
+        api.aet_destroy(h)
+
+
+def test_errors_are_reported_not_raised_by_the_device():
+    cfg = workloads.get_config("cfg1")
+    data, w0 = make(cfg)
+    h = api.aet_create(cfg)
+    try:
+        with pytest.raises(api.AetError) as e:
+            api.aet_run_rounds(h, 1)                      # no client data yet
+        assert e.value.status == 3
+        x, y = to_device(data)[0]
+        with pytest.raises(api.AetError) as e:
+            api.aet_load_client_data(h, 9, x, y)          # client out of range
+        assert e.value.status == 1
+        with pytest.raises(api.AetError) as e:
+            api.aet_set_global_model(h, w0[:100].copy())  # wrong length
+        assert e.value.status == 1
+        for c, (x, y) in enumerate(to_device(data)):
+            api.aet_load_client_data(h, c, x, y)
+        api.aet_run_rounds(h, 1)                          # and it still works afterwards
+        assert len(api.aet_get_event_log(h)[0]) == 4
+    finally:
+        api.aet_destroy(h)
+    with pytest.raises(api.AetError) as e:
+        api.aet_create(workloads.get_config("cfg1", dims=[784, 64]))   # too many classes
+    assert e.value.status == 2

@@ -1,0 +1,80 @@
+"""GPU parity of the minibatch MLP path (and of softmax regression shapes that
+go through it) against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sim
+from paper_2112_13935_b200 import api, workloads
+from gpu_helpers import U_TOL, check_against_oracle, check_round_U, make, rel_err, run_gpu, to_device
+
+pytestmark = pytest.mark.gpu
+
+BF16_U_TOL = 2e-3   # precision 1: an fp32-vs-fp64 sum can flip a bf16 rounding (2^-8 relative)
+
+
+def _small_cfg3(**kw):
+    base = dict(n_clients=6, n_rounds=4, data=dict(total=1200))
+    base.update(kw)
+    return workloads.get_config("cfg3", **base)
+
+
+def test_mlp_fp32_small_end_to_end_and_round_U():
+    cfg = _small_cfg3()
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for e in ref["events"][::5]:
+            check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
+
+
+@pytest.mark.parametrize("over", [
+    dict(dims=[784, 37, 10], batch=8, sched_a=8, sched_b=8),            # ragged widths, small batch
+    dict(dims=[784, 24, 12, 10], batch=16, sched_a=16, sched_b=16, l2=1e-3),  # three layers, l2
+    dict(model=0, dims=[50, 7], batch=1, sched_a=5, sched_b=3, data=dict(total=600, dim=50)),  # generic regression
+    dict(model=0, dims=[784, 10], batch=4, sched_a=4, sched_b=4, l2=1e-3),  # minibatch regression
+    dict(n_clients=40, n_rounds=2, data=dict(total=1600)),              # cluster size 2
+    dict(n_clients=2, n_rounds=3, data=dict(total=400)),                # cluster size 8
+])
+def test_mlp_shapes(over):
+    cfg = _small_cfg3(**over)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert rel_err(gpu["w"], ref["w"]) <= 2e-5
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        e = ref["events"][-1]
+        check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
+
+
+def test_mlp_bf16_small_end_to_end_and_round_U():
+    cfg = workloads.get_config("cfg4", n_clients=4, n_rounds=3, dims=[3072, 64, 32, 10],
+                               n_stragglers=1, data=dict(total=800))
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], BF16_U_TOL)
+                for e in ref["events"][::3]]
+    print("bf16 per-round U errors:", ["%.1e" % v for v in errs])
+
+
+def test_cfg3_full_size_log_invariant_and_sampled_rounds():
+    cfg = workloads.get_config("cfg3")
+    data, w0 = make(cfg)
+    from oracle import schedule
+    events, summary, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    gpu = run_gpu(cfg, data, w0)
+    assert gpu["blob"] == schedule.pack_events(events) and gpu["summary"] == summary
+    acc = w0.astype(np.float64)
+    for e in events:
+        acc -= sim.step_size(cfg, e["round"]) * gpu["U"][e["seq"]].astype(np.float64)
+    assert np.abs(acc - gpu["w"]).max() <= 2e-6 * max(1.0, np.abs(acc).max())
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for c, i in ((0, 0), (31, 7), (13, 39)):
+            check_round_U(cfg, data, s.h, c, i, gpu["w"])
