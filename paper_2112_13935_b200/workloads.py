@@ -55,7 +55,9 @@ CONFIGS = {
                  precision=1, sched_a=128, sched_b=128, n_rounds=30,
                  n_stragglers=8, straggler_factor=20.0,
                  data=dict(kind="dirichlet", total=50000, alpha=0.3, dim=3072)),
-    "cfg5": dict(_COMMON, n_clients=1024, model=0, dims=[784, 10], lr=0.01,
+    # lr None: the server sums (not averages) the clients' update sums, so the step
+    # size is scaled with the client count, lr = 0.02 / n_clients (see get_config).
+    "cfg5": dict(_COMMON, n_clients=1024, model=0, dims=[784, 10], lr=None,
                  sched_a=8, sched_b=8, n_rounds=10,
                  data=dict(kind="per_client", per_client=1024, dim=784)),
 }
@@ -68,6 +70,8 @@ def get_config(name: str, **overrides) -> dict:
     cfg.update(overrides)
     if data_over:
         cfg["data"].update(data_over)
+    if cfg["lr"] is None:
+        cfg["lr"] = 0.02 / cfg["n_clients"]
     cfg["name"] = name
     return cfg
 

@@ -34,7 +34,7 @@ def test_mlp_fp32_small_end_to_end_and_round_U():
 @pytest.mark.parametrize("over", [
     dict(dims=[784, 37, 10], batch=8, sched_a=8, sched_b=8),            # ragged widths, small batch
     dict(dims=[784, 24, 12, 10], batch=16, sched_a=16, sched_b=16, l2=1e-3),  # three layers, l2
-    dict(model=0, dims=[50, 7], batch=1, sched_a=5, sched_b=3, data=dict(total=600, dim=50)),  # generic regression
+    dict(model=0, dims=[50, 10], batch=1, sched_a=5, sched_b=3, data=dict(total=600, dim=50)),  # generic regression
     dict(model=0, dims=[784, 10], batch=4, sched_a=4, sched_b=4, l2=1e-3),  # minibatch regression
     dict(n_clients=40, n_rounds=2, data=dict(total=1600)),              # cluster size 2
     dict(n_clients=2, n_rounds=3, data=dict(total=400)),                # cluster size 8
