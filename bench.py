@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the AET-SGD hot path: client-SGD samples per second.
+
+One step = one pass of the whole path (schedule -> waves of local-SGD rounds ->
+ordered aggregation) over one workload: `aet_reset` + `aet_run_rounds(R)`.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+Prints one JSON line.  `value` is device-timed with the inputs resident in HBM;
+`e2e` goes through the C ABI from pinned host buffers; `roofline` is the
+local-SGD kernel against the measured HBM copy bandwidth; `cpu_baseline` is the
+CPU checker timed on this machine.  With several GPUs every rank runs an independent
+replica (own seed) and the job value is all samples over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "client_sgd_samples_per_sec"
+UNIT = "samples/s"
+CPU_BUDGET_S = 15.0      # CPU-baseline sample per run
+REF_STEP_BUDGET_S = 2.5  # --impl reference: CPU work per step
+
+DESCRIBE = {
+    "cfg1": "cfg1: 4 clients, softmax regression 784->10 fp32, l2 1e-4, s_i=10i+10, 5 rounds",
+    "cfg2": "cfg2: 16 clients, softmax regression 784->10 fp32, 60,000 samples Dirichlet(0.5), batch 1, "
+            "s_i=20i+20, 30 rounds, 2 stragglers x10",
+    "cfg3": "cfg3: 32 clients, MLP 784-128-10 fp32, batch 32, s_i=64i+64, 40 rounds",
+    "cfg4": "cfg4: 64 clients, MLP 3072-256-128-10 bf16 operands / fp32 accumulate, batch 64, s_i=128i+128, 30 rounds",
+    "cfg5": "cfg5: 1,024 clients, softmax regression 784->10 fp32, 1,024 samples/client, s_i=8i+8, 10 rounds",
+}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def algorithmic_bytes(cfg, events):
+    """Bytes the local-SGD kernel must move: per sample one row and its label,
+    per round-task the start model in and the update sum out."""
+    from paper_2112_13935_b200 import workloads
+    P = workloads.n_params(cfg["dims"])
+    elem = 2 if cfg["precision"] == 1 else 4
+    per_sample = elem * cfg["dims"][0] + 4
+    samples = sum(e["samples"] for e in events)
+    return samples * per_sample + len(events) * 8 * P
+
+
+def algorithmic_flops(cfg, events):
+    """Dense-contraction flops of the MLP path: forward and weight-gradient
+    products of every layer, input-gradient products of all but the first."""
+    d = cfg["dims"]
+    per_sample = sum(4 * d[l] * d[l + 1] for l in range(len(d) - 1)) + \
+        sum(2 * d[l] * d[l + 1] for l in range(1, len(d) - 1))
+    return per_sample * sum(e["samples"] for e in events)
+
+
+def measured_peak_tflops():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured, sustained bf16"
+    except Exception:
+        return 1400.0, "fallback, sustained bf16"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        try:
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm = [float(r[1]) for r in rows if len(r) >= 9]
+        if not sm:
+            return out
+        out["sm_mhz"] = float(np.median(sm))
+        out["sm_max_mhz"] = float(rows[0][2])
+        out["samples"] = len(sm)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for k, name in enumerate(names):
+            if any(len(r) >= 9 and r[5 + k].strip().lower().startswith("active") for r in rows):
+                out["reasons"].append(name)
+        return out
+
+
+def oracle_bounded(cfg, data, w0, budget_s):
+    """The CPU checker as it stands on a bounded sample of the workload: its
+    schedule, then round-tasks in start order until the time budget is spent."""
+    from oracle import schedule, sim
+    t0 = time.perf_counter()
+    events, _, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    order = sorted(events, key=lambda e: (e["t_start"], e["client"]))
+    w = np.asarray(w0, dtype=np.float64)
+    done_samples, done_tasks = 0, 0
+    for e in order:
+        sim.run_task(cfg, data[e["client"]], e["client"], e["round"], w)
+        done_samples += e["samples"]
+        done_tasks += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return done_samples / dt, done_samples, done_tasks, len(events), dt
+
+
+def blas_threads(cfg):
+    # batch-1 regression is matrix-vector work per sample: one thread does it all
+    return 1 if cfg["model"] == 0 and cfg["batch"] == 1 else (os.cpu_count() or 1)
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU checker, timed per step on a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from threadpoolctl import threadpool_limits
+    from paper_2112_13935_b200 import workloads
+    data = workloads.make_client_data(cfg)
+    w0 = workloads.make_start_model(cfg)
+    cores = blas_threads(cfg)
+    rates, sample = [], ""
+    with threadpool_limits(limits=cores):
+        for step in range(args.warmup + args.steps):
+            rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, REF_STEP_BUDGET_S)
+            if step >= args.warmup:
+                rates.append((n_s, dt))
+            sample = f"schedule + first {n_t} of {n_e} round-tasks in start order ({n_s} samples) per step"
+    total_s = sum(n for n, _ in rates)
+    total_t = sum(t for _, t in rates)
+    value = total_s / total_t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": DESCRIBE[cfg["name"]]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg2", choices=sorted(DESCRIBE))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+
+    from paper_2112_13935_b200 import workloads
+    rank = int(os.environ.get("RANK", "0"))
+    cfg = workloads.get_config(args.workload, seed=rank)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    from paper_2112_13935_b200 import api, dist
+    rank, world, local = dist.init_from_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    stream = torch.cuda.current_stream()
+
+    data = workloads.make_client_data(cfg)
+    w0 = workloads.make_start_model(cfg)
+    R = cfg["n_rounds"]
+    samples = workloads.total_samples(cfg)
+    dev = [(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()) for x, y in data]
+    w0_dev = torch.from_numpy(w0).cuda()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > L2 (126 MB)
+
+    sess = api.Session(cfg, dev, w0_dev)
+    for _ in range(args.warmup):
+        sess.reset()
+        sess.run(R)
+    torch.cuda.synchronize()
+    events, summary = sess.log()
+    assert summary["samples_total"] == samples
+    stats = api.aet_get_stats(sess.h)
+    launches_per_step = sum(stats["launches"])
+
+    # ---- timed region: K steps, each bracketed by events on the launching stream ----
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        for k in range(args.steps):
+            flush.fill_(k & 0xFF)                      # evict L2 between timed iterations
+            sess.reset()
+            starts[k].record(stream)
+            sess.run(R)
+            ends[k].record(stream)
+        torch.cuda.synchronize()
+    dist.barrier()
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    seconds = sum(step_ms) / 1e3
+    value = dist.job_throughput(samples * args.steps, seconds)
+    slowest = dist.max_over_ranks(seconds)
+
+    # ---- per-kernel device time (same steps again with events around every launch) ----
+    api.aet_set_kernel_timing(sess.h, True)
+    k_ms = [0.0, 0.0]
+    k_steps = min(args.steps, 5)
+    for k in range(k_steps):
+        flush.fill_(k & 0xFF)
+        sess.reset()
+        sess.run(R)
+        st = api.aet_get_stats(sess.h)
+        k_ms[0] += st["kernel_ms"][0]
+        k_ms[1] += st["kernel_ms"][1]
+    api.aet_set_kernel_timing(sess.h, False)
+    n_sgd_launches = stats["launches"][0]
+    alg_bytes = algorithmic_bytes(cfg, events)
+    sgd_ms_per_step = k_ms[0] / k_steps
+    achieved = alg_bytes / (sgd_ms_per_step * 1e-3) / 1e9
+    peak, peak_kind = measured_peak_gbs()
+    roof = {"bound": "hbm", "kernel": "local-SGD rounds", "achieved": achieved, "peak": peak,
+            "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind}
+    if cfg["model"] == 1:
+        tf = algorithmic_flops(cfg, events) / (sgd_ms_per_step * 1e-3) / 1e12
+        tpeak, tkind = measured_peak_tflops()
+        roof = {"bound": "tensor", "kernel": "local-SGD rounds (MLP)", "achieved": tf, "peak": tpeak,
+                "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "peak_kind": tkind,
+                "hbm_gbs_algorithmic": achieved}
+    roof.update(launches_per_step=n_sgd_launches, kernel_ms_per_step=sgd_ms_per_step,
+                aggregation_ms_per_step=k_ms[1] / k_steps, algorithmic_bytes_per_step=alg_bytes)
+    sess.close()
+    del dev
+
+    # ---- end to end through the C ABI from pinned host buffers ----
+    pinned = [(torch.from_numpy(x).pin_memory(), torch.from_numpy(y).pin_memory()) for x, y in data]
+    w0_pin = torch.from_numpy(w0).pin_memory()
+    out_pin = torch.empty(w0.size, dtype=torch.float32).pin_memory()
+    h2d = sum(x.numel() * 4 + y.numel() * 4 for x, y in pinned) + w0.size * 4
+    d2h = w0.size * 4
+    e2e_s = []
+    for k in range(args.e2e_steps + 1):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        h = api.aet_create(cfg)
+        api.aet_set_global_model(h, w0_pin)
+        for c, (x, y) in enumerate(pinned):
+            api.aet_load_client_data(h, c, x, y)
+        api.aet_run_rounds(h, R)
+        api.aet_get_global_model(h, out_pin)
+        ev, _ = api.aet_get_event_log(h)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        api.aet_destroy(h)
+        if k > 0:                                      # first one warms allocator and caches
+            e2e_s.append(dt)
+    e2e_value = dist.job_throughput(samples * len(e2e_s), sum(e2e_s))
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from threadpoolctl import threadpool_limits
+        cores = blas_threads(cfg)
+        with threadpool_limits(limits=cores):
+            rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, CPU_BUDGET_S)
+        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"schedule + first {n_t} of {n_e} round-tasks in start order ({n_s} samples, {dt:.1f} s)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * slowest / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == 1 else "f32",
+            "data": "synthetic",
+            "config": {"workload": DESCRIBE[args.workload], "n_clients": cfg["n_clients"], "rounds": R,
+                       "samples_per_step": samples, "events_per_step": len(events),
+                       "waves_per_step": stats["waves"], "l2": "flushed between timed steps (256 MB fill)",
+                       "multi_gpu": "independent replicas, one seed per rank"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": len(e2e_s)},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roof,
+            "cpu_baseline": cpu,
+            "plan_ms_first_run": stats["plan_ms"],
+        }
+        print(json.dumps(line))
+    dist.shutdown()
+
+
+if __name__ == "__main__":
+    main()
