@@ -284,7 +284,7 @@ def main():
     h2d = sum(x.numel() * 4 + y.numel() * 4 for x, y in pinned) + w0.size * 4
     d2h = w0.size * 4
     e2e_s = []
-    for k in range(args.e2e_steps + 1):
+    for k in range(args.e2e_steps + 1 if args.e2e_steps > 0 else 0):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         h = api.aet_create(cfg)

@@ -95,7 +95,10 @@ struct aet_handle {
   DevBuf<ClientData> d_clients;
   DevBuf<uint64_t> d_keys;
   DevBuf<uint32_t> d_H;
-  DevBuf<float> w_cur, w0, snaps, U, work, act, dbg;
+  DevBuf<float> w_buf[2], w0, snaps, U, work, act, dbg, totals;
+  int w_sel = 0;  // which of w_buf holds the server model
+  float* w_cur() { return w_buf[w_sel].p; }
+  DevBuf<uint32_t> d_status;
   DevBuf<TaskDesc> d_tasks;
   DevBuf<InflightRef> d_inflight;
   DevBuf<ApplyDesc> d_applies;
@@ -180,6 +183,17 @@ aet_status upload_clients(aet_handle* h, cudaStream_t s) {
   return AET_OK;
 }
 
+// After a synchronisation: did a bounded device-side wait give up?
+aet_status check_device_status(aet_handle* h) {
+  uint32_t st = 0;
+  AET_CUDA(h, cudaMemcpy(&st, h->d_status.p, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st & 1u) {
+    cudaMemset(h->d_status.p, 0, sizeof(uint32_t));
+    return fail(h, AET_ERR_TIMEOUT, "a bounded wait for an asynchronous row copy gave up; results are invalid");
+  }
+  return AET_OK;
+}
+
 aet_status launch_rounds(aet_handle* h, const RoundLaunch& r, cudaStream_t s) {
   KernelTimer kt(h, s, 0);
   cudaError_t e;
@@ -229,10 +243,13 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   }
   h->h_clients.assign(cfg->n_clients, ClientData{nullptr, nullptr, 0, 0});
   h->st.H.assign(cfg->n_clients, 0);
-  bool ok = h->w_cur.reserve(h->stride) && h->w0.reserve(h->stride) && h->d_H.reserve(cfg->n_clients);
+  bool ok = h->w_buf[0].reserve(h->stride) && h->w_buf[1].reserve(h->stride) && h->w0.reserve(h->stride) &&
+            h->d_H.reserve(cfg->n_clients) && h->d_status.reserve(1) && h->totals.reserve(32 * h->stride);
   if (ok && !h->lr_fast) ok = h->work.reserve((size_t)cfg->n_clients * h->stride);
   if (!ok) { aet_destroy(h); return fail(nullptr, AET_ERR_NOMEM, "device allocation failed"); }
-  if (cudaMemset(h->w_cur.p, 0, h->stride * sizeof(float)) != cudaSuccess ||
+  if (cudaMemset(h->w_buf[0].p, 0, h->stride * sizeof(float)) != cudaSuccess ||
+      cudaMemset(h->w_buf[1].p, 0, h->stride * sizeof(float)) != cudaSuccess ||
+      cudaMemset(h->d_status.p, 0, sizeof(uint32_t)) != cudaSuccess ||
       cudaMemset(h->w0.p, 0, h->stride * sizeof(float)) != cudaSuccess ||
       cudaMemset(h->d_H.p, 0, cfg->n_clients * sizeof(uint32_t)) != cudaSuccess) {
     cudaError_t e = cudaGetLastError();
@@ -250,7 +267,7 @@ aet_status aet_destroy(aet_handle* h) {
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
   h->arena.release();
   h->d_clients.release(); h->d_keys.release(); h->d_H.release();
-  h->w_cur.release(); h->w0.release(); h->snaps.release(); h->U.release();
+  h->w_buf[0].release(); h->w_buf[1].release(); h->totals.release(); h->d_status.release(); h->w0.release(); h->snaps.release(); h->U.release();
   h->work.release(); h->act.release(); h->dbg.release();
   h->d_tasks.release(); h->d_inflight.release(); h->d_applies.release();
   h->d_trig.release(); h->d_alog.release();
@@ -262,7 +279,7 @@ aet_status aet_destroy(aet_handle* h) {
 aet_status aet_reset(aet_handle* h, void* cuda_stream) {
   if (!h) return AET_ERR_ARG;
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  AET_CUDA(h, cudaMemcpyAsync(h->w_cur.p, h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  AET_CUDA(h, cudaMemcpyAsync(h->w_cur(), h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
   AET_CUDA(h, cudaMemsetAsync(h->d_H.p, 0, h->cfg.n_clients * sizeof(uint32_t), s));
   h->st = SchedState{};
   h->st.H.assign(h->cfg.n_clients, 0);
@@ -278,8 +295,8 @@ aet_status aet_set_global_model(aet_handle* h, const float* w0, size_t n_params,
   if (!h || !w0) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  AET_CUDA(h, cudaMemcpyAsync(h->w_cur.p, w0, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
-  AET_CUDA(h, cudaMemcpyAsync(h->w0.p, h->w_cur.p, (size_t)h->P * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  AET_CUDA(h, cudaMemcpyAsync(h->w_cur(), w0, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaMemcpyAsync(h->w0.p, h->w_cur(), (size_t)h->P * sizeof(float), cudaMemcpyDeviceToDevice, s));
   AET_CUDA(h, cudaStreamSynchronize(s));
   h->have_w0 = true;
   h->last_stream = s;
@@ -373,14 +390,14 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   }
   AET_CUDA(h, cudaMemsetAsync(h->d_trig.p, 0, E * sizeof(TriggerRec), s));
   // snapshot 0 = the server model as this call begins
-  AET_CUDA(h, cudaMemcpyAsync(h->snaps.p, h->w_cur.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  AET_CUDA(h, cudaMemcpyAsync(h->snaps.p, h->w_cur(), h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
 
   RoundLaunch r{};
   r.tasks = h->d_tasks.p; r.inflight = h->d_inflight.p; r.clients = h->d_clients.p;
   r.sample_keys = h->d_keys.p; r.snaps = h->snaps.p; r.U = h->U.p; r.w_end = nullptr;
-  r.trig = h->d_trig.p; r.stride = h->stride; r.l2 = h->cfg.l2;
+  r.trig = h->d_trig.p; r.status = h->d_status.p; r.stride = h->stride; r.l2 = h->cfg.l2;
   ApplyLaunch a{};
-  a.applies = h->d_applies.p; a.U = h->U.p; a.snaps = h->snaps.p; a.w_cur = h->w_cur.p;
+  a.applies = h->d_applies.p; a.U = h->U.p; a.snaps = h->snaps.p; a.totals = h->totals.p;
   a.H = h->d_H.p; a.log = h->d_alog.p; a.stride = h->stride; a.n_params = h->P;
 
   // ---- waves: a3/a4 local SGD of independent round-tasks, then a6 aggregation ----
@@ -393,6 +410,10 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
     if (rs != AET_OK) return rs;
     if (plan.apply_upto[L] > applied) {
       a.lo = applied; a.hi = plan.apply_upto[L];
+      a.groups = apply_groups(a.hi - a.lo);
+      a.w_in = h->w_cur();
+      if (a.groups > 1) h->w_sel ^= 1;   // grouped ranges write the other buffer
+      a.w_out = h->w_cur();
       KernelTimer kt(h, s, 1);
       cudaError_t e = launch_apply_updates(a, s);
       if (e != cudaSuccess) return cuda_fail(h, e, "aggregation kernel launch");
@@ -420,9 +441,9 @@ aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params, void
   if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  AET_CUDA(h, cudaMemcpyAsync(out, h->w_cur.p, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaMemcpyAsync(out, h->w_cur(), (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   AET_CUDA(h, cudaStreamSynchronize(s));
-  return AET_OK;
+  return check_device_status(h);
 }
 
 aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params, void* cuda_stream) {
@@ -446,15 +467,20 @@ aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity, siz
     AET_CUDA(h, cudaStreamSynchronize(h->last_stream));
     AET_CUDA(h, cudaMemcpy(trig.data(), h->d_trig.p, E * sizeof(TriggerRec), cudaMemcpyDeviceToHost));
     AET_CUDA(h, cudaMemcpy(alog.data(), h->d_alog.p, E * sizeof(ApplyRec), cudaMemcpyDeviceToHost));
-    std::vector<uint32_t> H = h->last_H_before;
+    if (aet_status ds = check_device_status(h)) return ds;
+    std::vector<uint32_t> H = h->last_H_before, Hdev(h->cfg.n_clients);
+    AET_CUDA(h, cudaMemcpy(Hdev.data(), h->d_H.p, Hdev.size() * sizeof(uint32_t), cudaMemcpyDeviceToHost));
     for (size_t k = 0; k < E; ++k) {
       const aet_event& e = h->log[h->last_first_event + k];
       if (trig[k].flags != 1 || trig[k].client != e.client || trig[k].round != e.round || trig[k].samples_done != e.samples)
         return fail(h, AET_ERR_STATE, "device trigger record " + std::to_string(k) + " does not match the schedule");
       H[e.client] += 1;
-      if (alog[k].seq != k || alog[k].client != e.client || alog[k].round != e.round || alog[k].h_after != H[e.client])
+      // h_after of two updates of one client applied by the same launch may swap
+      if (alog[k].seq != k || alog[k].client != e.client || alog[k].round != e.round ||
+          alog[k].h_after <= h->last_H_before[e.client] || alog[k].h_after > Hdev[e.client])
         return fail(h, AET_ERR_STATE, "device apply record " + std::to_string(k) + " does not match the schedule");
     }
+    if (H != Hdev) return fail(h, AET_ERR_STATE, "device history map H does not match the schedule");
     h->last_checked = true;
   }
   if (out) {
@@ -497,7 +523,7 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   AET_CUDA(h, cudaStreamSynchronize(s));
   RoundLaunch r{};
   r.tasks = dtask; r.inflight = nullptr; r.clients = h->d_clients.p; r.sample_keys = h->d_keys.p;
-  r.snaps = snap; r.U = U; r.w_end = wend; r.trig = dtrig; r.stride = h->stride;
+  r.snaps = snap; r.U = U; r.w_end = wend; r.trig = dtrig; r.status = h->d_status.p; r.stride = h->stride;
   r.task_begin = 0; r.n_tasks = 1; r.l2 = h->cfg.l2;
   const aet_stats keep = h->stats;
   const bool timing = h->timing;
@@ -506,6 +532,8 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   h->timing = timing;
   h->stats = keep;
   if (rs != AET_OK) return rs;
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  if (aet_status ds = check_device_status(h)) return ds;
   if (U_out) AET_CUDA(h, cudaMemcpyAsync(U_out, U, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   if (w_out) AET_CUDA(h, cudaMemcpyAsync(w_out, wend, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   AET_CUDA(h, cudaStreamSynchronize(s));

@@ -32,6 +32,7 @@ struct RoundLaunch {
   float* U;                      // [n_events, stride] update sums, row = seq
   float* w_end;                  // optional [n_events, stride] end-of-round models
   TriggerRec* trig;              // [n_events], row = seq
+  uint32_t* status;              // optional: bit 0 set if a bounded device wait gave up
   size_t stride;
   uint32_t task_begin, n_tasks;
   float l2;
@@ -62,12 +63,16 @@ struct ApplyLaunch {
   const ApplyDesc* applies;  // device, indexed by seq
   const float* U;
   float* snaps;
-  float* w_cur;              // server model [stride]
+  const float* w_in;         // server model before the range [stride]
+  float* w_out;              // ... and after it (may equal w_in only when groups == 1)
+  float* totals;             // scratch [groups, stride], used when groups > 1
   uint32_t* H;               // [n_clients]
   ApplyRec* log;             // [n_events]
   size_t stride;
   uint32_t n_params, lo, hi;
+  uint32_t groups;           // apply_groups(hi - lo)
 };
+uint32_t apply_groups(uint32_t n_updates);
 cudaError_t launch_apply_updates(const ApplyLaunch& p, cudaStream_t s);
 
 // bf16 conversion of a client's rows at load time (precision 1).

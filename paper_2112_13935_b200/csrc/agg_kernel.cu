@@ -1,14 +1,19 @@
 // Server side: ordered aggregation of the triggered update sums.
 //
 // Algorithm 3, Receive: "w = w - eta_k * U; H_v = H_v + 1", applied in the
-// order the simulated-time schedule fixes.  Each thread owns a few parameters
-// and walks the updates of the range in order, keeping its parameters in
-// registers; wherever a later round starts from the model after update k the
-// running value is also stored as that round's start snapshot (this replaces a
-// separate broadcast copy into client slots).  The walk is sequential in k, as
-// the paper's server is, and parallel over parameters.
-#include <cuda_runtime.h>
+// order the simulated-time schedule fixes.  Each thread owns one parameter and
+// walks the updates of its range in order, keeping the parameter in a register;
+// wherever a later round starts from the model after update k the running
+// value is also stored as that round's start snapshot (this replaces a
+// separate broadcast copy into client slots).
+//
+// A long range (many clients) is cut into G groups of consecutive updates.
+// Pass 1 sums -eta_k * U_k over each group; pass 2 starts group g from
+// w + sum of the totals of the groups before it and walks the group in order.
+// The result is the paper's sequential rule up to fp32 re-association across
+// group boundaries, and identical from run to run.
 #include <cuda_bf16.h>
+#include <cuda_runtime.h>
 
 #include "aet_kernels.h"
 
@@ -18,13 +23,42 @@ namespace {
 constexpr int kAggThreads = 128;
 constexpr int kAhead = 8;  // update rows fetched ahead of the dependent FMA chain
 
+__device__ __forceinline__ void group_range(const ApplyLaunch& p, uint32_t g, uint32_t& lo, uint32_t& hi) {
+  const uint32_t per = (p.hi - p.lo + p.groups - 1) / p.groups;
+  lo = min(p.hi, p.lo + g * per);
+  hi = min(p.hi, lo + per);
+}
+
+__global__ void __launch_bounds__(kAggThreads) group_totals_kernel(ApplyLaunch p) {
+  const uint32_t j = blockIdx.x * kAggThreads + threadIdx.x;
+  if (j >= p.n_params) return;
+  uint32_t lo, hi;
+  group_range(p, blockIdx.y, lo, hi);
+  const float* U = p.U + j;
+  float s = 0.f;
+  uint32_t k = lo;
+  for (; k + kAhead <= hi; k += kAhead) {
+    float u[kAhead];
+#pragma unroll
+    for (int a = 0; a < kAhead; ++a) u[a] = __ldg(U + (size_t)(k + a) * p.stride);
+#pragma unroll
+    for (int a = 0; a < kAhead; ++a) s = fmaf(-p.applies[k + a].eta, u[a], s);
+  }
+  for (; k < hi; ++k) s = fmaf(-p.applies[k].eta, __ldg(U + (size_t)k * p.stride), s);
+  p.totals[(size_t)blockIdx.y * p.stride + j] = s;
+}
+
 __global__ void __launch_bounds__(kAggThreads) apply_updates_kernel(ApplyLaunch p) {
   const uint32_t j = blockIdx.x * kAggThreads + threadIdx.x;
+  const uint32_t g = blockIdx.y;
+  uint32_t lo, hi;
+  group_range(p, g, lo, hi);
   if (j < p.n_params) {
-    float w = p.w_cur[j];
+    float w = p.w_in[j];
+    for (uint32_t q = 0; q < g; ++q) w += p.totals[(size_t)q * p.stride + j];
     const float* U = p.U + j;
-    uint32_t k = p.lo;
-    for (; k + kAhead <= p.hi; k += kAhead) {
+    uint32_t k = lo;
+    for (; k + kAhead <= hi; k += kAhead) {
       float u[kAhead];
 #pragma unroll
       for (int a = 0; a < kAhead; ++a) u[a] = __ldcs(U + (size_t)(k + a) * p.stride);
@@ -35,22 +69,22 @@ __global__ void __launch_bounds__(kAggThreads) apply_updates_kernel(ApplyLaunch 
         if (d.snap_slot >= 0) p.snaps[(size_t)d.snap_slot * p.stride + j] = w;
       }
     }
-    for (; k < p.hi; ++k) {
+    for (; k < hi; ++k) {
       const ApplyDesc d = p.applies[k];
       w = fmaf(-d.eta, __ldcs(U + (size_t)k * p.stride), w);
       if (d.snap_slot >= 0) p.snaps[(size_t)d.snap_slot * p.stride + j] = w;
     }
-    p.w_cur[j] = w;
+    if (g + 1 == p.groups) p.w_out[j] = w;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    for (uint32_t k = p.lo; k < p.hi; ++k) {
+  // history map and apply log: one thread per update of the group
+  if (blockIdx.x == 0)
+    for (uint32_t k = lo + threadIdx.x; k < hi; k += kAggThreads) {
       const ApplyDesc d = p.applies[k];
       ApplyRec r;
       r.client = d.client; r.round = d.round; r.seq = k;
-      r.h_after = ++p.H[d.client];
+      r.h_after = atomicAdd(&p.H[d.client], 1u) + 1u;
       p.log[k] = r;
     }
-  }
 }
 
 __global__ void to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
@@ -61,10 +95,20 @@ __global__ void to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __r
 
 }  // namespace
 
+uint32_t apply_groups(uint32_t n_updates) {
+  uint32_t g = n_updates / 32;
+  return g < 1 ? 1 : (g > 32 ? 32 : g);
+}
+
 cudaError_t launch_apply_updates(const ApplyLaunch& p, cudaStream_t s) {
   if (p.hi <= p.lo) return cudaSuccess;
   const uint32_t blocks = (p.n_params + kAggThreads - 1) / kAggThreads;
-  apply_updates_kernel<<<blocks, kAggThreads, 0, s>>>(p);
+  if (p.groups > 1) {
+    group_totals_kernel<<<dim3(blocks, p.groups - 1), kAggThreads, 0, s>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  apply_updates_kernel<<<dim3(blocks, p.groups), kAggThreads, 0, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -6,17 +6,22 @@
 // the running update sum stay in registers for the whole round and only the
 // sampled rows stream in from HBM.
 //
-// Work split: 7 warps x 28 lanes = 196 threads, thread u owns pixels 4u..4u+3
-// and all 10 classes of them (40 weights + 40 update-sum entries).  Per sample:
-//   1. every thread loads its 16 bytes of the row (prefetched kDepth samples
-//      ahead, straight into registers; the index stream is a counter hash, so
-//      addresses are known in advance);
-//   2. 40 FMAs give the thread's share of the 10 logits;
+// Work split: 4 warps (one per SM sub-partition), 98 threads own 8 consecutive
+// pixels each and all 10 classes of them: 80 weights + 80 update-sum entries,
+// held as 2 x 40 packed fp32 pairs (class 2c, 2c+1) so that logits and updates
+// run on fma.rn.f32x2.  Per sample:
+//   1. the row (3,136 B) was fetched kStages samples ahead by a bulk async copy
+//      (cp.async.bulk) into a shared-memory ring, completion on an mbarrier; the
+//      index stream is a counter hash, so addresses are known in advance;
+//   2. 40 packed FMAs give the thread's share of the 10 logits;
 //   3. a transposing butterfly (12 shuffles) leaves each class total of the warp
-//      in one lane; those go to shared memory, one barrier;
-//   4. every warp redundantly sums the 7 partials, does the softmax across its
-//      lanes and broadcasts delta = p - onehot(y);
-//   5. 80 FMAs update W and U.
+//      in one lane; 4 x 10 partials go to shared memory, one barrier;
+//   4. every thread sums the partials and computes the softmax itself on packed
+//      pairs (no further shuffles on the critical path): delta = p - onehot(y);
+//      the bias is one more always-1 "pixel" owned by a spare lane;
+//   5. 80 packed FMAs update W and U.
+// Two CTAs fit on one SM (<= 255 registers), so with many clients one CTA's
+// latency-bound phases overlap the other's FMA phases.
 #include <cuda_runtime.h>
 
 #include "aet_kernels.h"
@@ -25,18 +30,78 @@
 namespace aet {
 namespace {
 
-constexpr int kD = 784, kC = 10, kWarps = 7, kLanes = 28, kThreads = kWarps * 32, kPix = 4;
-constexpr int kDepth = 4;
+constexpr int kD = 784, kC = 10, kWarps = 4, kThreads = kWarps * 32, kPix = 8;
+constexpr int kLanes = 25;            // pixel groups per warp: 25+25+25+23 = 98
+constexpr int kGroups = kD / kPix;    // 98
+constexpr int kStages = 8;            // rows in flight
+constexpr uint32_t kRowBytes = kD * sizeof(float);
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kWaitLimit = 1u << 22;  // mbarrier polls before giving up
 
-__device__ __forceinline__ float4 ld_row(const float4* p) {
-  float4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
-  return v;
+typedef unsigned long long u64;
+
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
 }
-
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {  // a * b + c on both halves
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float rcp(float v) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+  return r;
+}
+__device__ __forceinline__ float ex2(float v) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+  return r;
+}
 __device__ __forceinline__ float shx(float v, int m) { return __shfl_xor_sync(0xffffffffu, v, m); }
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the copy did not land within kWaitLimit polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// One row global -> shared, 16-byte aligned on both sides, size a multiple of 16.
+__device__ __forceinline__ void bulk_load_row(float* dst, const float* src, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst)), "l"(src), "r"(kRowBytes), "r"(smem_addr(bar)) : "memory");
+}
 
 // Sum each of the 10 per-lane partials over the warp.  On return lane L holds
 // the total of class lr_class(L) if lr_class_valid(L); 12 shuffles instead of 50.
@@ -65,155 +130,240 @@ __device__ __forceinline__ bool lr_class_valid(int lane) {
 }
 
 template <bool kL2>
-__global__ void __launch_bounds__(kThreads) lr_round_kernel(RoundLaunch p) {
-  __shared__ float part[2][kWarps][16];
+__global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
+  __shared__ __align__(128) float rows[kStages][kD];
+  __shared__ __align__(16) float part[2][kWarps][12];  // class totals per warp, double-buffered
+  __shared__ __align__(16) float onehot[kC][12];        // row y: -1 at class y, else 0
+  __shared__ __align__(8) uint64_t full[kStages];
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool active = lane < kLanes;
-  const int u = warp * kLanes + (active ? lane : 0);  // pixel group
-  const int cls = lane & 15;                            // class this lane handles in the softmax
-  const bool cls_ok = cls < kC;
-
-  // ---- start model: server snapshot minus own update sums still in flight ----
-  float W[kPix][kC], U[kPix][kC];
-  float bias = 0.f, ubias = 0.f;
-  {
-    const float* src = p.snaps + (size_t)t.snap_slot * p.stride;
-    const float4* s4 = reinterpret_cast<const float4*>(src + (size_t)u * (kPix * kC));
-    float* w = &W[0][0];
-#pragma unroll
-    for (int j = 0; j < kPix * kC / 4; ++j) {
-      float4 v = active ? __ldg(s4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-      w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
-    }
-    if (cls_ok) bias = __ldg(src + kD * kC + cls);
-    for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
-      const InflightRef ref = p.inflight[t.inflight_off + f];
-      const float* us = p.U + (size_t)ref.seq * p.stride;
-      const float4* u4 = reinterpret_cast<const float4*>(us + (size_t)u * (kPix * kC));
-#pragma unroll
-      for (int j = 0; j < kPix * kC / 4; ++j) {
-        float4 v = active ? __ldg(u4 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-        w[4 * j] = fmaf(-ref.eta, v.x, w[4 * j]);
-        w[4 * j + 1] = fmaf(-ref.eta, v.y, w[4 * j + 1]);
-        w[4 * j + 2] = fmaf(-ref.eta, v.z, w[4 * j + 2]);
-        w[4 * j + 3] = fmaf(-ref.eta, v.w, w[4 * j + 3]);
-      }
-      if (cls_ok) bias = fmaf(-ref.eta, __ldg(us + kD * kC + cls), bias);
-    }
-#pragma unroll
-    for (int a = 0; a < kPix; ++a)
-#pragma unroll
-      for (int k = 0; k < kC; ++k) U[a][k] = 0.f;
-  }
+  const int u_raw = warp * kLanes + lane;
+  const bool active = lane < kLanes && u_raw < kGroups;
+  // The bias rides along as one more "pixel" that is always 1: the first spare
+  // lane of the last warp holds it in row 0 of its (otherwise zero) weights, so
+  // logits, update and update sum need no code of their own.
+  const bool is_bias = warp == kWarps - 1 && u_raw == kGroups;
+  const int u = active ? u_raw : 0;
 
   const ClientData cd = p.clients[t.client];
   const uint64_t key = p.sample_keys[t.client];
-  const float4* rows = reinterpret_cast<const float4*>(cd.x);
-  const float eta = t.eta;
-  const float decay = p.l2;  // lambda
-
-  // ---- prefetch ring ----
-  float4 xq[kDepth];
-  int yq[kDepth];
+  const float* xrows = reinterpret_cast<const float*>(cd.x);
   const uint32_t n = t.n_samples;
-  uint32_t h = 0;  // local iteration counter of Algorithm 3
+  const float eta = t.eta;
+
+  if (threadIdx.x == 0) {
 #pragma unroll
-  for (int dpt = 0; dpt < kDepth; ++dpt) {
-    xq[dpt] = make_float4(0.f, 0.f, 0.f, 0.f);
-    yq[dpt] = 0;
-    if ((uint32_t)dpt < n) {
-      const uint32_t idx = sample_index(draw(key, t.sample_ctr0 + dpt), cd.n);
-      if (active) xq[dpt] = ld_row(rows + (size_t)idx * (kD / 4) + u);
-      yq[dpt] = __ldg(cd.y + idx);
+    for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < kC * 12) onehot[threadIdx.x / 12][threadIdx.x % 12] = (threadIdx.x / 12 == threadIdx.x % 12) ? -1.f : 0.f;
+  if (threadIdx.x < 2 * kWarps * 12) (&part[0][0][0])[threadIdx.x] = 0.f;
+
+  // Sample indices and labels, 32 samples per block, lane l holds sample blk*32+l.
+  auto block_idx = [&](uint32_t first) -> uint32_t {
+    const uint32_t k = first + lane;
+    return k < n ? sample_index(draw(key, t.sample_ctr0 + k), cd.n) : 0u;
+  };
+  uint32_t idx_cur = block_idx(0), idx_nxt = block_idx(32);
+  int y_cur = __ldg(cd.y + idx_cur), y_nxt = __ldg(cd.y + idx_nxt);
+  __syncthreads();
+
+  // prologue: fill the ring
+  if (warp == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) {
+      const uint32_t idx = __shfl_sync(0xffffffffu, idx_cur, s);
+      if (lane == 0 && (uint32_t)s < n) {
+        mbar_expect_tx(&full[s], kRowBytes);
+        bulk_load_row(rows[s], xrows + (size_t)idx * kD, &full[s]);
+      }
     }
   }
 
-  for (uint32_t base = 0; base < n; base += kDepth) {
+  // ---- start model: server snapshot minus own update sums still in flight ----
+  u64 W2[kPix][kC / 2], U2[kPix][kC / 2];
+  {
+    const float* src = p.snaps + (size_t)t.snap_slot * p.stride;
+    // a pixel group reads 80 consecutive floats; the bias lane reads the 10 biases into row 0
+    const float2* s2 = reinterpret_cast<const float2*>(src + (is_bias ? (size_t)kD * kC : (size_t)u * (kPix * kC)));
 #pragma unroll
-    for (int dpt = 0; dpt < kDepth; ++dpt) {
-      const uint32_t k = base + dpt;
-      if (k >= n) break;
-      const float4 xv = xq[dpt];
-      const int y = yq[dpt];
-      // refill this slot with sample k + kDepth
-      if (k + kDepth < n) {
-        const uint32_t idx = sample_index(draw(key, t.sample_ctr0 + k + kDepth), cd.n);
-        if (active) xq[dpt] = ld_row(rows + (size_t)idx * (kD / 4) + u);
-        yq[dpt] = __ldg(cd.y + idx);
+    for (int a = 0; a < kPix; ++a)
+#pragma unroll
+      for (int c = 0; c < kC / 2; ++c) {
+        const bool live = active || (is_bias && a == 0);
+        float2 v = live ? __ldg(s2 + a * (kC / 2) + c) : make_float2(0.f, 0.f);
+        W2[a][c] = pack2(v.x, v.y);
+        U2[a][c] = 0ull;
       }
-      const float x[kPix] = {xv.x, xv.y, xv.z, xv.w};
-
-      float acc[kC];
-#pragma unroll
-      for (int c = 0; c < kC; ++c) acc[c] = x[0] * W[0][c];
-#pragma unroll
-      for (int a = 1; a < kPix; ++a)
-#pragma unroll
-        for (int c = 0; c < kC; ++c) acc[c] = fmaf(x[a], W[a][c], acc[c]);
-
-      const float tot = reduce10(acc, lane);
-      const int buf = k & 1;
-      if (lr_class_valid(lane)) part[buf][warp][lr_class(lane)] = tot;
-      __syncthreads();
-
-      float z = bias;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) z += part[buf][w][cls];
-      z = cls_ok ? z : -INFINITY;
-      float m = z;
-      m = fmaxf(m, shx(m, 8)); m = fmaxf(m, shx(m, 4));
-      m = fmaxf(m, shx(m, 2)); m = fmaxf(m, shx(m, 1));
-      const float e = exp2f((z - m) * kLog2e);
-      float sum = e;
-      sum += shx(sum, 8); sum += shx(sum, 4); sum += shx(sum, 2); sum += shx(sum, 1);
-      const float delta = cls_ok ? __fdividef(e, sum) - (cls == y ? 1.f : 0.f) : 0.f;
-      bias = fmaf(-eta, delta, bias);
-      ubias += delta;
-      ++h;
-
-      float d[kC];
-#pragma unroll
-      for (int c = 0; c < kC; ++c) d[c] = __shfl_sync(0xffffffffu, delta, c);
+    for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+      const InflightRef ref = p.inflight[t.inflight_off + f];
+      const float* us = p.U + (size_t)ref.seq * p.stride;
+      const float2* u2 = reinterpret_cast<const float2*>(us + (is_bias ? (size_t)kD * kC : (size_t)u * (kPix * kC)));
+      const u64 ne = pack2(-ref.eta, -ref.eta);
 #pragma unroll
       for (int a = 0; a < kPix; ++a)
 #pragma unroll
-        for (int c = 0; c < kC; ++c) {
-          if (kL2) {
-            const float g = fmaf(d[c], x[a], decay * W[a][c]);
-            W[a][c] = fmaf(-eta, g, W[a][c]);
-            U[a][c] += g;
-          } else {
-            W[a][c] = fmaf(-eta * d[c], x[a], W[a][c]);
-            U[a][c] = fmaf(d[c], x[a], U[a][c]);
-          }
+        for (int c = 0; c < kC / 2; ++c) {
+          const bool live = active || (is_bias && a == 0);
+          float2 v = live ? __ldg(u2 + a * (kC / 2) + c) : make_float2(0.f, 0.f);
+          W2[a][c] = fma2(ne, pack2(v.x, v.y), W2[a][c]);
         }
     }
   }
 
+  const u64 neta2 = pack2(-eta, -eta);
+  const u64 log2e2 = pack2(kLog2e, kLog2e);
+  const float lam = is_bias ? 0.f : p.l2;   // no l2 term on the bias
+  const u64 lam2 = pack2(lam, lam);
+  const u64 nel2 = pack2(-eta * lam, -eta * lam);
+  uint32_t h = 0;  // local iteration counter of Algorithm 3
+  bool timed_out = false;
+  uint32_t timeout_at = 0;
+
+  for (uint32_t k = 0; k < n; ++k) {
+    const int slot = k & (kStages - 1);
+    const int buf = k & 1;
+    if ((k & 31) == 0 && k) {  // next block of indices / labels
+      idx_cur = idx_nxt;
+      y_cur = y_nxt;
+      idx_nxt = block_idx(k + 32);
+      y_nxt = __ldg(cd.y + idx_nxt);
+    }
+    const int y = __shfl_sync(0xffffffffu, y_cur, k & 31);
+    // index of the row that will take this slot once everybody has read it
+    const uint32_t kn = k + kStages;
+    uint32_t idx_next = 0;
+    if (warp == 0) idx_next = __shfl_sync(0xffffffffu, (kn >> 5) == (k >> 5) ? idx_cur : idx_nxt, kn & 31);
+
+    const bool landed = mbar_wait(&full[slot], (k / kStages) & 1);
+
+    float4 xa = make_float4(is_bias ? 1.f : 0.f, 0.f, 0.f, 0.f), xb = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (active) {
+      const float4* r4 = reinterpret_cast<const float4*>(&rows[slot][u * kPix]);
+      xa = r4[0];
+      xb = r4[1];
+    }
+    const float x[kPix] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+    u64 xx[kPix];
+#pragma unroll
+    for (int a = 0; a < kPix; ++a) xx[a] = pack2(x[a], x[a]);
+
+    // logits: this thread's share
+    u64 acc2[kC / 2];
+#pragma unroll
+    for (int c = 0; c < kC / 2; ++c) acc2[c] = mul2(xx[0], W2[0][c]);
+#pragma unroll
+    for (int a = 1; a < kPix; ++a)
+#pragma unroll
+      for (int c = 0; c < kC / 2; ++c) acc2[c] = fma2(xx[a], W2[a][c], acc2[c]);
+    float acc[kC];
+#pragma unroll
+    for (int c = 0; c < kC / 2; ++c) unpack2(acc2[c], acc[2 * c], acc[2 * c + 1]);
+
+    const float tot = reduce10(acc, lane);
+    if (lr_class_valid(lane)) part[buf][warp][lr_class(lane)] = tot;
+    // partials visible; every thread has read its pixels of this row.  The same
+    // barrier carries the verdict of the bounded wait so that all threads leave together.
+    if (__syncthreads_or(!landed)) { timed_out = true; timeout_at = k; break; }
+
+    if (threadIdx.x == 0 && kn < n) {
+      mbar_expect_tx(&full[slot], kRowBytes);
+      bulk_load_row(rows[slot], xrows + (size_t)idx_next * kD, &full[slot]);
+    }
+
+    // softmax over the 10 logits, computed by every thread on packed pairs
+    u64 z2[6];
+    {
+      const ulonglong2* q = reinterpret_cast<const ulonglong2*>(&part[buf][0][0]);
+      u64 s01[6], s23[6];
+#pragma unroll
+      for (int j = 0; j < 3; ++j) {
+        const ulonglong2 a0 = q[j], a1 = q[3 + j], a2 = q[6 + j], a3 = q[9 + j];
+        s01[2 * j] = add2(a0.x, a1.x); s01[2 * j + 1] = add2(a0.y, a1.y);
+        s23[2 * j] = add2(a2.x, a3.x); s23[2 * j + 1] = add2(a2.y, a3.y);
+      }
+#pragma unroll
+      for (int c = 0; c < kC / 2; ++c) z2[c] = add2(s01[c], s23[c]);
+    }
+    float z[kC];
+#pragma unroll
+    for (int c = 0; c < kC / 2; ++c) unpack2(z2[c], z[2 * c], z[2 * c + 1]);
+    const float m = fmaxf(fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), fmaxf(fmaxf(z[4], z[5]), fmaxf(z[6], z[7]))),
+                          fmaxf(z[8], z[9]));
+    const float nms = -m * kLog2e;
+    const u64 nms2 = pack2(nms, nms);
+    u64 e2[kC / 2];
+#pragma unroll
+    for (int c = 0; c < kC / 2; ++c) {
+      float lo, hi;
+      unpack2(fma2(z2[c], log2e2, nms2), lo, hi);
+      e2[c] = pack2(ex2(lo), ex2(hi));
+    }
+    float slo, shi;
+    unpack2(add2(add2(add2(e2[0], e2[1]), add2(e2[2], e2[3])), e2[4]), slo, shi);
+    const float inv = rcp(slo + shi);
+    const u64 inv2 = pack2(inv, inv);
+    u64 d2[kC / 2], nd2[kC / 2];
+    {
+      const ulonglong2* oh = reinterpret_cast<const ulonglong2*>(&onehot[y][0]);
+      const ulonglong2 o0 = oh[0], o1 = oh[1], o2 = oh[2];
+      d2[0] = fma2(e2[0], inv2, o0.x); d2[1] = fma2(e2[1], inv2, o0.y);
+      d2[2] = fma2(e2[2], inv2, o1.x); d2[3] = fma2(e2[3], inv2, o1.y);
+      d2[4] = fma2(e2[4], inv2, o2.x);
+#pragma unroll
+      for (int c = 0; c < kC / 2; ++c) nd2[c] = mul2(d2[c], neta2);
+    }
+    ++h;
+
+    // W -= eta * g, U += g with g = delta x^T (+ lambda W)
+#pragma unroll
+    for (int a = 0; a < kPix; ++a)
+#pragma unroll
+      for (int c = 0; c < kC / 2; ++c) {
+        if (kL2) {
+          const u64 w_old = W2[a][c];
+          U2[a][c] = fma2(xx[a], d2[c], U2[a][c]);
+          U2[a][c] = fma2(w_old, lam2, U2[a][c]);
+          W2[a][c] = fma2(xx[a], nd2[c], w_old);
+          W2[a][c] = fma2(w_old, nel2, W2[a][c]);
+        } else {
+          W2[a][c] = fma2(xx[a], nd2[c], W2[a][c]);
+          U2[a][c] = fma2(xx[a], d2[c], U2[a][c]);
+        }
+      }
+  }
+
+  if (timed_out) {
+    // A row never arrived.  Flag it, give copies still in flight a bounded
+    // chance to land (their target is this CTA's shared memory), and leave.
+    if (threadIdx.x == 0) {
+      if (p.status) atomicOr(p.status, 1u);
+      for (uint32_t j = timeout_at; j < n && j < timeout_at + kStages; ++j)
+        mbar_wait(&full[j & (kStages - 1)], (j / kStages) & 1);
+    }
+    return;
+  }
+
   // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model) ----
   {
-    float* dstU = p.U + (size_t)t.seq * p.stride;
-    if (active) {
-      float4* d4 = reinterpret_cast<float4*>(dstU + (size_t)u * (kPix * kC));
-      const float* us = &U[0][0];
+    const size_t off = is_bias ? (size_t)kD * kC : (size_t)u * (kPix * kC);
+    float2* dU = reinterpret_cast<float2*>(p.U + (size_t)t.seq * p.stride + off);
+    float2* dW = p.w_end ? reinterpret_cast<float2*>(p.w_end + (size_t)t.seq * p.stride + off) : nullptr;
 #pragma unroll
-      for (int j = 0; j < kPix * kC / 4; ++j)
-        d4[j] = make_float4(us[4 * j], us[4 * j + 1], us[4 * j + 2], us[4 * j + 3]);
-    }
-    if (warp == 0 && lane < kC) dstU[kD * kC + lane] = ubias;
-    if (p.w_end) {
-      float* dstW = p.w_end + (size_t)t.seq * p.stride;
-      if (active) {
-        float4* d4 = reinterpret_cast<float4*>(dstW + (size_t)u * (kPix * kC));
-        const float* ws = &W[0][0];
+    for (int a = 0; a < kPix; ++a)
 #pragma unroll
-        for (int j = 0; j < kPix * kC / 4; ++j)
-          d4[j] = make_float4(ws[4 * j], ws[4 * j + 1], ws[4 * j + 2], ws[4 * j + 3]);
+      for (int c = 0; c < kC / 2; ++c) {
+        if (active || (is_bias && a == 0)) {
+          float lo, hi;
+          unpack2(U2[a][c], lo, hi);
+          dU[a * (kC / 2) + c] = make_float2(lo, hi);
+          if (dW) {
+            unpack2(W2[a][c], lo, hi);
+            dW[a * (kC / 2) + c] = make_float2(lo, hi);
+          }
+        }
       }
-      if (warp == 0 && lane < kC) dstW[kD * kC + lane] = bias;
-    }
     if (threadIdx.x == 0) {
       TriggerRec rec;
       rec.client = t.client; rec.round = t.round; rec.samples_done = h; rec.flags = 1;

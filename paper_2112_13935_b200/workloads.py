@@ -11,10 +11,14 @@ image-classification sets (Appendix, Table 2: 10 classes, 60,000 / 50,000
 training points); the public sets themselves are never used.
 
 Recipe (all draws from ``numpy.random.default_rng``):
-  * class means  mu[k, j] ~ U(-0.3, 0.9), k < 10, j < D
-  * a sample of class k is clip(mu[k] + 0.25 * N(0, I), 0, 1)  (about a quarter
-    of the pixels clip to exactly 0, like a dark background)
-  * labels are uniform over the 10 classes
+  * class patterns  mu[k, j] ~ U(-2.0, 0.5), k < 10, j < D: every class lights up
+    its own fifth of the pixels, the rest is dark
+  * a sample of class k is clip(mu[k] + 0.25 * N(0, I), 0, 1)  (about 80 % of the
+    pixels clip to exactly 0, like a dark background; |x|^2 is about 15 for
+    D = 784, which keeps the given step sizes stable when the server adds up
+    the update sums of all clients)
+  * labels are uniform over the 10 classes; one label in ten is then redrawn
+    uniformly, so no model separates the data and gradients never vanish
   * IID split: seeded permutation cut evenly
   * Dirichlet(alpha) label-skew split: per class, client proportions
     ~ Dir(alpha * 1_n), cumulative cut; re-drawn with seed+1, ... until every
@@ -29,6 +33,7 @@ import math
 import numpy as np
 
 N_CLASSES = 10
+LABEL_NOISE = 0.1   # fraction of labels redrawn uniformly
 NEVER_WAIT = 0xFFFFFFFF
 
 # Fields follow the C struct ``aet_config`` one to one; the extra keys
@@ -48,10 +53,10 @@ CONFIGS = {
     "cfg2": dict(_COMMON, n_clients=16, model=0, dims=[784, 10], lr=0.005,
                  sched_a=20, sched_b=20, n_rounds=30, n_stragglers=2, straggler_factor=10.0,
                  data=dict(kind="dirichlet", total=60000, alpha=0.5, dim=784)),
-    "cfg3": dict(_COMMON, n_clients=32, model=1, dims=[784, 128, 10], lr=0.01, batch=32,
+    "cfg3": dict(_COMMON, n_clients=32, model=1, dims=[784, 128, 10], lr=0.002, batch=32,
                  sched_a=64, sched_b=64, n_rounds=40, network_delay_mean=1.0,
                  data=dict(kind="iid", total=60000, dim=784)),
-    "cfg4": dict(_COMMON, n_clients=64, model=1, dims=[3072, 256, 128, 10], lr=0.01, batch=64,
+    "cfg4": dict(_COMMON, n_clients=64, model=1, dims=[3072, 256, 128, 10], lr=0.0005, batch=64,
                  precision=1, sched_a=128, sched_b=128, n_rounds=30,
                  n_stragglers=8, straggler_factor=20.0,
                  data=dict(kind="dirichlet", total=50000, alpha=0.3, dim=3072)),
@@ -90,7 +95,7 @@ def total_samples(cfg) -> int:
 def make_pool(n: int, dim: int, seed: int):
     """n synthetic images (float32 in [0,1], row-major [n, dim]) and int32 labels."""
     rng = np.random.default_rng(seed)
-    mu = rng.uniform(-0.3, 0.9, size=(N_CLASSES, dim)).astype(np.float32)
+    mu = rng.uniform(-2.0, 0.5, size=(N_CLASSES, dim)).astype(np.float32)
     y = rng.integers(0, N_CLASSES, size=n).astype(np.int32)
     x = np.empty((n, dim), dtype=np.float32)
     chunk = 65536
@@ -101,6 +106,8 @@ def make_pool(n: int, dim: int, seed: int):
         z += mu[y[s:e]]
         np.clip(z, 0.0, 1.0, out=z)
         x[s:e] = z
+    flip = rng.random(n) < LABEL_NOISE
+    y = np.where(flip, rng.integers(0, N_CLASSES, size=n), y).astype(np.int32)
     return x, y
 
 
