@@ -191,6 +191,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg2", choices=sorted(DESCRIBE))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--clients", type=int, default=0, help="override the workload's client count (cfg5 sweep)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -198,7 +199,8 @@ def main():
 
     from paper_2112_13935_b200 import workloads
     rank = int(os.environ.get("RANK", "0"))
-    cfg = workloads.get_config(args.workload, seed=rank)
+    over = dict(n_clients=args.clients) if args.clients else {}
+    cfg = workloads.get_config(args.workload, seed=rank, **over)
     if args.impl == "reference":
         run_reference(args, cfg)
         return

@@ -129,11 +129,15 @@ __device__ __forceinline__ bool lr_class_valid(int lane) {
   return (b3 ? !b2 : !(b2 && b1)) && !(lane & 1);
 }
 
-template <bool kL2>
+// kShared: one warp (rotating) computes the softmax and hands delta to the others
+// through shared memory (a second barrier): fewer instructions per sample, more
+// latency - used when enough CTAs share an SM to hide it.
+template <bool kL2, bool kShared>
 __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
   __shared__ __align__(128) float rows[kStages][kD];
   __shared__ __align__(16) float part[2][kWarps][12];  // class totals per warp, double-buffered
   __shared__ __align__(16) float onehot[kC][12];        // row y: -1 at class y, else 0
+  __shared__ __align__(16) float dsm[2][12];            // delta of the current sample (kShared)
   __shared__ __align__(8) uint64_t full[kStages];
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
@@ -159,6 +163,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
   }
   if (threadIdx.x < kC * 12) onehot[threadIdx.x / 12][threadIdx.x % 12] = (threadIdx.x / 12 == threadIdx.x % 12) ? -1.f : 0.f;
   if (threadIdx.x < 2 * kWarps * 12) (&part[0][0][0])[threadIdx.x] = 0.f;
+  if (threadIdx.x < 24) (&dsm[0][0])[threadIdx.x] = 0.f;
 
   // Sample indices and labels, 32 samples per block, lane l holds sample blk*32+l.
   auto block_idx = [&](uint32_t first) -> uint32_t {
@@ -272,6 +277,26 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
       bulk_load_row(rows[slot], xrows + (size_t)idx_next * kD, &full[slot]);
     }
 
+    u64 d2[kC / 2], nd2[kC / 2];
+    if (kShared) {
+      if (warp == (int)(k & (kWarps - 1))) {
+        const int cls = lane & 15;
+        float z = -INFINITY;
+        if (cls < kC) z = (part[buf][0][cls] + part[buf][1][cls]) + (part[buf][2][cls] + part[buf][3][cls]);
+        float m = z;
+        m = fmaxf(m, shx(m, 8)); m = fmaxf(m, shx(m, 4)); m = fmaxf(m, shx(m, 2)); m = fmaxf(m, shx(m, 1));
+        const float e = ex2((z - m) * kLog2e);
+        float sum = e;
+        sum += shx(sum, 8); sum += shx(sum, 4); sum += shx(sum, 2); sum += shx(sum, 1);
+        if (lane < kC) dsm[buf][lane] = fmaf(e, rcp(sum), lane == y ? -1.f : 0.f);
+      }
+      __syncthreads();
+      const ulonglong2* dq = reinterpret_cast<const ulonglong2*>(&dsm[buf][0]);
+      const ulonglong2 q0 = dq[0], q1 = dq[1], q2 = dq[2];
+      d2[0] = q0.x; d2[1] = q0.y; d2[2] = q1.x; d2[3] = q1.y; d2[4] = q2.x;
+#pragma unroll
+      for (int c = 0; c < kC / 2; ++c) nd2[c] = mul2(d2[c], neta2);
+    } else {
     // softmax over the 10 logits, computed by every thread on packed pairs
     u64 z2[6];
     {
@@ -304,7 +329,6 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
     unpack2(add2(add2(add2(e2[0], e2[1]), add2(e2[2], e2[3])), e2[4]), slo, shi);
     const float inv = rcp(slo + shi);
     const u64 inv2 = pack2(inv, inv);
-    u64 d2[kC / 2], nd2[kC / 2];
     {
       const ulonglong2* oh = reinterpret_cast<const ulonglong2*>(&onehot[y][0]);
       const ulonglong2 o0 = oh[0], o1 = oh[1], o2 = oh[2];
@@ -313,6 +337,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
       d2[4] = fma2(e2[4], inv2, o2.x);
 #pragma unroll
       for (int c = 0; c < kC / 2; ++c) nd2[c] = mul2(d2[c], neta2);
+    }
     }
     ++h;
 
@@ -376,10 +401,15 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
 
 cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s) {
   if (p.n_tasks == 0) return cudaSuccess;
-  if (p.l2 != 0.f)
-    lr_round_kernel<true><<<p.n_tasks, kThreads, 0, s>>>(p);
-  else
-    lr_round_kernel<false><<<p.n_tasks, kThreads, 0, s>>>(p);
+  // enough round-tasks to put two CTAs on every SM: trade latency for instruction count
+  const bool shared = p.n_tasks >= 2 * 148;
+  if (p.l2 != 0.f) {
+    if (shared) lr_round_kernel<true, true><<<p.n_tasks, kThreads, 0, s>>>(p);
+    else lr_round_kernel<true, false><<<p.n_tasks, kThreads, 0, s>>>(p);
+  } else {
+    if (shared) lr_round_kernel<false, true><<<p.n_tasks, kThreads, 0, s>>>(p);
+    else lr_round_kernel<false, false><<<p.n_tasks, kThreads, 0, s>>>(p);
+  }
   return cudaGetLastError();
 }
 

@@ -62,6 +62,19 @@ def test_cfg5_shape_64_clients_end_to_end():
     assert np.abs(gpu["w"] - ref["w"]).max() <= 2e-5
 
 
+@pytest.mark.parametrize("l2", [0.0, 1e-3])
+def test_many_clients_take_the_kernel_variant_for_crowded_waves(l2):
+    # >= 296 round-tasks in a wave switch the kernel to its one-warp softmax
+    cfg = workloads.get_config("cfg5", n_clients=320, n_rounds=3, l2=l2, data=dict(per_client=64))
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    for k in (0, 400, 959):
+        assert rel_err(gpu["U"][k], ref["U"][k]) <= 1e-4
+
+
 @pytest.mark.parametrize("over", [
     dict(max_lag_d=0), dict(max_lag_d=workloads.NEVER_WAIT, network_delay_mean=20.0),
     dict(n_clients=1), dict(lr_beta=0.05, l2=0.0), dict(delay_dist=1, n_stragglers=1, straggler_factor=30.0),
