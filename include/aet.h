@@ -176,6 +176,32 @@ size_t aet_n_params(const aet_handle* h);
  * the last aet_create failure of the calling thread. */
 const char* aet_last_error(const aet_handle* h);
 
+/* One round-task with no handle and no allocation (the paper has no counterpart;
+ * this serves callers that may not allocate device memory while they run, e.g.
+ * a process whose memory was handed to a pool at start-up, or one that must keep
+ * the device-wide synchronisation of cudaMalloc off its latency path).  It does
+ * what aet_debug_run_client_round does for fp32 models: round `round` of client
+ * `client` (Algorithm 3, MainComputeNode) from the model w_in, writing the update
+ * sum U_out and the end-of-round model w_out.  x [n, dims[0]] fp32, y [n] int32,
+ * w_in, U_out, w_out (n_params floats each) are DEVICE pointers owned by the
+ * caller.  The kernel's scratch (descriptors, the working model, activations)
+ * is a fixed array inside the library image: every GPU that loads the library
+ * holds about 1 MB for it until the process exits.  Limits: precision 0, at most
+ * 131,072 parameters and 131,072 floats of activation scratch (about
+ * 10 x batch x sum of layer widths); larger requests return AET_ERR_CONFIG
+ * with the sizes in aet_last_error(NULL).  The call is asynchronous on
+ * `cuda_stream`, launches two kernels and calls neither cudaMalloc nor
+ * cudaFree.  Its first call on a device looks the array's device address up
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * All calls share the one array and what the last call left in it (the entry
+ * point clears what must start at zero), so two calls whose kernels could
+ * overlap on the GPU - different streams, different threads - race: keep them
+ * ordered on one stream or synchronise between them. */
+aet_status aet_round_no_alloc(const aet_config* cfg, uint32_t client, uint32_t round,
+                              const float* x, const int32_t* y, uint32_t n,
+                              const float* w_in, float* U_out, float* w_out,
+                              void* cuda_stream);
+
 /* ---- host-only helpers (no GPU needed) -------------------------------- */
 
 /* The integer schedule alone: what aet_run_rounds(n_rounds) on a fresh handle

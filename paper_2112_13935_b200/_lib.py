@@ -68,6 +68,8 @@ PROTOTYPES = {
     "aet_get_stats": (C.c_int, [C.c_void_p, C.POINTER(AetStats)]),
     "aet_n_params": (C.c_size_t, [C.c_void_p]),
     "aet_last_error": (C.c_char_p, [C.c_void_p]),
+    "aet_round_no_alloc": (C.c_int, [C.POINTER(AetConfig), C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
+                                     C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "aet_schedule_only": (C.c_int, [C.POINTER(AetConfig), C.c_uint32, C.POINTER(AetEvent), C.c_size_t,
                                     C.POINTER(C.c_size_t), C.POINTER(AetSummary)]),
     "aet_debug_draw": (C.c_uint64, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64]),

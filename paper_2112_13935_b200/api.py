@@ -142,6 +142,16 @@ def aet_debug_run_client_round(h, client: int, rnd: int, w_in, U_out=None, w_out
     return U_out, w_out
 
 
+def aet_round_no_alloc(cfg, client: int, rnd: int, x, y, w_in, U_out, w_out, stream=None):
+    """One round-task from caller-owned DEVICE buffers, using only the scratch
+    array built into the library: for callers that may not allocate device
+    memory while they run.  Asynchronous on the stream; calls that could overlap
+    on the GPU race on the shared scratch."""
+    conf = cfg if isinstance(cfg, AetConfig) else make_config(cfg)
+    _check(None, _lib.load().aet_round_no_alloc(C.byref(conf), client, rnd, _ptr(x), _ptr(y), x.shape[0],
+                                                _ptr(w_in), _ptr(U_out), _ptr(w_out), _stream(stream)))
+
+
 def aet_set_kernel_timing(h, enable: bool):
     _check(h, _lib.load().aet_set_kernel_timing(h, int(enable)))
 

@@ -76,6 +76,11 @@ struct CachedPlan {
 
 }  // namespace
 
+namespace aet {
+// Lets other translation units of the library set the text aet_last_error(NULL) returns.
+void set_thread_error(const std::string& msg) { g_create_error = msg; }
+}  // namespace aet
+
 struct aet_handle {
   aet_config cfg{};
   uint32_t P = 0;
