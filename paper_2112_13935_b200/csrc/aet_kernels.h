@@ -56,6 +56,9 @@ cudaError_t launch_mlp_rounds(const MlpLaunch& p, cudaStream_t s);
 size_t mlp_act_floats(const MlpShape& shape);
 uint32_t mlp_pick_cluster(const MlpShape& shape, uint32_t n_clients);
 const char* mlp_check_shape(const MlpShape& shape);  // null if the kernel can run it
+// bf16 models whose first layer fits the tensor-core kernel (tcgen05 + TMEM)
+bool mlp_tc_eligible(const MlpShape& shape);
+cudaError_t launch_mlp_tc_rounds(const MlpLaunch& p, cudaStream_t s);
 
 // Ordered aggregation: for seq in [lo, hi): w -= eta_seq * U[seq]; keep a copy
 // where a later round starts from it; bump H and log the apply.

@@ -21,45 +21,16 @@
 
 #include "aet_kernels.h"
 #include "aet_rng.h"
+#include "mlp_common.cuh"
 
 namespace aet {
 namespace {
 
+using namespace mlp;
+
 constexpr int kThreads = 256;
 constexpr int kRC = 32;        // rows of W_l staged per chunk
 constexpr int kMaxTiles = 4;   // 4x4 output micro-tiles per thread in the forward product
-
-__device__ __forceinline__ void cluster_sync(bool clustered) {
-  if (clustered) {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-  } else {
-    __threadfence_block();
-    __syncthreads();
-  }
-}
-__device__ __forceinline__ uint32_t cluster_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ float q_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
-__device__ __forceinline__ int up4(int v) { return (v + 3) & ~3; }
-
-struct Layout {  // offsets (in floats) into the per-task global scratch
-  size_t part[AET_MAX_LAYERS], dz[AET_MAX_LAYERS], a[AET_MAX_LAYERS], total;
-};
-__host__ __device__ inline Layout make_layout(const MlpShape& s) {
-  Layout L{};
-  size_t o = 0;
-  for (uint32_t l = 0; l < s.n_layers; ++l) {
-    const size_t bn = (size_t)s.batch * s.dims[l + 1];
-    L.part[l] = o; o += (size_t)s.cluster * bn;
-    L.dz[l] = o; o += bn;
-    L.a[l] = o; o += bn;
-  }
-  L.total = (o + 31) & ~(size_t)31;
-  return L;
-}
 
 struct Smem {  // offsets (in floats) into dynamic shared memory
   int idx, As, AsT, Ws, dzs, dzq, zs, total;
@@ -421,6 +392,7 @@ uint32_t mlp_pick_cluster(const MlpShape& shape, uint32_t n_clients) {
 
 cudaError_t launch_mlp_rounds(const MlpLaunch& p, cudaStream_t s) {
   if (p.r.n_tasks == 0) return cudaSuccess;
+  if (mlp_tc_eligible(p.shape)) return launch_mlp_tc_rounds(p, s);
   const Smem m = make_smem(p.shape);
   const size_t smem = (size_t)m.total * sizeof(float);
   static size_t configured = 0;

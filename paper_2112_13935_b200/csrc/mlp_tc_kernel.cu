@@ -1,0 +1,629 @@
+// Local-SGD round of one client for a bf16-operand ReLU MLP: the two products
+// of the wide first layer run on the 5th-generation tensor cores.
+//
+// Algorithm 3, MainComputeNode, inner loop with xi a minibatch (mean gradient;
+// w_c -= eta_i g; U_i += g).  Same cluster structure as the fp32 kernel: every
+// W_l is split by input rows over the CTAs of the round-task's cluster.  What
+// changes is layer 0, which carries ~95 % of the flops of a 3072-256-128-10 net:
+//   forward   Z0^T[out0 x B] += W0[rows]^T . X[:, rows]^T   chunks of 64 input rows:
+//             A = bf16(W0 chunk)^T [out0 x 64] (converted from the fp32 master on
+//             the way into shared memory), B = X chunk [B x 64]; tcgen05.mma
+//             M = 128 (x out0/128), N = B, K = 16 x 4, fp32 accumulators in TMEM;
+//             operand tiles double-buffered, completion by tcgen05.commit on mbarriers;
+//   backward  G[128 rows x out0] = X[:, rows]^T . dZ0       chunks of 128 input rows:
+//             A = X chunk^T [128 x B], B = bf16(dZ0)^T [out0 x B]; M = 128, N = out0,
+//             K = B; two TMEM accumulators so the MMAs of chunk c+1 run while the
+//             epilogue of chunk c reads its tile back (tcgen05.ld) and does
+//             g = G + lambda W, W -= eta g, U += g on the fp32 master in HBM/L2.
+// Operand tiles use the K-major, no-swizzle core-matrix layout (8 rows x 16 bytes
+// contiguous; LBO = stride between core matrices along K, SBO = along M/N).
+// The narrow layers (l >= 1), softmax and bias updates run on plain FMAs.
+// Every mbarrier wait is bounded; after a timeout the CTA flags `status`, stops
+// polling and keeps to the barrier schedule so that its cluster peers never block.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "aet_kernels.h"
+#include "aet_rng.h"
+#include "mlp_common.cuh"
+
+namespace aet {
+namespace {
+
+using namespace mlp;
+
+constexpr int kThreads = 256;
+constexpr int kRC = 32;        // rows per chunk of the FMA layers
+constexpr int kMaxTiles = 4;
+constexpr int kKC = 64;        // input rows per forward chunk
+constexpr int kMT = 128;       // input rows per backward chunk (M of the MMA)
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+struct TcSmem {  // byte offsets into dynamic shared memory
+  int tiles, idx, As, AsT, Ws, dzs, dzq, zs, total;
+};
+__host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
+  const int B = (int)s.batch, out0 = (int)s.dims[1];
+  int nmax = 0;
+  for (uint32_t l = 1; l < s.n_layers; ++l) nmax = max(nmax, (int)((s.dims[l + 1] + 3) & ~3u));
+  const int fwd = 2 * out0 * kKC * 2 + 2 * B * kKC * 2;
+  const int bwd = 2 * kMT * B * 2 + out0 * B * 2;
+  TcSmem m{};
+  int o = 0;
+  m.tiles = o; o += max(fwd, bwd);
+  m.idx = o; o += B * 4;
+  m.As = o; o += kRC * B * 4;
+  m.AsT = o; o += B * kRC * 4;
+  m.Ws = o; o += kRC * (nmax + 4) * 4;
+  m.dzs = o; o += B * nmax * 4;
+  m.dzq = o; o += B * nmax * 4;
+  m.zs = o; o += B * 32 * 4;
+  m.total = o;
+  return m;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Shared-memory matrix descriptor: K-major, no swizzle.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major.
+__device__ __forceinline__ uint32_t umma_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// One mbarrier that tcgen05.commit arrives on, with the bookkeeping that keeps
+// waits and completions paired (never more than one completion ahead).
+struct CommitBar {
+  uint64_t* bar;
+  uint32_t issued, waited;
+};
+__device__ __forceinline__ void bar_drain(CommitBar& b, bool& failed) {
+  while (b.waited < b.issued) {
+    const uint32_t parity = b.waited & 1u;
+    bool ok = failed;  // after a timeout: stop polling, keep the counters moving
+    for (uint32_t i = 0; i < kWaitLimit && !ok; ++i) {
+      uint32_t p;
+      asm volatile("{\n\t.reg .pred q;\n\tmbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                   : "=r"(p) : "r"(smem_u32(b.bar)), "r"(parity) : "memory");
+      ok = p != 0;
+    }
+    if (!ok) failed = true;
+    ++b.waited;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
+  extern __shared__ __align__(1024) unsigned char smraw[];
+  __shared__ __align__(8) uint64_t bars[4];
+  __shared__ uint32_t tmem_base_s;
+
+  const MlpShape& S = p.shape;
+  const int C = (int)S.cluster;
+  const bool clustered = C > 1;
+  const int rank = clustered ? (int)cluster_rank() : 0;
+  const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / C];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int L = (int)S.n_layers, B = (int)S.batch;
+  const int D0 = (int)S.dims[0], out0 = (int)S.dims[1];
+  const TcSmem M = make_tc_smem(S);
+  const Layout G = make_layout(S);
+  unsigned char* tiles = smraw + M.tiles;
+  int* idx = reinterpret_cast<int*>(smraw + M.idx);
+  float* As = reinterpret_cast<float*>(smraw + M.As);
+  float* AsT = reinterpret_cast<float*>(smraw + M.AsT);
+  float* Ws = reinterpret_cast<float*>(smraw + M.Ws);
+  float* dzs = reinterpret_cast<float*>(smraw + M.dzs);
+  float* dzq = reinterpret_cast<float*>(smraw + M.dzq);
+  float* zs = reinterpret_cast<float*>(smraw + M.zs);
+
+  float* act = p.act + (size_t)(blockIdx.x / C) * p.act_stride;
+  float* work = p.work + (size_t)t.client * p.r.stride;
+  float* Urow = p.r.U + (size_t)t.seq * p.r.stride;
+  const ClientData cd = p.r.clients[t.client];
+  const __nv_bfloat16* xdata = reinterpret_cast<const __nv_bfloat16*>(cd.x);
+  const uint64_t key = p.r.sample_keys[t.client];
+  const float eta = t.eta, lambda = p.r.l2;
+
+  size_t woff[AET_MAX_LAYERS], boff[AET_MAX_LAYERS];
+  int r0[AET_MAX_LAYERS], r1[AET_MAX_LAYERS];
+  {
+    size_t o = 0;
+    for (int l = 0; l < L; ++l) {
+      woff[l] = o; o += (size_t)S.dims[l] * S.dims[l + 1];
+      boff[l] = o; o += S.dims[l + 1];
+      r0[l] = (int)(((long long)S.dims[l] * rank) / C);
+      r1[l] = (int)(((long long)S.dims[l] * (rank + 1)) / C);
+    }
+  }
+
+  // ---- barriers and tensor memory ----
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[i])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = tmem_base_s;
+  CommitBar fbar[2] = {{&bars[0], 0, 0}, {&bars[1], 0, 0}};
+  CommitBar bbar[2] = {{&bars[2], 0, 0}, {&bars[3], 0, 0}};
+  bool failed = false;
+
+  // ---- start model into the client's work row: snapshot - own in-flight sums ----
+  {
+    const float* snap = p.r.snaps + (size_t)t.snap_slot * p.r.stride;
+    for (int l = 0; l < L; ++l) {
+      const int N = (int)S.dims[l + 1];
+      const size_t lo = woff[l] + (size_t)r0[l] * N, hi = woff[l] + (size_t)r1[l] * N;
+      for (size_t j = lo + tid; j < hi; j += kThreads) {
+        float w = snap[j];
+        for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+          const InflightRef ref = p.r.inflight[t.inflight_off + f];
+          w = fmaf(-ref.eta, p.r.U[(size_t)ref.seq * p.r.stride + j], w);
+        }
+        work[j] = w;
+        Urow[j] = 0.f;
+      }
+      if (rank == l % C)
+        for (int j = tid; j < N; j += kThreads) {
+          float w = snap[boff[l] + j];
+          for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+            const InflightRef ref = p.r.inflight[t.inflight_off + f];
+            w = fmaf(-ref.eta, p.r.U[(size_t)ref.seq * p.r.stride + boff[l] + j], w);
+          }
+          work[boff[l] + j] = w;
+          Urow[boff[l] + j] = 0.f;
+        }
+    }
+  }
+  cluster_sync(clustered);
+
+  const int R0 = r1[0] - r0[0];
+  const uint32_t sbo_k64 = (kKC / 8) * 128;   // tiles with K = 64: next 8-row group after 8 core matrices
+  const uint32_t sbo_kB = (B / 8) * 128;      // tiles with K = B
+  uint32_t h = 0;
+
+  for (uint32_t it = 0; it < t.steps; ++it) {
+    for (int b = tid; b < B; b += kThreads)
+      idx[b] = (int)sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * B + b), cd.n);
+    __syncthreads();
+
+    // ================= forward, layer 0 (tensor cores) =================
+    {
+      const int n_mt = out0 / 128;
+      const uint32_t idesc = umma_idesc(128, B);
+      const int a_bytes = out0 * kKC * 2, b_bytes = B * kKC * 2;
+      for (int c = 0; c * kKC < R0; ++c) {
+        const int s = c & 1, c0 = r0[0] + c * kKC;
+        unsigned char* tA = tiles + s * a_bytes;
+        unsigned char* tB = tiles + 2 * a_bytes + s * b_bytes;
+        bar_drain(fbar[s], failed);  // the MMAs that last read this buffer are done
+        // A: bf16(W0[c0 + k, j]) as element (row j, col k)
+        for (int e = tid; e < out0 * (kKC / 8); e += kThreads) {
+          const int j = e % out0, kg = e / out0;
+          const float* src = work + woff[0] + (size_t)(c0 + kg * 8) * out0 + j;
+          uint4 v;
+          v.x = pack_bf16(src[0], src[out0]);
+          v.y = pack_bf16(src[2 * (size_t)out0], src[3 * (size_t)out0]);
+          v.z = pack_bf16(src[4 * (size_t)out0], src[5 * (size_t)out0]);
+          v.w = pack_bf16(src[6 * (size_t)out0], src[7 * (size_t)out0]);
+          *reinterpret_cast<uint4*>(tA + (j >> 3) * sbo_k64 + kg * 128 + (j & 7) * 16) = v;
+        }
+        // B: X[idx[b], c0 + k] as element (row b, col k); already bf16 in HBM
+        for (int e = tid; e < B * (kKC / 8); e += kThreads) {
+          const int kg = e % (kKC / 8), b = e / (kKC / 8);
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(xdata + (size_t)idx[b] * D0 + c0 + kg * 8));
+          *reinterpret_cast<uint4*>(tB + (b >> 3) * sbo_k64 + kg * 128 + (b & 7) * 16) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          for (int mt = 0; mt < n_mt; ++mt)
+            for (int j = 0; j < kKC / 16; ++j)
+              umma_bf16(tmem + mt * B,
+                        umma_desc(smem_u32(tA) + mt * 16 * sbo_k64 + j * 256, 128, sbo_k64),
+                        umma_desc(smem_u32(tB) + j * 256, 128, sbo_k64), idesc, (c > 0 || j > 0) ? 1u : 0u);
+          umma_commit(fbar[s].bar);
+        }
+        ++fbar[s].issued;
+      }
+      bar_drain(fbar[0], failed);
+      bar_drain(fbar[1], failed);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      // partial Z0^T (lane = hidden unit, column = batch index) -> global scratch [b][n]
+      {
+        float* part = act + G.part[0] + (size_t)rank * B * out0;
+        const int span = n_mt * B, half = span / 2;
+        for (int cc0 = (warp >> 2) * half; cc0 < ((warp >> 2) + 1) * half; cc0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + cc0, v);
+          const int mt = cc0 / B, b0 = cc0 % B;
+          const int n = mt * 128 + (warp & 3) * 32 + lane;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) part[(size_t)(b0 + i) * out0 + n] = __uint_as_float(v[i]);
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      cluster_sync(clustered);
+      // bias + ReLU + bf16 rounding of the columns this CTA feeds into layer 1
+      {
+        const float* part0 = act + G.part[0];
+        const float* bias = work + boff[0];
+        const int c_lo = r0[1], c_n = r1[1] - r0[1];
+        for (int e = tid; e < B * c_n; e += kThreads) {
+          const int b = e / c_n, n = c_lo + e % c_n;
+          float z = bias[n];
+          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * out0 + n];
+          act[G.a[0] + (size_t)b * out0 + n] = q_bf16(fmaxf(z, 0.f));
+        }
+        __syncthreads();
+      }
+    }
+
+    // ================= forward, layers >= 1 (FMA) =================
+    for (int l = 1; l < L; ++l) {
+      const int N = (int)S.dims[l + 1], Np = up4(N), ldw = Np + 4;
+      const int tiles_n = Np / 4, ntile = (B / 4) * tiles_n;
+      float acc[kMaxTiles][16];
+#pragma unroll
+      for (int q = 0; q < kMaxTiles; ++q)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[q][e] = 0.f;
+      for (int c0 = r0[l]; c0 < r1[l]; c0 += kRC) {
+        const int rc = min(kRC, r1[l] - c0);
+        __syncthreads();
+        for (int e = tid; e < kRC * B; e += kThreads) {
+          const int b = e / kRC, ic = e % kRC;
+          As[ic * B + b] = ic < rc ? act[G.a[l - 1] + (size_t)b * S.dims[l] + c0 + ic] : 0.f;
+        }
+        for (int e = tid; e < kRC * Np; e += kThreads) {
+          const int ic = e / Np, j = e % Np;
+          Ws[ic * ldw + j] = (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kMaxTiles; ++q) {
+          const int mt = tid + q * kThreads;
+          if (mt < ntile) {
+            const int bt = mt / tiles_n, jt = mt % tiles_n;
+            for (int ic = 0; ic < rc; ++ic) {
+              const float4 a = *reinterpret_cast<const float4*>(As + ic * B + 4 * bt);
+              const float4 w = *reinterpret_cast<const float4*>(Ws + ic * ldw + 4 * jt);
+              const float av[4] = {a.x, a.y, a.z, a.w}, wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[q][4 * i + j] = fmaf(av[i], wv[j], acc[q][4 * i + j]);
+            }
+          }
+        }
+      }
+      {
+        float* part = act + G.part[l] + (size_t)rank * B * N;
+#pragma unroll
+        for (int q = 0; q < kMaxTiles; ++q) {
+          const int mt = tid + q * kThreads;
+          if (mt < ntile) {
+            const int bt = mt / tiles_n, jt = mt % tiles_n;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int n = 4 * jt + j;
+                if (n < N) part[(size_t)(4 * bt + i) * N + n] = acc[q][4 * i + j];
+              }
+          }
+        }
+      }
+      cluster_sync(clustered);
+      const float* part0 = act + G.part[l];
+      const float* bias = work + boff[l];
+      if (l < L - 1) {
+        const int c_lo = r0[l + 1], c_n = r1[l + 1] - r0[l + 1];
+        for (int e = tid; e < B * c_n; e += kThreads) {
+          const int b = e / c_n, n = c_lo + e % c_n;
+          float z = bias[n];
+          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
+          act[G.a[l] + (size_t)b * N + n] = q_bf16(fmaxf(z, 0.f));
+        }
+        __syncthreads();
+      } else {
+        for (int e = tid; e < B * N; e += kThreads) {
+          const int b = e / N, n = e % N;
+          float z = bias[n];
+          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
+          zs[b * 32 + n] = z;
+        }
+        __syncthreads();
+        for (int b = tid; b < B; b += kThreads) {
+          float m = -INFINITY;
+          for (int n = 0; n < N; ++n) m = fmaxf(m, zs[b * 32 + n]);
+          float sum = 0.f;
+          for (int n = 0; n < N; ++n) sum += __expf(zs[b * 32 + n] - m);
+          const int y = cd.y[idx[b]];
+          const float inv = 1.f / sum, invB = 1.f / (float)B;
+          for (int n = 0; n < Np; ++n) {
+            float d = 0.f;
+            if (n < N) d = (__expf(zs[b * 32 + n] - m) * inv - (n == y ? 1.f : 0.f)) * invB;
+            dzs[b * Np + n] = d;
+            dzq[b * Np + n] = q_bf16(d);
+          }
+        }
+        __syncthreads();
+      }
+    }
+
+    // ================= backward + update, layers >= 1 (FMA) =================
+    for (int l = L - 1; l >= 1; --l) {
+      const int N = (int)S.dims[l + 1], Np = up4(N), ldw = Np + 4;
+      const int K = (int)S.dims[l];
+      for (int c0 = r0[l]; c0 < r1[l]; c0 += kRC) {
+        const int rc = min(kRC, r1[l] - c0);
+        __syncthreads();
+        for (int e = tid; e < kRC * B; e += kThreads) {
+          const int b = e / kRC, ic = e % kRC;
+          AsT[b * kRC + ic] = ic < rc ? act[G.a[l - 1] + (size_t)b * K + c0 + ic] : 0.f;
+        }
+        for (int e = tid; e < kRC * Np; e += kThreads) {
+          const int ic = e / Np, j = e % Np;
+          Ws[ic * ldw + j] = (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f;
+        }
+        __syncthreads();
+        for (int e = tid; e < B * rc; e += kThreads) {
+          const int b = e / rc, ic = e % rc;
+          float s = 0.f;
+          for (int j = 0; j < Np; j += 4) {
+            const float4 d = *reinterpret_cast<const float4*>(dzq + b * Np + j);
+            const float4 w = *reinterpret_cast<const float4*>(Ws + ic * ldw + j);
+            s = fmaf(d.x, w.x, s); s = fmaf(d.y, w.y, s); s = fmaf(d.z, w.z, s); s = fmaf(d.w, w.w, s);
+          }
+          act[G.dz[l - 1] + (size_t)b * K + c0 + ic] = AsT[b * kRC + ic] > 0.f ? s : 0.f;
+        }
+        {
+          const int tiles_n = Np / 4, ntile = (kRC / 4) * tiles_n;
+          for (int mt = tid; mt < ntile; mt += kThreads) {
+            const int it4 = mt / tiles_n, jt = mt % tiles_n;
+            float g[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) g[e] = 0.f;
+            for (int b = 0; b < B; ++b) {
+              const float4 a = *reinterpret_cast<const float4*>(AsT + b * kRC + 4 * it4);
+              const float4 d = *reinterpret_cast<const float4*>(dzq + b * Np + 4 * jt);
+              const float av[4] = {a.x, a.y, a.z, a.w}, dv[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) g[4 * i + j] = fmaf(av[i], dv[j], g[4 * i + j]);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int ic = 4 * it4 + i;
+              if (ic >= rc) continue;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int n = 4 * jt + j;
+                if (n >= N) continue;
+                const size_t o = woff[l] + (size_t)(c0 + ic) * N + n;
+                const float w = work[o];
+                const float gg = fmaf(lambda, w, g[4 * i + j]);
+                work[o] = fmaf(-eta, gg, w);
+                Urow[o] += gg;
+              }
+            }
+          }
+        }
+      }
+      cluster_sync(clustered);
+      if (rank == l % C)
+        for (int n = tid; n < N; n += kThreads) {
+          float gb = 0.f;
+          for (int b = 0; b < B; ++b) gb += dzs[b * Np + n];
+          work[boff[l] + n] = fmaf(-eta, gb, work[boff[l] + n]);
+          Urow[boff[l] + n] += gb;
+        }
+      if (l > 1) {
+        __syncthreads();
+        const int Nm = (int)S.dims[l], Nmp = up4(Nm);
+        for (int e = tid; e < B * Nmp; e += kThreads) {
+          const int b = e / Nmp, n = e % Nmp;
+          const float d = n < Nm ? act[G.dz[l - 1] + (size_t)b * Nm + n] : 0.f;
+          dzs[b * Nmp + n] = d;
+          dzq[b * Nmp + n] = q_bf16(d);
+        }
+        __syncthreads();
+      }
+    }
+
+    // ================= backward + update, layer 0 (tensor cores) =================
+    {
+      const float* dz0 = act + G.dz[0];          // full dZ0 [B, out0], fp32, visible after the barrier above
+      const int a_bytes = kMT * B * 2;
+      unsigned char* tBd = tiles + 2 * a_bytes;  // bf16(dZ0)^T: element (row j, col b)
+      const uint32_t idesc = umma_idesc(128, out0);
+      __syncthreads();
+      for (int e = tid; e < out0 * (B / 8); e += kThreads) {
+        const int j = e % out0, bg = e / out0;
+        const float* src = dz0 + (size_t)(bg * 8) * out0 + j;
+        uint4 v;
+        v.x = pack_bf16(src[0], src[out0]);
+        v.y = pack_bf16(src[2 * (size_t)out0], src[3 * (size_t)out0]);
+        v.z = pack_bf16(src[4 * (size_t)out0], src[5 * (size_t)out0]);
+        v.w = pack_bf16(src[6 * (size_t)out0], src[7 * (size_t)out0]);
+        *reinterpret_cast<uint4*>(tBd + (j >> 3) * sbo_kB + bg * 128 + (j & 7) * 16) = v;
+      }
+      const int nch = R0 / kMT;
+      auto stage_and_issue = [&](int c) {
+        const int s = c & 1, c0 = r0[0] + c * kMT;
+        unsigned char* tA = tiles + s * a_bytes;  // X^T chunk: element (row i, col b)
+        for (int e = tid; e < kMT * (B / 8); e += kThreads) {
+          const int i = e % kMT, bg = e / kMT;
+          const __nv_bfloat16* col = xdata + c0 + i;
+          unsigned short q[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) q[k] = __ldg(reinterpret_cast<const unsigned short*>(col + (size_t)idx[bg * 8 + k] * D0));
+          uint4 v;
+          v.x = q[0] | ((uint32_t)q[1] << 16); v.y = q[2] | ((uint32_t)q[3] << 16);
+          v.z = q[4] | ((uint32_t)q[5] << 16); v.w = q[6] | ((uint32_t)q[7] << 16);
+          *reinterpret_cast<uint4*>(tA + (i >> 3) * sbo_kB + bg * 128 + (i & 7) * 16) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          for (int j = 0; j < B / 16; ++j)
+            umma_bf16(tmem + s * 256, umma_desc(smem_u32(tA) + j * 256, 128, sbo_kB),
+                      umma_desc(smem_u32(tBd) + j * 256, 128, sbo_kB), idesc, j > 0 ? 1u : 0u);
+          umma_commit(bbar[s].bar);
+        }
+        ++bbar[s].issued;
+      };
+      if (nch > 0) stage_and_issue(0);
+      for (int c = 0; c < nch; ++c) {
+        const int s = c & 1, c0 = r0[0] + c * kMT;
+        if (c + 1 < nch) stage_and_issue(c + 1);   // its buffer and accumulator were released by chunk c-1
+        bar_drain(bbar[s], failed);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // epilogue: thread = one row of W0, half of its columns
+        const size_t row = woff[0] + (size_t)(c0 + (warp & 3) * 32 + lane) * out0;
+        const int half = out0 / 2;
+        for (int j0 = (warp >> 2) * half; j0 < ((warp >> 2) + 1) * half; j0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + s * 256 + j0, v);
+          float4* wp = reinterpret_cast<float4*>(work + row + j0);
+          float4* up = reinterpret_cast<float4*>(Urow + row + j0);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 w = wp[q], u = up[q];
+            const float g0 = fmaf(lambda, w.x, __uint_as_float(v[4 * q])), g1 = fmaf(lambda, w.y, __uint_as_float(v[4 * q + 1]));
+            const float g2 = fmaf(lambda, w.z, __uint_as_float(v[4 * q + 2])), g3 = fmaf(lambda, w.w, __uint_as_float(v[4 * q + 3]));
+            w.x = fmaf(-eta, g0, w.x); w.y = fmaf(-eta, g1, w.y); w.z = fmaf(-eta, g2, w.z); w.w = fmaf(-eta, g3, w.w);
+            u.x += g0; u.y += g1; u.z += g2; u.w += g3;
+            wp[q] = w;
+            up[q] = u;
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      }
+      cluster_sync(clustered);
+      if (rank == 0)
+        for (int n = tid; n < out0; n += kThreads) {
+          float gb = 0.f;
+          for (int b = 0; b < B; ++b) gb += dz0[(size_t)b * out0 + n];
+          work[boff[0] + n] = fmaf(-eta, gb, work[boff[0] + n]);
+          Urow[boff[0] + n] += gb;
+        }
+    }
+    h += (uint32_t)B;
+  }
+
+  // ---- event trigger: publish (c, U_i, i) ----
+  cluster_sync(clustered);
+  if (p.r.w_end) {
+    float* dst = p.r.w_end + (size_t)t.seq * p.r.stride;
+    for (int l = 0; l < L; ++l) {
+      const int N = (int)S.dims[l + 1];
+      const size_t lo = woff[l] + (size_t)r0[l] * N, hi = woff[l] + (size_t)r1[l] * N;
+      for (size_t j = lo + tid; j < hi; j += kThreads) dst[j] = work[j];
+      if (rank == l % C)
+        for (int j = tid; j < N; j += kThreads) dst[boff[l] + j] = work[boff[l] + j];
+    }
+  }
+  if (failed && tid == 0 && p.r.status) atomicOr(p.r.status, 1u);
+  if (rank == 0 && tid == 0) {
+    TriggerRec rec;
+    rec.client = t.client; rec.round = t.round; rec.samples_done = h; rec.flags = 1;
+    p.r.trig[t.seq] = rec;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+}  // namespace
+
+bool mlp_tc_eligible(const MlpShape& s) {
+  if (s.precision != 1 || s.n_layers < 2 || s.cluster == 0) return false;
+  const uint32_t out0 = s.dims[1], B = s.batch;
+  if (out0 != 128 && out0 != 256) return false;
+  if (B != 32 && B != 64) return false;
+  if (s.dims[0] % (s.cluster * 128)) return false;           // every CTA owns whole 128-row chunks
+  for (uint32_t l = 1; l < s.n_layers; ++l)
+    if (((B + 3) / 4) * ((s.dims[l + 1] + 3) / 4) > (uint32_t)(kMaxTiles * kThreads)) return false;
+  if (s.dims[s.n_layers] > 32) return false;
+  return (size_t)make_tc_smem(s).total <= 227 * 1024;
+}
+
+cudaError_t launch_mlp_tc_rounds(const MlpLaunch& p, cudaStream_t s) {
+  if (p.r.n_tasks == 0) return cudaSuccess;
+  // More than half of an SM's shared memory: never two of these CTAs on one SM, so the
+  // 512-column tensor-memory allocation of one can never wait on a cluster peer.
+  size_t smem = (size_t)make_tc_smem(p.shape).total;
+  if (smem < 120 * 1024) smem = 120 * 1024;
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(p.r.n_tasks * p.shape.cluster, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = p.shape.cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, mlp_tc_kernel, p);
+}
+
+}  // namespace aet

@@ -64,6 +64,25 @@ def test_mlp_bf16_small_end_to_end_and_round_U():
     print("bf16 per-round U errors:", ["%.1e" % v for v in errs])
 
 
+@pytest.mark.parametrize("over", [
+    dict(n_clients=4, n_rounds=3, dims=[3072, 128, 32, 10], n_stragglers=1, data=dict(total=800)),                 # cluster of 8
+    dict(n_clients=40, n_rounds=2, dims=[3072, 256, 128, 10], n_stragglers=3, data=dict(kind="iid", total=4000)),  # cluster of 2
+    dict(n_clients=20, n_rounds=2, dims=[3072, 256, 10], batch=32, sched_a=32, sched_b=32, l2=1e-3, n_stragglers=0,
+         data=dict(kind="iid", total=2000)),                                                                    # cluster of 4, two layers
+])
+def test_mlp_bf16_tensor_core_path(over):
+    cfg = workloads.get_config("cfg4", **over)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert rel_err(gpu["w"], ref["w"]) <= 1e-3
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], BF16_U_TOL)
+                for e in ref["events"][::max(1, len(ref["events"]) // 6)]]
+    print("tensor-core path per-round U errors:", ["%.1e" % v for v in errs])
+
+
 def test_cfg3_full_size_log_invariant_and_sampled_rounds():
     cfg = workloads.get_config("cfg3")
     data, w0 = make(cfg)
