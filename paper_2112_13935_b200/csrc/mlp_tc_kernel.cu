@@ -38,10 +38,11 @@ constexpr int kMaxTiles = 4;
 constexpr int kKC = 64;        // input rows per forward chunk
 constexpr int kMT = 128;       // input rows per backward chunk (M of the MMA)
 constexpr uint32_t kTmemCols = 512;
+constexpr int kTrLd = 36;     // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 struct TcSmem {  // byte offsets into dynamic shared memory
-  int tiles, idx, As, AsT, Ws, dzs, dzq, zs, total;
+  int tiles, idx, As, AsT, Ws, dzs, dzq, zs, tr, total;
 };
 __host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
   const int B = (int)s.batch, out0 = (int)s.dims[1];
@@ -59,6 +60,9 @@ __host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
   m.dzs = o; o += B * nmax * 4;
   m.dzq = o; o += B * nmax * 4;
   m.zs = o; o += B * 32 * 4;
+  // the transposes reuse the FMA layers' staging area (idle during the layer-0 backward pass)
+  m.tr = m.As;
+  if (o - m.As < (kThreads / 32) * 32 * kTrLd * 4) o = m.As + (kThreads / 32) * 32 * kTrLd * 4;
   m.total = o;
   return m;
 }
@@ -111,6 +115,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Element-wise copy with four loads in flight per thread before the first store
+// (the compiler cannot reorder global loads across shared-memory stores itself).
+template <class Load, class Store>
+__device__ __forceinline__ void staged_copy(int total, int tid, Load ld, Store st) {
+  for (int e0 = tid; e0 < total; e0 += 4 * kThreads) {
+    float v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { const int e = e0 + u * kThreads; v[u] = e < total ? ld(e) : 0.f; }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { const int e = e0 + u * kThreads; if (e < total) st(e, v[u]); }
+  }
+}
+
 // One mbarrier that tcgen05.commit arrives on, with the bookkeeping that keeps
 // waits and completions paired (never more than one completion ahead).
 struct CommitBar {
@@ -155,6 +172,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   float* dzs = reinterpret_cast<float*>(smraw + M.dzs);
   float* dzq = reinterpret_cast<float*>(smraw + M.dzq);
   float* zs = reinterpret_cast<float*>(smraw + M.zs);
+  float* trbuf = reinterpret_cast<float*>(smraw + M.tr);   // per-warp transpose buffers of the layer-0 epilogue
 
   float* act = p.act + (size_t)(blockIdx.x / C) * p.act_stride;
   float* work = p.work + (size_t)t.client * p.r.stride;
@@ -243,15 +261,23 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         unsigned char* tB = tiles + 2 * a_bytes + s * b_bytes;
         bar_drain(fbar[s], failed);  // the MMAs that last read this buffer are done
         // A: bf16(W0[c0 + k, j]) as element (row j, col k)
-        for (int e = tid; e < out0 * (kKC / 8); e += kThreads) {
-          const int j = e % out0, kg = e / out0;
-          const float* src = work + woff[0] + (size_t)(c0 + kg * 8) * out0 + j;
-          uint4 v;
-          v.x = pack_bf16(src[0], src[out0]);
-          v.y = pack_bf16(src[2 * (size_t)out0], src[3 * (size_t)out0]);
-          v.z = pack_bf16(src[4 * (size_t)out0], src[5 * (size_t)out0]);
-          v.w = pack_bf16(src[6 * (size_t)out0], src[7 * (size_t)out0]);
-          *reinterpret_cast<uint4*>(tA + (j >> 3) * sbo_k64 + kg * 128 + (j & 7) * 16) = v;
+        for (int e0 = tid; e0 < out0 * (kKC / 8); e0 += 4 * kThreads) {
+          float f[4][8];
+#pragma unroll
+          for (int u4 = 0; u4 < 4; ++u4) {   // out0 * 8 is a multiple of 4 * kThreads: no tail
+            const int e = e0 + u4 * kThreads, j = e % out0, kg = e / out0;
+            const float* src = work + woff[0] + (size_t)(c0 + kg * 8) * out0 + j;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) f[u4][k] = src[(size_t)k * out0];
+          }
+#pragma unroll
+          for (int u4 = 0; u4 < 4; ++u4) {
+            const int e = e0 + u4 * kThreads, j = e % out0, kg = e / out0;
+            uint4 v;
+            v.x = pack_bf16(f[u4][0], f[u4][1]); v.y = pack_bf16(f[u4][2], f[u4][3]);
+            v.z = pack_bf16(f[u4][4], f[u4][5]); v.w = pack_bf16(f[u4][6], f[u4][7]);
+            *reinterpret_cast<uint4*>(tA + (j >> 3) * sbo_k64 + kg * 128 + (j & 7) * 16) = v;
+          }
         }
         // B: X[idx[b], c0 + k] as element (row b, col k); already bf16 in HBM
         for (int e = tid; e < B * (kKC / 8); e += kThreads) {
@@ -295,12 +321,12 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         const float* part0 = act + G.part[0];
         const float* bias = work + boff[0];
         const int c_lo = r0[1], c_n = r1[1] - r0[1];
-        for (int e = tid; e < B * c_n; e += kThreads) {
-          const int b = e / c_n, n = c_lo + e % c_n;
-          float z = bias[n];
-          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * out0 + n];
-          act[G.a[0] + (size_t)b * out0 + n] = q_bf16(fmaxf(z, 0.f));
-        }
+        staged_copy(B * c_n, tid,
+                    [&](int e) { const int b = e / c_n, n = c_lo + e % c_n;
+                                 float z = bias[n];
+                                 for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * out0 + n];
+                                 return z; },
+                    [&](int e, float z) { act[G.a[0] + (size_t)(e / c_n) * out0 + c_lo + e % c_n] = q_bf16(fmaxf(z, 0.f)); });
         __syncthreads();
       }
     }
@@ -317,14 +343,14 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       for (int c0 = r0[l]; c0 < r1[l]; c0 += kRC) {
         const int rc = min(kRC, r1[l] - c0);
         __syncthreads();
-        for (int e = tid; e < kRC * B; e += kThreads) {
-          const int b = e / kRC, ic = e % kRC;
-          As[ic * B + b] = ic < rc ? act[G.a[l - 1] + (size_t)b * S.dims[l] + c0 + ic] : 0.f;
-        }
-        for (int e = tid; e < kRC * Np; e += kThreads) {
-          const int ic = e / Np, j = e % Np;
-          Ws[ic * ldw + j] = (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f;
-        }
+        staged_copy(kRC * B, tid,
+                    [&](int e) { const int b = e / kRC, ic = e % kRC;
+                                 return ic < rc ? act[G.a[l - 1] + (size_t)b * S.dims[l] + c0 + ic] : 0.f; },
+                    [&](int e, float v) { As[(e % kRC) * B + e / kRC] = v; });
+        staged_copy(kRC * Np, tid,
+                    [&](int e) { const int ic = e / Np, j = e % Np;
+                                 return (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f; },
+                    [&](int e, float v) { Ws[(e / Np) * ldw + e % Np] = v; });
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kMaxTiles; ++q) {
@@ -365,20 +391,20 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       const float* bias = work + boff[l];
       if (l < L - 1) {
         const int c_lo = r0[l + 1], c_n = r1[l + 1] - r0[l + 1];
-        for (int e = tid; e < B * c_n; e += kThreads) {
-          const int b = e / c_n, n = c_lo + e % c_n;
-          float z = bias[n];
-          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
-          act[G.a[l] + (size_t)b * N + n] = q_bf16(fmaxf(z, 0.f));
-        }
+        staged_copy(B * c_n, tid,
+                    [&](int e) { const int b = e / c_n, n = c_lo + e % c_n;
+                                 float z = bias[n];
+                                 for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
+                                 return z; },
+                    [&](int e, float z) { act[G.a[l] + (size_t)(e / c_n) * N + c_lo + e % c_n] = q_bf16(fmaxf(z, 0.f)); });
         __syncthreads();
       } else {
-        for (int e = tid; e < B * N; e += kThreads) {
-          const int b = e / N, n = e % N;
-          float z = bias[n];
-          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
-          zs[b * 32 + n] = z;
-        }
+        staged_copy(B * N, tid,
+                    [&](int e) { const int b = e / N, n = e % N;
+                                 float z = bias[n];
+                                 for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
+                                 return z; },
+                    [&](int e, float z) { zs[(e / N) * 32 + e % N] = z; });
         __syncthreads();
         for (int b = tid; b < B; b += kThreads) {
           float m = -INFINITY;
@@ -405,14 +431,14 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       for (int c0 = r0[l]; c0 < r1[l]; c0 += kRC) {
         const int rc = min(kRC, r1[l] - c0);
         __syncthreads();
-        for (int e = tid; e < kRC * B; e += kThreads) {
-          const int b = e / kRC, ic = e % kRC;
-          AsT[b * kRC + ic] = ic < rc ? act[G.a[l - 1] + (size_t)b * K + c0 + ic] : 0.f;
-        }
-        for (int e = tid; e < kRC * Np; e += kThreads) {
-          const int ic = e / Np, j = e % Np;
-          Ws[ic * ldw + j] = (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f;
-        }
+        staged_copy(kRC * B, tid,
+                    [&](int e) { const int b = e / kRC, ic = e % kRC;
+                                 return ic < rc ? act[G.a[l - 1] + (size_t)b * K + c0 + ic] : 0.f; },
+                    [&](int e, float v) { AsT[e] = v; });
+        staged_copy(kRC * Np, tid,
+                    [&](int e) { const int ic = e / Np, j = e % Np;
+                                 return (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f; },
+                    [&](int e, float v) { Ws[(e / Np) * ldw + e % Np] = v; });
         __syncthreads();
         for (int e = tid; e < B * rc; e += kThreads) {
           const int b = e / rc, ic = e % rc;
@@ -428,7 +454,17 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
           const int tiles_n = Np / 4, ntile = (kRC / 4) * tiles_n;
           for (int mt = tid; mt < ntile; mt += kThreads) {
             const int it4 = mt / tiles_n, jt = mt % tiles_n;
-            float g[16];
+            float g[16], wv[16], uv[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)     // master and update-sum entries first: in flight during the FMAs
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int ic = 4 * it4 + i, n = 4 * jt + j;
+                const bool live = ic < rc && n < N;
+                const size_t o = woff[l] + (size_t)(c0 + ic) * N + n;
+                wv[4 * i + j] = live ? work[o] : 0.f;
+                uv[4 * i + j] = live ? Urow[o] : 0.f;
+              }
 #pragma unroll
             for (int e = 0; e < 16; ++e) g[e] = 0.f;
             for (int b = 0; b < B; ++b) {
@@ -441,20 +477,17 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
                 for (int j = 0; j < 4; ++j) g[4 * i + j] = fmaf(av[i], dv[j], g[4 * i + j]);
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int ic = 4 * it4 + i;
-              if (ic >= rc) continue;
+            for (int i = 0; i < 4; ++i)
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const int n = 4 * jt + j;
-                if (n >= N) continue;
-                const size_t o = woff[l] + (size_t)(c0 + ic) * N + n;
-                const float w = work[o];
-                const float gg = fmaf(lambda, w, g[4 * i + j]);
-                work[o] = fmaf(-eta, gg, w);
-                Urow[o] += gg;
+                const int ic = 4 * it4 + i, n = 4 * jt + j;
+                if (ic < rc && n < N) {
+                  const size_t o = woff[l] + (size_t)(c0 + ic) * N + n;
+                  const float gg = fmaf(lambda, wv[4 * i + j], g[4 * i + j]);
+                  work[o] = fmaf(-eta, gg, wv[4 * i + j]);
+                  Urow[o] = uv[4 * i + j] + gg;
+                }
               }
-            }
           }
         }
       }
@@ -469,12 +502,10 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       if (l > 1) {
         __syncthreads();
         const int Nm = (int)S.dims[l], Nmp = up4(Nm);
-        for (int e = tid; e < B * Nmp; e += kThreads) {
-          const int b = e / Nmp, n = e % Nmp;
-          const float d = n < Nm ? act[G.dz[l - 1] + (size_t)b * Nm + n] : 0.f;
-          dzs[b * Nmp + n] = d;
-          dzq[b * Nmp + n] = q_bf16(d);
-        }
+        staged_copy(B * Nmp, tid,
+                    [&](int e) { const int b = e / Nmp, n = e % Nmp;
+                                 return n < Nm ? act[G.dz[l - 1] + (size_t)b * Nm + n] : 0.f; },
+                    [&](int e, float d) { dzs[e] = d; dzq[e] = q_bf16(d); });
         __syncthreads();
       }
     }
@@ -529,23 +560,40 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         if (c + 1 < nch) stage_and_issue(c + 1);   // its buffer and accumulator were released by chunk c-1
         bar_drain(bbar[s], failed);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // epilogue: thread = one row of W0, half of its columns
-        const size_t row = woff[0] + (size_t)(c0 + (warp & 3) * 32 + lane) * out0;
+        // epilogue: a warp owns 32 rows of W0 and half of the columns.  The accumulator
+        // block comes out of tensor memory one row per lane; a per-warp transpose through
+        // shared memory lets every global access cover 4 rows x 128 contiguous bytes.
+        float* tr = trbuf + warp * (32 * kTrLd);
         const int half = out0 / 2;
+        const int rr = lane >> 3, cg = (lane & 7) * 4;
         for (int j0 = (warp >> 2) * half; j0 < ((warp >> 2) + 1) * half; j0 += 32) {
           uint32_t v[32];
           tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + s * 256 + j0, v);
-          float4* wp = reinterpret_cast<float4*>(work + row + j0);
-          float4* up = reinterpret_cast<float4*>(Urow + row + j0);
+          __syncwarp();
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<float4*>(tr + lane * kTrLd + 4 * q) =
+                make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          __syncwarp();
+          const size_t base = woff[0] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + j0 + cg;
+          float4 w[8], u[8], g[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: 16 independent 16-byte loads in flight
+            w[q] = *reinterpret_cast<const float4*>(work + base + (size_t)(4 * q) * out0);
+            u[q] = *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0);
+            g[q] = *reinterpret_cast<const float4*>(tr + (4 * q + rr) * kTrLd + cg);
+          }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            float4 w = wp[q], u = up[q];
-            const float g0 = fmaf(lambda, w.x, __uint_as_float(v[4 * q])), g1 = fmaf(lambda, w.y, __uint_as_float(v[4 * q + 1]));
-            const float g2 = fmaf(lambda, w.z, __uint_as_float(v[4 * q + 2])), g3 = fmaf(lambda, w.w, __uint_as_float(v[4 * q + 3]));
-            w.x = fmaf(-eta, g0, w.x); w.y = fmaf(-eta, g1, w.y); w.z = fmaf(-eta, g2, w.z); w.w = fmaf(-eta, g3, w.w);
-            u.x += g0; u.y += g1; u.z += g2; u.w += g3;
-            wp[q] = w;
-            up[q] = u;
+            const float g0 = fmaf(lambda, w[q].x, g[q].x), g1 = fmaf(lambda, w[q].y, g[q].y);
+            const float g2 = fmaf(lambda, w[q].z, g[q].z), g3 = fmaf(lambda, w[q].w, g[q].w);
+            w[q].x = fmaf(-eta, g0, w[q].x); w[q].y = fmaf(-eta, g1, w[q].y); w[q].z = fmaf(-eta, g2, w[q].z); w[q].w = fmaf(-eta, g3, w[q].w);
+            u[q].x += g0; u[q].y += g1; u[q].z += g2; u[q].w += g3;
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            *reinterpret_cast<float4*>(work + base + (size_t)(4 * q) * out0) = w[q];
+            *reinterpret_cast<float4*>(Urow + base + (size_t)(4 * q) * out0) = u[q];
           }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
