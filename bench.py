@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(DESCRIBE))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--clients", type=int, default=0, help="override the workload's client count (cfg5 sweep)")
+    ap.add_argument("--rounds", type=int, default=0, help="override the number of rounds (profiling on a smaller case)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -200,6 +201,8 @@ def main():
     from paper_2112_13935_b200 import workloads
     rank = int(os.environ.get("RANK", "0"))
     over = dict(n_clients=args.clients) if args.clients else {}
+    if args.rounds:
+        over["n_rounds"] = args.rounds
     cfg = workloads.get_config(args.workload, seed=rank, **over)
     if args.impl == "reference":
         run_reference(args, cfg)

@@ -115,16 +115,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Element-wise copy with four loads in flight per thread before the first store
-// (the compiler cannot reorder global loads across shared-memory stores itself).
+// Element-wise copy with kInFlight loads in flight per thread before the first
+// store (the compiler cannot reorder global loads across shared-memory stores
+// itself, and a dependent round trip to L2 costs about a microsecond).
+constexpr int kInFlight = 8;
 template <class Load, class Store>
 __device__ __forceinline__ void staged_copy(int total, int tid, Load ld, Store st) {
-  for (int e0 = tid; e0 < total; e0 += 4 * kThreads) {
-    float v[4];
+  for (int e0 = tid; e0 < total; e0 += kInFlight * kThreads) {
+    float v[kInFlight];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) { const int e = e0 + u * kThreads; v[u] = e < total ? ld(e) : 0.f; }
+    for (int u = 0; u < kInFlight; ++u) { const int e = e0 + u * kThreads; v[u] = e < total ? ld(e) : 0.f; }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) { const int e = e0 + u * kThreads; if (e < total) st(e, v[u]); }
+    for (int u = 0; u < kInFlight; ++u) { const int e = e0 + u * kThreads; if (e < total) st(e, v[u]); }
   }
 }
 
@@ -440,15 +442,34 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
                                  return (ic < rc && j < N) ? q_bf16(work[woff[l] + (size_t)(c0 + ic) * N + j]) : 0.f; },
                     [&](int e, float v) { Ws[(e / Np) * ldw + e % Np] = v; });
         __syncthreads();
-        for (int e = tid; e < B * rc; e += kThreads) {
-          const int b = e / rc, ic = e % rc;
-          float s = 0.f;
-          for (int j = 0; j < Np; j += 4) {
-            const float4 d = *reinterpret_cast<const float4*>(dzq + b * Np + j);
-            const float4 w = *reinterpret_cast<const float4*>(Ws + ic * ldw + j);
-            s = fmaf(d.x, w.x, s); s = fmaf(d.y, w.y, s); s = fmaf(d.z, w.z, s); s = fmaf(d.w, w.w, s);
+        for (int e0 = tid; e0 < B * rc; e0 += 8 * kThreads) {   // eight independent dot products per thread
+          float s8[8];
+          const float* dp[8];
+          const float* wq[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int e = min(e0 + q * kThreads, B * rc - 1);
+            s8[q] = 0.f;
+            dp[q] = dzq + (e / rc) * Np;
+            wq[q] = Ws + (e % rc) * ldw;
           }
-          act[G.dz[l - 1] + (size_t)b * K + c0 + ic] = AsT[b * kRC + ic] > 0.f ? s : 0.f;
+          for (int j = 0; j < Np; j += 4) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 d = *reinterpret_cast<const float4*>(dp[q] + j);
+              const float4 w = *reinterpret_cast<const float4*>(wq[q] + j);
+              s8[q] = fmaf(d.x, w.x, s8[q]); s8[q] = fmaf(d.y, w.y, s8[q]);
+              s8[q] = fmaf(d.z, w.z, s8[q]); s8[q] = fmaf(d.w, w.w, s8[q]);
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int e = e0 + q * kThreads;
+            if (e < B * rc) {
+              const int b = e / rc, ic = e % rc;
+              act[G.dz[l - 1] + (size_t)b * K + c0 + ic] = AsT[b * kRC + ic] > 0.f ? s8[q] : 0.f;
+            }
+          }
         }
         {
           const int tiles_n = Np / 4, ntile = (kRC / 4) * tiles_n;
