@@ -41,5 +41,20 @@ __host__ __device__ inline Layout make_layout(const MlpShape& s) {
   return L;
 }
 
+// Element-wise copy with kInFlight loads in flight per thread before the first
+// store (the compiler cannot reorder global loads across shared-memory stores
+// itself, and a dependent round trip to L2 costs about a microsecond).
+constexpr int kInFlight = 8;
+template <int kThreadsT, class Load, class Store>
+__device__ __forceinline__ void staged_copy_t(int total, int tid, Load ld, Store st) {
+  for (int e0 = tid; e0 < total; e0 += kInFlight * kThreadsT) {
+    float v[kInFlight];
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) { const int e = e0 + u * kThreadsT; v[u] = e < total ? ld(e) : 0.f; }
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) { const int e = e0 + u * kThreadsT; if (e < total) st(e, v[u]); }
+  }
+}
+
 }  // namespace mlp
 }  // namespace aet

@@ -51,6 +51,11 @@ __host__ __device__ inline Smem make_smem(const MlpShape& s) {
   return m;
 }
 
+template <class Load, class Store>
+__device__ __forceinline__ void staged_copy(int total, int tid, Load ld, Store st) {
+  staged_copy_t<kThreads>(total, tid, ld, st);
+}
+
 __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
   extern __shared__ __align__(16) float sm[];
   const MlpShape& S = p.shape;
@@ -140,29 +145,24 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
         const int rc = min(kRC, r1[l] - c0);
         __syncthreads();
         // stage A chunk as As[ic][b] and W chunk as Ws[ic][j]
-        for (int e = tid; e < kRC * Bp; e += kThreads) {
-          const int b = e / kRC, ic = e % kRC;
-          float v = 0.f;
-          if (b < B && ic < rc) {
-            if (l == 0) {
-              const size_t off = (size_t)idx[b] * S.dims[0] + c0 + ic;
-              v = bf ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(cd.x)[off])
-                     : reinterpret_cast<const float*>(cd.x)[off];
-            } else {
-              v = act[G.a[l - 1] + (size_t)b * S.dims[l] + c0 + ic];
-            }
-          }
-          As[ic * Bp + b] = v;
-        }
-        for (int e = tid; e < kRC * Np; e += kThreads) {
-          const int ic = e / Np, j = e % Np;
-          float v = 0.f;
-          if (ic < rc && j < N) {
-            v = work[woff[l] + (size_t)(c0 + ic) * N + j];
-            if (bf) v = q_bf16(v);
-          }
-          Ws[ic * ldw + j] = v;
-        }
+        staged_copy(kRC * Bp, tid,
+                    [&](int e) {
+                      const int b = e / kRC, ic = e % kRC;
+                      if (b >= B || ic >= rc) return 0.f;
+                      if (l > 0) return act[G.a[l - 1] + (size_t)b * S.dims[l] + c0 + ic];
+                      const size_t off = (size_t)idx[b] * S.dims[0] + c0 + ic;
+                      return bf ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(cd.x)[off])
+                                : reinterpret_cast<const float*>(cd.x)[off];
+                    },
+                    [&](int e, float v) { As[(e % kRC) * Bp + e / kRC] = v; });
+        staged_copy(kRC * Np, tid,
+                    [&](int e) {
+                      const int ic = e / Np, j = e % Np;
+                      if (ic >= rc || j >= N) return 0.f;
+                      const float v = work[woff[l] + (size_t)(c0 + ic) * N + j];
+                      return bf ? q_bf16(v) : v;
+                    },
+                    [&](int e, float v) { Ws[(e / Np) * ldw + e % Np] = v; });
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kMaxTiles; ++q) {
@@ -205,22 +205,27 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
       if (l < L - 1) {
         // columns this CTA feeds into the next layer
         const int c_lo = r0[l + 1], c_n = r1[l + 1] - r0[l + 1];
-        for (int e = tid; e < B * c_n; e += kThreads) {
-          const int b = e / c_n, n = c_lo + e % c_n;
-          float z = bias[n];
-          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
-          float a = fmaxf(z, 0.f);
-          if (bf) a = q_bf16(a);
-          act[G.a[l] + (size_t)b * N + n] = a;
-        }
+        staged_copy(B * c_n, tid,
+                    [&](int e) {
+                      const int b = e / c_n, n = c_lo + e % c_n;
+                      float z = bias[n];
+                      for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
+                      return z;
+                    },
+                    [&](int e, float z) {
+                      const float a = fmaxf(z, 0.f);
+                      act[G.a[l] + (size_t)(e / c_n) * N + c_lo + e % c_n] = bf ? q_bf16(a) : a;
+                    });
         __syncthreads();
       } else {
-        for (int e = tid; e < B * N; e += kThreads) {
-          const int b = e / N, n = e % N;
-          float z = bias[n];
-          for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
-          zs[b * 32 + n] = z;
-        }
+        staged_copy(B * N, tid,
+                    [&](int e) {
+                      const int b = e / N, n = e % N;
+                      float z = bias[n];
+                      for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * N + n];
+                      return z;
+                    },
+                    [&](int e, float z) { zs[(e / N) * 32 + e % N] = z; });
         __syncthreads();
         // softmax cross-entropy: dZ = (p - onehot(y)) / B
         for (int b = tid; b < Bp; b += kThreads) {
@@ -252,30 +257,25 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
       for (int c0 = r0[l]; c0 < r1[l]; c0 += kRC) {
         const int rc = min(kRC, r1[l] - c0);
         __syncthreads();
-        for (int e = tid; e < kRC * Bp; e += kThreads) {
-          const int b = e / kRC, ic = e % kRC;
-          float v = 0.f;
-          if (b < B && ic < rc) {
-            if (l == 0) {
-              const size_t off = (size_t)idx[b] * S.dims[0] + c0 + ic;
-              v = bf ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(cd.x)[off])
-                     : reinterpret_cast<const float*>(cd.x)[off];
-            } else {
-              v = act[G.a[l - 1] + (size_t)b * K + c0 + ic];
-            }
-          }
-          AsT[b * kRC + ic] = v;
-        }
+        staged_copy(kRC * Bp, tid,
+                    [&](int e) {
+                      const int b = e / kRC, ic = e % kRC;
+                      if (b >= B || ic >= rc) return 0.f;
+                      if (l > 0) return act[G.a[l - 1] + (size_t)b * K + c0 + ic];
+                      const size_t off = (size_t)idx[b] * S.dims[0] + c0 + ic;
+                      return bf ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(cd.x)[off])
+                                : reinterpret_cast<const float*>(cd.x)[off];
+                    },
+                    [&](int e, float v) { AsT[e] = v; });
         if (l > 0)
-          for (int e = tid; e < kRC * Np; e += kThreads) {
-            const int ic = e / Np, j = e % Np;
-            float v = 0.f;
-            if (ic < rc && j < N) {
-              v = work[woff[l] + (size_t)(c0 + ic) * N + j];
-              if (bf) v = q_bf16(v);
-            }
-            Ws[ic * ldw + j] = v;
-          }
+          staged_copy(kRC * Np, tid,
+                      [&](int e) {
+                        const int ic = e / Np, j = e % Np;
+                        if (ic >= rc || j >= N) return 0.f;
+                        const float v = work[woff[l] + (size_t)(c0 + ic) * N + j];
+                        return bf ? q_bf16(v) : v;
+                      },
+                      [&](int e, float v) { Ws[(e / Np) * ldw + e % Np] = v; });
         __syncthreads();
         if (l > 0) {
           // dZ_{l-1}[b, c0+ic] = relu'(A_{l-1}) * sum_j dZq_l[b, j] W_l[c0+ic, j]
@@ -296,7 +296,17 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
           const int tiles_n = Np / 4, tiles = (kRC / 4) * tiles_n;
           for (int mt = tid; mt < tiles; mt += kThreads) {
             const int it4 = mt / tiles_n, jt = mt % tiles_n;
-            float g[16];
+            float g[16], wv[16], uv[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)     // master and update-sum entries first: in flight during the FMAs
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int ic = 4 * it4 + i, n = 4 * jt + j;
+                const bool live = ic < rc && n < N;
+                const size_t o = woff[l] + (size_t)(c0 + ic) * N + n;
+                wv[4 * i + j] = live ? work[o] : 0.f;
+                uv[4 * i + j] = live ? Urow[o] : 0.f;
+              }
 #pragma unroll
             for (int e = 0; e < 16; ++e) g[e] = 0.f;
             for (int b = 0; b < B; ++b) {
@@ -317,10 +327,10 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
                 const int n = 4 * jt + j;
                 if (n >= N) continue;
                 const size_t o = woff[l] + (size_t)(c0 + ic) * N + n;
-                const float w = work[o];
+                const float w = wv[4 * i + j];
                 const float gg = fmaf(lambda, w, g[4 * i + j]);
                 work[o] = fmaf(-eta, gg, w);
-                Urow[o] += gg;
+                Urow[o] = uv[4 * i + j] + gg;
               }
             }
           }
@@ -338,12 +348,12 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
       if (l > 0) {
         __syncthreads();
         const int Nm = (int)S.dims[l], Nmp = up4(Nm);
-        for (int e = tid; e < Bp * Nmp; e += kThreads) {
-          const int b = e / Nmp, n = e % Nmp;
-          const float d = (b < B && n < Nm) ? act[G.dz[l - 1] + (size_t)b * Nm + n] : 0.f;
-          dzs[b * Nmp + n] = d;
-          if (bf) dzq[b * Nmp + n] = q_bf16(d);
-        }
+        staged_copy(Bp * Nmp, tid,
+                    [&](int e) {
+                      const int b = e / Nmp, n = e % Nmp;
+                      return (b < B && n < Nm) ? act[G.dz[l - 1] + (size_t)b * Nm + n] : 0.f;
+                    },
+                    [&](int e, float d) { dzs[e] = d; if (bf) dzq[e] = q_bf16(d); });
         __syncthreads();
       }
     }

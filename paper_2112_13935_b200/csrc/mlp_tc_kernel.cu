@@ -115,19 +115,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Element-wise copy with kInFlight loads in flight per thread before the first
-// store (the compiler cannot reorder global loads across shared-memory stores
-// itself, and a dependent round trip to L2 costs about a microsecond).
-constexpr int kInFlight = 8;
 template <class Load, class Store>
 __device__ __forceinline__ void staged_copy(int total, int tid, Load ld, Store st) {
-  for (int e0 = tid; e0 < total; e0 += kInFlight * kThreads) {
-    float v[kInFlight];
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) { const int e = e0 + u * kThreads; v[u] = e < total ? ld(e) : 0.f; }
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) { const int e = e0 + u * kThreads; if (e < total) st(e, v[u]); }
-  }
+  staged_copy_t<kThreads>(total, tid, ld, st);
 }
 
 // One mbarrier that tcgen05.commit arrives on, with the bookkeeping that keeps
