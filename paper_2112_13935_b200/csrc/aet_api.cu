@@ -243,7 +243,7 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   h->shape.batch = cfg->batch;
   h->shape.precision = cfg->precision;
   h->shape.cluster = mlp_pick_cluster(h->shape, cfg->n_clients);
-  if (!h->lr_fast) {
+  if (!h->lr_fast && !mlp_tc_eligible(h->shape)) {
     if (const char* why = mlp_check_shape(h->shape)) { delete h; return fail(nullptr, AET_ERR_CONFIG, why); }
   }
   h->h_clients.assign(cfg->n_clients, ClientData{nullptr, nullptr, 0, 0});
