@@ -193,6 +193,8 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--clients", type=int, default=0, help="override the workload's client count (cfg5 sweep)")
     ap.add_argument("--rounds", type=int, default=0, help="override the number of rounds (profiling on a smaller case)")
+    ap.add_argument("--net-delay", type=float, default=None, help="override the mean network delay (time units)")
+    ap.add_argument("--max-lag", type=int, default=None, help="override the checkpoint threshold d (-1 = never wait)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -203,6 +205,10 @@ def main():
     over = dict(n_clients=args.clients) if args.clients else {}
     if args.rounds:
         over["n_rounds"] = args.rounds
+    if args.net_delay is not None:
+        over["network_delay_mean"] = args.net_delay
+    if args.max_lag is not None:
+        over["max_lag_d"] = workloads.NEVER_WAIT if args.max_lag < 0 else args.max_lag
     cfg = workloads.get_config(args.workload, seed=rank, **over)
     if args.impl == "reference":
         run_reference(args, cfg)
@@ -322,6 +328,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == 1 else "f32",
             "data": "synthetic",
             "config": {"workload": DESCRIBE[args.workload], "n_clients": cfg["n_clients"], "rounds": R,
+                       "network_delay_mean": cfg["network_delay_mean"],
+                       "max_lag_d": "never wait" if cfg["max_lag_d"] == workloads.NEVER_WAIT else cfg["max_lag_d"],
                        "samples_per_step": samples, "events_per_step": len(events),
                        "waves_per_step": stats["waves"], "l2": "flushed between timed steps (256 MB fill)",
                        "multi_gpu": "independent replicas, one seed per rank"},
