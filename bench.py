@@ -43,6 +43,15 @@ DESCRIBE = {
 }
 
 
+# DRAM bytes (read + write) over algorithmic bytes of one launch of the round kernel, from the
+# ncu captures summarised under profiles/ (traffic grows in proportion to the samples of a launch).
+# Set an entry to None when its kernel changes after the counters were taken.
+TRAFFIC_RATIO = {
+    "cfg2": (28.4029 / 29.6420, "profiles/lr_round_kernel_cfg2.md"),
+    "cfg5": (45.3678 / 36.4115, "profiles/lr_round_kernel_cfg5_512clients.md"),
+}
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -275,8 +284,12 @@ def main():
     sgd_ms_per_step = k_ms[0] / k_steps
     achieved = alg_bytes / (sgd_ms_per_step * 1e-3) / 1e9
     peak, peak_kind = measured_peak_gbs()
+    ratio = TRAFFIC_RATIO.get(args.workload)
+    traffic = ratio[0] * alg_bytes / n_sgd_launches if ratio and ratio[0] and not args.rounds else None
     roof = {"bound": "hbm", "kernel": "local-SGD rounds", "achieved": achieved, "peak": peak,
-            "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind}
+            "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+            "traffic_source": ratio[1] if traffic else None, "peak_kind": peak_kind,
+            "algorithmic_bytes_per_launch": alg_bytes / n_sgd_launches}
     if cfg["model"] == 1:
         tf = algorithmic_flops(cfg, events) / (sgd_ms_per_step * 1e-3) / 1e12
         tpeak, tkind = measured_peak_tflops()
