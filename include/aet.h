@@ -165,6 +165,15 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
                                       const float* w_in, float* U_out, float* w_out,
                                       void* cuda_stream);
 
+/* Failure-detection aid: runs the give-up path of the kernels' bounded waits on
+ * purpose.  One CTA polls a barrier that nothing signals at most max_polls times
+ * (1 .. 2^24; a few milliseconds at most), flags the handle's device status word
+ * as a round kernel would after a lost asynchronous copy, and returns normally.
+ * The call synchronises `cuda_stream` and returns AET_ERR_TIMEOUT; the handle
+ * and the CUDA context stay usable.  (The paper assumes messages are never lost,
+ * Section 3.3.1; this guards the library's own asynchronous copies.) */
+aet_status aet_debug_wait_probe(aet_handle* h, uint32_t max_polls, void* cuda_stream);
+
 /* Record CUDA events around every kernel of later runs (adds a little launch
  * overhead) so that aet_get_stats can report device time per kernel. */
 aet_status aet_set_kernel_timing(aet_handle* h, int enable);

@@ -64,6 +64,7 @@ PROTOTYPES = {
     "aet_get_update_sum": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]),
     "aet_debug_run_client_round": (C.c_int, [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p]),
+    "aet_debug_wait_probe": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p]),
     "aet_set_kernel_timing": (C.c_int, [C.c_void_p, C.c_int]),
     "aet_get_stats": (C.c_int, [C.c_void_p, C.POINTER(AetStats)]),
     "aet_n_params": (C.c_size_t, [C.c_void_p]),

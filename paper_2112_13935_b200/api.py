@@ -152,6 +152,11 @@ def aet_round_no_alloc(cfg, client: int, rnd: int, x, y, w_in, U_out, w_out, str
                                                 _ptr(w_in), _ptr(U_out), _ptr(w_out), _stream(stream)))
 
 
+def aet_debug_wait_probe(h, max_polls: int = 1 << 12, stream=None):
+    """Makes a bounded device wait run out on purpose; raises AetError(AET_ERR_TIMEOUT)."""
+    _check(h, _lib.load().aet_debug_wait_probe(h, max_polls, _stream(stream)))
+
+
 def aet_set_kernel_timing(h, enable: bool):
     _check(h, _lib.load().aet_set_kernel_timing(h, int(enable)))
 

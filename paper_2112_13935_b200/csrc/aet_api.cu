@@ -545,6 +545,16 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   return AET_OK;
 }
 
+aet_status aet_debug_wait_probe(aet_handle* h, uint32_t max_polls, void* cuda_stream) {
+  if (!h) return AET_ERR_ARG;
+  if (max_polls == 0 || max_polls > (1u << 24)) return fail(h, AET_ERR_ARG, "max_polls must be in [1, 2^24]");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  cudaError_t e = launch_wait_probe(h->d_status.p, max_polls, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "wait probe launch");
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  return check_device_status(h);
+}
+
 aet_status aet_set_kernel_timing(aet_handle* h, int enable) {
   if (!h) return AET_ERR_ARG;
   h->timing = enable != 0;

@@ -38,6 +38,9 @@ struct RoundLaunch {
   float l2;
 };
 
+// One CTA waits (at most max_polls polls) on a barrier nobody signals, then sets bit 0 of *status.
+cudaError_t launch_wait_probe(uint32_t* status, uint32_t max_polls, cudaStream_t s);
+
 // Softmax regression 784 -> 10, batch 1: one CTA per round-task.
 cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s);
 

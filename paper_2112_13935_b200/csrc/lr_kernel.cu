@@ -91,12 +91,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the copy did not land within kWaitLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i)
+// Bounded wait: false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) { return mbar_wait_limit(bar, parity, kWaitLimit); }
 // One row global -> shared, 16-byte aligned on both sides, size a multiple of 16.
 __device__ __forceinline__ void bulk_load_row(float* dst, const float* src, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -397,7 +398,26 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
   }
 }
 
+// Exercises the give-up path of the bounded wait without any faulty hardware:
+// an mbarrier that nothing ever arrives on is polled `max_polls` times, then the
+// CTA flags `status` exactly as a round kernel does and returns normally.
+__global__ void wait_probe_kernel(uint32_t* status, uint32_t max_polls) {
+  __shared__ __align__(8) uint64_t never;
+  if (threadIdx.x == 0) {
+    mbar_init(&never, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool landed = mbar_wait_limit(&never, 0, max_polls);
+  if (__syncthreads_or(!landed) && threadIdx.x == 0) atomicOr(status, 1u);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_probe(uint32_t* status, uint32_t max_polls, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(status, max_polls);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s) {
   if (p.n_tasks == 0) return cudaSuccess;

@@ -74,6 +74,11 @@ def test_schedule_is_bit_identical_to_the_checker(name):
     dict(max_lag_d=0), dict(max_lag_d=workloads.NEVER_WAIT), dict(n_clients=1),
     dict(delay_dist=1), dict(n_stragglers=3, straggler_factor=37.5, max_lag_d=2),
     dict(round_base=1, sched_b=0, lr_beta=0.01), dict(network_delay_mean=50.0, n_clients=9, max_lag_d=3),
+    # constant, equal delays: every START coincides with APPLYs (tie rule) and with other STARTs
+    dict(n_clients=3, sched_a=0, sched_b=1, delay_dist=1, compute_delay_lo=5 / 2 ** 20, compute_delay_hi=5 / 2 ** 20,
+         network_delay_lo=5 / 2 ** 20, network_delay_hi=5 / 2 ** 20, max_lag_d=workloads.NEVER_WAIT),
+    dict(n_clients=3, sched_a=0, sched_b=2, delay_dist=1, compute_delay_lo=4 / 2 ** 20, compute_delay_hi=4 / 2 ** 20,
+         network_delay_lo=8 / 2 ** 20, network_delay_hi=8 / 2 ** 20, max_lag_d=1),
 ])
 def test_schedule_variants_match_the_checker(over):
     cfg = workloads.get_config("cfg1", **over)

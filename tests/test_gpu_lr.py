@@ -150,6 +150,31 @@ def test_host_buffers_are_accepted():
         api.aet_destroy(h)
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_survives():
+    cfg = workloads.get_config("cfg1", n_rounds=2)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0)
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        with pytest.raises(api.AetError) as e:
+            api.aet_debug_wait_probe(s.h, 1 << 10)        # nothing ever signals that barrier
+        assert e.value.status == 6                        # AET_ERR_TIMEOUT
+        s.run()                                           # status was cleared; the context is intact
+        assert np.abs(s.model() - ref["w"]).max() <= 1e-5
+        with pytest.raises(api.AetError) as e:
+            api.aet_debug_wait_probe(s.h, 0)
+        assert e.value.status == 1
+
+
+def test_zero_rounds_is_a_no_op():
+    cfg = workloads.get_config("cfg1")
+    data, w0 = make(cfg)
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        s.run(0)
+        events, summary = s.log()
+        assert events == [] and summary["messages_up"] == 0
+        assert s.model().tobytes() == w0.tobytes()
+
+
 def test_errors_are_reported_not_raised_by_the_device():
     cfg = workloads.get_config("cfg1")
     data, w0 = make(cfg)

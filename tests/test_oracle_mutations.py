@@ -1,0 +1,110 @@
+"""Do the pins bite?  Each case plants one plausible mistake in the CPU checker
+(never in the CUDA path) and expects the named pin to fail."""
+import numpy as np
+import pytest
+
+import test_oracle_models as tm
+import test_oracle_rng as tr
+import test_oracle_schedule as ts
+import test_oracle_sim as tsim
+from oracle import models, rng, schedule, sim
+
+
+def _fails(fn, *args):
+    with pytest.raises((AssertionError, IndexError, ValueError)):
+        fn(*args)
+
+
+def test_dropped_l2_term_is_caught(monkeypatch):
+    real = models.loss_and_grad
+
+    def no_l2_in_grad(w, X, y, dims, l2=0.0, precision=0):
+        loss, _ = real(w, X, y, dims, l2, precision)
+        return loss, real(w, X, y, dims, 0.0, precision)[1]
+    monkeypatch.setattr(models, "loss_and_grad", no_l2_in_grad)
+    _fails(tm.test_gradient_matches_central_differences, [9, 6, 10], 4, 0.05)
+    _fails(tm.test_matches_torch_autograd_mlp)
+
+
+def test_bias_gradient_scaled_wrongly_is_caught(monkeypatch):
+    real = models.loss_and_grad
+
+    def bad(w, X, y, dims, l2=0.0, precision=0):
+        loss, g = real(w, X, y, dims, l2, precision)
+        g = g.copy()
+        g[-dims[-1]:] /= X.shape[0]
+        return loss, g
+    monkeypatch.setattr(models, "loss_and_grad", bad)
+    _fails(tm.test_gradient_matches_central_differences, [7, 10], 5, 0.0)
+
+
+def test_wrong_sign_of_the_local_step_is_caught(monkeypatch):
+    real = sim.run_task
+
+    def ascent(cfg, client_data, c, i, w_start):
+        U, w_end = real(cfg, client_data, c, i, w_start)
+        return U, 2 * np.asarray(w_start, dtype=np.float64) - w_end
+    monkeypatch.setattr(sim, "run_task", ascent)
+    _fails(tsim.test_update_sum_identity_U_equals_model_difference_over_eta)
+
+
+def test_forgotten_in_flight_correction_is_caught(monkeypatch):
+    real = sim.step_size
+    calls = {"n": 0}
+
+    # the correction is the only caller of step_size between a START and its run_task;
+    # make own in-flight sums count for nothing by zeroing U rows through a patched run
+    def run_without_correction(cfg, data, w0, n_rounds=None, keep=False, state=None):
+        n_rounds = cfg["n_rounds"] if n_rounds is None else n_rounds
+        events, summary, after = schedule.simulate(cfg, n_rounds, state)
+        order = sorted([(e["t_apply"], 0, e["client"], e["round"], e) for e in events] +
+                       [(e["t_start"], 1, e["client"], e["round"], e) for e in events], key=lambda r: r[:4])
+        w_g = np.array(w0, dtype=np.float64)
+        U = [None] * len(events)
+        for _, kind, c, i, e in order:
+            if kind == 1:
+                U[e["seq"]] = sim.run_task(cfg, data[c], c, i, w_g.copy())[0]     # no own-update correction
+            else:
+                w_g -= real(cfg, i) * U[e["seq"]]
+        return dict(events=events, summary=summary, w=w_g, U=U, w_start=[None] * len(events), state=after)
+    monkeypatch.setattr(sim, "run", run_without_correction)
+    _fails(tsim.test_one_client_is_plain_sgd_whatever_the_delays)
+
+
+def test_start_before_apply_on_ties_is_caught(monkeypatch):
+    monkeypatch.setattr(schedule, "APPLY", 1)
+    monkeypatch.setattr(schedule, "START", 0)
+    _fails(ts.test_apply_precedes_start_on_equal_ticks)
+
+
+def test_round_size_off_by_one_is_caught(monkeypatch):
+    monkeypatch.setattr(schedule, "sample_size", lambda a, b, i: a * (i + 1) + b)
+    _fails(ts.test_round_counts_printed_in_the_paper, ("linear", 60000, 10, 0, 1, 110))
+    _fails(ts.test_sample_totals_closed_form, "cfg2", 9300, 148800, 480)
+
+
+def test_checkpoint_that_counts_the_client_itself_is_caught(monkeypatch):
+    real = schedule.simulate
+
+    def lenient(cfg, n_rounds, state=None):
+        return real(dict(cfg, max_lag_d=schedule.NEVER_WAIT), n_rounds, state)
+    monkeypatch.setattr(schedule, "simulate", lenient)
+    _fails(ts.test_d0_every_client_waits_for_all_previous_rounds)
+    _fails(ts.test_two_client_timeline_worked_by_hand)
+
+
+def test_log2_instead_of_ln_is_caught(monkeypatch):
+    monkeypatch.setattr(rng, "LN2_Q32", 1 << 32)
+    _fails(tr.test_exp_scales_with_mean_and_floors_at_one_tick)
+    _fails(tr.test_exp_draws_have_the_right_distribution)
+
+
+def test_low_word_sample_index_is_caught(monkeypatch):
+    monkeypatch.setattr(rng, "sample_index", lambda r, n: ((r & 0xFFFFFFFF) * n) >> 32)
+    _fails(tsim.test_one_client_is_plain_sgd_whatever_the_delays)
+
+
+def test_wrong_mixing_constant_is_caught(monkeypatch):
+    real = rng.mix64
+    monkeypatch.setattr(rng, "mix64", lambda z: real(z) ^ 1)
+    _fails(tr.test_mix_matches_published_splitmix64_sequence)

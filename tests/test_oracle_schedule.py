@@ -147,6 +147,22 @@ def test_two_client_timeline_worked_by_hand():
     assert summary["messages_if_per_sample"] == 12 and summary["messages_if_constant_b"] == 12
 
 
+def test_apply_precedes_start_on_equal_ticks():
+    # Two equal clients, one sample per round, 5 ticks per iteration and per message, no waiting:
+    # rounds start at 0, 5, 10, ...; the updates of round i arrive at 5 i + 10, exactly when
+    # round i + 2 starts.  By the tie rule the server applies them first, so round i + 2 sees them.
+    tick = 1.0 / (1 << 20)
+    cfg = workloads.get_config("cfg1", n_clients=2, sched_a=0, sched_b=1, delay_dist=1,
+                               compute_delay_lo=5 * tick, compute_delay_hi=5 * tick,
+                               network_delay_lo=5 * tick, network_delay_hi=5 * tick,
+                               max_lag_d=schedule.NEVER_WAIT)
+    events, _, _ = schedule.simulate(cfg, 4)
+    for e in events:
+        assert (e["t_start"], e["t_trigger"], e["t_apply"]) == (5 * e["round"], 5 * e["round"] + 5, 5 * e["round"] + 10)
+        assert e["seen"] == 2 * max(0, e["round"] - 1)
+        assert e["seq"] == 2 * e["round"] + e["client"]
+
+
 def test_communication_cost_ratio_of_the_papers_setting():
     # K = 60,000 per node with s_i = 10 i from round 1: 110 messages per node
     # against 60,000 (one per sample) and 6,000 (constant s = 10, Table 5).
