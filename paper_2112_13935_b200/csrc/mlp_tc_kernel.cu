@@ -32,9 +32,10 @@ namespace {
 
 using namespace mlp;
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;   // 16 warps: enough loads in flight to cover HBM/L2 latency
+constexpr int kColSplit = kThreads / 128;  // warps sharing one 32-lane quarter of tensor memory split the columns
 constexpr int kRC = 32;        // rows per chunk of the FMA layers
-constexpr int kMaxTiles = 4;
+constexpr int kMaxTiles = 2;
 constexpr int kKC = 64;        // input rows per forward chunk
 constexpr int kMT = 128;       // input rows per backward chunk (M of the MMA)
 constexpr uint32_t kTmemCols = 512;
@@ -253,17 +254,17 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         unsigned char* tB = tiles + 2 * a_bytes + s * b_bytes;
         bar_drain(fbar[s], failed);  // the MMAs that last read this buffer are done
         // A: bf16(W0[c0 + k, j]) as element (row j, col k)
-        for (int e0 = tid; e0 < out0 * (kKC / 8); e0 += 4 * kThreads) {
-          float f[4][8];
+        for (int e0 = tid; e0 < out0 * (kKC / 8); e0 += 2 * kThreads) {
+          float f[2][8];
 #pragma unroll
-          for (int u4 = 0; u4 < 4; ++u4) {   // out0 * 8 is a multiple of 4 * kThreads: no tail
+          for (int u4 = 0; u4 < 2; ++u4) {   // out0 * 8 is a multiple of 2 * kThreads: no tail
             const int e = e0 + u4 * kThreads, j = e % out0, kg = e / out0;
             const float* src = work + woff[0] + (size_t)(c0 + kg * 8) * out0 + j;
 #pragma unroll
             for (int k = 0; k < 8; ++k) f[u4][k] = src[(size_t)k * out0];
           }
 #pragma unroll
-          for (int u4 = 0; u4 < 4; ++u4) {
+          for (int u4 = 0; u4 < 2; ++u4) {
             const int e = e0 + u4 * kThreads, j = e % out0, kg = e / out0;
             uint4 v;
             v.x = pack_bf16(f[u4][0], f[u4][1]); v.y = pack_bf16(f[u4][2], f[u4][3]);
@@ -296,8 +297,9 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       // partial Z0^T (lane = hidden unit, column = batch index) -> global scratch [b][n]
       {
         float* part = act + G.part[0] + (size_t)rank * B * out0;
-        const int span = n_mt * B, half = span / 2;
-        for (int cc0 = (warp >> 2) * half; cc0 < ((warp >> 2) + 1) * half; cc0 += 16) {
+        const int span = n_mt * B;
+        const int nsplit = min(kColSplit, span / 16), half = span / nsplit;
+        for (int cc0 = (warp >> 2) * half; (warp >> 2) < nsplit && cc0 < ((warp >> 2) + 1) * half; cc0 += 16) {
           uint32_t v[16];
           tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + cc0, v);
           const int mt = cc0 / B, b0 = cc0 % B;
@@ -575,7 +577,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         // block comes out of tensor memory one row per lane; a per-warp transpose through
         // shared memory lets every global access cover 4 rows x 128 contiguous bytes.
         float* tr = trbuf + warp * (32 * kTrLd);
-        const int half = out0 / 2;
+        const int half = out0 / kColSplit;   // 64 or 32 columns per warp
         const int rr = lane >> 3, cg = (lane & 7) * 4;
         for (int j0 = (warp >> 2) * half; j0 < ((warp >> 2) + 1) * half; j0 += 32) {
           uint32_t v[32];
@@ -587,17 +589,17 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
                 make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
           __syncwarp();
           const size_t base = woff[0] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + j0 + cg;
-          float4 w[8], u[8], g[8];
+          float4 w[8], u[8];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: 16 independent 16-byte loads in flight
             w[q] = *reinterpret_cast<const float4*>(work + base + (size_t)(4 * q) * out0);
             u[q] = *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0);
-            g[q] = *reinterpret_cast<const float4*>(tr + (4 * q + rr) * kTrLd + cg);
           }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
-            const float g0 = fmaf(lambda, w[q].x, g[q].x), g1 = fmaf(lambda, w[q].y, g[q].y);
-            const float g2 = fmaf(lambda, w[q].z, g[q].z), g3 = fmaf(lambda, w[q].w, g[q].w);
+            const float4 gq = *reinterpret_cast<const float4*>(tr + (4 * q + rr) * kTrLd + cg);
+            const float g0 = fmaf(lambda, w[q].x, gq.x), g1 = fmaf(lambda, w[q].y, gq.y);
+            const float g2 = fmaf(lambda, w[q].z, gq.z), g3 = fmaf(lambda, w[q].w, gq.w);
             w[q].x = fmaf(-eta, g0, w[q].x); w[q].y = fmaf(-eta, g1, w[q].y); w[q].z = fmaf(-eta, g2, w[q].z); w[q].w = fmaf(-eta, g3, w[q].w);
             u[q].x += g0; u[q].y += g1; u[q].z += g2; u[q].w += g3;
           }
