@@ -68,6 +68,19 @@ __host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
   return m;
 }
 
+// Can layer l of this shape use the tensor-core path?  (Rows are split evenly over the cluster.)
+__host__ __device__ inline bool tc_layer_ok(const MlpShape& s, int l) {
+  const int out = (int)s.dims[l + 1], rows = (int)(s.dims[l] / s.cluster), B = (int)s.batch;
+  if (l == 0) return true;                       // checked by mlp_tc_eligible
+  if (l == (int)s.n_layers - 1) return false;    // the class layer is too narrow for a 128-row tile
+  if (out != 128 && out != 256) return false;
+  if (s.dims[l] % s.cluster || rows % 128) return false;
+  const int out0 = (int)s.dims[1];
+  const int region = max(2 * out0 * kKC * 2 + 2 * B * kKC * 2, 2 * kMT * B * 2 + out0 * B * 2);
+  return (128 + B) * out * 2 <= region && 2 * out * kKC * 2 + 2 * B * kKC * 2 <= region &&
+         2 * kMT * B * 2 + out * B * 2 <= region;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // Shared-memory matrix descriptor: K-major, no swizzle.
@@ -154,7 +167,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / C];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int L = (int)S.n_layers, B = (int)S.batch;
-  const int D0 = (int)S.dims[0], out0 = (int)S.dims[1];
+  const int D0 = (int)S.dims[0];
   const TcSmem M = make_tc_smem(S);
   const Layout G = make_layout(S);
   unsigned char* tiles = smraw + M.tiles;
@@ -233,7 +246,10 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   }
   cluster_sync(clustered);
 
-  const int R0 = r1[0] - r0[0];
+  // Layers whose products run on tensor cores: layer 0 always; a hidden layer when its width
+  // and this CTA's slice of its rows fit the 128-row tiles and the operand tile region.
+  bool tc_layer[AET_MAX_LAYERS];
+  for (int l = 0; l < L; ++l) tc_layer[l] = tc_layer_ok(S, l);
   const uint32_t sbo_k64 = (kKC / 8) * 128;   // tiles with K = 64: next 8-row group after 8 core matrices
   const uint32_t sbo_kB = (B / 8) * 128;      // tiles with K = B
   uint32_t h = 0;
@@ -243,13 +259,14 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       idx[b] = (int)sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * B + b), cd.n);
     __syncthreads();
 
-    // ================= forward, layer 0 (tensor cores) =================
-    {
+    // ================= forward of one layer on tensor cores =================
+    auto fwd_tc = [&](const int l) {
+      const int out0 = (int)S.dims[l + 1], Kin = (int)S.dims[l], R0 = r1[l] - r0[l];
       const int n_mt = out0 / 128;
       const uint32_t idesc = umma_idesc(128, B);
       const int a_bytes = out0 * kKC * 2, b_bytes = B * kKC * 2;
       for (int c = 0; c * kKC < R0; ++c) {
-        const int s = c & 1, c0 = r0[0] + c * kKC;
+        const int s = c & 1, c0 = r0[l] + c * kKC;
         unsigned char* tA = tiles + s * a_bytes;
         unsigned char* tB = tiles + 2 * a_bytes + s * b_bytes;
         bar_drain(fbar[s], failed);  // the MMAs that last read this buffer are done
@@ -259,7 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
 #pragma unroll
           for (int u4 = 0; u4 < 2; ++u4) {   // out0 * 8 is a multiple of 2 * kThreads: no tail
             const int e = e0 + u4 * kThreads, j = e % out0, kg = e / out0;
-            const float* src = work + woff[0] + (size_t)(c0 + kg * 8) * out0 + j;
+            const float* src = work + woff[l] + (size_t)(c0 + kg * 8) * out0 + j;
 #pragma unroll
             for (int k = 0; k < 8; ++k) f[u4][k] = src[(size_t)k * out0];
           }
@@ -272,10 +289,17 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
             *reinterpret_cast<uint4*>(tA + (j >> 3) * sbo_k64 + kg * 128 + (j & 7) * 16) = v;
           }
         }
-        // B: X[idx[b], c0 + k] as element (row b, col k); already bf16 in HBM
+        // B: the layer's input, element (row b, col k): X[idx[b], c0 + k] (bf16 in HBM) or A_{l-1}[b, c0 + k]
         for (int e = tid; e < B * (kKC / 8); e += kThreads) {
           const int kg = e % (kKC / 8), b = e / (kKC / 8);
-          const uint4 v = __ldg(reinterpret_cast<const uint4*>(xdata + (size_t)idx[b] * D0 + c0 + kg * 8));
+          uint4 v;
+          if (l == 0) {
+            v = __ldg(reinterpret_cast<const uint4*>(xdata + (size_t)idx[b] * D0 + c0 + kg * 8));
+          } else {
+            const float4* src = reinterpret_cast<const float4*>(act + G.a[l - 1] + (size_t)b * Kin + c0 + kg * 8);
+            const float4 lo = src[0], hi = src[1];
+            v.x = pack_bf16(lo.x, lo.y); v.y = pack_bf16(lo.z, lo.w); v.z = pack_bf16(hi.x, hi.y); v.w = pack_bf16(hi.z, hi.w);
+          }
           *reinterpret_cast<uint4*>(tB + (b >> 3) * sbo_k64 + kg * 128 + (b & 7) * 16) = v;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -296,7 +320,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       // partial Z0^T (lane = hidden unit, column = batch index) -> global scratch [b][n]
       {
-        float* part = act + G.part[0] + (size_t)rank * B * out0;
+        float* part = act + G.part[l] + (size_t)rank * B * out0;
         const int span = n_mt * B;
         const int nsplit = min(kColSplit, span / 16), half = span / nsplit;
         for (int cc0 = (warp >> 2) * half; (warp >> 2) < nsplit && cc0 < ((warp >> 2) + 1) * half; cc0 += 16) {
@@ -310,23 +334,25 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       cluster_sync(clustered);
-      // bias + ReLU + bf16 rounding of the columns this CTA feeds into layer 1
+      // bias + ReLU + bf16 rounding of the columns this CTA feeds into the next layer
       {
-        const float* part0 = act + G.part[0];
-        const float* bias = work + boff[0];
-        const int c_lo = r0[1], c_n = r1[1] - r0[1];
+        const float* part0 = act + G.part[l];
+        const float* bias = work + boff[l];
+        const int c_lo = r0[l + 1], c_n = r1[l + 1] - r0[l + 1];
         staged_copy(B * c_n, tid,
                     [&](int e) { const int b = e / c_n, n = c_lo + e % c_n;
                                  float z = bias[n];
                                  for (int r = 0; r < C; ++r) z += part0[((size_t)r * B + b) * out0 + n];
                                  return z; },
-                    [&](int e, float z) { act[G.a[0] + (size_t)(e / c_n) * out0 + c_lo + e % c_n] = q_bf16(fmaxf(z, 0.f)); });
+                    [&](int e, float z) { act[G.a[l] + (size_t)(e / c_n) * out0 + c_lo + e % c_n] = q_bf16(fmaxf(z, 0.f)); });
         __syncthreads();
       }
-    }
+    };
+    fwd_tc(0);
 
     // ================= forward, layers >= 1 (FMA) =================
     for (int l = 1; l < L; ++l) {
+      if (tc_layer[l]) { fwd_tc(l); continue; }
       const int N = (int)S.dims[l + 1], Np = up4(N), ldw = Np + 4;
       const int tiles_n = Np / 4, ntile = (B / 4) * tiles_n;
       float acc[kMaxTiles][16];
@@ -418,8 +444,182 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       }
     }
 
+    // ================= backward + update of one layer on tensor cores =================
+    auto bwd_tc = [&](const int l) {
+      const int out0 = (int)S.dims[l + 1], Kin = (int)S.dims[l], R0 = r1[l] - r0[l];
+      const float* dz0 = act + G.dz[l];          // full dZ_l [B, out], fp32, visible after a cluster barrier
+      if (l > 0) {
+        // dZ_{l-1}[b, i] = relu'(A_{l-1}[b, i]) * sum_j W_l[i, j] bf16(dZ_l)[b, j] for the rows i this CTA owns,
+        // from the weights as they are before this iteration's update:
+        // D[128 rows x B] = bf16(W_l chunk)[128 x out] . bf16(dZ_l)[B x out]^T
+        const uint32_t sbo_ko = (out0 / 8) * 128;
+        unsigned char* tW = tiles;
+        unsigned char* tD = tiles + 128 * out0 * 2;
+        const uint32_t idesc_a = umma_idesc(128, B);
+        __syncthreads();
+        for (int e = tid; e < B * (out0 / 8); e += kThreads) {
+          const int kg = e % (out0 / 8), b = e / (out0 / 8);
+          const float4* src = reinterpret_cast<const float4*>(dz0 + (size_t)b * out0 + kg * 8);
+          const float4 lo = src[0], hi = src[1];
+          uint4 v;
+          v.x = pack_bf16(lo.x, lo.y); v.y = pack_bf16(lo.z, lo.w); v.z = pack_bf16(hi.x, hi.y); v.w = pack_bf16(hi.z, hi.w);
+          *reinterpret_cast<uint4*>(tD + (b >> 3) * sbo_ko + kg * 128 + (b & 7) * 16) = v;
+        }
+        for (int c0 = r0[l]; c0 < r1[l]; c0 += kMT) {
+          for (int e = tid; e < kMT * (out0 / 8); e += kThreads) {
+            const int kg = e % (out0 / 8), i = e / (out0 / 8);
+            const float4* src = reinterpret_cast<const float4*>(work + woff[l] + (size_t)(c0 + i) * out0 + kg * 8);
+            const float4 lo = src[0], hi = src[1];
+            uint4 v;
+            v.x = pack_bf16(lo.x, lo.y); v.y = pack_bf16(lo.z, lo.w); v.z = pack_bf16(hi.x, hi.y); v.w = pack_bf16(hi.z, hi.w);
+            *reinterpret_cast<uint4*>(tW + (i >> 3) * sbo_ko + kg * 128 + (i & 7) * 16) = v;
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncthreads();
+          if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            for (int j = 0; j < out0 / 16; ++j)
+              umma_bf16(tmem, umma_desc(smem_u32(tW) + j * 256, 128, sbo_ko),
+                        umma_desc(smem_u32(tD) + j * 256, 128, sbo_ko), idesc_a, j > 0 ? 1u : 0u);
+            umma_commit(fbar[0].bar);
+          }
+          ++fbar[0].issued;
+          bar_drain(fbar[0], failed);
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          {
+            const int nsplit = min(kColSplit, B / 16), half = B / nsplit;
+            const int i = c0 + (warp & 3) * 32 + lane;   // lane = row of the chunk, columns = batch index
+            for (int b0 = (warp >> 2) * half; (warp >> 2) < nsplit && b0 < ((warp >> 2) + 1) * half; b0 += 16) {
+              uint32_t v[16];
+              tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + b0, v);
+              float a[16];
+#pragma unroll
+              for (int q = 0; q < 16; ++q) a[q] = act[G.a[l - 1] + (size_t)(b0 + q) * Kin + i];
+#pragma unroll
+              for (int q = 0; q < 16; ++q)
+                act[G.dz[l - 1] + (size_t)(b0 + q) * Kin + i] = a[q] > 0.f ? __uint_as_float(v[q]) : 0.f;
+            }
+          }
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncthreads();   // the tile and the accumulator are free again
+        }
+      }
+      const int a_bytes = kMT * B * 2;
+      unsigned char* tBd = tiles + 2 * a_bytes;  // bf16(dZ0)^T: element (row j, col b)
+      const uint32_t idesc = umma_idesc(128, out0);
+      __syncthreads();
+      for (int e = tid; e < out0 * (B / 8); e += kThreads) {
+        const int j = e % out0, bg = e / out0;
+        const float* src = dz0 + (size_t)(bg * 8) * out0 + j;
+        uint4 v;
+        v.x = pack_bf16(src[0], src[out0]);
+        v.y = pack_bf16(src[2 * (size_t)out0], src[3 * (size_t)out0]);
+        v.z = pack_bf16(src[4 * (size_t)out0], src[5 * (size_t)out0]);
+        v.w = pack_bf16(src[6 * (size_t)out0], src[7 * (size_t)out0]);
+        *reinterpret_cast<uint4*>(tBd + (j >> 3) * sbo_kB + bg * 128 + (j & 7) * 16) = v;
+      }
+      const int nch = R0 / kMT;
+      auto stage_and_issue = [&](int c) {
+        const int s = c & 1, c0 = r0[l] + c * kMT;
+        unsigned char* tA = tiles + s * a_bytes;  // the layer's input, transposed: element (row i, col b)
+        for (int e = tid; e < kMT * (B / 8); e += kThreads) {
+          const int i = e % kMT, bg = e / kMT;
+          uint4 v;
+          if (l == 0) {
+            const __nv_bfloat16* col = xdata + c0 + i;
+            unsigned short q[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) q[k] = __ldg(reinterpret_cast<const unsigned short*>(col + (size_t)idx[bg * 8 + k] * D0));
+            v.x = q[0] | ((uint32_t)q[1] << 16); v.y = q[2] | ((uint32_t)q[3] << 16);
+            v.z = q[4] | ((uint32_t)q[5] << 16); v.w = q[6] | ((uint32_t)q[7] << 16);
+          } else {
+            const float* col = act + G.a[l - 1] + (size_t)(bg * 8) * Kin + c0 + i;
+            float f[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) f[k] = col[(size_t)k * Kin];
+            v.x = pack_bf16(f[0], f[1]); v.y = pack_bf16(f[2], f[3]); v.z = pack_bf16(f[4], f[5]); v.w = pack_bf16(f[6], f[7]);
+          }
+          *reinterpret_cast<uint4*>(tA + (i >> 3) * sbo_kB + bg * 128 + (i & 7) * 16) = v;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          for (int j = 0; j < B / 16; ++j)
+            umma_bf16(tmem + s * 256, umma_desc(smem_u32(tA) + j * 256, 128, sbo_kB),
+                      umma_desc(smem_u32(tBd) + j * 256, 128, sbo_kB), idesc, j > 0 ? 1u : 0u);
+          umma_commit(bbar[s].bar);
+        }
+        ++bbar[s].issued;
+      };
+      if (nch > 0) stage_and_issue(0);
+      for (int c = 0; c < nch; ++c) {
+        const int s = c & 1, c0 = r0[l] + c * kMT;
+        if (c + 1 < nch) stage_and_issue(c + 1);   // its buffer and accumulator were released by chunk c-1
+        bar_drain(bbar[s], failed);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // epilogue: a warp owns 32 rows of W0 and half of the columns.  The accumulator
+        // block comes out of tensor memory one row per lane; a per-warp transpose through
+        // shared memory lets every global access cover 4 rows x 128 contiguous bytes.
+        float* tr = trbuf + warp * (32 * kTrLd);
+        const int half = out0 / kColSplit;   // 64 or 32 columns per warp
+        const int rr = lane >> 3, cg = (lane & 7) * 4;
+        for (int j0 = (warp >> 2) * half; j0 < ((warp >> 2) + 1) * half; j0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + s * 256 + j0, v);
+          __syncwarp();
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<float4*>(tr + lane * kTrLd + 4 * q) =
+                make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          __syncwarp();
+          const size_t base = woff[l] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + j0 + cg;
+          float4 w[8], u[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: 16 independent 16-byte loads in flight
+            w[q] = *reinterpret_cast<const float4*>(work + base + (size_t)(4 * q) * out0);
+            u[q] = *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0);
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 gq = *reinterpret_cast<const float4*>(tr + (4 * q + rr) * kTrLd + cg);
+            const float g0 = fmaf(lambda, w[q].x, gq.x), g1 = fmaf(lambda, w[q].y, gq.y);
+            const float g2 = fmaf(lambda, w[q].z, gq.z), g3 = fmaf(lambda, w[q].w, gq.w);
+            w[q].x = fmaf(-eta, g0, w[q].x); w[q].y = fmaf(-eta, g1, w[q].y); w[q].z = fmaf(-eta, g2, w[q].z); w[q].w = fmaf(-eta, g3, w[q].w);
+            u[q].x += g0; u[q].y += g1; u[q].z += g2; u[q].w += g3;
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            *reinterpret_cast<float4*>(work + base + (size_t)(4 * q) * out0) = w[q];
+            *reinterpret_cast<float4*>(Urow + base + (size_t)(4 * q) * out0) = u[q];
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      }
+      cluster_sync(clustered);
+      if (rank == l % C)
+        for (int n = tid; n < out0; n += kThreads) {
+          float gb = 0.f;
+          for (int b = 0; b < B; ++b) gb += dz0[(size_t)b * out0 + n];
+          work[boff[l] + n] = fmaf(-eta, gb, work[boff[l] + n]);
+          Urow[boff[l] + n] += gb;
+        }
+      if (l > 1 && !tc_layer[l - 1]) {   // the FMA layer below reads dZ_{l-1} from shared memory
+        __syncthreads();
+        const int Nm = (int)S.dims[l], Nmp = up4(Nm);
+        staged_copy(B * Nmp, tid,
+                    [&](int e) { const int b = e / Nmp, n = e % Nmp;
+                                 return n < Nm ? act[G.dz[l - 1] + (size_t)b * Nm + n] : 0.f; },
+                    [&](int e, float d) { dzs[e] = d; dzq[e] = q_bf16(d); });
+        __syncthreads();
+      }
+    };
+
     // ================= backward + update, layers >= 1 (FMA) =================
     for (int l = L - 1; l >= 1; --l) {
+      if (tc_layer[l]) { bwd_tc(l); continue; }
       const int N = (int)S.dims[l + 1], Np = up4(N), ldw = Np + 4;
       const int K = (int)S.dims[l];
       for (int c0 = r0[l]; c0 < r1[l]; c0 += kRC) {
@@ -512,7 +712,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
           work[boff[l] + n] = fmaf(-eta, gb, work[boff[l] + n]);
           Urow[boff[l] + n] += gb;
         }
-      if (l > 1) {
+      if (l > 1 && !tc_layer[l - 1]) {
         __syncthreads();
         const int Nm = (int)S.dims[l], Nmp = up4(Nm);
         staged_copy(B * Nmp, tid,
@@ -523,103 +723,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       }
     }
 
-    // ================= backward + update, layer 0 (tensor cores) =================
-    {
-      const float* dz0 = act + G.dz[0];          // full dZ0 [B, out0], fp32, visible after the barrier above
-      const int a_bytes = kMT * B * 2;
-      unsigned char* tBd = tiles + 2 * a_bytes;  // bf16(dZ0)^T: element (row j, col b)
-      const uint32_t idesc = umma_idesc(128, out0);
-      __syncthreads();
-      for (int e = tid; e < out0 * (B / 8); e += kThreads) {
-        const int j = e % out0, bg = e / out0;
-        const float* src = dz0 + (size_t)(bg * 8) * out0 + j;
-        uint4 v;
-        v.x = pack_bf16(src[0], src[out0]);
-        v.y = pack_bf16(src[2 * (size_t)out0], src[3 * (size_t)out0]);
-        v.z = pack_bf16(src[4 * (size_t)out0], src[5 * (size_t)out0]);
-        v.w = pack_bf16(src[6 * (size_t)out0], src[7 * (size_t)out0]);
-        *reinterpret_cast<uint4*>(tBd + (j >> 3) * sbo_kB + bg * 128 + (j & 7) * 16) = v;
-      }
-      const int nch = R0 / kMT;
-      auto stage_and_issue = [&](int c) {
-        const int s = c & 1, c0 = r0[0] + c * kMT;
-        unsigned char* tA = tiles + s * a_bytes;  // X^T chunk: element (row i, col b)
-        for (int e = tid; e < kMT * (B / 8); e += kThreads) {
-          const int i = e % kMT, bg = e / kMT;
-          const __nv_bfloat16* col = xdata + c0 + i;
-          unsigned short q[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) q[k] = __ldg(reinterpret_cast<const unsigned short*>(col + (size_t)idx[bg * 8 + k] * D0));
-          uint4 v;
-          v.x = q[0] | ((uint32_t)q[1] << 16); v.y = q[2] | ((uint32_t)q[3] << 16);
-          v.z = q[4] | ((uint32_t)q[5] << 16); v.w = q[6] | ((uint32_t)q[7] << 16);
-          *reinterpret_cast<uint4*>(tA + (i >> 3) * sbo_kB + bg * 128 + (i & 7) * 16) = v;
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (tid == 0) {
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          for (int j = 0; j < B / 16; ++j)
-            umma_bf16(tmem + s * 256, umma_desc(smem_u32(tA) + j * 256, 128, sbo_kB),
-                      umma_desc(smem_u32(tBd) + j * 256, 128, sbo_kB), idesc, j > 0 ? 1u : 0u);
-          umma_commit(bbar[s].bar);
-        }
-        ++bbar[s].issued;
-      };
-      if (nch > 0) stage_and_issue(0);
-      for (int c = 0; c < nch; ++c) {
-        const int s = c & 1, c0 = r0[0] + c * kMT;
-        if (c + 1 < nch) stage_and_issue(c + 1);   // its buffer and accumulator were released by chunk c-1
-        bar_drain(bbar[s], failed);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // epilogue: a warp owns 32 rows of W0 and half of the columns.  The accumulator
-        // block comes out of tensor memory one row per lane; a per-warp transpose through
-        // shared memory lets every global access cover 4 rows x 128 contiguous bytes.
-        float* tr = trbuf + warp * (32 * kTrLd);
-        const int half = out0 / kColSplit;   // 64 or 32 columns per warp
-        const int rr = lane >> 3, cg = (lane & 7) * 4;
-        for (int j0 = (warp >> 2) * half; j0 < ((warp >> 2) + 1) * half; j0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + s * 256 + j0, v);
-          __syncwarp();
-#pragma unroll
-          for (int q = 0; q < 8; ++q)
-            *reinterpret_cast<float4*>(tr + lane * kTrLd + 4 * q) =
-                make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
-          __syncwarp();
-          const size_t base = woff[0] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + j0 + cg;
-          float4 w[8], u[8];
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: 16 independent 16-byte loads in flight
-            w[q] = *reinterpret_cast<const float4*>(work + base + (size_t)(4 * q) * out0);
-            u[q] = *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0);
-          }
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const float4 gq = *reinterpret_cast<const float4*>(tr + (4 * q + rr) * kTrLd + cg);
-            const float g0 = fmaf(lambda, w[q].x, gq.x), g1 = fmaf(lambda, w[q].y, gq.y);
-            const float g2 = fmaf(lambda, w[q].z, gq.z), g3 = fmaf(lambda, w[q].w, gq.w);
-            w[q].x = fmaf(-eta, g0, w[q].x); w[q].y = fmaf(-eta, g1, w[q].y); w[q].z = fmaf(-eta, g2, w[q].z); w[q].w = fmaf(-eta, g3, w[q].w);
-            u[q].x += g0; u[q].y += g1; u[q].z += g2; u[q].w += g3;
-          }
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            *reinterpret_cast<float4*>(work + base + (size_t)(4 * q) * out0) = w[q];
-            *reinterpret_cast<float4*>(Urow + base + (size_t)(4 * q) * out0) = u[q];
-          }
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      }
-      cluster_sync(clustered);
-      if (rank == 0)
-        for (int n = tid; n < out0; n += kThreads) {
-          float gb = 0.f;
-          for (int b = 0; b < B; ++b) gb += dz0[(size_t)b * out0 + n];
-          work[boff[0] + n] = fmaf(-eta, gb, work[boff[0] + n]);
-          Urow[boff[0] + n] += gb;
-        }
-    }
+    bwd_tc(0);
     h += (uint32_t)B;
   }
 
