@@ -28,9 +28,9 @@ namespace {
 
 using namespace mlp;
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kRC = 32;        // rows of W_l staged per chunk
-constexpr int kMaxTiles = 4;   // 4x4 output micro-tiles per thread in the forward product
+constexpr int kMaxTiles = 2;   // 4x4 output micro-tiles per thread in the forward product
 
 struct Smem {  // offsets (in floats) into dynamic shared memory
   int idx, As, AsT, Ws, dzs, dzq, zs, total;
