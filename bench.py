@@ -30,8 +30,8 @@ import numpy as np  # noqa: E402
 
 METRIC = "client_sgd_samples_per_sec"
 UNIT = "samples/s"
-CPU_BUDGET_S = 15.0      # CPU-baseline sample per run
-REF_STEP_BUDGET_S = 2.5  # --impl reference: CPU work per step
+CPU_LIMIT_S = 15.0      # CPU-baseline sample per run
+REF_STEP_LIMIT_S = 2.5  # --impl reference: CPU work per step
 
 DESCRIBE = {
     "cfg1": "cfg1: 4 clients, softmax regression 784->10 fp32, l2 1e-4, s_i=10i+10, 5 rounds",
@@ -137,9 +137,9 @@ class ClockSampler:
         return out
 
 
-def oracle_bounded(cfg, data, w0, budget_s):
+def oracle_bounded(cfg, data, w0, limit_s):
     """The CPU checker as it stands on a bounded sample of the workload: its
-    schedule, then round-tasks in start order until the time budget is spent."""
+    schedule, then round-tasks in start order until the time limit is reached."""
     from oracle import schedule, sim
     t0 = time.perf_counter()
     events, _, _ = schedule.simulate(cfg, cfg["n_rounds"])
@@ -150,7 +150,7 @@ def oracle_bounded(cfg, data, w0, budget_s):
         sim.run_task(cfg, data[e["client"]], e["client"], e["round"], w)
         done_samples += e["samples"]
         done_tasks += 1
-        if time.perf_counter() - t0 > budget_s:
+        if time.perf_counter() - t0 > limit_s:
             break
     dt = time.perf_counter() - t0
     return done_samples / dt, done_samples, done_tasks, len(events), dt
@@ -174,7 +174,7 @@ def run_reference(args, cfg):
     rates, sample = [], ""
     with threadpool_limits(limits=cores):
         for step in range(args.warmup + args.steps):
-            rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, REF_STEP_BUDGET_S)
+            rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, REF_STEP_LIMIT_S)
             if step >= args.warmup:
                 rates.append((n_s, dt))
             sample = f"schedule + first {n_t} of {n_e} round-tasks in start order ({n_s} samples) per step"
@@ -330,7 +330,7 @@ def main():
         from threadpoolctl import threadpool_limits
         cores = blas_threads(cfg)
         with threadpool_limits(limits=cores):
-            rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, CPU_BUDGET_S)
+            rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, CPU_LIMIT_S)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"schedule + first {n_t} of {n_e} round-tasks in start order ({n_s} samples, {dt:.1f} s)"}
 

@@ -5,7 +5,7 @@ Python-integer arithmetic, so results are bit-reproducible.
 
 The paper fixes no generator: it samples "uniformly at random xi from D_c"
 (Algorithm 3) and injects random compute / network delays (Section 3.3.2,
-Section 5 "System delay").  The convention used by this build:
+Section 5 "System delay").  The convention used here:
 
 * mixing function = the SplitMix64 output function (Steele, Lea, Flood 2014);
 * a stream key is derived from (seed, stream id, client), a draw from

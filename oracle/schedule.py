@@ -21,7 +21,7 @@ Follows the paper as below.
 Client-server form of Section 1: the server applies update sums in arrival
 order; a client pulls the server's model when its round starts.
 
-Conventions the paper leaves open (fixed for this build):
+Conventions the paper leaves open (fixed here):
 * time is integer ticks, 2^20 per unit; ties are ordered by
   (tick, APPLY before START, client, round);
 * H_c counts the updates of client c the server has applied (Algorithm 3 bumps

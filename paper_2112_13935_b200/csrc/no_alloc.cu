@@ -1,7 +1,7 @@
 // aet_round_no_alloc: one round-task without a handle and without any allocation.
 //
 // Some hosts of this library may not allocate device memory while they run: a
-// service that has handed its whole memory budget to a pool at start-up, code
+// service that has handed all of its device memory to a pool at start-up, code
 // running between a framework's allocator snapshots, or a process that must keep
 // cudaMalloc (which synchronises the device) off its latency path.  For them the
 // scratch the round kernel needs - the task and client descriptors, the client's
