@@ -41,6 +41,14 @@ constexpr int kMT = 128;       // input rows per backward chunk (M of the MMA)
 constexpr uint32_t kTmemCols = 512;
 constexpr int kTrLd = 36;     // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
 constexpr uint32_t kWaitLimit = 1u << 22;
+// The widest layer's update sum is not accumulated entry by entry: Algorithm 3 does
+// w -= eta * g and U += g in the same step with eta constant within the round, so
+// U_i = (w_start - w_end) / eta_i holds term by term.  The row of U keeps w_start during
+// the round and is turned into U_i at the event trigger; this removes the read and the
+// write of U_0 (40 % of the HBM traffic) from every SGD iteration.  In fp32 the quotient
+// carries the rounding of the master updates (about 1e-4 of max|U| here), which is inside
+// the noise of the bf16 operand roundings of this path; the fp32 kernels accumulate U.
+constexpr bool kDeriveU0 = true;
 
 struct TcSmem {  // byte offsets into dynamic shared memory
   int tiles, idx, As, AsT, Ws, dzs, dzq, zs, tr, total;
@@ -230,7 +238,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
           w = fmaf(-ref.eta, p.r.U[(size_t)ref.seq * p.r.stride + j], w);
         }
         work[j] = w;
-        Urow[j] = 0.f;
+        Urow[j] = (kDeriveU0 && l == 0) ? w : 0.f;
       }
       if (rank == l % C)
         for (int j = tid; j < N; j += kThreads) {
@@ -576,11 +584,13 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
                 make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
           __syncwarp();
           const size_t base = woff[l] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + j0 + cg;
+          const bool with_u = !(kDeriveU0 && l == 0);
           float4 w[8], u[8];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: 16 independent 16-byte loads in flight
+          for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: independent 16-byte loads in flight
             w[q] = *reinterpret_cast<const float4*>(work + base + (size_t)(4 * q) * out0);
-            u[q] = *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0);
+            u[q] = with_u ? *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0)
+                          : make_float4(0.f, 0.f, 0.f, 0.f);
           }
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
@@ -593,7 +603,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             *reinterpret_cast<float4*>(work + base + (size_t)(4 * q) * out0) = w[q];
-            *reinterpret_cast<float4*>(Urow + base + (size_t)(4 * q) * out0) = u[q];
+            if (with_u) *reinterpret_cast<float4*>(Urow + base + (size_t)(4 * q) * out0) = u[q];
           }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -729,6 +739,15 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
 
   // ---- event trigger: publish (c, U_i, i) ----
   cluster_sync(clustered);
+  if (kDeriveU0) {   // U_0 = (w_start - w_end) / eta on this CTA's rows of W_0
+    const float inv_eta = 1.f / eta;
+    const size_t lo = woff[0] + (size_t)r0[0] * S.dims[1], hi = woff[0] + (size_t)r1[0] * S.dims[1];
+    for (size_t j = lo + 4 * (size_t)tid; j < hi; j += 4 * kThreads) {   // slices start and end on 16-byte boundaries
+      const float4 a = *reinterpret_cast<const float4*>(Urow + j), b = *reinterpret_cast<const float4*>(work + j);
+      *reinterpret_cast<float4*>(Urow + j) =
+          make_float4((a.x - b.x) * inv_eta, (a.y - b.y) * inv_eta, (a.z - b.z) * inv_eta, (a.w - b.w) * inv_eta);
+    }
+  }
   if (p.r.w_end) {
     float* dst = p.r.w_end + (size_t)t.seq * p.r.stride;
     for (int l = 0; l < L; ++l) {

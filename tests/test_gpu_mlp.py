@@ -97,3 +97,18 @@ def test_cfg3_full_size_log_invariant_and_sampled_rounds():
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
         for c, i in ((0, 0), (31, 7), (13, 39)):
             check_round_U(cfg, data, s.h, c, i, gpu["w"])
+
+
+def test_cfg4_full_size_log_and_sampled_rounds():
+    # full size, the launch configuration bench.py times: clusters of 2, all layers with 128-row slices on tensor cores
+    cfg = workloads.get_config("cfg4")
+    data, w0 = make(cfg)
+    from oracle import schedule
+    events, summary, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    gpu = run_gpu(cfg, data, w0, want_U=False)
+    assert gpu["blob"] == schedule.pack_events(events) and gpu["summary"] == summary
+    assert summary["samples_total"] == 3809280 and len(events) == 1920
+    assert np.isfinite(gpu["w"]).all()
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for c, i in ((0, 0), (63, 3), (17, 29)):
+            check_round_U(cfg, data, s.h, c, i, gpu["w"], BF16_U_TOL)
