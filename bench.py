@@ -239,9 +239,12 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > L2 (126 MB)
 
     sess = api.Session(cfg, dev, w0_dev)
+    plan_ms = None
     for _ in range(args.warmup):
         sess.reset()
         sess.run(R)
+        if plan_ms is None:   # host time of the integer schedule + launch plan; later runs reuse the cached plan
+            plan_ms = api.aet_get_stats(sess.h)["plan_ms"]
     torch.cuda.synchronize()
     events, summary = sess.log()
     assert summary["samples_total"] == samples
@@ -352,7 +355,7 @@ def main():
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roof,
             "cpu_baseline": cpu,
-            "plan_ms_first_run": stats["plan_ms"],
+            "schedule_and_plan_ms_first_run": plan_ms,
         }
         print(json.dumps(line))
     dist.shutdown()
