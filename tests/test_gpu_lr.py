@@ -62,16 +62,16 @@ def test_cfg5_shape_64_clients_end_to_end():
     assert np.abs(gpu["w"] - ref["w"]).max() <= 2e-5
 
 
-@pytest.mark.parametrize("l2", [0.0, 1e-3])
-def test_many_clients_take_the_kernel_variant_for_crowded_waves(l2):
+@pytest.mark.parametrize("n_clients,l2", [(320, 0.0), (320, 1e-3), (480, 0.0), (480, 1e-3)])
+def test_many_clients_take_the_kernel_variant_for_crowded_waves(n_clients, l2):
     # >= 296 round-tasks in a wave switch the kernel to its one-warp softmax
-    cfg = workloads.get_config("cfg5", n_clients=320, n_rounds=3, l2=l2, data=dict(per_client=64))
+    cfg = workloads.get_config("cfg5", n_clients=n_clients, n_rounds=3, l2=l2, data=dict(per_client=64))
     data, w0 = make(cfg)
     ref = sim.run(cfg, data, w0, keep=True)
     gpu = run_gpu(cfg, data, w0)
     check_against_oracle(cfg, data, w0, gpu, ref)
     assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
-    for k in (0, 400, 959):
+    for k in (0, 400, 3 * n_clients - 1):
         assert rel_err(gpu["U"][k], ref["U"][k]) <= 1e-4
 
 
