@@ -5,16 +5,18 @@
 // w_c -= eta_i g; U_i += g).  Same cluster structure as the fp32 kernel: every
 // W_l is split by input rows over the CTAs of the round-task's cluster.  What
 // changes is layer 0, which carries ~95 % of the flops of a 3072-256-128-10 net:
-//   forward   Z0^T[out0 x B] += W0[rows]^T . X[:, rows]^T   chunks of 64 input rows:
-//             A = bf16(W0 chunk)^T [out0 x 64] (converted from the fp32 master on
-//             the way into shared memory), B = X chunk [B x 64]; tcgen05.mma
-//             M = 128 (x out0/128), N = B, K = 16 x 4, fp32 accumulators in TMEM;
-//             operand tiles double-buffered, completion by tcgen05.commit on mbarriers;
-//   backward  G[128 rows x out0] = X[:, rows]^T . dZ0       chunks of 128 input rows:
-//             A = X chunk^T [128 x B], B = bf16(dZ0)^T [out0 x B]; M = 128, N = out0,
-//             K = B; two TMEM accumulators so the MMAs of chunk c+1 run while the
-//             epilogue of chunk c reads its tile back (tcgen05.ld) and does
-//             g = G + lambda W, W -= eta g, U += g on the fp32 master in HBM/L2.
+//   forward   Z0^T[out0 x B] += W0[rows]^T . X[:, rows]^T: A = bf16(W0 chunk)^T, B = X chunk
+//             [B x rows]; tcgen05.mma M = 128 (x out0/128), N = B, fp32 accumulators in TMEM.
+//             Only the first iteration of a round runs it as a pass of its own (chunks of 64
+//             rows converted from the fp32 master, tiles double-buffered, completion by
+//             tcgen05.commit on mbarriers); afterwards the product for iteration t + 1 is
+//             issued from inside the backward pass of iteration t, chunk by chunk, from the
+//             weights that pass has just updated, so W0 is read once per iteration, not twice;
+//   backward  G[128 rows x out0] = X[:, rows]^T . dZ0       chunks of 128 input rows, in units
+//             of 128 columns: A = X chunk^T [128 x B], B = bf16(dZ0)^T [128 x B]; M = 128,
+//             N = 128, K = B; two TMEM slots so the MMAs of unit u+1 run while the epilogue
+//             of unit u reads its tile back (tcgen05.ld) and does g = G + lambda W,
+//             W -= eta g on the fp32 master in HBM/L2.
 // Operand tiles use the K-major, no-swizzle core-matrix layout (8 rows x 16 bytes
 // contiguous; LBO = stride between core matrices along K, SBO = along M/N).
 // The narrow layers (l >= 1), softmax and bias updates run on plain FMAs.
@@ -39,6 +41,7 @@ constexpr int kMaxTiles = 2;
 constexpr int kKC = 64;        // input rows per forward chunk
 constexpr int kMT = 128;       // input rows per backward chunk (M of the MMA)
 constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kFwdCol = 256;   // tensor-memory columns [256, 384): layer-0 forward accumulators
 constexpr int kTrLd = 36;     // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
 constexpr uint32_t kWaitLimit = 1u << 22;
 // The widest layer's update sum is not accumulated entry by entry: Algorithm 3 does
@@ -51,18 +54,25 @@ constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr bool kDeriveU0 = true;
 
 struct TcSmem {  // byte offsets into dynamic shared memory
-  int tiles, idx, As, AsT, Ws, dzs, dzq, zs, tr, total;
+  int tiles, idx, As, AsT, Ws, dzs, dzq, zs, tr, x2, total;
 };
-__host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
+// Operand-tile region: the larger of the stand-alone forward pass (two A and two B tiles of 64
+// input rows) and the layer-0 backward pass (two X^T tiles, bf16(dZ0)^T, and for the forward
+// product of the next iteration one tile of updated weights and one tile of next-batch inputs).
+__host__ __device__ inline int tc_tiles_bytes(const MlpShape& s) {
   const int B = (int)s.batch, out0 = (int)s.dims[1];
+  const int fwd = 2 * out0 * kKC * 2 + 2 * B * kKC * 2;
+  const int bwd = 2 * kMT * B * 2 + out0 * B * 2 + 128 * kMT * 2 + B * kMT * 2;
+  return max(fwd, bwd);
+}
+__host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
+  const int B = (int)s.batch;
   int nmax = 0;
   for (uint32_t l = 1; l < s.n_layers; ++l) nmax = max(nmax, (int)((s.dims[l + 1] + 3) & ~3u));
-  const int fwd = 2 * out0 * kKC * 2 + 2 * B * kKC * 2;
-  const int bwd = 2 * kMT * B * 2 + out0 * B * 2;
   TcSmem m{};
   int o = 0;
-  m.tiles = o; o += max(fwd, bwd);
-  m.idx = o; o += B * 4;
+  m.tiles = o; o += tc_tiles_bytes(s);
+  m.idx = o; o += 2 * B * 4;   // sample indices of this iteration and of the next
   m.As = o; o += kRC * B * 4;
   m.AsT = o; o += B * kRC * 4;
   m.Ws = o; o += kRC * (nmax + 4) * 4;
@@ -70,8 +80,10 @@ __host__ __device__ inline TcSmem make_tc_smem(const MlpShape& s) {
   m.dzq = o; o += B * nmax * 4;
   m.zs = o; o += B * 32 * 4;
   // the transposes reuse the FMA layers' staging area (idle during the layer-0 backward pass)
+  // and are followed by the second tile of next-batch inputs
   m.tr = m.As;
-  if (o - m.As < (kThreads / 32) * 32 * kTrLd * 4) o = m.As + (kThreads / 32) * 32 * kTrLd * 4;
+  m.x2 = m.As + (kThreads / 32) * 32 * kTrLd * 4;
+  if (o < m.x2 + B * kMT * 2) o = m.x2 + B * kMT * 2;
   m.total = o;
   return m;
 }
@@ -83,8 +95,7 @@ __host__ __device__ inline bool tc_layer_ok(const MlpShape& s, int l) {
   if (l == (int)s.n_layers - 1) return false;    // the class layer is too narrow for a 128-row tile
   if (out != 128 && out != 256) return false;
   if (s.dims[l] % s.cluster || rows % 128) return false;
-  const int out0 = (int)s.dims[1];
-  const int region = max(2 * out0 * kKC * 2 + 2 * B * kKC * 2, 2 * kMT * B * 2 + out0 * B * 2);
+  const int region = tc_tiles_bytes(s);
   return (128 + B) * out * 2 <= region && 2 * out * kKC * 2 + 2 * B * kKC * 2 <= region &&
          2 * kMT * B * 2 + out * B * 2 <= region;
 }
@@ -165,7 +176,7 @@ __device__ __forceinline__ void bar_drain(CommitBar& b, bool& failed) {
 
 __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   extern __shared__ __align__(1024) unsigned char smraw[];
-  __shared__ __align__(8) uint64_t bars[4];
+  __shared__ __align__(8) uint64_t bars[5];
   __shared__ uint32_t tmem_base_s;
 
   const MlpShape& S = p.shape;
@@ -179,7 +190,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   const TcSmem M = make_tc_smem(S);
   const Layout G = make_layout(S);
   unsigned char* tiles = smraw + M.tiles;
-  int* idx = reinterpret_cast<int*>(smraw + M.idx);
+  int* idxbuf = reinterpret_cast<int*>(smraw + M.idx);
   float* As = reinterpret_cast<float*>(smraw + M.As);
   float* AsT = reinterpret_cast<float*>(smraw + M.AsT);
   float* Ws = reinterpret_cast<float*>(smraw + M.Ws);
@@ -210,7 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
 
   // ---- barriers and tensor memory ----
   if (tid == 0) {
-    for (int i = 0; i < 4; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[i])));
+    for (int i = 0; i < 5; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[i])));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -223,6 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   const uint32_t tmem = tmem_base_s;
   CommitBar fbar[2] = {{&bars[0], 0, 0}, {&bars[1], 0, 0}};
   CommitBar bbar[2] = {{&bars[2], 0, 0}, {&bars[3], 0, 0}};
+  CommitBar fwbar = {&bars[4], 0, 0};   // forward MMAs issued from inside the layer-0 backward pass
   bool failed = false;
 
   // ---- start model into the client's work row: snapshot - own in-flight sums ----
@@ -263,17 +275,26 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   uint32_t h = 0;
 
   for (uint32_t it = 0; it < t.steps; ++it) {
-    for (int b = tid; b < B; b += kThreads)
-      idx[b] = (int)sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * B + b), cd.n);
+    // The forward product of layer 0 for iteration it + 1 is folded into the backward pass of
+    // iteration it (see bwd0), so the next batch's sample indices are drawn one iteration early.
+    int* idx = idxbuf + (it & 1) * B;
+    int* idxn = idxbuf + ((it + 1) & 1) * B;
+    const bool fuse = it + 1 < t.steps;
+    for (int b = tid; b < B; b += kThreads) {
+      if (it == 0) idx[b] = (int)sample_index(draw(key, t.sample_ctr0 + b), cd.n);
+      if (fuse) idxn[b] = (int)sample_index(draw(key, t.sample_ctr0 + (uint64_t)(it + 1) * B + b), cd.n);
+    }
     __syncthreads();
 
     // ================= forward of one layer on tensor cores =================
-    auto fwd_tc = [&](const int l) {
+    // acc_ready: the accumulators were already filled (layer 0, by the previous backward pass)
+    auto fwd_tc = [&](const int l, const bool acc_ready) {
       const int out0 = (int)S.dims[l + 1], Kin = (int)S.dims[l], R0 = r1[l] - r0[l];
       const int n_mt = out0 / 128;
       const uint32_t idesc = umma_idesc(128, B);
       const int a_bytes = out0 * kKC * 2, b_bytes = B * kKC * 2;
-      for (int c = 0; c * kKC < R0; ++c) {
+      const uint32_t dcol = l == 0 ? kFwdCol : 0u;
+      for (int c = 0; !acc_ready && c * kKC < R0; ++c) {
         const int s = c & 1, c0 = r0[l] + c * kKC;
         unsigned char* tA = tiles + s * a_bytes;
         unsigned char* tB = tiles + 2 * a_bytes + s * b_bytes;
@@ -316,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           for (int mt = 0; mt < n_mt; ++mt)
             for (int j = 0; j < kKC / 16; ++j)
-              umma_bf16(tmem + mt * B,
+              umma_bf16(tmem + dcol + mt * B,
                         umma_desc(smem_u32(tA) + mt * 16 * sbo_k64 + j * 256, 128, sbo_k64),
                         umma_desc(smem_u32(tB) + j * 256, 128, sbo_k64), idesc, (c > 0 || j > 0) ? 1u : 0u);
           umma_commit(fbar[s].bar);
@@ -333,7 +354,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         const int nsplit = min(kColSplit, span / 16), half = span / nsplit;
         for (int cc0 = (warp >> 2) * half; (warp >> 2) < nsplit && cc0 < ((warp >> 2) + 1) * half; cc0 += 16) {
           uint32_t v[16];
-          tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + cc0, v);
+          tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + dcol + cc0, v);
           const int mt = cc0 / B, b0 = cc0 % B;
           const int n = mt * 128 + (warp & 3) * 32 + lane;
 #pragma unroll
@@ -356,11 +377,11 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         __syncthreads();
       }
     };
-    fwd_tc(0);
+    fwd_tc(0, it > 0);
 
     // ================= forward, layers >= 1 (FMA) =================
     for (int l = 1; l < L; ++l) {
-      if (tc_layer[l]) { fwd_tc(l); continue; }
+      if (tc_layer[l]) { fwd_tc(l, false); continue; }
       const int N = (int)S.dims[l + 1], Np = up4(N), ldw = Np + 4;
       const int tiles_n = Np / 4, ntile = (B / 4) * tiles_n;
       float acc[kMaxTiles][16];
@@ -452,11 +473,11 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       }
     }
 
-    // ================= backward + update of one layer on tensor cores =================
+    // ================= backward + update of a hidden layer l >= 1 on tensor cores =================
     auto bwd_tc = [&](const int l) {
       const int out0 = (int)S.dims[l + 1], Kin = (int)S.dims[l], R0 = r1[l] - r0[l];
       const float* dz0 = act + G.dz[l];          // full dZ_l [B, out], fp32, visible after a cluster barrier
-      if (l > 0) {
+      {
         // dZ_{l-1}[b, i] = relu'(A_{l-1}[b, i]) * sum_j W_l[i, j] bf16(dZ_l)[b, j] for the rows i this CTA owns,
         // from the weights as they are before this iteration's update:
         // D[128 rows x B] = bf16(W_l chunk)[128 x out] . bf16(dZ_l)[B x out]^T
@@ -534,20 +555,11 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         for (int e = tid; e < kMT * (B / 8); e += kThreads) {
           const int i = e % kMT, bg = e / kMT;
           uint4 v;
-          if (l == 0) {
-            const __nv_bfloat16* col = xdata + c0 + i;
-            unsigned short q[8];
+          const float* col = act + G.a[l - 1] + (size_t)(bg * 8) * Kin + c0 + i;
+          float f[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) q[k] = __ldg(reinterpret_cast<const unsigned short*>(col + (size_t)idx[bg * 8 + k] * D0));
-            v.x = q[0] | ((uint32_t)q[1] << 16); v.y = q[2] | ((uint32_t)q[3] << 16);
-            v.z = q[4] | ((uint32_t)q[5] << 16); v.w = q[6] | ((uint32_t)q[7] << 16);
-          } else {
-            const float* col = act + G.a[l - 1] + (size_t)(bg * 8) * Kin + c0 + i;
-            float f[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) f[k] = col[(size_t)k * Kin];
-            v.x = pack_bf16(f[0], f[1]); v.y = pack_bf16(f[2], f[3]); v.z = pack_bf16(f[4], f[5]); v.w = pack_bf16(f[6], f[7]);
-          }
+          for (int k = 0; k < 8; ++k) f[k] = col[(size_t)k * Kin];
+          v.x = pack_bf16(f[0], f[1]); v.y = pack_bf16(f[2], f[3]); v.z = pack_bf16(f[4], f[5]); v.w = pack_bf16(f[6], f[7]);
           *reinterpret_cast<uint4*>(tA + (i >> 3) * sbo_kB + bg * 128 + (i & 7) * 16) = v;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -584,7 +596,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
                 make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
           __syncwarp();
           const size_t base = woff[l] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + j0 + cg;
-          const bool with_u = !(kDeriveU0 && l == 0);
+          const bool with_u = true;
           float4 w[8], u[8];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: independent 16-byte loads in flight
@@ -625,6 +637,173 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
                     [&](int e, float d) { dzs[e] = d; dzq[e] = q_bf16(d); });
         __syncthreads();
       }
+    };
+
+    // ========== layer 0: backward + update, fused with the next iteration's forward product ==========
+    // The gradient G[128 rows x out0] of a chunk is computed in units of 128 columns, two
+    // tensor-memory slots of 128 columns taking turns: the MMAs of unit u + 1 run while unit u
+    // is read back and applied to the fp32 master.  A unit's updated weights are what the next
+    // iteration's forward pass would read again from HBM, so they go, rounded to bf16, from the
+    // registers of the epilogue into one more operand tile, and Z0^T[unit's columns x B] +=
+    // bf16(W0_new[chunk rows, unit's columns])^T . X_next[:, chunk rows]^T is issued right away into
+    // the forward accumulators (columns kFwdCol...).  Chunk by chunk this is the same sum, in the
+    // same order, as the stand-alone forward pass, which only the first iteration of a round runs.
+    auto bwd0 = [&]() {
+      const int out0 = (int)S.dims[1], R0 = r1[0] - r0[0];
+      const float* dz0 = act + G.dz[0];
+      const int NH = out0 / 128, nch = R0 / kMT, NU = nch * NH;
+      const int a_bytes = kMT * B * 2;
+      unsigned char* tBd = tiles + 2 * a_bytes;                 // bf16(dZ0)^T: element (row j, col b)
+      unsigned char* tWf = tBd + out0 * B * 2;                  // bf16(W0_new) of one unit: element (row j, col i)
+      unsigned char* tXf0 = tWf + 128 * kMT * 2;                // next batch's inputs of a chunk: element (row b, col i)
+      unsigned char* tXf1 = smraw + M.x2;                       // ... and of the chunk after it
+      const uint32_t idesc_b = umma_idesc(128, 128), idesc_f = umma_idesc(128, B);
+      const uint32_t sbo_kM = (kMT / 8) * 128;                  // tiles with K = 128
+      __syncthreads();
+      for (int e = tid; e < out0 * (B / 8); e += kThreads) {
+        const int j = e % out0, bg = e / out0;
+        const float* src = dz0 + (size_t)(bg * 8) * out0 + j;
+        uint4 v;
+        v.x = pack_bf16(src[0], src[out0]);
+        v.y = pack_bf16(src[2 * (size_t)out0], src[3 * (size_t)out0]);
+        v.z = pack_bf16(src[4 * (size_t)out0], src[5 * (size_t)out0]);
+        v.w = pack_bf16(src[6 * (size_t)out0], src[7 * (size_t)out0]);
+        *reinterpret_cast<uint4*>(tBd + (j >> 3) * sbo_kB + bg * 128 + (j & 7) * 16) = v;
+      }
+      auto stage = [&](int c) {   // operand tiles of chunk c; ends with a block barrier
+        const int c0 = r0[0] + c * kMT;
+        unsigned char* tA = tiles + (c & 1) * a_bytes;   // this batch's inputs, transposed: element (row i, col b)
+        for (int e = tid; e < kMT * (B / 8); e += kThreads) {
+          const int i = e % kMT, bg = e / kMT;
+          const __nv_bfloat16* col = xdata + c0 + i;
+          unsigned short q[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) q[k] = __ldg(reinterpret_cast<const unsigned short*>(col + (size_t)idx[bg * 8 + k] * D0));
+          uint4 v;
+          v.x = q[0] | ((uint32_t)q[1] << 16); v.y = q[2] | ((uint32_t)q[3] << 16);
+          v.z = q[4] | ((uint32_t)q[5] << 16); v.w = q[6] | ((uint32_t)q[7] << 16);
+          *reinterpret_cast<uint4*>(tA + (i >> 3) * sbo_kB + bg * 128 + (i & 7) * 16) = v;
+        }
+        if (fuse) {
+          unsigned char* tX = (c & 1) ? tXf1 : tXf0;
+          for (int e = tid; e < B * (kMT / 8); e += kThreads) {
+            const int kg = e % (kMT / 8), b = e / (kMT / 8);
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(xdata + (size_t)idxn[b] * D0 + c0 + kg * 8));
+            *reinterpret_cast<uint4*>(tX + (b >> 3) * sbo_kM + kg * 128 + (b & 7) * 16) = v;
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+      };
+      auto issue_bwd = [&](int u) {   // thread 0: gradient MMAs of unit u into slot u & 1
+        const int c = u / NH, hh = u % NH;
+        unsigned char* tA = tiles + (c & 1) * a_bytes;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int j = 0; j < B / 16; ++j)
+          umma_bf16(tmem + (u & 1) * 128, umma_desc(smem_u32(tA) + j * 256, 128, sbo_kB),
+                    umma_desc(smem_u32(tBd) + hh * 16 * sbo_kB + j * 256, 128, sbo_kB), idesc_b, j > 0 ? 1u : 0u);
+        umma_commit(bbar[u & 1].bar);
+      };
+      if (NU > 0) {
+        stage(0);
+        if (tid == 0) issue_bwd(0);
+        ++bbar[0].issued;
+      }
+      float* tr = trbuf + warp * (32 * kTrLd);
+      const int rr = lane >> 3, cg = (lane & 7) * 4;
+      for (int u = 0; u < NU; ++u) {
+        const int c = u / NH, hh = u % NH, sl = u & 1, c0 = r0[0] + c * kMT;
+        if (u + 1 < NU) {
+          // slot (u + 1) & 1 was read back by unit u - 1, before the barrier that ended its turn
+          if ((u + 1) % NH == 0) {
+            if (fuse) bar_drain(fwbar, failed);   // the forward MMAs that read the input tile being replaced
+            stage(c + 1);
+          }
+          if (tid == 0) issue_bwd(u + 1);
+          ++bbar[(u + 1) & 1].issued;
+        }
+        bar_drain(bbar[sl], failed);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // epilogue: a warp owns 32 rows x 32 columns of the unit.  The accumulator block comes
+        // out of tensor memory one row per lane; a per-warp transpose through shared memory
+        // lets every global access cover 4 rows x 128 contiguous bytes.
+        {
+          const int jl = (warp >> 2) * 32;          // first column within the unit
+          uint32_t v[32];
+          tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + sl * 128 + jl, v);
+          __syncwarp();
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<float4*>(tr + lane * kTrLd + 4 * q) =
+                make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+          __syncwarp();
+          const size_t base = woff[0] + (size_t)(c0 + (warp & 3) * 32 + rr) * out0 + hh * 128 + jl + cg;
+          float4 w[8], uu[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {   // rows rr, rr + 4, ...: independent 16-byte loads in flight
+            w[q] = *reinterpret_cast<const float4*>(work + base + (size_t)(4 * q) * out0);
+            uu[q] = kDeriveU0 ? make_float4(0.f, 0.f, 0.f, 0.f)
+                              : *reinterpret_cast<const float4*>(Urow + base + (size_t)(4 * q) * out0);
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 gq = *reinterpret_cast<const float4*>(tr + (4 * q + rr) * kTrLd + cg);
+            const float g0 = fmaf(lambda, w[q].x, gq.x), g1 = fmaf(lambda, w[q].y, gq.y);
+            const float g2 = fmaf(lambda, w[q].z, gq.z), g3 = fmaf(lambda, w[q].w, gq.w);
+            w[q].x = fmaf(-eta, g0, w[q].x); w[q].y = fmaf(-eta, g1, w[q].y); w[q].z = fmaf(-eta, g2, w[q].z); w[q].w = fmaf(-eta, g3, w[q].w);
+            uu[q].x += g0; uu[q].y += g1; uu[q].z += g2; uu[q].w += g3;
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            *reinterpret_cast<float4*>(work + base + (size_t)(4 * q) * out0) = w[q];
+            if (!kDeriveU0) *reinterpret_cast<float4*>(Urow + base + (size_t)(4 * q) * out0) = uu[q];
+          }
+          if (fuse) {
+            // the new weights go back through the transpose buffer: a lane then holds 8 consecutive
+            // input rows of one column = one 16-byte entry of the K-major operand tile
+            bar_drain(fwbar, failed);   // the previous unit's forward MMAs have read the tile
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < 8; ++q) *reinterpret_cast<float4*>(tr + (4 * q + rr) * kTrLd + cg) = w[q];
+            __syncwarp();
+            const int j = jl + lane;
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8) {
+              float f[8];
+#pragma unroll
+              for (int r = 0; r < 8; ++r) f[r] = tr[(8 * g8 + r) * kTrLd + lane];
+              uint4 pk;
+              pk.x = pack_bf16(f[0], f[1]); pk.y = pack_bf16(f[2], f[3]); pk.z = pack_bf16(f[4], f[5]); pk.w = pack_bf16(f[6], f[7]);
+              const int kg = (warp & 3) * 4 + g8;
+              *reinterpret_cast<uint4*>(tWf + (j >> 3) * sbo_kM + kg * 128 + (j & 7) * 16) = pk;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();   // the slot is free again; the weight tile is complete
+        if (fuse) {
+          if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            for (int j = 0; j < kMT / 16; ++j)
+              umma_bf16(tmem + kFwdCol + hh * B, umma_desc(smem_u32(tWf) + j * 256, 128, sbo_kM),
+                        umma_desc(smem_u32((c & 1) ? tXf1 : tXf0) + j * 256, 128, sbo_kM), idesc_f, (c > 0 || j > 0) ? 1u : 0u);
+            umma_commit(fwbar.bar);
+          }
+          ++fwbar.issued;
+        }
+      }
+      bar_drain(fwbar, failed);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      cluster_sync(clustered);
+      if (rank == 0)
+        for (int n = tid; n < out0; n += kThreads) {
+          float gb = 0.f;
+          for (int b = 0; b < B; ++b) gb += dz0[(size_t)b * out0 + n];
+          work[boff[0] + n] = fmaf(-eta, gb, work[boff[0] + n]);
+          Urow[boff[0] + n] += gb;
+        }
     };
 
     // ================= backward + update, layers >= 1 (FMA) =================
@@ -733,7 +912,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
       }
     }
 
-    bwd_tc(0);
+    bwd0();
     h += (uint32_t)B;
   }
 
