@@ -406,40 +406,43 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
 // block, delta_s = softmax(z_s) - onehot(y_s) and G[s][t] = x_s . x_t + 1 (the
 // 1 is the bias), step t of the block sees the logits
 //     z_t = W x_t + b - eta * sum_{s<t} delta_s G[s][t],
-// because W_t = W - eta * sum_{s<t} delta_s x_s^T.  So per block:
-//   P1  Z0 = W X (every thread: its 7 pixels x 10 classes x kM samples), summed
-//       over the CTA by a transposing shuffle butterfly and 4 partials in shared
-//       memory;
+// because W_t = W - eta * sum_{s<t} delta_s x_s^T.  And since eta is constant
+// within a round and lambda = 0, W = W_start - eta * U at every block boundary,
+// so only U is updated sample by sample.  Per block:
+//   P1  W = W_start - eta U (registers, one FMA per parameter), Z0 = W X (every
+//       thread: 14 pixels x 5 classes x kM samples), summed over the CTA by a
+//       transposing shuffle butterfly and 4 per-warp partials in shared memory;
 //   R   one warp (rotating) walks the kM samples: lane t owns sample t, takes the
 //       softmax of its corrected logits and hands -eta*delta_t to the later
-//       samples' lanes by shuffle; delta and -eta*delta go to shared memory;
-//       meanwhile the other three warps compute the Gram matrix of the NEXT block
-//       (it does not depend on W) and one of them issues the bulk copies of the
-//       block after that;
-//   P3  W += (-eta delta_t) x_t^T and U += delta_t x_t^T for the block's samples.
+//       samples' lanes by shuffle; delta goes to shared memory; meanwhile the
+//       other three warps compute the Gram matrix of the NEXT block (it does not
+//       depend on W) and one of them issues the bulk copies of the block after it;
+//   P3  U += delta_t x_t^T for the block's samples.
 // The result equals the step-by-step recursion up to fp32 rounding order.  One
 // barrier pair per kM samples instead of one per sample, and the latency-bound
 // softmax chain of one block overlaps the FMA phases of the CTA sharing the SM.
+// All FMAs here are scalar: on this part fma.rn.f32x2 with three distinct
+// register pairs issues every ~3 cycles, a scalar fma every cycle.
 //
-// Work split: 4 warps x 28 lanes x 7 consecutive pixels = 784; lane 28 of the
-// last warp carries the bias as an always-1 pixel.  W and U stay in registers
-// (2 x 35 packed pairs).  Rows arrive by cp.async.bulk into a ring of 3 blocks,
-// issued two blocks ahead; every mbarrier wait is bounded.
+// Work split: lane = 2 * (pixel group) + (class half).  4 warps x 14 groups x
+// 14 consecutive pixels = 784; lanes 28, 29 of the last warp carry the bias as
+// an always-1 pixel.  W_start and U stay in registers (2 x 70).  Rows arrive by
+// cp.async.bulk into a ring of 3 blocks, issued two blocks ahead; every
+// mbarrier wait is bounded.
 constexpr int kM = 8;                  // samples per block
 constexpr int kSlots = 3;              // blocks of rows in shared memory
-constexpr int kPx = 7, kAct = 28;      // pixels per thread, pixel-owning lanes per warp
-constexpr int kQ = 4;                  // samples per accumulator group in P1
+constexpr int kPx = 14, kPl = 14;      // pixels per thread, pixel groups per warp
+constexpr int kCh = kC / 2;            // classes per thread
 constexpr int kPairs = kM * (kM - 1) / 2;
-static_assert(kAct * kWarps * kPx == kD, "pixel split");
-static_assert(kM % kQ == 0 && kM <= 8, "block shape");
+static_assert(kPl * kWarps * kPx == kD, "pixel split");
+static_assert(kM == 8, "lane-per-sample recurrence and butterfly widths assume 8");
 
 struct __align__(128) BlkSmem {
   float rows[kSlots][kM][kD];
   float partZ[kWarps][kM * kC];       // per-warp totals of Z0, index t*10 + c
   float partG[2][kWarps][32];         // per-warp totals of the Gram pairs, double-buffered by block parity
-  float dbuf[kM][24];                 // [0..9] delta_t, [12..21] -eta*delta_t
-  float onehot[kC][12];               // row y: -1 at class y, else 0
-  float consts[16];                   // [0..6] = 1,0,0,0,0,0,0 (bias lane's "row"); [8..14] = 0 (idle lanes)
+  float dbuf[kM][16];                 // delta_t: classes 0..4 at [0..4], 5..9 at [8..12]
+  float consts[32];                   // [0..13] = 1,0,...,0 (bias lanes' "row"); [16..29] = 0 (idle lanes)
   int ys[kSlots][kM];
   uint64_t full[kSlots];
 };
@@ -462,7 +465,7 @@ template <int N> struct BflyDims {
 };
 // Sums v[i] over the 32 lanes for every i; lane L ends with n5 totals in o[].
 template <int N>
-__device__ __forceinline__ void bfly_reduce(const float (&v)[N], float (&o)[BflyDims<N>::n5], int lane) {
+__device__ __forceinline__ void bfly_reduce5(const float (&v)[N], float (&o)[BflyDims<N>::n5], int lane) {
   typedef BflyDims<N> D;
   float a[D::n1], b[D::n2], c[D::n3], d[D::n4];
   bfly_stage<N>(v, a, 16, lane & 16);
@@ -473,7 +476,7 @@ __device__ __forceinline__ void bfly_reduce(const float (&v)[N], float (&o)[Bfly
 }
 // Which v[] index the lane's i-th total belongs to (-1: padding).
 template <int N>
-__device__ __forceinline__ int bfly_index(int lane, int i) {
+__device__ __forceinline__ int bfly_index5(int lane, int i) {
   typedef BflyDims<N> D;
   const int i4 = i + ((lane & 1) ? D::n5 : 0);
   const int i3 = i4 + ((lane & 2) ? D::n4 : 0);
@@ -481,6 +484,26 @@ __device__ __forceinline__ int bfly_index(int lane, int i) {
   const int i1 = i2 + ((lane & 8) ? D::n2 : 0);
   const int i0 = i1 + ((lane & 16) ? D::n1 : 0);
   const bool ok = i4 < D::n4 && i3 < D::n3 && i2 < D::n2 && i1 < D::n1 && i0 < N;
+  return ok ? i0 : -1;
+}
+// The same over the 16 lanes that share bit 0 (masks 16, 8, 4, 2): n4 totals per lane.
+template <int N>
+__device__ __forceinline__ void bfly_reduce4(const float (&v)[N], float (&o)[BflyDims<N>::n4], int lane) {
+  typedef BflyDims<N> D;
+  float a[D::n1], b[D::n2], c[D::n3];
+  bfly_stage<N>(v, a, 16, lane & 16);
+  bfly_stage<D::n1>(a, b, 8, lane & 8);
+  bfly_stage<D::n2>(b, c, 4, lane & 4);
+  bfly_stage<D::n3>(c, o, 2, lane & 2);
+}
+template <int N>
+__device__ __forceinline__ int bfly_index4(int lane, int i) {
+  typedef BflyDims<N> D;
+  const int i3 = i + ((lane & 2) ? D::n4 : 0);
+  const int i2 = i3 + ((lane & 4) ? D::n3 : 0);
+  const int i1 = i2 + ((lane & 8) ? D::n2 : 0);
+  const int i0 = i1 + ((lane & 16) ? D::n1 : 0);
+  const bool ok = i3 < D::n3 && i2 < D::n2 && i1 < D::n1 && i0 < N;
   return ok ? i0 : -1;
 }
 __device__ __forceinline__ constexpr int pair_index(int s, int t) { return t * (t - 1) / 2 + s; }  // s < t
@@ -491,24 +514,24 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool active = lane < kAct;
-  const bool is_bias = warp == kWarps - 1 && lane == kAct;
-  const int g = warp * kAct + (active ? lane : 0);   // pixel group: pixels 7g .. 7g+6
+  const int cg = lane & 1, pl = lane >> 1;
+  const bool active = pl < kPl;
+  const bool is_bias = warp == kWarps - 1 && pl == kPl;
+  const int pg = warp * kPl + (active ? pl : 0);     // pixel group: pixels 14 pg .. 14 pg + 13
 
   const ClientData cd = p.clients[t.client];
   const uint64_t key = p.sample_keys[t.client];
   const float* xrows = reinterpret_cast<const float*>(cd.x);
   const uint32_t n = t.n_samples;
   const uint32_t nblk = (n + kM - 1) / kM;
-  const float eta = t.eta;
+  const float neta = -t.eta;
 
   if (threadIdx.x == 0) {
 #pragma unroll
     for (int s = 0; s < kSlots; ++s) mbar_init(&sm.full[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (threadIdx.x < kC * 12) sm.onehot[threadIdx.x / 12][threadIdx.x % 12] = (threadIdx.x / 12 == threadIdx.x % 12) ? -1.f : 0.f;
-  if (threadIdx.x < 16) sm.consts[threadIdx.x] = threadIdx.x == 0 ? 1.f : 0.f;
+  if (threadIdx.x < 32) sm.consts[threadIdx.x] = threadIdx.x == 0 ? 1.f : 0.f;
   __syncthreads();
 
   // Producer step: the rows and labels of block kb into ring slot kb % kSlots.
@@ -529,46 +552,47 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
   }
 
   // ---- start model: server snapshot minus own update sums still in flight ----
-  u64 W2[kPx][kC / 2], U2[kPx][kC / 2];
+  // Ws[a][c] = W[14 pg + a][5 cg + c]; the bias lanes hold b[5 cg + c] in row 0.
+  float Ws[kPx][kCh], U[kPx][kCh];
   const bool owns = active || is_bias;
-  const size_t poff = is_bias ? (size_t)kD * kC : (size_t)g * (kPx * kC);
+  const size_t poff = (is_bias ? (size_t)kD * kC : (size_t)pg * (kPx * kC)) + (size_t)cg * kCh;
   {
-    const float2* s2 = reinterpret_cast<const float2*>(p.snaps + (size_t)t.snap_slot * p.stride + poff);
+    const float* src = p.snaps + (size_t)t.snap_slot * p.stride + poff;
 #pragma unroll
     for (int a = 0; a < kPx; ++a)
 #pragma unroll
-      for (int c = 0; c < kC / 2; ++c) {
+      for (int c = 0; c < kCh; ++c) {
         const bool live = active || (is_bias && a == 0);
-        const float2 v = live ? __ldg(s2 + a * (kC / 2) + c) : make_float2(0.f, 0.f);
-        W2[a][c] = pack2(v.x, v.y);
-        U2[a][c] = 0ull;
+        Ws[a][c] = live ? __ldg(src + a * kC + c) : 0.f;
+        U[a][c] = 0.f;
       }
     for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
       const InflightRef ref = p.inflight[t.inflight_off + f];
-      const float2* u2 = reinterpret_cast<const float2*>(p.U + (size_t)ref.seq * p.stride + poff);
-      const u64 ne = pack2(-ref.eta, -ref.eta);
+      const float* us = p.U + (size_t)ref.seq * p.stride + poff;
 #pragma unroll
       for (int a = 0; a < kPx; ++a)
 #pragma unroll
-        for (int c = 0; c < kC / 2; ++c) {
+        for (int c = 0; c < kCh; ++c) {
           const bool live = active || (is_bias && a == 0);
-          const float2 v = live ? __ldg(u2 + a * (kC / 2) + c) : make_float2(0.f, 0.f);
-          W2[a][c] = fma2(ne, pack2(v.x, v.y), W2[a][c]);
+          Ws[a][c] = fmaf(-ref.eta, live ? __ldg(us + a * kC + c) : 0.f, Ws[a][c]);
         }
     }
   }
 
   // Where this thread reads "its pixels" of sample (slot, t): pixel-owning lanes
-  // from the row, the bias lane from {1,0,...}, idle lanes from zeros (row stride 0).
-  const float* xbase = active ? &sm.rows[0][0][g * kPx] : (is_bias ? &sm.consts[0] : &sm.consts[8]);
+  // from the row, the bias lanes from {1,0,...}, idle lanes from zeros (row stride 0).
+  const float* xbase = active ? &sm.rows[0][0][pg * kPx] : (is_bias ? &sm.consts[0] : &sm.consts[16]);
   const int rs = active ? kD : 0;
 
   // where the lane's butterfly totals go
-  int zidx[2], gidx;
-  zidx[0] = bfly_index<kQ * kC>(lane, 0);
-  zidx[1] = bfly_index<kQ * kC>(lane, 1);
-  gidx = bfly_index<kPairs>(lane, 0);
-  static_assert(BflyDims<kQ * kC>::n5 == 2 && BflyDims<kPairs>::n5 == 1, "butterfly widths");
+  static_assert(BflyDims<kM * kCh>::n4 == 3 && BflyDims<kPairs>::n5 == 1, "butterfly widths");
+  int zidx[3];
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    const int v = bfly_index4<kM * kCh>(lane, i);       // v = s * 5 + c
+    zidx[i] = v < 0 ? -1 : (v / kCh) * kC + cg * kCh + (v % kCh);
+  }
+  const int gidx = bfly_index5<kPairs>(lane, 0);
 
   // Gram pairs of block kb over this warp's share of the pixels (rank r of 3).
   auto gram_partial = [&](uint32_t kb, int r) {
@@ -589,12 +613,10 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
       }
     }
     float o[1];
-    bfly_reduce<kPairs>(gacc, o, lane);
+    bfly_reduce5<kPairs>(gacc, o, lane);
     if (gidx >= 0) sm.partG[kb & 1][warp][gidx] = o[0];
   };
 
-  const u64 neta2 = pack2(-eta, -eta);
-  const u64 log2e2 = pack2(kLog2e, kLog2e);
   bool ok = true;
   bool timed_out = false;
   uint32_t timeout_at = 0;
@@ -611,28 +633,37 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     ok = mbar_wait(&sm.full[slot], (k / kSlots) & 1) && ok;
     const float* xslot = xbase + (size_t)slot * kM * rs;
 
-    // ---- P1: this thread's share of Z0 = W X, kQ samples at a time ----
+    // ---- P1: W = W_start - eta U; this thread's share of Z0 = W X ----
+    {
+      float acc[kM][kCh];
 #pragma unroll
-    for (int q = 0; q < kM / kQ; ++q) {
-      u64 acc[kQ][kC / 2];
+      for (int a2 = 0; a2 < kPx / 2; ++a2) {
+        float w0[kCh], w1[kCh];
 #pragma unroll
-      for (int a = 0; a < kPx; ++a)
-#pragma unroll
-        for (int s = 0; s < kQ; ++s) {
-          const float x = xslot[(q * kQ + s) * rs + a];
-          const u64 xs = pack2(x, x);
-#pragma unroll
-          for (int c = 0; c < kC / 2; ++c) acc[s][c] = a == 0 ? mul2(xs, W2[0][c]) : fma2(xs, W2[a][c], acc[s][c]);
+        for (int c = 0; c < kCh; ++c) {
+          w0[c] = fmaf(neta, U[2 * a2][c], Ws[2 * a2][c]);
+          w1[c] = fmaf(neta, U[2 * a2 + 1][c], Ws[2 * a2 + 1][c]);
         }
-      float v[kQ * kC];
 #pragma unroll
-      for (int s = 0; s < kQ; ++s)
+        for (int s = 0; s < kM; ++s) {
+          const float2 x = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
 #pragma unroll
-        for (int c = 0; c < kC / 2; ++c) unpack2(acc[s][c], v[s * kC + 2 * c], v[s * kC + 2 * c + 1]);
-      float o[2];
-      bfly_reduce<kQ * kC>(v, o, lane);
-      if (zidx[0] >= 0) sm.partZ[warp][q * kQ * kC + zidx[0]] = o[0];
-      if (zidx[1] >= 0) sm.partZ[warp][q * kQ * kC + zidx[1]] = o[1];
+          for (int c = 0; c < kCh; ++c) {
+            acc[s][c] = a2 == 0 ? x.x * w0[c] : fmaf(x.x, w0[c], acc[s][c]);
+            acc[s][c] = fmaf(x.y, w1[c], acc[s][c]);
+          }
+        }
+      }
+      float v[kM * kCh];
+#pragma unroll
+      for (int s = 0; s < kM; ++s)
+#pragma unroll
+        for (int c = 0; c < kCh; ++c) v[s * kCh + c] = acc[s][c];
+      float o[3];
+      bfly_reduce4<kM * kCh>(v, o, lane);
+#pragma unroll
+      for (int i = 0; i < 3; ++i)
+        if (zidx[i] >= 0) sm.partZ[warp][zidx[i]] = o[i];
     }
     // barrier A: partials visible, rows of block k-1 no longer read by anyone; it
     // also carries the verdict of the bounded waits so that all threads leave together
@@ -642,81 +673,65 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     if (warp == rwarp) {
       // ---- R: the block's kM dependent softmax steps, lane j owns sample j ----
       const int j = lane & (kM - 1);
-      u64 z[kC / 2];
+      float z[kC];
       {
-        const u64* z0 = reinterpret_cast<const u64*>(&sm.partZ[0][j * kC]);
-        const u64* z1 = reinterpret_cast<const u64*>(&sm.partZ[1][j * kC]);
-        const u64* z2 = reinterpret_cast<const u64*>(&sm.partZ[2][j * kC]);
-        const u64* z3 = reinterpret_cast<const u64*>(&sm.partZ[3][j * kC]);
+        const float2* z0 = reinterpret_cast<const float2*>(&sm.partZ[0][j * kC]);
+        const float2* z1 = reinterpret_cast<const float2*>(&sm.partZ[1][j * kC]);
+        const float2* z2 = reinterpret_cast<const float2*>(&sm.partZ[2][j * kC]);
+        const float2* z3 = reinterpret_cast<const float2*>(&sm.partZ[3][j * kC]);
 #pragma unroll
-        for (int c = 0; c < kC / 2; ++c) z[c] = add2(add2(z0[c], z1[c]), add2(z2[c], z3[c]));
+        for (int c = 0; c < kC / 2; ++c) {
+          const float2 a0 = z0[c], a1 = z1[c], a2 = z2[c], a3 = z3[c];
+          z[2 * c] = (a0.x + a1.x) + (a2.x + a3.x);
+          z[2 * c + 1] = (a0.y + a1.y) + (a2.y + a3.y);
+        }
       }
-      // column j of the Gram matrix: G[s][j], s < j; the warp that ran R for block k-1 has no share in it
+      // column j of the Gram matrix: G[s][j], s < j (0 for the others: a finished
+      // sample takes no correction); the warp that ran R for block k-1 has no share in it
       float Gj[kM - 1];
       {
         const int skip = (k + kWarps - 1) & (kWarps - 1);
+        const int w0 = skip == 0 ? 1 : 0, w1 = skip <= 1 ? 2 : 1, w2 = skip <= 2 ? 3 : 2;
+        const float* g0 = sm.partG[k & 1][w0];
+        const float* g1 = sm.partG[k & 1][w1];
+        const float* g2 = sm.partG[k & 1][w2];
         const int base = j * (j - 1) / 2;
 #pragma unroll
         for (int s = 0; s < kM - 1; ++s) {
           const int idx = s < j ? base + s : 0;
-          float acc = 1.f;   // the bias "pixel"
-#pragma unroll
-          for (int w = 0; w < kWarps; ++w)
-            if (w != skip) acc += sm.partG[k & 1][w][idx];
-          Gj[s] = acc;
+          const float gsum = (1.f + g0[idx]) + (g1[idx] + g2[idx]);   // 1 = the bias "pixel"
+          Gj[s] = s < j ? gsum : 0.f;
         }
       }
       const int y = sm.ys[slot][j];
-      u64 oh[kC / 2];
-      {
-        const ulonglong2* q = reinterpret_cast<const ulonglong2*>(&sm.onehot[((unsigned)y < (unsigned)kC) ? y : 0][0]);
-        const ulonglong2 o0 = q[0], o1 = q[1], o2 = q[2];
-        oh[0] = o0.x; oh[1] = o0.y; oh[2] = o1.x; oh[3] = o1.y; oh[4] = o2.x;
-      }
+      float oh[kC];
+#pragma unroll
+      for (int c = 0; c < kC; ++c) oh[c] = c == y ? -1.f : 0.f;
 #pragma unroll
       for (int s = 0; s < kM; ++s) {
         if ((uint32_t)s < nv) {      // uniform
-          float zf[kC];
-#pragma unroll
-          for (int c = 0; c < kC / 2; ++c) unpack2(z[c], zf[2 * c], zf[2 * c + 1]);
-          const float m = fmaxf(fmaxf(fmaxf(fmaxf(zf[0], zf[1]), fmaxf(zf[2], zf[3])), fmaxf(fmaxf(zf[4], zf[5]), fmaxf(zf[6], zf[7]))),
-                                fmaxf(zf[8], zf[9]));
+          const float m = fmaxf(fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), fmaxf(fmaxf(z[4], z[5]), fmaxf(z[6], z[7]))),
+                                fmaxf(z[8], z[9]));
           const float nms = -m * kLog2e;
-          const u64 nms2 = pack2(nms, nms);
-          u64 e2[kC / 2];
+          float e[kC];
 #pragma unroll
-          for (int c = 0; c < kC / 2; ++c) {
-            float lo, hi;
-            unpack2(fma2(z[c], log2e2, nms2), lo, hi);
-            e2[c] = pack2(ex2(lo), ex2(hi));
-          }
-          float slo, shi;
-          unpack2(add2(add2(add2(e2[0], e2[1]), add2(e2[2], e2[3])), e2[4]), slo, shi);
-          const float inv = rcp(slo + shi);
-          const u64 inv2 = pack2(inv, inv);
-          u64 d2[kC / 2], nd2[kC / 2];
+          for (int c = 0; c < kC; ++c) e[c] = ex2(fmaf(z[c], kLog2e, nms));
+          const float sum = (((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]))) + (e[8] + e[9]);
+          const float inv = rcp(sum);
+          float d[kC];
 #pragma unroll
-          for (int c = 0; c < kC / 2; ++c) {
-            d2[c] = fma2(e2[c], inv2, oh[c]);
-            nd2[c] = mul2(d2[c], neta2);
-          }
+          for (int c = 0; c < kC; ++c) d[c] = fmaf(e[c], inv, oh[c]);
           if (lane == s) {
-            ulonglong2* dq = reinterpret_cast<ulonglong2*>(&sm.dbuf[s][0]);
-            dq[0] = make_ulonglong2(d2[0], d2[1]);
-            dq[1] = make_ulonglong2(d2[2], d2[3]);
-            dq[2] = make_ulonglong2(d2[4], 0ull);
-            dq[3] = make_ulonglong2(nd2[0], nd2[1]);
-            dq[4] = make_ulonglong2(nd2[2], nd2[3]);
-            dq[5] = make_ulonglong2(nd2[4], 0ull);
+            float4* dq = reinterpret_cast<float4*>(&sm.dbuf[s][0]);
+            dq[0] = make_float4(d[0], d[1], d[2], d[3]);
+            dq[1] = make_float4(d[4], 0.f, 0.f, 0.f);
+            dq[2] = make_float4(d[5], d[6], d[7], d[8]);
+            dq[3] = make_float4(d[9], 0.f, 0.f, 0.f);
           }
           if (s + 1 < kM) {
-            const float gs = Gj[s < kM - 1 ? s : 0];
-            const u64 g2 = j > s ? pack2(gs, gs) : 0ull;   // earlier samples are done: no correction
+            const float gs = Gj[s < kM - 1 ? s : 0] * neta;
 #pragma unroll
-            for (int c = 0; c < kC / 2; ++c) {
-              const u64 nds = __shfl_sync(0xffffffffu, nd2[c], s);
-              z[c] = fma2(nds, g2, z[c]);
-            }
+            for (int c = 0; c < kC; ++c) z[c] = fmaf(__shfl_sync(0xffffffffu, d[c], s), gs, z[c]);
           }
         }
       }
@@ -730,20 +745,18 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     }
     __syncthreads();   // barrier B: delta of the block is in shared memory
 
-    // ---- P3: W -= eta * delta_t x_t^T, U += delta_t x_t^T ----
+    // ---- P3: U += delta_t x_t^T ----
     auto apply_sample = [&](int s) {
-      const ulonglong2* dq = reinterpret_cast<const ulonglong2*>(&sm.dbuf[s][0]);
-      const ulonglong2 q0 = dq[0], q1 = dq[1], q2 = dq[2], q3 = dq[3], q4 = dq[4], q5 = dq[5];
-      const u64 d2[kC / 2] = {q0.x, q0.y, q1.x, q1.y, q2.x};
-      const u64 nd2[kC / 2] = {q3.x, q3.y, q4.x, q4.y, q5.x};
+      const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
+      const float d4 = sm.dbuf[s][cg * 8 + 4];
+      const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, d4};
 #pragma unroll
-      for (int a = 0; a < kPx; ++a) {
-        const float x = xslot[s * rs + a];
-        const u64 xs = pack2(x, x);
+      for (int a2 = 0; a2 < kPx / 2; ++a2) {
+        const float2 x = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
 #pragma unroll
-        for (int c = 0; c < kC / 2; ++c) {
-          U2[a][c] = fma2(xs, d2[c], U2[a][c]);
-          W2[a][c] = fma2(xs, nd2[c], W2[a][c]);
+        for (int c = 0; c < kCh; ++c) {
+          U[2 * a2][c] = fmaf(x.x, d[c], U[2 * a2][c]);
+          U[2 * a2 + 1][c] = fmaf(x.y, d[c], U[2 * a2 + 1][c]);
         }
       }
     };
@@ -765,22 +778,17 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     return;
   }
 
-  // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model) ----
+  // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model W_start - eta U) ----
   if (owns) {
-    float2* dU = reinterpret_cast<float2*>(p.U + (size_t)t.seq * p.stride + poff);
-    float2* dW = p.w_end ? reinterpret_cast<float2*>(p.w_end + (size_t)t.seq * p.stride + poff) : nullptr;
+    float* dU = p.U + (size_t)t.seq * p.stride + poff;
+    float* dW = p.w_end ? p.w_end + (size_t)t.seq * p.stride + poff : nullptr;
 #pragma unroll
     for (int a = 0; a < kPx; ++a)
 #pragma unroll
-      for (int c = 0; c < kC / 2; ++c) {
+      for (int c = 0; c < kCh; ++c) {
         if (active || a == 0) {
-          float lo, hi;
-          unpack2(U2[a][c], lo, hi);
-          dU[a * (kC / 2) + c] = make_float2(lo, hi);
-          if (dW) {
-            unpack2(W2[a][c], lo, hi);
-            dW[a * (kC / 2) + c] = make_float2(lo, hi);
-          }
+          dU[a * kC + c] = U[a][c];
+          if (dW) dW[a * kC + c] = fmaf(neta, U[a][c], Ws[a][c]);
         }
       }
   }
