@@ -686,54 +686,49 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
           z[2 * c + 1] = (a0.y + a1.y) + (a2.y + a3.y);
         }
       }
-      // column j of the Gram matrix: G[s][j], s < j (0 for the others: a finished
-      // sample takes no correction); the warp that ran R for block k-1 has no share in it
-      float Gj[kM - 1];
-      {
-        const int skip = (k + kWarps - 1) & (kWarps - 1);
-        const int w0 = skip == 0 ? 1 : 0, w1 = skip <= 1 ? 2 : 1, w2 = skip <= 2 ? 3 : 2;
-        const float* g0 = sm.partG[k & 1][w0];
-        const float* g1 = sm.partG[k & 1][w1];
-        const float* g2 = sm.partG[k & 1][w2];
-        const int base = j * (j - 1) / 2;
-#pragma unroll
-        for (int s = 0; s < kM - 1; ++s) {
-          const int idx = s < j ? base + s : 0;
-          const float gsum = (1.f + g0[idx]) + (g1[idx] + g2[idx]);   // 1 = the bias "pixel"
-          Gj[s] = s < j ? gsum : 0.f;
-        }
-      }
+      // column j of the Gram matrix, one entry per step: -eta * G[s][j] for s < j, 0 for
+      // the others (a finished sample takes no correction); the warp that ran R for block
+      // k-1 has no share in the Gram partials.  Loaded one step ahead of its use.
+      const int skip = (k + kWarps - 1) & (kWarps - 1);
+      const float* g0 = sm.partG[k & 1][skip == 0 ? 1 : 0];
+      const float* g1 = sm.partG[k & 1][skip <= 1 ? 2 : 1];
+      const float* g2 = sm.partG[k & 1][skip <= 2 ? 3 : 2];
+      const int gbase = j * (j - 1) / 2;
+      auto corr = [&](int s) -> float {
+        const int idx = s < j ? gbase + s : 0;
+        const float gsum = (1.f + g0[idx]) + (g1[idx] + g2[idx]);   // 1 = the bias "pixel"
+        return s < j ? gsum * neta : 0.f;
+      };
       const int y = sm.ys[slot][j];
       float oh[kC];
 #pragma unroll
       for (int c = 0; c < kC; ++c) oh[c] = c == y ? -1.f : 0.f;
+      float gs = corr(0);
+      // The loop stays rolled: the whole per-block body has to fit the instruction cache.
+#pragma unroll 1
+      for (int s = 0; s < (int)nv; ++s) {
+        const float gnext = corr(s + 1);
+        const float m = fmaxf(fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), fmaxf(fmaxf(z[4], z[5]), fmaxf(z[6], z[7]))),
+                              fmaxf(z[8], z[9]));
+        const float nms = -m * kLog2e;
+        float e[kC];
 #pragma unroll
-      for (int s = 0; s < kM; ++s) {
-        if ((uint32_t)s < nv) {      // uniform
-          const float m = fmaxf(fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), fmaxf(fmaxf(z[4], z[5]), fmaxf(z[6], z[7]))),
-                                fmaxf(z[8], z[9]));
-          const float nms = -m * kLog2e;
-          float e[kC];
+        for (int c = 0; c < kC; ++c) e[c] = ex2(fmaf(z[c], kLog2e, nms));
+        const float sum = (((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]))) + (e[8] + e[9]);
+        const float inv = rcp(sum);
+        float d[kC];
 #pragma unroll
-          for (int c = 0; c < kC; ++c) e[c] = ex2(fmaf(z[c], kLog2e, nms));
-          const float sum = (((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]))) + (e[8] + e[9]);
-          const float inv = rcp(sum);
-          float d[kC];
-#pragma unroll
-          for (int c = 0; c < kC; ++c) d[c] = fmaf(e[c], inv, oh[c]);
-          if (lane == s) {
-            float4* dq = reinterpret_cast<float4*>(&sm.dbuf[s][0]);
-            dq[0] = make_float4(d[0], d[1], d[2], d[3]);
-            dq[1] = make_float4(d[4], 0.f, 0.f, 0.f);
-            dq[2] = make_float4(d[5], d[6], d[7], d[8]);
-            dq[3] = make_float4(d[9], 0.f, 0.f, 0.f);
-          }
-          if (s + 1 < kM) {
-            const float gs = Gj[s < kM - 1 ? s : 0] * neta;
-#pragma unroll
-            for (int c = 0; c < kC; ++c) z[c] = fmaf(__shfl_sync(0xffffffffu, d[c], s), gs, z[c]);
-          }
+        for (int c = 0; c < kC; ++c) d[c] = fmaf(e[c], inv, oh[c]);
+        if (lane == s) {
+          float4* dq = reinterpret_cast<float4*>(&sm.dbuf[s][0]);
+          dq[0] = make_float4(d[0], d[1], d[2], d[3]);
+          dq[1] = make_float4(d[4], 0.f, 0.f, 0.f);
+          dq[2] = make_float4(d[5], d[6], d[7], d[8]);
+          dq[3] = make_float4(d[9], 0.f, 0.f, 0.f);
         }
+#pragma unroll
+        for (int c = 0; c < kC; ++c) z[c] = fmaf(__shfl_sync(0xffffffffu, d[c], s), gs, z[c]);
+        gs = gnext;
       }
     } else {
       const int rank = ((warp - rwarp) & (kWarps - 1)) - 1;   // 0..2 among the three other warps
@@ -745,26 +740,33 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     }
     __syncthreads();   // barrier B: delta of the block is in shared memory
 
-    // ---- P3: U += delta_t x_t^T ----
-    auto apply_sample = [&](int s) {
-      const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
-      const float d4 = sm.dbuf[s][cg * 8 + 4];
-      const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, d4};
+    // ---- P3: U += delta_t x_t^T (rolled; the next sample's operands are loaded ahead) ----
+    {
+      float2 xn[kPx / 2];
+      float4 dn4;
+      float dn1;
+      auto load_sample = [&](int s) {
+        dn4 = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
+        dn1 = sm.dbuf[s][cg * 8 + 4];
 #pragma unroll
-      for (int a2 = 0; a2 < kPx / 2; ++a2) {
-        const float2 x = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
+        for (int a2 = 0; a2 < kPx / 2; ++a2) xn[a2] = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
+      };
+      load_sample(0);
+#pragma unroll 1
+      for (int s = 0; s < (int)nv; ++s) {
+        float2 x[kPx / 2];
 #pragma unroll
-        for (int c = 0; c < kCh; ++c) {
-          U[2 * a2][c] = fmaf(x.x, d[c], U[2 * a2][c]);
-          U[2 * a2 + 1][c] = fmaf(x.y, d[c], U[2 * a2 + 1][c]);
-        }
+        for (int a2 = 0; a2 < kPx / 2; ++a2) x[a2] = xn[a2];
+        const float d[kCh] = {dn4.x, dn4.y, dn4.z, dn4.w, dn1};
+        load_sample(s + 1 < kM ? s + 1 : s);
+#pragma unroll
+        for (int a2 = 0; a2 < kPx / 2; ++a2)
+#pragma unroll
+          for (int c = 0; c < kCh; ++c) {
+            U[2 * a2][c] = fmaf(x[a2].x, d[c], U[2 * a2][c]);
+            U[2 * a2 + 1][c] = fmaf(x[a2].y, d[c], U[2 * a2 + 1][c]);
+          }
       }
-    };
-    if (nv == kM) {
-#pragma unroll
-      for (int s = 0; s < kM; ++s) apply_sample(s);
-    } else {
-      for (uint32_t s = 0; s < nv; ++s) apply_sample((int)s);
     }
   }
 
