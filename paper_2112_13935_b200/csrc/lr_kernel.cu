@@ -104,6 +104,17 @@ __device__ __forceinline__ void bulk_load_row(float* dst, const float* src, uint
                ::"r"(smem_addr(dst)), "l"(src), "r"(kRowBytes), "r"(smem_addr(bar)) : "memory");
 }
 
+// n bytes global -> shared and shared -> global (both 16-byte aligned, n a multiple of 16).
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_store_and_wait(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_addr(src)), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the source may be reused after this
+}
+
 // Sum each of the 10 per-lane partials over the warp.  On return lane L holds
 // the total of class lr_class(L) if lr_class_valid(L); 12 shuffles instead of 50.
 __device__ __forceinline__ float reduce10(const float (&a)[kC], int lane) {
@@ -434,6 +445,8 @@ constexpr int kSlots = 3;              // blocks of rows in shared memory
 constexpr int kPx = 14, kPl = 14;      // pixels per thread, pixel groups per warp
 constexpr int kCh = kC / 2;            // classes per thread
 constexpr int kPairs = kM * (kM - 1) / 2;
+constexpr int kParams = kD * kC + kC;                 // 7,850
+constexpr int kStageFloats = (kParams + 31) / 32 * 32;   // a model row as the arrays store it (128-byte multiple)
 static_assert(kPl * kWarps * kPx == kD, "pixel split");
 static_assert(kM == 8, "lane-per-sample recurrence and butterfly widths assume 8");
 
@@ -445,6 +458,8 @@ struct __align__(128) BlkSmem {
   float consts[32];                   // [0..13] = 1,0,...,0 (bias lanes' "row"); [16..29] = 0 (idle lanes)
   int ys[kSlots][kM];
   uint64_t full[kSlots];
+  uint64_t staged;                    // completion of a bulk copy into stage[]
+  float stage[kStageFloats];          // one model row on its way in (snapshot, in-flight sums) or out (U, end model)
 };
 
 // One stage of a transposing reduction: N values per lane in, ceil(N/2) out; the
@@ -529,6 +544,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
   if (threadIdx.x == 0) {
 #pragma unroll
     for (int s = 0; s < kSlots; ++s) mbar_init(&sm.full[s], 1);
+    mbar_init(&sm.staged, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (threadIdx.x < 32) sm.consts[threadIdx.x] = threadIdx.x == 0 ? 1.f : 0.f;
@@ -553,28 +569,45 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
 
   // ---- start model: server snapshot minus own update sums still in flight ----
   // Ws[a][c] = W[14 pg + a][5 cg + c]; the bias lanes hold b[5 cg + c] in row 0.
+  // A thread's 70 parameters are 20-byte pieces 40 bytes apart: each row comes in
+  // as one bulk copy and the threads pick their pieces out of shared memory.
   float Ws[kPx][kCh], U[kPx][kCh];
   const bool owns = active || is_bias;
   const size_t poff = (is_bias ? (size_t)kD * kC : (size_t)pg * (kPx * kC)) + (size_t)cg * kCh;
+  const bool whole_rows = p.stride == (size_t)kStageFloats;   // rows as this kernel stages them
+  bool ok = true;
   {
-    const float* src = p.snaps + (size_t)t.snap_slot * p.stride + poff;
 #pragma unroll
     for (int a = 0; a < kPx; ++a)
 #pragma unroll
-      for (int c = 0; c < kCh; ++c) {
-        const bool live = active || (is_bias && a == 0);
-        Ws[a][c] = live ? __ldg(src + a * kC + c) : 0.f;
-        U[a][c] = 0.f;
+      for (int c = 0; c < kCh; ++c) { Ws[a][c] = 0.f; U[a][c] = 0.f; }
+    for (uint32_t f = 0; f <= t.inflight_cnt; ++f) {   // f = 0: the snapshot, then the sums in flight
+      const float* row;
+      float scale;
+      if (f == 0) {
+        row = p.snaps + (size_t)t.snap_slot * p.stride;
+        scale = 1.f;
+      } else {
+        const InflightRef ref = p.inflight[t.inflight_off + f - 1];
+        row = p.U + (size_t)ref.seq * p.stride;
+        scale = -ref.eta;
       }
-    for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
-      const InflightRef ref = p.inflight[t.inflight_off + f];
-      const float* us = p.U + (size_t)ref.seq * p.stride + poff;
+      if (whole_rows) {
+        if (f) __syncthreads();   // everybody has taken the previous row out of stage[]
+        if (threadIdx.x == 0) {
+          mbar_expect_tx(&sm.staged, kStageFloats * sizeof(float));
+          bulk_load(sm.stage, row, kStageFloats * sizeof(float), &sm.staged);
+        }
+        ok = mbar_wait(&sm.staged, f & 1) && ok;
+        row = sm.stage;
+      }
 #pragma unroll
       for (int a = 0; a < kPx; ++a)
 #pragma unroll
         for (int c = 0; c < kCh; ++c) {
           const bool live = active || (is_bias && a == 0);
-          Ws[a][c] = fmaf(-ref.eta, live ? __ldg(us + a * kC + c) : 0.f, Ws[a][c]);
+          const float v = live ? (whole_rows ? row[poff + a * kC + c] : __ldg(row + poff + a * kC + c)) : 0.f;
+          Ws[a][c] = fmaf(scale, v, Ws[a][c]);
         }
     }
   }
@@ -617,13 +650,12 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     if (gidx >= 0) sm.partG[kb & 1][warp][gidx] = o[0];
   };
 
-  bool ok = true;
   bool timed_out = false;
   uint32_t timeout_at = 0;
 
   // Gram matrix of block 0: warps 0..2 (the rotation below treats warp 3 as busy before block 0)
   if (warp != kWarps - 1) {
-    ok = mbar_wait(&sm.full[0], 0);
+    ok = mbar_wait(&sm.full[0], 0) && ok;
     gram_partial(0, warp);
   }
 
@@ -740,32 +772,19 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     }
     __syncthreads();   // barrier B: delta of the block is in shared memory
 
-    // ---- P3: U += delta_t x_t^T (rolled; the next sample's operands are loaded ahead) ----
-    {
-      float2 xn[kPx / 2];
-      float4 dn4;
-      float dn1;
-      auto load_sample = [&](int s) {
-        dn4 = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
-        dn1 = sm.dbuf[s][cg * 8 + 4];
+    // ---- P3: U += delta_t x_t^T (two samples per trip: the loop has to stay small, see R) ----
+#pragma unroll 2
+    for (int s = 0; s < (int)nv; ++s) {
+      const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
+      const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, sm.dbuf[s][cg * 8 + 4]};
 #pragma unroll
-        for (int a2 = 0; a2 < kPx / 2; ++a2) xn[a2] = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
-      };
-      load_sample(0);
-#pragma unroll 1
-      for (int s = 0; s < (int)nv; ++s) {
-        float2 x[kPx / 2];
+      for (int a2 = 0; a2 < kPx / 2; ++a2) {
+        const float2 x = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
 #pragma unroll
-        for (int a2 = 0; a2 < kPx / 2; ++a2) x[a2] = xn[a2];
-        const float d[kCh] = {dn4.x, dn4.y, dn4.z, dn4.w, dn1};
-        load_sample(s + 1 < kM ? s + 1 : s);
-#pragma unroll
-        for (int a2 = 0; a2 < kPx / 2; ++a2)
-#pragma unroll
-          for (int c = 0; c < kCh; ++c) {
-            U[2 * a2][c] = fmaf(x[a2].x, d[c], U[2 * a2][c]);
-            U[2 * a2 + 1][c] = fmaf(x[a2].y, d[c], U[2 * a2 + 1][c]);
-          }
+        for (int c = 0; c < kCh; ++c) {
+          U[2 * a2][c] = fmaf(x.x, d[c], U[2 * a2][c]);
+          U[2 * a2 + 1][c] = fmaf(x.y, d[c], U[2 * a2 + 1][c]);
+        }
       }
     }
   }
@@ -776,23 +795,31 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     if (threadIdx.x == 0) {
       if (p.status) atomicOr(p.status, 1u);
       for (uint32_t j = timeout_at; j < nblk && j < timeout_at + 2; ++j) mbar_wait(&sm.full[j % kSlots], (j / kSlots) & 1);
+      if (whole_rows) mbar_wait(&sm.staged, t.inflight_cnt & 1);   // the last row staged at the start
     }
     return;
   }
 
   // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model W_start - eta U) ----
-  if (owns) {
-    float* dU = p.U + (size_t)t.seq * p.stride + poff;
-    float* dW = p.w_end ? p.w_end + (size_t)t.seq * p.stride + poff : nullptr;
+  for (int pass = 0; pass < (p.w_end ? 2 : 1); ++pass) {
+    float* dst = (pass == 0 ? p.U : p.w_end) + (size_t)t.seq * p.stride;
+    float* out = whole_rows ? sm.stage : dst;
+    if (whole_rows) {
+      if (pass) __syncthreads();   // the previous row has left stage[]
+      if (threadIdx.x < kStageFloats - kParams) sm.stage[kParams + threadIdx.x] = 0.f;   // the row's padding
+    }
+    if (owns) {
 #pragma unroll
-    for (int a = 0; a < kPx; ++a)
+      for (int a = 0; a < kPx; ++a)
 #pragma unroll
-      for (int c = 0; c < kCh; ++c) {
-        if (active || a == 0) {
-          dU[a * kC + c] = U[a][c];
-          if (dW) dW[a * kC + c] = fmaf(neta, U[a][c], Ws[a][c]);
-        }
-      }
+        for (int c = 0; c < kCh; ++c)
+          if (active || a == 0) out[poff + a * kC + c] = pass == 0 ? U[a][c] : fmaf(neta, U[a][c], Ws[a][c]);
+    }
+    if (whole_rows) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads what the threads wrote
+      __syncthreads();
+      if (threadIdx.x == 0) bulk_store_and_wait(dst, sm.stage, kStageFloats * sizeof(float));
+    }
   }
   if (threadIdx.x == 0) {
     TriggerRec rec;
