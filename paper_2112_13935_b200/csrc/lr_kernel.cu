@@ -562,11 +562,6 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
       sm.ys[sb][lane] = __ldg(cd.y + idx);
     }
   };
-  if (warp == 0) {
-    produce(0);
-    if (nblk > 1) produce(1);
-  }
-
   // ---- start model: server snapshot minus own update sums still in flight ----
   // Ws[a][c] = W[14 pg + a][5 cg + c]; the bias lanes hold b[5 cg + c] in row 0.
   // A thread's 70 parameters are 20-byte pieces 40 bytes apart: each row comes in
@@ -598,6 +593,12 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
           mbar_expect_tx(&sm.staged, kStageFloats * sizeof(float));
           bulk_load(sm.stage, row, kStageFloats * sizeof(float), &sm.staged);
         }
+      }
+      if (f == 0 && warp == 0) {   // the first two blocks of rows, right behind the snapshot
+        produce(0);
+        if (nblk > 1) produce(1);
+      }
+      if (whole_rows) {
         ok = mbar_wait(&sm.staged, f & 1) && ok;
         row = sm.stage;
       }
