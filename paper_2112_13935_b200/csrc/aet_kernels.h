@@ -59,6 +59,9 @@ cudaError_t launch_mlp_rounds(const MlpLaunch& p, cudaStream_t s);
 size_t mlp_act_floats(const MlpShape& shape);
 uint32_t mlp_pick_cluster(const MlpShape& shape, uint32_t n_clients);
 const char* mlp_check_shape(const MlpShape& shape);  // null if the kernel can run it
+// fp32 784-128-C models, batch 32: the model stays on-chip for the whole round (4-CTA cluster)
+bool mlp_res_eligible(const MlpLaunch& p);
+cudaError_t launch_mlp_res_rounds(const MlpLaunch& p, cudaStream_t s);
 // bf16 models whose first layer fits the tensor-core kernel (tcgen05 + TMEM)
 bool mlp_tc_eligible(const MlpShape& shape);
 cudaError_t launch_mlp_tc_rounds(const MlpLaunch& p, cudaStream_t s);

@@ -1,0 +1,444 @@
+// Local-SGD round of one client for the fp32 ReLU MLP 784 -> 128 -> C (C <= 12),
+// minibatch 32, with the model resident on-chip for the whole round.
+//
+// Algorithm 3, MainComputeNode, inner loop with xi a minibatch of B samples:
+// g = mean gradient (+ lambda W); w_c -= eta_i * g; U_i += g.  One cluster of
+// four CTAs runs one round-task.  CTA r owns input rows [196 r, 196 r + 196) of
+// W0 - in its shared memory from the first iteration to the trigger - and the
+// same slice of U0 in registers; it also owns hidden columns [32 r, 32 r + 32):
+// their bias, their rows of W1 and the matching update sums.  Nothing of the
+// model touches global memory between the start of the round and the trigger.
+// Per SGD iteration (three hardware cluster barriers, no polling):
+//   forward   hp = X[:, rows_r] W0[rows_r, :]                      (K split over the CTAs)
+//     barrier 1
+//             h[:, cols_r] = relu(b0 + sum_q hp_q[:, cols_r])      (peers' partials over DSMEM)
+//             z1p = h[:, cols_r] W1[cols_r, :]
+//     barrier 2
+//             z = b1 + sum_q z1p_q; dZ1 = (softmax(z) - onehot) / B (every CTA, identically)
+//             dZ0[:, cols_r] = (dZ1 W1[cols_r, :]^T) * relu'        -> pushed into all four CTAs
+//             W1[cols_r, :], b1: gradient, update, update sum
+//     barrier 3
+//   backward  G = X[:, rows_r]^T dZ0; W0 -= eta (G + lambda W0); U0 += ...   (registers + shared memory)
+// The minibatch rows (this CTA's 196 columns of each) arrive by cp.async.bulk,
+// one iteration ahead, completion on an mbarrier with a bounded wait.  A wait
+// that runs out flags `status`; the CTA then keeps to the barrier schedule so
+// that its peers never block, and the host reports the time-out.
+#include <cuda_runtime.h>
+
+#include "aet_kernels.h"
+#include "aet_rng.h"
+#include "mlp_common.cuh"
+
+namespace aet {
+namespace {
+
+using namespace mlp;
+
+constexpr int kT = 512, kCL = 4, kB = 32, kD0 = 784, kH = 128, kCP = 12;
+constexpr int kR = kD0 / kCL;        // 196 input rows per CTA
+constexpr int kHS = kH / kCL;        // 32 hidden columns per CTA
+constexpr int kRW = 14;              // rows of the gradient tile per warp; 14 warps x 14 rows = 196
+constexpr int kGW = kR / kRW;        // warps that own a tile of W0 / U0
+constexpr int kKH = kR / 2;          // the forward product splits K once more inside the CTA
+constexpr uint32_t kWaitLimit = 1u << 22;
+static_assert(kGW * kRW == kR && kGW <= kT / 32 - 1, "gradient tiling");
+
+struct __align__(128) ResSmem {
+  float W0[kR][kH];        // this CTA's rows of W0, current
+  float xs[2][kB][kR];     // this CTA's columns of the minibatch rows, double-buffered
+  float hp[kB][kH];        // partial pre-activations from this CTA's K slice (read by the peers)
+  float dz0[kB][kH];       // dZ0, every CTA's columns (written by the peers); scratch inside the forward product
+  float hs[kB][kHS + 1];   // activations of the owned hidden columns
+  float W1[kHS][kCP];      // owned rows of W1 (columns >= C stay zero)
+  float U1[kHS][kCP];
+  float z1p[kB][kCP];      // partial logits from the owned hidden columns (read by the peers)
+  float dz1[kB][kCP];      // logits, then dZ1
+  float b0[kHS], Ub0[kHS], b1[kCP], Ub1[kCP];
+  int ys[2][kB];
+  uint64_t full[2], wbar;
+};
+
+__device__ __forceinline__ uint32_t saddr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(saddr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(saddr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {   // bounded
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(saddr(bar)), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+// global -> this CTA's shared memory; both 16-byte aligned, size a multiple of 16
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(saddr(dst)), "l"(src), "r"(bytes), "r"(saddr(bar)) : "memory");
+}
+// the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t peer(uint32_t a, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_peer4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ float ld_peer(uint32_t a) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_peer(uint32_t a, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  ResSmem& sm = *reinterpret_cast<ResSmem*>(smem_raw);
+
+  const int rank = (int)cluster_rank();
+  const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / kCL];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int C = (int)p.shape.dims[2];
+  const ClientData cd = p.r.clients[t.client];
+  const uint64_t key = p.r.sample_keys[t.client];
+  const float* xrows = reinterpret_cast<const float*>(cd.x);
+  const float eta = t.eta, lambda = p.r.l2, invB = 1.f / (float)kB;
+
+  // parameter vector: W0 [784,128], b0 [128], W1 [128,C], b1 [C]
+  const size_t woff0 = 0, boff0 = (size_t)kD0 * kH, woff1 = boff0 + kH, boff1 = woff1 + (size_t)kH * C;
+  const size_t w0_mine = woff0 + (size_t)rank * kR * kH;
+  const float* snap = p.r.snaps + (size_t)t.snap_slot * p.r.stride;
+
+  if (tid == 0) {
+    mbar_init(&sm.full[0], 1);
+    mbar_init(&sm.full[1], 1);
+    mbar_init(&sm.wbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // The minibatch of iteration `it`: this CTA's 196 columns of each of the 32 sampled rows.
+  auto issue_rows = [&](uint32_t it, int buf) {
+    if (warp == 0) {
+      if (lane == 0) mbar_expect_tx(&sm.full[buf], kB * kR * sizeof(float));
+      __syncwarp();
+      const uint32_t idx = sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * kB + lane), cd.n);
+      bulk_load(&sm.xs[buf][lane][0], xrows + (size_t)idx * kD0 + (size_t)rank * kR, kR * sizeof(float), &sm.full[buf]);
+      sm.ys[buf][lane] = __ldg(cd.y + idx);
+    }
+  };
+
+  // ---- start model: server snapshot minus own update sums still in flight ----
+  if (tid == 0) {
+    mbar_expect_tx(&sm.wbar, kR * kH * sizeof(float));
+    bulk_load(&sm.W0[0][0], snap + w0_mine, kR * kH * sizeof(float), &sm.wbar);
+  }
+  if (t.steps) issue_rows(0, 0);
+  auto start_value = [&](size_t j) {
+    float w = __ldg(snap + j);
+    for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+      const InflightRef ref = p.r.inflight[t.inflight_off + f];
+      w = fmaf(-ref.eta, __ldg(p.r.U + (size_t)ref.seq * p.r.stride + j), w);
+    }
+    return w;
+  };
+  for (int e = tid; e < kHS * kCP; e += kT) {
+    const int jl = e / kCP, c = e % kCP;
+    sm.W1[jl][c] = c < C ? start_value(woff1 + (size_t)(rank * kHS + jl) * C + c) : 0.f;
+    sm.U1[jl][c] = 0.f;
+  }
+  if (tid < kHS) { sm.b0[tid] = start_value(boff0 + rank * kHS + tid); sm.Ub0[tid] = 0.f; }
+  if (tid < kCP) { sm.b1[tid] = tid < C ? start_value(boff1 + tid) : 0.f; sm.Ub1[tid] = 0.f; }
+  bool ok = mbar_wait(&sm.wbar, 0);
+  for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+    const InflightRef ref = p.r.inflight[t.inflight_off + f];
+    const float4* us = reinterpret_cast<const float4*>(p.r.U + (size_t)ref.seq * p.r.stride + w0_mine);
+    float4* w4 = reinterpret_cast<float4*>(&sm.W0[0][0]);
+    for (int e = tid; e < kR * kH / 4; e += kT) {
+      const float4 u = __ldg(us + e);
+      float4 w = w4[e];
+      w.x = fmaf(-ref.eta, u.x, w.x); w.y = fmaf(-ref.eta, u.y, w.y);
+      w.z = fmaf(-ref.eta, u.z, w.z); w.w = fmaf(-ref.eta, u.w, w.w);
+      w4[e] = w;
+    }
+  }
+  // this thread's tile of U0: rows 14 warp .. 14 warp + 13, columns 4 lane .. 4 lane + 3
+  float U0[kRW][4];
+#pragma unroll
+  for (int i = 0; i < kRW; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) U0[i][j] = 0.f;
+  __syncthreads();
+  cluster_barrier();   // every CTA of the cluster is set up before any of them is written to
+
+  // forward-product roles: K half, 4 batch rows, 4 hidden columns
+  const int half = tid >> 8, t2 = tid & 255, bt = t2 >> 5, jt = t2 & 31;
+  uint32_t h = 0;   // local sample counter of Algorithm 3
+
+  for (uint32_t it = 0; it < t.steps; ++it) {
+    const int buf = it & 1;
+    if (it + 1 < t.steps) issue_rows(it + 1, buf ^ 1);   // that buffer was last read before the previous trip's closing barrier
+    ok = mbar_wait(&sm.full[buf], (it >> 1) & 1) && ok;
+
+    // ---------------- forward: hp = X[:, rows] W0[rows, :] ----------------
+    {
+      float acc[4][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+      const float* xb = &sm.xs[buf][4 * bt][kKH * half];
+      const float* wb = &sm.W0[kKH * half][4 * jt];
+#pragma unroll 7
+      for (int k = 0; k < kKH; k += 2) {
+        const float4 w0 = *reinterpret_cast<const float4*>(wb + k * kH);
+        const float4 w1 = *reinterpret_cast<const float4*>(wb + (k + 1) * kH);
+        const float wa[4] = {w0.x, w0.y, w0.z, w0.w}, wc[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 x = *reinterpret_cast<const float2*>(xb + i * kR + k);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(x.y, wc[j], fmaf(x.x, wa[j], acc[i][j]));
+        }
+      }
+      float4* scratch = reinterpret_cast<float4*>(&sm.dz0[0][0]);   // free until the peers pass barrier 2
+      if (half == 1) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) scratch[i * 256 + t2] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+      }
+      __syncthreads();
+      if (half == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 o = scratch[i * 256 + t2];
+          *reinterpret_cast<float4*>(&sm.hp[4 * bt + i][4 * jt]) =
+              make_float4(acc[i][0] + o.x, acc[i][1] + o.y, acc[i][2] + o.z, acc[i][3] + o.w);
+        }
+      }
+    }
+    cluster_barrier();   // 1: every CTA's partial pre-activations are in place
+
+    // owned hidden columns: bias + the four partials, ReLU
+    if (tid < kB * kHS / 4) {
+      const int b = tid >> 3, j4 = (tid & 7) * 4;
+      const uint32_t a = saddr(&sm.hp[b][rank * kHS + j4]);
+      float4 z = make_float4(sm.b0[j4], sm.b0[j4 + 1], sm.b0[j4 + 2], sm.b0[j4 + 3]);
+#pragma unroll
+      for (int q = 0; q < kCL; ++q) {
+        const float4 v = ld_peer4(peer(a, q));
+        z.x += v.x; z.y += v.y; z.z += v.z; z.w += v.w;
+      }
+      sm.hs[b][j4] = fmaxf(z.x, 0.f); sm.hs[b][j4 + 1] = fmaxf(z.y, 0.f);
+      sm.hs[b][j4 + 2] = fmaxf(z.z, 0.f); sm.hs[b][j4 + 3] = fmaxf(z.w, 0.f);
+    }
+    __syncthreads();
+    if (tid < kB * kCP) {   // partial logits from the owned columns
+      const int b = tid / kCP, c = tid % kCP;
+      float s = 0.f;
+#pragma unroll 8
+      for (int jl = 0; jl < kHS; ++jl) s = fmaf(sm.hs[b][jl], sm.W1[jl][c], s);
+      sm.z1p[b][c] = s;
+    }
+    cluster_barrier();   // 2: every CTA's partial logits are in place; dz0 is no longer anybody's scratch
+
+    if (tid < kB * kCP) {
+      const int b = tid / kCP, c = tid % kCP;
+      const uint32_t a = saddr(&sm.z1p[b][c]);
+      float z = sm.b1[c];
+#pragma unroll
+      for (int q = 0; q < kCL; ++q) z += ld_peer(peer(a, q));
+      sm.dz1[b][c] = z;
+    }
+    __syncthreads();
+    if (warp == 0) {   // softmax cross-entropy, one sample per lane: dZ1 = (p - onehot(y)) / B
+      const int b = lane, y = sm.ys[buf][b];
+      float m = -INFINITY;
+      for (int c = 0; c < C; ++c) m = fmaxf(m, sm.dz1[b][c]);
+      float e[kCP], sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < kCP; ++c) { e[c] = c < C ? __expf(sm.dz1[b][c] - m) : 0.f; sum += e[c]; }
+      const float inv = 1.f / sum;
+#pragma unroll
+      for (int c = 0; c < kCP; ++c) sm.dz1[b][c] = c < C ? (e[c] * inv - (c == y ? 1.f : 0.f)) * invB : 0.f;
+    }
+    __syncthreads();
+    // dZ0 for the owned columns, into every CTA of the cluster
+#pragma unroll
+    for (int u = 0; u < kB * kHS / kT; ++u) {
+      const int e = tid + u * kT, b = e >> 5, jl = e & 31;
+      float s = 0.f;
+#pragma unroll
+      for (int c = 0; c < kCP; ++c) s = fmaf(sm.dz1[b][c], sm.W1[jl][c], s);
+      const float v = sm.hs[b][jl] > 0.f ? s : 0.f;
+      const uint32_t a = saddr(&sm.dz0[b][rank * kHS + jl]);
+#pragma unroll
+      for (int q = 0; q < kCL; ++q) st_peer(peer(a, q), v);
+    }
+    __syncthreads();   // W1 has been read by everybody
+    if (tid < kHS * kCP) {   // W1 rows of the owned columns
+      const int jl = tid / kCP, c = tid % kCP;
+      float g = 0.f;
+#pragma unroll 8
+      for (int b = 0; b < kB; ++b) g = fmaf(sm.hs[b][jl], sm.dz1[b][c], g);
+      const float w = sm.W1[jl][c];
+      g = fmaf(lambda, w, g);
+      sm.W1[jl][c] = fmaf(-eta, g, w);
+      sm.U1[jl][c] += g;
+    } else if (tid < kHS * kCP + kCP) {   // b1: every CTA keeps its own, identical copy
+      const int c = tid - kHS * kCP;
+      float g = 0.f;
+      for (int b = 0; b < kB; ++b) g += sm.dz1[b][c];
+      sm.b1[c] = fmaf(-eta, g, sm.b1[c]);
+      sm.Ub1[c] += g;
+    }
+    cluster_barrier();   // 3: dZ0 is complete in every CTA
+
+    // ---------------- backward: G = X[:, rows]^T dZ0, update of W0 and U0 ----------------
+    if (warp < kGW) {
+      const int row0 = warp * kRW;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        float g[7][4];
+#pragma unroll
+        for (int i = 0; i < 7; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) g[i][j] = 0.f;
+        const float* xr = &sm.xs[buf][0][row0 + 7 * hh];
+#pragma unroll 4
+        for (int b = 0; b < kB; ++b) {
+          const float4 d = *reinterpret_cast<const float4*>(&sm.dz0[b][4 * lane]);
+          const float dv[4] = {d.x, d.y, d.z, d.w};
+          float x[7];
+          if (hh == 0) {   // the tile's first row is even: pairs first
+            const float2 p0 = *reinterpret_cast<const float2*>(xr + b * kR), p1 = *reinterpret_cast<const float2*>(xr + b * kR + 2),
+                         p2 = *reinterpret_cast<const float2*>(xr + b * kR + 4);
+            x[0] = p0.x; x[1] = p0.y; x[2] = p1.x; x[3] = p1.y; x[4] = p2.x; x[5] = p2.y; x[6] = xr[b * kR + 6];
+          } else {
+            const float2 p0 = *reinterpret_cast<const float2*>(xr + b * kR + 1), p1 = *reinterpret_cast<const float2*>(xr + b * kR + 3),
+                         p2 = *reinterpret_cast<const float2*>(xr + b * kR + 5);
+            x[0] = xr[b * kR]; x[1] = p0.x; x[2] = p0.y; x[3] = p1.x; x[4] = p1.y; x[5] = p2.x; x[6] = p2.y;
+          }
+#pragma unroll
+          for (int i = 0; i < 7; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) g[i][j] = fmaf(x[i], dv[j], g[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 7; ++i) {
+          float4* wp = reinterpret_cast<float4*>(&sm.W0[row0 + 7 * hh + i][4 * lane]);
+          float4 w = *wp;
+          const float g0 = fmaf(lambda, w.x, g[i][0]), g1 = fmaf(lambda, w.y, g[i][1]),
+                      g2 = fmaf(lambda, w.z, g[i][2]), g3 = fmaf(lambda, w.w, g[i][3]);
+          w.x = fmaf(-eta, g0, w.x); w.y = fmaf(-eta, g1, w.y); w.z = fmaf(-eta, g2, w.z); w.w = fmaf(-eta, g3, w.w);
+          *wp = w;
+          U0[7 * hh + i][0] += g0; U0[7 * hh + i][1] += g1; U0[7 * hh + i][2] += g2; U0[7 * hh + i][3] += g3;
+        }
+      }
+    } else if (warp == kGW) {   // b0 of the owned columns
+      float g = 0.f;
+      for (int b = 0; b < kB; ++b) g += sm.dz0[b][rank * kHS + lane];
+      sm.b0[lane] = fmaf(-eta, g, sm.b0[lane]);
+      sm.Ub0[lane] += g;
+    }
+    h += kB;
+    __syncthreads();   // W0 and b0 updated; the row buffer may be refilled
+  }
+
+  if (!ok) {
+    // A bulk copy never completed.  Report it; give what may still be in flight a
+    // bounded chance to land in this CTA's shared memory before it goes away.
+    if (tid == 0) {
+      if (p.r.status) atomicOr(p.r.status, 1u);
+      mbar_wait(&sm.wbar, 0);
+      for (uint32_t it = t.steps >= 2 ? t.steps - 2 : 0; it < t.steps; ++it) mbar_wait(&sm.full[it & 1], (it >> 1) & 1);
+    }
+  }
+
+  // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model) ----
+  {
+    float* Urow = p.r.U + (size_t)t.seq * p.r.stride;
+    float* Wend = p.r.w_end ? p.r.w_end + (size_t)t.seq * p.r.stride : nullptr;
+    if (warp < kGW) {
+#pragma unroll
+      for (int i = 0; i < kRW; ++i) {
+        const size_t o = w0_mine + (size_t)(warp * kRW + i) * kH + 4 * lane;
+        *reinterpret_cast<float4*>(Urow + o) = make_float4(U0[i][0], U0[i][1], U0[i][2], U0[i][3]);
+        if (Wend) *reinterpret_cast<float4*>(Wend + o) = *reinterpret_cast<const float4*>(&sm.W0[warp * kRW + i][4 * lane]);
+      }
+    }
+    for (int e = tid; e < kHS * C; e += kT) {
+      const int jl = e / C, c = e % C;
+      const size_t o = woff1 + (size_t)(rank * kHS + jl) * C + c;
+      Urow[o] = sm.U1[jl][c];
+      if (Wend) Wend[o] = sm.W1[jl][c];
+    }
+    if (tid < kHS) {
+      Urow[boff0 + rank * kHS + tid] = sm.Ub0[tid];
+      if (Wend) Wend[boff0 + rank * kHS + tid] = sm.b0[tid];
+    }
+    if (rank == 0 && tid < C) {
+      Urow[boff1 + tid] = sm.Ub1[tid];
+      if (Wend) Wend[boff1 + tid] = sm.b1[tid];
+    }
+    if (rank == 0 && tid == 0) {
+      TriggerRec rec;
+      rec.client = t.client; rec.round = t.round; rec.samples_done = h; rec.flags = 1;
+      p.r.trig[t.seq] = rec;
+    }
+  }
+  cluster_barrier();   // nobody leaves while a peer could still address its shared memory
+}
+
+}  // namespace
+
+// Shapes the resident kernel runs; rows of the model arrays must be whole (stride != 0:
+// the handle's 128-byte aligned rows), since the model slices come in by bulk copy.
+bool mlp_res_eligible(const MlpLaunch& p) {
+  const MlpShape& s = p.shape;
+  return s.precision == 0 && s.n_layers == 2 && s.batch == kB && s.dims[0] == kD0 && s.dims[1] == kH &&
+         s.dims[2] >= 1 && s.dims[2] <= kCP && p.r.stride != 0 && p.r.stride % 4 == 0 &&
+         (reinterpret_cast<uintptr_t>(p.r.snaps) & 15) == 0 && (reinterpret_cast<uintptr_t>(p.r.U) & 15) == 0 &&
+         (p.r.w_end == nullptr || (reinterpret_cast<uintptr_t>(p.r.w_end) & 15) == 0);
+}
+
+cudaError_t launch_mlp_res_rounds(const MlpLaunch& p, cudaStream_t s) {
+  if (p.r.n_tasks == 0) return cudaSuccess;
+  static bool opted_in[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+    e = cudaFuncSetAttribute(mlp_res_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ResSmem));
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) opted_in[dev] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(p.r.n_tasks * kCL, 1, 1);
+  cfg.blockDim = dim3(kT, 1, 1);
+  cfg.dynamicSmemBytes = sizeof(ResSmem);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kCL;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, mlp_res_kernel, p);
+}
+
+}  // namespace aet
