@@ -81,6 +81,28 @@ def algorithmic_flops(cfg, events):
     return per_sample * sum(e["samples"] for e in events)
 
 
+def fp32_fma_peak_tflops():
+    """Plain fp32 FMA peak from the unit counts and the maximum SM clock:
+    148 SMs x 128 fp32 lanes x 2 flops x clock (a register-only FMA loop measured 126 of the
+    128 lanes per clock on this part)."""
+    mhz = 1965.0
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            mhz = float(json.load(f).get("sm_max_mhz", mhz))
+    except Exception:
+        pass
+    return 148 * 128 * 2 * mhz * 1e6 / 1e12, f"derived: 148 SMs x 128 fp32 lanes x 2 x {mhz:.0f} MHz"
+
+
+def regression_flops(cfg, events):
+    """Softmax regression, batch 1: logits, model update and update sum are one FMA per
+    parameter and sample each (the l2 term adds two more per weight)."""
+    from paper_2112_13935_b200 import workloads
+    P = workloads.n_params(cfg["dims"])
+    per_sample = 2 * (3 + (2 if cfg["l2"] else 0)) * P
+    return per_sample * sum(e["samples"] for e in events)
+
+
 def measured_peak_tflops():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -295,10 +317,20 @@ def main():
             "algorithmic_bytes_per_launch": alg_bytes / n_sgd_launches}
     if cfg["model"] == 1:
         tf = algorithmic_flops(cfg, events) / (sgd_ms_per_step * 1e-3) / 1e12
-        tpeak, tkind = measured_peak_tflops()
-        roof = {"bound": "tensor", "kernel": "local-SGD rounds (MLP)", "achieved": tf, "peak": tpeak,
+        if cfg["precision"] == 1:     # bf16 operands: the dense contraction runs on the tensor cores
+            tpeak, tkind = measured_peak_tflops()
+            bound = "tensor"
+        else:                         # fp32 model: plain FMAs
+            tpeak, tkind = fp32_fma_peak_tflops()
+            bound = "alu"
+        roof = {"bound": bound, "kernel": "local-SGD rounds (MLP)", "achieved": tf, "peak": tpeak,
                 "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "peak_kind": tkind,
                 "hbm_gbs_algorithmic": achieved}
+    else:
+        # the batch-1 regression kernel sits on the FMA / HBM ridge: its fp32 FMA rate beside the HBM figure
+        apeak, akind = fp32_fma_peak_tflops()
+        atf = regression_flops(cfg, events) / (sgd_ms_per_step * 1e-3) / 1e12
+        roof.update(alu_tflops=atf, alu_peak=apeak, alu_frac=atf / apeak, alu_peak_kind=akind)
     roof.update(launches_per_step=n_sgd_launches, kernel_ms_per_step=sgd_ms_per_step,
                 aggregation_ms_per_step=k_ms[1] / k_steps, algorithmic_bytes_per_step=alg_bytes)
     sess.close()

@@ -39,9 +39,10 @@ constexpr int kR = kD0 / kCL;        // 196 input rows per CTA
 constexpr int kHS = kH / kCL;        // 32 hidden columns per CTA
 constexpr int kRW = 14;              // rows of the gradient tile per warp; 14 warps x 14 rows = 196
 constexpr int kGW = kR / kRW;        // warps that own a tile of W0 / U0
-constexpr int kKH = kR / 2;          // the forward product splits K once more inside the CTA
+constexpr int kKH = 100;             // the forward product splits K once more inside the CTA: rows [0,100) and [100,196)
 constexpr uint32_t kWaitLimit = 1u << 22;
-static_assert(kGW * kRW == kR && kGW <= kT / 32 - 1, "gradient tiling");
+static_assert(kGW * kRW == kR && kGW + 2 <= kT / 32, "gradient tiling: two warps stay free for the bias and the row copies");
+static_assert(kKH % 4 == 0 && (kR - kKH) % 4 == 0, "forward K split");
 
 struct __align__(128) ResSmem {
   float W0[kR][kH];        // this CTA's rows of W0, current
@@ -52,7 +53,8 @@ struct __align__(128) ResSmem {
   float W1[kHS][kCP];      // owned rows of W1 (columns >= C stay zero)
   float U1[kHS][kCP];
   float z1p[kB][kCP];      // partial logits from the owned hidden columns (read by the peers)
-  float dz1[kB][kCP];      // logits, then dZ1
+  float z1[kB][kCP];       // logits
+  float dz1[kB][kCP];
   float b0[kHS], Ub0[kHS], b1[kCP], Ub1[kCP];
   int ys[2][kB];
   uint64_t full[2], wbar;
@@ -132,14 +134,14 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
   __syncthreads();
 
   // The minibatch of iteration `it`: this CTA's 196 columns of each of the 32 sampled rows.
-  auto issue_rows = [&](uint32_t it, int buf) {
-    if (warp == 0) {
-      if (lane == 0) mbar_expect_tx(&sm.full[buf], kB * kR * sizeof(float));
-      __syncwarp();
-      const uint32_t idx = sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * kB + lane), cd.n);
-      bulk_load(&sm.xs[buf][lane][0], xrows + (size_t)idx * kD0 + (size_t)rank * kR, kR * sizeof(float), &sm.full[buf]);
-      sm.ys[buf][lane] = __ldg(cd.y + idx);
-    }
+  // One warp; returns lane b's label.  Issuing 32 bulk copies keeps a warp busy for a few
+  // thousand cycles, so inside the loop it is the job of a warp with nothing else to do.
+  auto issue_rows = [&](uint32_t it, int buf) -> int {
+    if (lane == 0) mbar_expect_tx(&sm.full[buf], kB * kR * sizeof(float));
+    __syncwarp();
+    const uint32_t idx = sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * kB + lane), cd.n);
+    bulk_load(&sm.xs[buf][lane][0], xrows + (size_t)idx * kD0 + (size_t)rank * kR, kR * sizeof(float), &sm.full[buf]);
+    return __ldg(cd.y + idx);
   };
 
   // ---- start model: server snapshot minus own update sums still in flight ----
@@ -147,7 +149,7 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
     mbar_expect_tx(&sm.wbar, kR * kH * sizeof(float));
     bulk_load(&sm.W0[0][0], snap + w0_mine, kR * kH * sizeof(float), &sm.wbar);
   }
-  if (t.steps) issue_rows(0, 0);
+  if (warp == 0 && t.steps) sm.ys[0][lane] = issue_rows(0, 0);
   auto start_value = [&](size_t j) {
     float w = __ldg(snap + j);
     for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
@@ -191,7 +193,6 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
 
   for (uint32_t it = 0; it < t.steps; ++it) {
     const int buf = it & 1;
-    if (it + 1 < t.steps) issue_rows(it + 1, buf ^ 1);   // that buffer was last read before the previous trip's closing barrier
     ok = mbar_wait(&sm.full[buf], (it >> 1) & 1) && ok;
 
     // ---------------- forward: hp = X[:, rows] W0[rows, :] ----------------
@@ -203,16 +204,21 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
       const float* xb = &sm.xs[buf][4 * bt][kKH * half];
       const float* wb = &sm.W0[kKH * half][4 * jt];
-#pragma unroll 7
-      for (int k = 0; k < kKH; k += 2) {
-        const float4 w0 = *reinterpret_cast<const float4*>(wb + k * kH);
-        const float4 w1 = *reinterpret_cast<const float4*>(wb + (k + 1) * kH);
-        const float wa[4] = {w0.x, w0.y, w0.z, w0.w}, wc[4] = {w1.x, w1.y, w1.z, w1.w};
+      const int kn = half ? kR - kKH : kKH;
+#pragma unroll 4
+      for (int k = 0; k < kn; k += 4) {
+        float w[4][4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 v = *reinterpret_cast<const float4*>(wb + (k + q) * kH);
+          w[q][0] = v.x; w[q][1] = v.y; w[q][2] = v.z; w[q][3] = v.w;
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float2 x = *reinterpret_cast<const float2*>(xb + i * kR + k);
+          const float4 x = *reinterpret_cast<const float4*>(xb + i * kR + k);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(x.y, wc[j], fmaf(x.x, wa[j], acc[i][j]));
+          for (int j = 0; j < 4; ++j)
+            acc[i][j] = fmaf(x.w, w[3][j], fmaf(x.z, w[2][j], fmaf(x.y, w[1][j], fmaf(x.x, w[0][j], acc[i][j]))));
         }
       }
       float4* scratch = reinterpret_cast<float4*>(&sm.dz0[0][0]);   // free until the peers pass barrier 2
@@ -261,19 +267,25 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
       float z = sm.b1[c];
 #pragma unroll
       for (int q = 0; q < kCL; ++q) z += ld_peer(peer(a, q));
-      sm.dz1[b][c] = z;
+      sm.z1[b][c] = z;
     }
     __syncthreads();
-    if (warp == 0) {   // softmax cross-entropy, one sample per lane: dZ1 = (p - onehot(y)) / B
-      const int b = lane, y = sm.ys[buf][b];
+    if (tid < kB * kCP) {   // softmax cross-entropy: dZ1 = (p - onehot(y)) / B; every thread sums its sample's row itself
+      const int b = tid / kCP, c = tid % kCP;
+      const float4 r0 = *reinterpret_cast<const float4*>(&sm.z1[b][0]), r1 = *reinterpret_cast<const float4*>(&sm.z1[b][4]),
+                   r2 = *reinterpret_cast<const float4*>(&sm.z1[b][8]);
+      const float z[kCP] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w, r2.x, r2.y, r2.z, r2.w};
       float m = -INFINITY;
-      for (int c = 0; c < C; ++c) m = fmaxf(m, sm.dz1[b][c]);
-      float e[kCP], sum = 0.f;
 #pragma unroll
-      for (int c = 0; c < kCP; ++c) { e[c] = c < C ? __expf(sm.dz1[b][c] - m) : 0.f; sum += e[c]; }
-      const float inv = 1.f / sum;
+      for (int k = 0; k < kCP; ++k) m = k < C ? fmaxf(m, z[k]) : m;
+      float sum = 0.f, mine = 0.f;
 #pragma unroll
-      for (int c = 0; c < kCP; ++c) sm.dz1[b][c] = c < C ? (e[c] * inv - (c == y ? 1.f : 0.f)) * invB : 0.f;
+      for (int k = 0; k < kCP; ++k) {
+        const float e = k < C ? __expf(z[k] - m) : 0.f;
+        sum += e;
+        mine = k == c ? e : mine;
+      }
+      sm.dz1[b][c] = c < C ? (mine / sum - (c == sm.ys[buf][b] ? 1.f : 0.f)) * invB : 0.f;
     }
     __syncthreads();
     // dZ0 for the owned columns, into every CTA of the cluster
@@ -348,6 +360,9 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
           U0[7 * hh + i][0] += g0; U0[7 * hh + i][1] += g1; U0[7 * hh + i][2] += g2; U0[7 * hh + i][3] += g3;
         }
       }
+    } else if (warp == kT / 32 - 1) {
+      // the next minibatch; its buffer was last read before the previous trip's closing barrier
+      if (it + 1 < t.steps) sm.ys[buf ^ 1][lane] = issue_rows(it + 1, buf ^ 1);
     } else if (warp == kGW) {   // b0 of the owned columns
       float g = 0.f;
       for (int b = 0; b < kB; ++b) g += sm.dz0[b][rank * kHS + lane];
