@@ -89,6 +89,28 @@ def test_variants_end_to_end(over):
     assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
 
 
+@pytest.mark.parametrize("over", [
+    dict(sched_a=3, sched_b=1, n_rounds=9),                       # rounds of 1, 4, 7, ... 25 samples: every tail length
+    dict(sched_a=1, sched_b=1, n_rounds=7, n_clients=3),          # rounds shorter than one block of 8
+    dict(sched_a=5, sched_b=11, n_rounds=6, max_lag_d=0),         # odd sizes, everybody waits for everybody
+    dict(n_clients=1, n_rounds=6),                                # one client: plain SGD
+    dict(n_clients=2, n_rounds=6, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=500.0),   # own sums in flight
+    dict(lr_beta=0.05, sched_a=7, sched_b=2),                     # step size changes from round to round
+])
+def test_blocked_kernel_variants_without_l2(over):
+    # lambda = 0 takes the kernel that runs eight steps per block; check ragged tails and start-model cases on it
+    cfg = workloads.get_config("cfg1", l2=0.0, data=dict(per_client=300), **over)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        worst = max(check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
+                    for e in ref["events"])
+    assert worst <= U_TOL
+
+
 def test_many_own_updates_in_flight():
     # a slow network keeps several of a client's own sums in flight at round start
     cfg = workloads.get_config("cfg1", n_clients=2, n_rounds=6, max_lag_d=workloads.NEVER_WAIT,
