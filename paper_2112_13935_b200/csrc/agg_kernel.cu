@@ -49,6 +49,11 @@ __global__ void __launch_bounds__(kAggThreads) group_totals_kernel(ApplyLaunch p
 }
 
 __global__ void __launch_bounds__(kAggThreads) apply_updates_kernel(ApplyLaunch p) {
+  // The round kernel that follows in the stream may be launched with programmatic stream
+  // serialisation: let its CTAs start their set-up (descriptors, first rows) while this grid
+  // runs.  They read nothing this grid writes before their own griddepcontrol.wait, which
+  // returns only once this grid has finished and its writes are visible.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t j = blockIdx.x * kAggThreads + threadIdx.x;
   const uint32_t g = blockIdx.y;
   uint32_t lo, hi;

@@ -576,6 +576,14 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     for (int a = 0; a < kPx; ++a)
 #pragma unroll
       for (int c = 0; c < kCh; ++c) { Ws[a][c] = 0.f; U[a][c] = 0.f; }
+    // Everything above reads only what earlier, finished grids and the host wrote.  The snapshot
+    // is written by the aggregation kernel launched just before this grid, which may still be
+    // running when this grid was launched with programmatic stream serialisation.
+    if (warp == 0) {   // the first two blocks of rows
+      produce(0);
+      if (nblk > 1) produce(1);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (uint32_t f = 0; f <= t.inflight_cnt; ++f) {   // f = 0: the snapshot, then the sums in flight
       const float* row;
       float scale;
@@ -593,10 +601,6 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
           mbar_expect_tx(&sm.staged, kStageFloats * sizeof(float));
           bulk_load(sm.stage, row, kStageFloats * sizeof(float), &sm.staged);
         }
-      }
-      if (f == 0 && warp == 0) {   // the first two blocks of rows, right behind the snapshot
-        produce(0);
-        if (nblk > 1) produce(1);
       }
       if (whole_rows) {
         ok = mbar_wait(&sm.staged, f & 1) && ok;
@@ -863,8 +867,20 @@ cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s) {
       if (e != cudaSuccess) return e;
       if (dev >= 0 && dev < 64) opted_in[dev] = true;
     }
-    lr_block_kernel<<<p.n_tasks, kThreads, sizeof(BlkSmem), s>>>(p);
-    return cudaGetLastError();
+    // Programmatic stream serialisation: the grid may start while the kernel before it in the
+    // stream (the aggregation of the previous wave) is still running; lr_block_kernel waits
+    // (griddepcontrol.wait) before it reads anything that kernel writes.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(p.n_tasks, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = sizeof(BlkSmem);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, lr_block_kernel, p);
   }
   // lambda != 0 couples the steps of a block through the decay of W: step by step.
   // Enough round-tasks to put two CTAs on every SM: trade latency for instruction count.
