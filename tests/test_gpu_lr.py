@@ -62,6 +62,23 @@ def test_cfg5_shape_64_clients_end_to_end():
     assert np.abs(gpu["w"] - ref["w"]).max() <= 2e-5
 
 
+def test_cfg5_full_size_log_invariant_and_sampled_rounds():
+    # 1,024 clients: the configuration the roofline figure is quoted on (waves of up to 1,024 round-tasks)
+    cfg = workloads.get_config("cfg5")
+    data, w0 = make(cfg)
+    events, summary, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    assert len(events) == 10240 and summary["samples_total"] == 450560
+    gpu = run_gpu(cfg, data, w0)
+    assert gpu["blob"] == schedule.pack_events(events) and gpu["summary"] == summary
+    acc = w0.astype(np.float64)
+    for e in events:
+        acc -= sim.step_size(cfg, e["round"]) * gpu["U"][e["seq"]].astype(np.float64)
+    assert np.abs(acc - gpu["w"]).max() <= 2e-6 * max(1.0, np.abs(acc).max())
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for c, i in ((0, 0), (1023, 9), (517, 4), (64, 7)):
+            check_round_U(cfg, data, s.h, c, i, gpu["w"])
+
+
 @pytest.mark.parametrize("n_clients,l2", [(320, 0.0), (320, 1e-3), (480, 0.0), (480, 1e-3)])
 def test_many_clients_take_the_kernel_variant_for_crowded_waves(n_clients, l2):
     # >= 296 round-tasks in a wave switch the kernel to its one-warp softmax
