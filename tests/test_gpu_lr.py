@@ -113,18 +113,23 @@ def test_variants_end_to_end(over):
     dict(n_clients=1, n_rounds=6),                                # one client: plain SGD
     dict(n_clients=2, n_rounds=6, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=500.0),   # own sums in flight
     dict(lr_beta=0.05, sched_a=7, sched_b=2),                     # step size changes from round to round
+    dict(n_clients=330, n_rounds=4, sched_a=3, sched_b=2, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=50.0,
+         data=dict(per_client=64)),   # more round-tasks than CTAs: a CTA runs several in a row, with sums in flight and ragged tails
 ])
 def test_blocked_kernel_variants_without_l2(over):
     # lambda = 0 takes the kernel that runs eight steps per block; check ragged tails and start-model cases on it
-    cfg = workloads.get_config("cfg1", l2=0.0, data=dict(per_client=300), **over)
+    over = dict(over)
+    cfg = workloads.get_config("cfg1", l2=0.0, data=over.pop("data", dict(per_client=300)), **over)
     data, w0 = make(cfg)
     ref = sim.run(cfg, data, w0, keep=True)
     gpu = run_gpu(cfg, data, w0)
     check_against_oracle(cfg, data, w0, gpu, ref)
     assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    for k in range(0, len(ref["events"]), max(1, len(ref["events"]) // 40)):   # update sums of the run itself
+        assert rel_err(gpu["U"][k], ref["U"][k]) <= 1e-4, k
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
         worst = max(check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
-                    for e in ref["events"])
+                    for e in ref["events"][::max(1, len(ref["events"]) // 60)])
     assert worst <= U_TOL
 
 
