@@ -5,18 +5,19 @@
 // g = mean gradient (+ lambda W); w_c -= eta_i * g; U_i += g.  One cluster of
 // four CTAs runs one round-task.  CTA r owns input rows [196 r, 196 r + 196) of
 // W0 - in its shared memory from the first iteration to the trigger - and the
-// same slice of U0 in registers.  The small parameters (b0, W1, b1) and their
-// update sums are kept by every CTA, identically: all four run the narrow part
-// of the network on the same numbers in the same order.  Nothing of the model
-// touches global memory between the start of the round and the trigger.
-// Per SGD iteration:
-//   forward   hp = X[:, rows_r] W0[rows_r, :]        (K split over the CTAs, and four ways inside one)
-//     cluster barrier A (hardware, blocking): every CTA's partial is in place
-//             h = relu(b0 + sum_q hp_q)              (all 128 columns, peers' partials over DSMEM)
-//     cluster barrier B, arrive only: "I have read my peers' partials"; its wait
-//             sits just before hp is written again, one iteration later
-//             z = b1 + h W1; dZ1 = (softmax(z) - onehot) / B; dZ0 = (dZ1 W1^T) * relu'
-//             W1, b1: gradient, update, update sum
+// same slice of U0 in registers; it also owns hidden columns [32 r, 32 r + 32):
+// their bias, their rows of W1 and the matching update sums.  Nothing of the
+// model touches global memory between the start of the round and the trigger.
+// Per SGD iteration (three hardware cluster barriers, no polling):
+//   forward   hp = X[:, rows_r] W0[rows_r, :]                      (K split over the CTAs)
+//     barrier 1
+//             h[:, cols_r] = relu(b0 + sum_q hp_q[:, cols_r])      (peers' partials over DSMEM)
+//             z1p = h[:, cols_r] W1[cols_r, :]
+//     barrier 2
+//             z = b1 + sum_q z1p_q; dZ1 = (softmax(z) - onehot) / B (every CTA, identically)
+//             dZ0[:, cols_r] = (dZ1 W1[cols_r, :]^T) * relu'        -> pushed into all four CTAs
+//             W1[cols_r, :], b1: gradient, update, update sum
+//     barrier 3
 //   backward  G = X[:, rows_r]^T dZ0; W0 -= eta (G + lambda W0); U0 += ...   (registers + shared memory)
 // The minibatch rows (this CTA's 196 columns of each) arrive by cp.async.bulk,
 // one iteration ahead, completion on an mbarrier with a bounded wait.  A wait
@@ -38,26 +39,26 @@ constexpr int kR = kD0 / kCL;        // 196 input rows per CTA
 constexpr int kHS = kH / kCL;        // 32 hidden columns per CTA
 constexpr int kRW = 14;              // rows of the gradient tile per warp; 14 warps x 14 rows = 196
 constexpr int kGW = kR / kRW;        // warps that own a tile of W0 / U0
-constexpr int kKQ = 48;              // the forward product splits K four ways inside the CTA: 48 + 48 + 48 + 52 rows
+constexpr int kKH = 100;             // the forward product splits K once more inside the CTA: rows [0,100) and [100,196)
 constexpr uint32_t kWaitLimit = 1u << 22;
 static_assert(kGW * kRW == kR && kGW + 2 <= kT / 32, "gradient tiling: two warps stay free for the bias and the row copies");
-static_assert(kKQ % 4 == 0 && (kR - 3 * kKQ) % 4 == 0, "forward K split");
+static_assert(kKH % 4 == 0 && (kR - kKH) % 4 == 0, "forward K split");
 
 struct __align__(128) ResSmem {
   float W0[kR][kH];        // this CTA's rows of W0, current
   float xs[2][kB][kR];     // this CTA's columns of the minibatch rows, double-buffered
   float hp[kB][kH];        // partial pre-activations from this CTA's K slice (read by the peers)
-  float hf[kB][kH];        // activations, all columns; scratch inside the forward product
-  float dz0[kB][kH];       // dZ0, all columns; scratch inside the forward product
-  float W1[kH][kCP];       // columns >= C stay zero
-  float U1[kH][kCP];
-  float z1q[4][kB][kCP];   // logits, partial over a quarter of the hidden columns
+  float dz0[kB][kH];       // dZ0, every CTA's columns (written by the peers); scratch inside the forward product
+  float hs[kB][kHS + 1];   // activations of the owned hidden columns
+  float W1[kHS][kCP];      // owned rows of W1 (columns >= C stay zero)
+  float U1[kHS][kCP];
+  float z1p[kB][kCP];      // partial logits from the owned hidden columns (read by the peers)
+  float z1[kB][kCP];       // logits
   float dz1[kB][kCP];
-  float b0[kH], Ub0[kH], b1[kCP], Ub1[kCP];
+  float b0[kHS], Ub0[kHS], b1[kCP], Ub1[kCP];
   int ys[2][kB];
   uint64_t full[2], wbar;
 };
-static_assert(sizeof(ResSmem) <= 227 * 1024, "shared memory of one CTA");
 
 __device__ __forceinline__ uint32_t saddr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -94,11 +95,17 @@ __device__ __forceinline__ float4 ld_peer4(uint32_t a) {
   asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
   return v;
 }
+__device__ __forceinline__ float ld_peer(uint32_t a) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_peer(uint32_t a, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
 __device__ __forceinline__ void cluster_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -151,12 +158,12 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
     }
     return w;
   };
-  for (int e = tid; e < kH * kCP; e += kT) {
-    const int j = e / kCP, c = e % kCP;
-    sm.W1[j][c] = c < C ? start_value(woff1 + (size_t)j * C + c) : 0.f;
-    sm.U1[j][c] = 0.f;
+  for (int e = tid; e < kHS * kCP; e += kT) {
+    const int jl = e / kCP, c = e % kCP;
+    sm.W1[jl][c] = c < C ? start_value(woff1 + (size_t)(rank * kHS + jl) * C + c) : 0.f;
+    sm.U1[jl][c] = 0.f;
   }
-  if (tid < kH) { sm.b0[tid] = start_value(boff0 + tid); sm.Ub0[tid] = 0.f; }
+  if (tid < kHS) { sm.b0[tid] = start_value(boff0 + rank * kHS + tid); sm.Ub0[tid] = 0.f; }
   if (tid < kCP) { sm.b1[tid] = tid < C ? start_value(boff1 + tid) : 0.f; sm.Ub1[tid] = 0.f; }
   bool ok = mbar_wait(&sm.wbar, 0);
   for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
@@ -180,8 +187,8 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
   __syncthreads();
   cluster_barrier();   // every CTA of the cluster is set up before any of them is written to
 
-  // forward-product roles: K quarter, 8 batch rows, 4 hidden columns
-  const int kq = tid >> 7, t3 = tid & 127, bt = t3 >> 5, jt = t3 & 31;
+  // forward-product roles: K half, 4 batch rows, 4 hidden columns
+  const int half = tid >> 8, t2 = tid & 255, bt = t2 >> 5, jt = t2 & 31;
   uint32_t h = 0;   // local sample counter of Algorithm 3
 
   for (uint32_t it = 0; it < t.steps; ++it) {
@@ -190,15 +197,15 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
 
     // ---------------- forward: hp = X[:, rows] W0[rows, :] ----------------
     {
-      float acc[8][4];
+      float acc[4][4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-      const float* xb = &sm.xs[buf][8 * bt][kKQ * kq];
-      const float* wb = &sm.W0[kKQ * kq][4 * jt];
-      const int kn = kq == 3 ? kR - 3 * kKQ : kKQ;
-#pragma unroll 1
+      const float* xb = &sm.xs[buf][4 * bt][kKH * half];
+      const float* wb = &sm.W0[kKH * half][4 * jt];
+      const int kn = half ? kR - kKH : kKH;
+#pragma unroll 4
       for (int k = 0; k < kn; k += 4) {
         float w[4][4];
 #pragma unroll
@@ -207,88 +214,67 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
           w[q][0] = v.x; w[q][1] = v.y; w[q][2] = v.z; w[q][3] = v.w;
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {
           const float4 x = *reinterpret_cast<const float4*>(xb + i * kR + k);
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             acc[i][j] = fmaf(x.w, w[3][j], fmaf(x.z, w[2][j], fmaf(x.y, w[1][j], fmaf(x.x, w[0][j], acc[i][j]))));
         }
       }
-      // the four K quarters meet in two steps; hf and dz0 are nobody's yet in this iteration
-      float4* s1 = reinterpret_cast<float4*>(&sm.dz0[0][0]);
-      float4* s2 = reinterpret_cast<float4*>(&sm.hf[0][0]);
-      if (kq & 1) {
-        float4* dst = kq == 1 ? s1 : s2;
+      float4* scratch = reinterpret_cast<float4*>(&sm.dz0[0][0]);   // free until the peers pass barrier 2
+      if (half == 1) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) dst[i * 128 + t3] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        for (int i = 0; i < 4; ++i) scratch[i * 256 + t2] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
       }
       __syncthreads();
-      if (!(kq & 1)) {
-        const float4* src = kq == 0 ? s1 : s2;
+      if (half == 0) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float4 o = src[i * 128 + t3];
-          acc[i][0] += o.x; acc[i][1] += o.y; acc[i][2] += o.z; acc[i][3] += o.w;
-        }
-        if (kq == 2) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) s2[i * 128 + t3] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-        }
-      }
-      __syncthreads();
-      if (it) cluster_wait();   // B of the previous iteration: every peer has read the old hp
-      if (kq == 0) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float4 o = s2[i * 128 + t3];
-          *reinterpret_cast<float4*>(&sm.hp[8 * bt + i][4 * jt]) =
+        for (int i = 0; i < 4; ++i) {
+          const float4 o = scratch[i * 256 + t2];
+          *reinterpret_cast<float4*>(&sm.hp[4 * bt + i][4 * jt]) =
               make_float4(acc[i][0] + o.x, acc[i][1] + o.y, acc[i][2] + o.z, acc[i][3] + o.w);
         }
       }
     }
-    cluster_barrier();   // A: every CTA's partial pre-activations are in place
-    __syncthreads();     // ... and this CTA is done with its forward scratch
+    cluster_barrier();   // 1: every CTA's partial pre-activations are in place
 
-    // every hidden column: bias + the four partials (same order in every CTA), ReLU
-#pragma unroll
-    for (int u = 0; u < kB * kH / 4 / kT; ++u) {
-      const int e = tid + u * kT, b = e >> 5, j4 = (e & 31) * 4;
-      const uint32_t a = saddr(&sm.hp[b][j4]);
-      float4 z = *reinterpret_cast<const float4*>(&sm.b0[j4]);
+    // owned hidden columns: bias + the four partials, ReLU
+    if (tid < kB * kHS / 4) {
+      const int b = tid >> 3, j4 = (tid & 7) * 4;
+      const uint32_t a = saddr(&sm.hp[b][rank * kHS + j4]);
+      float4 z = make_float4(sm.b0[j4], sm.b0[j4 + 1], sm.b0[j4 + 2], sm.b0[j4 + 3]);
 #pragma unroll
       for (int q = 0; q < kCL; ++q) {
         const float4 v = ld_peer4(peer(a, q));
         z.x += v.x; z.y += v.y; z.z += v.z; z.w += v.w;
       }
-      *reinterpret_cast<float4*>(&sm.hf[b][j4]) = make_float4(fmaxf(z.x, 0.f), fmaxf(z.y, 0.f), fmaxf(z.z, 0.f), fmaxf(z.w, 0.f));
+      sm.hs[b][j4] = fmaxf(z.x, 0.f); sm.hs[b][j4 + 1] = fmaxf(z.y, 0.f);
+      sm.hs[b][j4 + 2] = fmaxf(z.z, 0.f); sm.hs[b][j4 + 3] = fmaxf(z.w, 0.f);
     }
-    cluster_arrive();    // B: this CTA has read its peers' partials (the wait is in the next forward pass)
     __syncthreads();
-    if (tid < kB * kCP) {   // logits, partial over a quarter of the hidden columns: 4 classes x 32 columns per thread
-      const int b = tid / kCP, r = tid % kCP, c4 = (r % 3) * 4, jq = r / 3;
-      float z[4] = {0.f, 0.f, 0.f, 0.f};
+    if (tid < kB * kCP) {   // partial logits from the owned columns
+      const int b = tid / kCP, c = tid % kCP;
+      float s = 0.f;
 #pragma unroll 8
-      for (int j = jq * 32; j < jq * 32 + 32; ++j) {
-        const float a = sm.hf[b][j];
-        const float4 w = *reinterpret_cast<const float4*>(&sm.W1[j][c4]);
-        z[0] = fmaf(a, w.x, z[0]); z[1] = fmaf(a, w.y, z[1]); z[2] = fmaf(a, w.z, z[2]); z[3] = fmaf(a, w.w, z[3]);
-      }
-      *reinterpret_cast<float4*>(&sm.z1q[jq][b][c4]) = make_float4(z[0], z[1], z[2], z[3]);
+      for (int jl = 0; jl < kHS; ++jl) s = fmaf(sm.hs[b][jl], sm.W1[jl][c], s);
+      sm.z1p[b][c] = s;
+    }
+    cluster_barrier();   // 2: every CTA's partial logits are in place; dz0 is no longer anybody's scratch
+
+    if (tid < kB * kCP) {
+      const int b = tid / kCP, c = tid % kCP;
+      const uint32_t a = saddr(&sm.z1p[b][c]);
+      float z = sm.b1[c];
+#pragma unroll
+      for (int q = 0; q < kCL; ++q) z += ld_peer(peer(a, q));
+      sm.z1[b][c] = z;
     }
     __syncthreads();
     if (tid < kB * kCP) {   // softmax cross-entropy: dZ1 = (p - onehot(y)) / B; every thread sums its sample's row itself
       const int b = tid / kCP, c = tid % kCP;
-      float z[kCP];
-#pragma unroll
-      for (int k4 = 0; k4 < kCP; k4 += 4) {
-        float4 v = *reinterpret_cast<const float4*>(&sm.b1[k4]);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float4 o = *reinterpret_cast<const float4*>(&sm.z1q[q][b][k4]);
-          v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-        }
-        z[k4] = v.x; z[k4 + 1] = v.y; z[k4 + 2] = v.z; z[k4 + 3] = v.w;
-      }
+      const float4 r0 = *reinterpret_cast<const float4*>(&sm.z1[b][0]), r1 = *reinterpret_cast<const float4*>(&sm.z1[b][4]),
+                   r2 = *reinterpret_cast<const float4*>(&sm.z1[b][8]);
+      const float z[kCP] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w, r2.x, r2.y, r2.z, r2.w};
       float m = -INFINITY;
 #pragma unroll
       for (int k = 0; k < kCP; ++k) m = k < C ? fmaxf(m, z[k]) : m;
@@ -302,48 +288,36 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
       sm.dz1[b][c] = c < C ? (mine / sum - (c == sm.ys[buf][b] ? 1.f : 0.f)) * invB : 0.f;
     }
     __syncthreads();
-    {   // dZ0 = (dZ1 W1^T) * relu'(h): one sample, 8 columns per thread
-      const int b = tid >> 4, j0 = (tid & 15) * 8;
-      const float4 d0 = *reinterpret_cast<const float4*>(&sm.dz1[b][0]), d1 = *reinterpret_cast<const float4*>(&sm.dz1[b][4]),
-                   d2 = *reinterpret_cast<const float4*>(&sm.dz1[b][8]);
-      float v[8];
+    // dZ0 for the owned columns, into every CTA of the cluster
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float4 w0 = *reinterpret_cast<const float4*>(&sm.W1[j0 + i][0]), w1 = *reinterpret_cast<const float4*>(&sm.W1[j0 + i][4]),
-                     w2 = *reinterpret_cast<const float4*>(&sm.W1[j0 + i][8]);
-        float sacc = d0.x * w0.x;
-        sacc = fmaf(d0.y, w0.y, sacc); sacc = fmaf(d0.z, w0.z, sacc); sacc = fmaf(d0.w, w0.w, sacc);
-        sacc = fmaf(d1.x, w1.x, sacc); sacc = fmaf(d1.y, w1.y, sacc); sacc = fmaf(d1.z, w1.z, sacc); sacc = fmaf(d1.w, w1.w, sacc);
-        sacc = fmaf(d2.x, w2.x, sacc); sacc = fmaf(d2.y, w2.y, sacc); sacc = fmaf(d2.z, w2.z, sacc); sacc = fmaf(d2.w, w2.w, sacc);
-        v[i] = sm.hf[b][j0 + i] > 0.f ? sacc : 0.f;
-      }
-      *reinterpret_cast<float4*>(&sm.dz0[b][j0]) = make_float4(v[0], v[1], v[2], v[3]);
-      *reinterpret_cast<float4*>(&sm.dz0[b][j0 + 4]) = make_float4(v[4], v[5], v[6], v[7]);
+    for (int u = 0; u < kB * kHS / kT; ++u) {
+      const int e = tid + u * kT, b = e >> 5, jl = e & 31;
+      float s = 0.f;
+#pragma unroll
+      for (int c = 0; c < kCP; ++c) s = fmaf(sm.dz1[b][c], sm.W1[jl][c], s);
+      const float v = sm.hs[b][jl] > 0.f ? s : 0.f;
+      const uint32_t a = saddr(&sm.dz0[b][rank * kHS + jl]);
+#pragma unroll
+      for (int q = 0; q < kCL; ++q) st_peer(peer(a, q), v);
     }
-    __syncthreads();   // W1 has been read by everybody; dZ0 is complete
-    if (tid < kH * 3) {   // W1: one hidden column, 4 classes per thread
-      const int j = tid / 3, c4 = (tid % 3) * 4;
-      float g[4] = {0.f, 0.f, 0.f, 0.f};
+    __syncthreads();   // W1 has been read by everybody
+    if (tid < kHS * kCP) {   // W1 rows of the owned columns
+      const int jl = tid / kCP, c = tid % kCP;
+      float g = 0.f;
 #pragma unroll 8
-      for (int b = 0; b < kB; ++b) {
-        const float a = sm.hf[b][j];
-        const float4 d = *reinterpret_cast<const float4*>(&sm.dz1[b][c4]);
-        g[0] = fmaf(a, d.x, g[0]); g[1] = fmaf(a, d.y, g[1]); g[2] = fmaf(a, d.z, g[2]); g[3] = fmaf(a, d.w, g[3]);
-      }
-      float4 w = *reinterpret_cast<const float4*>(&sm.W1[j][c4]);
-      float4 uu = *reinterpret_cast<const float4*>(&sm.U1[j][c4]);
-      g[0] = fmaf(lambda, w.x, g[0]); g[1] = fmaf(lambda, w.y, g[1]); g[2] = fmaf(lambda, w.z, g[2]); g[3] = fmaf(lambda, w.w, g[3]);
-      w.x = fmaf(-eta, g[0], w.x); w.y = fmaf(-eta, g[1], w.y); w.z = fmaf(-eta, g[2], w.z); w.w = fmaf(-eta, g[3], w.w);
-      uu.x += g[0]; uu.y += g[1]; uu.z += g[2]; uu.w += g[3];
-      *reinterpret_cast<float4*>(&sm.W1[j][c4]) = w;
-      *reinterpret_cast<float4*>(&sm.U1[j][c4]) = uu;
-    } else if (tid < kH * 3 + kCP) {   // b1
-      const int c = tid - kH * 3;
+      for (int b = 0; b < kB; ++b) g = fmaf(sm.hs[b][jl], sm.dz1[b][c], g);
+      const float w = sm.W1[jl][c];
+      g = fmaf(lambda, w, g);
+      sm.W1[jl][c] = fmaf(-eta, g, w);
+      sm.U1[jl][c] += g;
+    } else if (tid < kHS * kCP + kCP) {   // b1: every CTA keeps its own, identical copy
+      const int c = tid - kHS * kCP;
       float g = 0.f;
       for (int b = 0; b < kB; ++b) g += sm.dz1[b][c];
       sm.b1[c] = fmaf(-eta, g, sm.b1[c]);
       sm.Ub1[c] += g;
     }
+    cluster_barrier();   // 3: dZ0 is complete in every CTA
 
     // ---------------- backward: G = X[:, rows]^T dZ0, update of W0 and U0 ----------------
     if (warp < kGW) {
@@ -389,24 +363,15 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
     } else if (warp == kT / 32 - 1) {
       // the next minibatch; its buffer was last read before the previous trip's closing barrier
       if (it + 1 < t.steps) sm.ys[buf ^ 1][lane] = issue_rows(it + 1, buf ^ 1);
-    } else if (warp == kGW) {   // b0: four columns per lane
-      float g[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-      for (int b = 0; b < kB; ++b) {
-        const float4 d = *reinterpret_cast<const float4*>(&sm.dz0[b][4 * lane]);
-        g[0] += d.x; g[1] += d.y; g[2] += d.z; g[3] += d.w;
-      }
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        sm.b0[4 * lane + j] = fmaf(-eta, g[j], sm.b0[4 * lane + j]);
-        sm.Ub0[4 * lane + j] += g[j];
-      }
+    } else if (warp == kGW) {   // b0 of the owned columns
+      float g = 0.f;
+      for (int b = 0; b < kB; ++b) g += sm.dz0[b][rank * kHS + lane];
+      sm.b0[lane] = fmaf(-eta, g, sm.b0[lane]);
+      sm.Ub0[lane] += g;
     }
     h += kB;
     __syncthreads();   // W0 and b0 updated; the row buffer may be refilled
   }
-
-  if (t.steps) cluster_wait();   // the last iteration's B
 
   if (!ok) {
     // A bulk copy never completed.  Report it; give what may still be in flight a
@@ -430,16 +395,15 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
         if (Wend) *reinterpret_cast<float4*>(Wend + o) = *reinterpret_cast<const float4*>(&sm.W0[warp * kRW + i][4 * lane]);
       }
     }
-    for (int e = tid; e < kHS * C; e += kT) {   // the small parameters are identical in all four CTAs: each writes a quarter
-      const int j = rank * kHS + e / C, c = e % C;
-      const size_t o = woff1 + (size_t)j * C + c;
-      Urow[o] = sm.U1[j][c];
-      if (Wend) Wend[o] = sm.W1[j][c];
+    for (int e = tid; e < kHS * C; e += kT) {
+      const int jl = e / C, c = e % C;
+      const size_t o = woff1 + (size_t)(rank * kHS + jl) * C + c;
+      Urow[o] = sm.U1[jl][c];
+      if (Wend) Wend[o] = sm.W1[jl][c];
     }
     if (tid < kHS) {
-      const int j = rank * kHS + tid;
-      Urow[boff0 + j] = sm.Ub0[j];
-      if (Wend) Wend[boff0 + j] = sm.b0[j];
+      Urow[boff0 + rank * kHS + tid] = sm.Ub0[tid];
+      if (Wend) Wend[boff0 + rank * kHS + tid] = sm.b0[tid];
     }
     if (rank == 0 && tid < C) {
       Urow[boff1 + tid] = sm.Ub1[tid];

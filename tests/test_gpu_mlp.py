@@ -39,6 +39,7 @@ def test_mlp_fp32_small_end_to_end_and_round_U():
     dict(n_clients=40, n_rounds=2, data=dict(total=1600)),              # cluster size 2
     dict(n_clients=2, n_rounds=3, data=dict(total=400)),                # cluster size 8
     dict(l2=1e-3, n_rounds=3),                                          # resident 784-128-10 kernel with the l2 term
+    dict(dims=[784, 128, 12], n_rounds=3),                              # ... with all 12 class columns in use
     dict(n_clients=2, n_rounds=5, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=500.0,
          data=dict(total=400)),                                         # ... with own update sums in flight at round start
 ])
