@@ -523,16 +523,29 @@ __device__ __forceinline__ int bfly_index4(int lane, int i) {
 }
 __device__ __forceinline__ constexpr int pair_index(int s, int t) { return t * (t - 1) / 2 + s; }  // s < t
 
-__global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
+// kDed: two more warps that own no pixels.  Warp 4 runs R and hands each delta_t to the four
+// pixel warps through a hardware named barrier of its own, so that P3 streams under R instead
+// of following it; warps 5 and 6 compute the Gram matrix of the next block, warp 7 issues the row
+// copies (fetching their labels stalls it for an HBM round trip).  255 registers x 256 threads leave room for one such CTA per SM: the variant for launches
+// with at most one round-task per SM, where a round-task's latency is all that counts.
+__device__ __forceinline__ void named_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void named_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+
+template <bool kDed>
+__global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) lr_block_kernel(RoundLaunch p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   BlkSmem& sm = *reinterpret_cast<BlkSmem*>(smem_raw);
+  constexpr int kHand = kThreads + 32;                    // threads meeting at a delta hand-over: pixel warps + R warp
+  constexpr int kGramRanks = kDed ? 2 : kWarps - 1;       // warps sharing the Gram matrix of a block
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool rw = kDed && warp >= kWarps;            // the warps without pixels: R (warp 4), Gram and row copies (warp 5)
+  const bool gw = kDed && (warp == kWarps + 1 || warp == kWarps + 2);   // warps 5 and 6
   const int cg = lane & 1, pl = lane >> 1;
-  const bool active = pl < kPl;
+  const bool active = !rw && pl < kPl;
   const bool is_bias = warp == kWarps - 1 && pl == kPl;
-  const int pg = warp * kPl + (active ? pl : 0);     // pixel group: pixels 14 pg .. 14 pg + 13
+  const int pg = rw ? 0 : warp * kPl + (active ? pl : 0);     // pixel group: pixels 14 pg .. 14 pg + 13
 
   const ClientData cd = p.clients[t.client];
   const uint64_t key = p.sample_keys[t.client];
@@ -638,7 +651,8 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     float gacc[kPairs];
 #pragma unroll
     for (int i = 0; i < kPairs; ++i) gacc[i] = 0.f;
-    for (int chunk = r; chunk * 32 < kD; chunk += 3) {
+#pragma unroll 2
+    for (int chunk = r; chunk * 32 < kD; chunk += kGramRanks) {
       const int px = chunk * 32 + lane;
       if (px < kD) {
         float x[kM];
@@ -652,16 +666,17 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     }
     float o[1];
     bfly_reduce5<kPairs>(gacc, o, lane);
-    if (gidx >= 0) sm.partG[kb & 1][warp][gidx] = o[0];
+    if (gidx >= 0) sm.partG[kb & 1][kDed ? r : warp][gidx] = o[0];
   };
 
   bool timed_out = false;
   uint32_t timeout_at = 0;
 
-  // Gram matrix of block 0: warps 0..2 (the rotation below treats warp 3 as busy before block 0)
-  if (warp != kWarps - 1) {
+  // Gram matrix of block 0: warps 0..2 (the rotation below treats warp 3 as busy before block 0),
+  // or the Gram warp alone
+  if (kDed ? gw : warp != kWarps - 1) {
     ok = mbar_wait(&sm.full[0], 0) && ok;
-    gram_partial(0, warp);
+    gram_partial(0, kDed ? warp - (kWarps + 1) : warp);
   }
 
   for (uint32_t k = 0; k < nblk; ++k) {
@@ -671,7 +686,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     const float* xslot = xbase + (size_t)slot * kM * rs;
 
     // ---- P1: W = W_start - eta U; this thread's share of Z0 = W X ----
-    {
+    if (!rw) {
       float acc[kM][kCh];
 #pragma unroll
       for (int a2 = 0; a2 < kPx / 2; ++a2) {
@@ -706,7 +721,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
     // also carries the verdict of the bounded waits so that all threads leave together
     if (__syncthreads_or(!ok)) { timed_out = true; timeout_at = k; break; }
 
-    const int rwarp = k & (kWarps - 1);
+    const int rwarp = kDed ? kWarps : (int)(k & (kWarps - 1));
     if (warp == rwarp) {
       // ---- R: the block's kM dependent softmax steps, lane j owns sample j ----
       const int j = lane & (kM - 1);
@@ -726,14 +741,14 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
       // column j of the Gram matrix, one entry per step: -eta * G[s][j] for s < j, 0 for
       // the others (a finished sample takes no correction); the warp that ran R for block
       // k-1 has no share in the Gram partials.  Loaded one step ahead of its use.
-      const int skip = (k + kWarps - 1) & (kWarps - 1);
+      const int skip = kDed ? kWarps : (int)((k + kWarps - 1) & (kWarps - 1));
       const float* g0 = sm.partG[k & 1][skip == 0 ? 1 : 0];
       const float* g1 = sm.partG[k & 1][skip <= 1 ? 2 : 1];
       const float* g2 = sm.partG[k & 1][skip <= 2 ? 3 : 2];
       const int gbase = j * (j - 1) / 2;
       auto corr = [&](int s) -> float {
         const int idx = s < j ? gbase + s : 0;
-        const float gsum = (1.f + g0[idx]) + (g1[idx] + g2[idx]);   // 1 = the bias "pixel"
+        const float gsum = kDed ? (1.f + g0[idx]) + g1[idx] : (1.f + g0[idx]) + (g1[idx] + g2[idx]);   // 1 = the bias "pixel"
         return s < j ? gsum * neta : 0.f;
       };
       const int y = sm.ys[slot][j];
@@ -763,32 +778,41 @@ __global__ void __launch_bounds__(kThreads, 2) lr_block_kernel(RoundLaunch p) {
           dq[2] = make_float4(d[5], d[6], d[7], d[8]);
           dq[3] = make_float4(d[9], 0.f, 0.f, 0.f);
         }
+        if (kDed) named_arrive(1 + s, kHand);   // delta_s is out: the pixel warps may apply it
 #pragma unroll
         for (int c = 0; c < kC; ++c) z[c] = fmaf(__shfl_sync(0xffffffffu, d[c], s), gs, z[c]);
         gs = gnext;
       }
     } else {
-      const int rank = ((warp - rwarp) & (kWarps - 1)) - 1;   // 0..2 among the three other warps
-      if (rank == 0 && k + 2 < nblk) produce(k + 2);          // its slot held block k-1: free since barrier A
-      if (k + 1 < nblk) {
+      // 0..2 among the three other warps; kDed: the Gram warp alone does this part
+      const int rank = kDed ? warp - (kWarps + 1) : ((warp - rwarp) & (kWarps - 1)) - 1;
+      const bool producer = kDed ? warp == kWarps + 3 : rank == 0;
+      // block k+2's slot held block k-1: free since barrier A.  The copies' labels take an HBM round
+      // trip, so the Gram warps (whose result R needs at the next barrier) fetch after their share.
+      if (!kDed && producer && k + 2 < nblk) produce(k + 2);
+      if ((!kDed || gw) && k + 1 < nblk) {
         ok = mbar_wait(&sm.full[(k + 1) % kSlots], ((k + 1) / kSlots) & 1) && ok;
         gram_partial(k + 1, rank);
       }
+      if (kDed && producer && k + 2 < nblk) produce(k + 2);
     }
-    __syncthreads();   // barrier B: delta of the block is in shared memory
+    if (!kDed) __syncthreads();   // barrier B: delta of the block is in shared memory
 
     // ---- P3: U += delta_t x_t^T (two samples per trip: the loop has to stay small, see R) ----
+    if (!rw) {
 #pragma unroll 2
-    for (int s = 0; s < (int)nv; ++s) {
-      const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
-      const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, sm.dbuf[s][cg * 8 + 4]};
+      for (int s = 0; s < (int)nv; ++s) {
+        if (kDed) named_sync(1 + s, kHand);   // delta_s has been written
+        const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
+        const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, sm.dbuf[s][cg * 8 + 4]};
 #pragma unroll
-      for (int a2 = 0; a2 < kPx / 2; ++a2) {
-        const float2 x = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
+        for (int a2 = 0; a2 < kPx / 2; ++a2) {
+          const float2 x = *reinterpret_cast<const float2*>(xslot + s * rs + 2 * a2);
 #pragma unroll
-        for (int c = 0; c < kCh; ++c) {
-          U[2 * a2][c] = fmaf(x.x, d[c], U[2 * a2][c]);
-          U[2 * a2 + 1][c] = fmaf(x.y, d[c], U[2 * a2 + 1][c]);
+          for (int c = 0; c < kCh; ++c) {
+            U[2 * a2][c] = fmaf(x.x, d[c], U[2 * a2][c]);
+            U[2 * a2 + 1][c] = fmaf(x.y, d[c], U[2 * a2 + 1][c]);
+          }
         }
       }
     }
@@ -859,20 +883,28 @@ cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s) {
   if (p.l2 == 0.f) {
     // more than 48 KB of shared memory has to be asked for once per device
     static bool opted_in[64] = {};
+    static int sm_count[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !opted_in[dev]) {
-      e = cudaFuncSetAttribute(lr_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BlkSmem));
+    const bool known = dev >= 0 && dev < 64;
+    int sms = known ? sm_count[dev] : 0;
+    if (!known || !opted_in[dev]) {
+      e = cudaFuncSetAttribute(lr_block_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BlkSmem));
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(lr_block_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BlkSmem));
+      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
       if (e != cudaSuccess) return e;
-      if (dev >= 0 && dev < 64) opted_in[dev] = true;
+      if (known) { opted_in[dev] = true; sm_count[dev] = sms; }
     }
+    // At most one round-task per SM: the variant with a warp of its own for the softmax recurrence.
+    const bool dedicated = p.n_tasks <= (uint32_t)sms;
     // Programmatic stream serialisation: the grid may start while the kernel before it in the
     // stream (the aggregation of the previous wave) is still running; lr_block_kernel waits
     // (griddepcontrol.wait) before it reads anything that kernel writes.
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(p.n_tasks, 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(dedicated ? 2 * kThreads : kThreads, 1, 1);
     cfg.dynamicSmemBytes = sizeof(BlkSmem);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -880,7 +912,7 @@ cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, lr_block_kernel, p);
+    return dedicated ? cudaLaunchKernelEx(&cfg, lr_block_kernel<true>, p) : cudaLaunchKernelEx(&cfg, lr_block_kernel<false>, p);
   }
   // lambda != 0 couples the steps of a block through the decay of W: step by step.
   // Enough round-tasks to put two CTAs on every SM: trade latency for instruction count.
