@@ -799,10 +799,9 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
     if (!kDed) __syncthreads();   // barrier B: delta of the block is in shared memory
 
     // ---- P3: U += delta_t x_t^T (two samples per trip: the loop has to stay small, see R) ----
-    if (!rw) {
+    if (!rw && !kDed) {
 #pragma unroll 2
       for (int s = 0; s < (int)nv; ++s) {
-        if (kDed) named_sync(1 + s, kHand);   // delta_s has been written
         const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
         const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, sm.dbuf[s][cg * 8 + 4]};
 #pragma unroll
@@ -813,6 +812,31 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
             U[2 * a2][c] = fmaf(x.x, d[c], U[2 * a2][c]);
             U[2 * a2 + 1][c] = fmaf(x.y, d[c], U[2 * a2 + 1][c]);
           }
+        }
+      }
+    }
+    if (!rw && kDed) {
+      // streaming under R: a sample's pixels are fetched before the wait for its delta
+      float2 x[kPx / 2];
+#pragma unroll
+      for (int a2 = 0; a2 < kPx / 2; ++a2) x[a2] = *reinterpret_cast<const float2*>(xslot + 2 * a2);
+#pragma unroll 1
+      for (int s = 0; s < (int)nv; ++s) {
+        named_sync(1 + s, kHand);   // delta_s has been written
+        const float4 dq = *reinterpret_cast<const float4*>(&sm.dbuf[s][cg * 8]);
+        const float d[kCh] = {dq.x, dq.y, dq.z, dq.w, sm.dbuf[s][cg * 8 + 4]};
+        float2 xn[kPx / 2];
+        const int sn = s + 1 < kM ? s + 1 : s;
+#pragma unroll
+        for (int a2 = 0; a2 < kPx / 2; ++a2) xn[a2] = *reinterpret_cast<const float2*>(xslot + sn * rs + 2 * a2);
+#pragma unroll
+        for (int a2 = 0; a2 < kPx / 2; ++a2) {
+#pragma unroll
+          for (int c = 0; c < kCh; ++c) {
+            U[2 * a2][c] = fmaf(x[a2].x, d[c], U[2 * a2][c]);
+            U[2 * a2 + 1][c] = fmaf(x[a2].y, d[c], U[2 * a2 + 1][c]);
+          }
+          x[a2] = xn[a2];
         }
       }
     }
