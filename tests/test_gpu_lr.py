@@ -162,6 +162,18 @@ def test_two_runs_are_bit_identical_and_reset_replays():
     assert all(u.tobytes() == v.tobytes() for u, v in zip(a["U"], run_gpu(cfg, data, w0)["U"]))
 
 
+@pytest.mark.parametrize("n_clients", [6, 330])
+def test_blocked_kernel_runs_are_bit_identical(n_clients):
+    # 6 clients: the 8-warp instance (one round-task per SM); 330: the 4-warp instance, two CTAs per SM
+    cfg = workloads.get_config("cfg1", l2=0.0, n_clients=n_clients, n_rounds=4, sched_a=5, sched_b=3,
+                               data=dict(per_client=64))
+    data, w0 = make(cfg)
+    a = run_gpu(cfg, data, w0)
+    b = run_gpu(cfg, data, w0)
+    assert a["w"].tobytes() == b["w"].tobytes() and a["blob"] == b["blob"]
+    assert all(u.tobytes() == v.tobytes() for u, v in zip(a["U"], b["U"]))
+
+
 def test_run_in_two_calls_matches_the_checker_continued():
     cfg = workloads.get_config("cfg1")
     data, w0 = make(cfg)
