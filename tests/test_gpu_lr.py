@@ -133,6 +133,23 @@ def test_blocked_kernel_variants_without_l2(over):
     assert worst <= U_TOL
 
 
+@pytest.mark.parametrize("l2", [0.0, 1e-4])
+def test_the_papers_schedule_shape_end_to_end(l2):
+    # Table 2 / Appendix A.2 of the paper: five nodes, s_i = 10 i counted from round 1, eta_0 = 0.01 with
+    # beta = 0.01 (step size constant within a round), d = 1; 12 rounds here instead of 110
+    cfg = workloads.get_config("cfg1", n_clients=5, sched_a=10, sched_b=0, round_base=1, n_rounds=12, lr=0.01,
+                               lr_beta=0.01, l2=l2, max_lag_d=1, data=dict(per_client=400))
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    assert [e["samples"] for e in ref["events"] if e["client"] == 0] == [10 * i for i in range(1, 13)]
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for e in ref["events"][::7]:
+            check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
+
+
 def test_many_own_updates_in_flight():
     # a slow network keeps several of a client's own sums in flight at round start
     cfg = workloads.get_config("cfg1", n_clients=2, n_rounds=6, max_lag_d=workloads.NEVER_WAIT,
