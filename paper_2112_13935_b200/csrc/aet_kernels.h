@@ -41,7 +41,9 @@ struct RoundLaunch {
 // One CTA waits (at most max_polls polls) on a barrier nobody signals, then sets bit 0 of *status.
 cudaError_t launch_wait_probe(uint32_t* status, uint32_t max_polls, cudaStream_t s);
 
-// Softmax regression 784 -> 10, batch 1: one CTA per round-task.
+// Softmax regression 784 -> 10, batch 1: one CTA per round-task; the kernel is picked by lambda and by
+// how many round-tasks the launch holds.  Asynchronous on s; may start under the tail of the previous kernel in s
+// (programmatic stream serialisation) and waits on the device before reading that kernel's output.
 cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s);
 
 struct MlpShape {

@@ -6,7 +6,12 @@
 // the running update sum stay in registers for the whole round and only the
 // sampled rows stream in from HBM.
 //
-// Work split: 4 warps (one per SM sub-partition), 98 threads own 8 consecutive
+// Two kernels live here.  lr_round_kernel takes the steps one by one and serves
+// lambda != 0; lr_block_kernel (further down, with its own description) takes
+// eight steps per block and serves lambda = 0, in a 4-warp instance for crowded
+// launches and an 8-warp instance for launches with an SM per round-task.
+//
+// lr_round_kernel.  Work split: 4 warps (one per SM sub-partition), 98 threads own 8 consecutive
 // pixels each and all 10 classes of them: 80 weights + 80 update-sum entries,
 // held as 2 x 40 packed fp32 pairs (class 2c, 2c+1) so that logits and updates
 // run on fma.rn.f32x2.  Per sample:
