@@ -29,7 +29,13 @@ __device__ __forceinline__ void group_range(const ApplyLaunch& p, uint32_t g, ui
   hi = min(p.hi, lo + per);
 }
 
+// Both kernels are launched with programmatic stream serialisation: their CTAs may become resident
+// while the kernel ahead of them in the stream (the round kernel, then group_totals_kernel) is
+// draining, and they read and write nothing before griddepcontrol.wait, which returns once that
+// kernel - and, because it waited the same way, every kernel before it - has finished.
 __global__ void __launch_bounds__(kAggThreads) group_totals_kernel(ApplyLaunch p) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t j = blockIdx.x * kAggThreads + threadIdx.x;
   if (j >= p.n_params) return;
   uint32_t lo, hi;
@@ -54,6 +60,7 @@ __global__ void __launch_bounds__(kAggThreads) apply_updates_kernel(ApplyLaunch 
   // runs.  They read nothing this grid writes before their own griddepcontrol.wait, which
   // returns only once this grid has finished and its writes are visible.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t j = blockIdx.x * kAggThreads + threadIdx.x;
   const uint32_t g = blockIdx.y;
   uint32_t lo, hi;
@@ -108,13 +115,22 @@ uint32_t apply_groups(uint32_t n_updates) {
 cudaError_t launch_apply_updates(const ApplyLaunch& p, cudaStream_t s) {
   if (p.hi <= p.lo) return cudaSuccess;
   const uint32_t blocks = (p.n_params + kAggThreads - 1) / kAggThreads;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.blockDim = dim3(kAggThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (p.groups > 1) {
-    group_totals_kernel<<<dim3(blocks, p.groups - 1), kAggThreads, 0, s>>>(p);
-    cudaError_t e = cudaGetLastError();
+    cfg.gridDim = dim3(blocks, p.groups - 1, 1);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, group_totals_kernel, p);
     if (e != cudaSuccess) return e;
   }
-  apply_updates_kernel<<<dim3(blocks, p.groups), kAggThreads, 0, s>>>(p);
-  return cudaGetLastError();
+  cfg.gridDim = dim3(blocks, p.groups, 1);
+  return cudaLaunchKernelEx(&cfg, apply_updates_kernel, p);
 }
 
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t n, cudaStream_t s) {

@@ -858,6 +858,9 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
     return;
   }
 
+  // The aggregation kernel behind this grid in the stream may become resident from here on (it
+  // touches nothing until this grid has finished and its writes are visible).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model W_start - eta U) ----
   for (int pass = 0; pass < (p.w_end ? 2 : 1); ++pass) {
     float* dst = (pass == 0 ? p.U : p.w_end) + (size_t)t.seq * p.stride;
