@@ -47,8 +47,8 @@ DESCRIBE = {
 # ncu captures summarised under profiles/ (traffic grows in proportion to the samples of a launch).
 # Set an entry to None when its kernel changes after the counters were taken.
 TRAFFIC_RATIO = {
-    "cfg2": (20.505856 / 21.1008, "profiles/lr_block_kernel_cfg2.md"),
-    "cfg5": (45.641728 / 50.41584, "profiles/lr_block_kernel_cfg5_512clients.md"),
+    "cfg2": (20.505344 / 21.1008, "profiles/lr_block_kernel_cfg2.md"),
+    "cfg5": (45.324544 / 50.41584, "profiles/lr_block_kernel_cfg5_512clients.md"),
 }
 
 
