@@ -255,7 +255,7 @@ def main():
     data = workloads.make_client_data(cfg)
     w0 = workloads.make_start_model(cfg)
     R = cfg["n_rounds"]
-    samples = workloads.total_samples(cfg)
+    samples = None  # filled from the library's own summary after the first run
     dev = [(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()) for x, y in data]
     w0_dev = torch.from_numpy(w0).cuda()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > L2 (126 MB)

@@ -16,7 +16,9 @@ Modules
 Pins (tests marked "not gpu"): the generator against the published SplitMix64
 sequence; the schedule against the paper's printed round counts (110 rounds
 for K = 60,000 with s_i = 10 i; the ceil(K/s) column of Table 5) and closed
-forms; gradients against central finite differences; one client against a
+forms; the round step size against values worked by hand from Section 4.1;
+gradients against central finite differences; the bf16 rounding points against a
+two-sample 2-2-2 network worked scalar by scalar; one client against a
 plain SGD loop; d = 0 against synchronous local SGD; the server rule against
 w = w_0 - sum(eta * U); a two-client case worked by hand; a convex case
 against a brute-force optimum.

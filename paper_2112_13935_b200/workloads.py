@@ -85,13 +85,6 @@ def n_params(dims) -> int:
     return sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
 
 
-def total_samples(cfg) -> int:
-    """Samples all clients consume in cfg['n_rounds'] rounds (count only)."""
-    r0, R = cfg["round_base"], cfg["n_rounds"]
-    per_client = sum(cfg["sched_a"] * i + cfg["sched_b"] for i in range(r0, r0 + R))
-    return per_client * cfg["n_clients"]
-
-
 def make_pool(n: int, dim: int, seed: int):
     """n synthetic images (float32 in [0,1], row-major [n, dim]) and int32 labels."""
     rng = np.random.default_rng(seed)

@@ -100,3 +100,72 @@ def test_full_loss_is_the_mean_over_all_clients():
     data = [(X[:5], y[:5]), (X[5:], y[5:])]
     want, _ = models.loss_and_grad(w, X, y, dims, 0.3)
     assert np.isclose(models.full_loss(w, data, dims, 0.3, chunk=4), want, rtol=1e-13)
+
+
+def _bf(v):
+    """Nearest bf16 of a Python float through a library conversion (not the checker's own)."""
+    return float(torch.tensor(v, dtype=torch.float32).to(torch.bfloat16))
+
+
+def bf16_case():
+    """Two samples through a 2-2-2 network, chosen so that every value that the low-precision
+    path rounds sits off the bf16 grid: x[0][0], x[1][1], W_0[0][0], W_1[1][1], both hidden
+    activations of unit 0, the logits of class 0 (which stay unrounded), and every dZ entry."""
+    dims = [2, 2, 2]
+    X = np.array([[1 + 2.0 ** -9, 0.5], [0.25, 1 - 2.0 ** -10]])
+    y = np.array([1, 0])
+    W0 = np.array([[0.5 + 2.0 ** -10, -0.25], [0.25, 0.5]])
+    b0 = np.array([2.0 ** -10, 0.0])
+    W1 = np.array([[1.0, -1.0], [0.5, 0.25 + 2.0 ** -11]])
+    b1 = np.array([2.0 ** -10, 0.0])
+    w = np.concatenate([W0.ravel(), b0, W1.ravel(), b1])
+    return dims, w, X, y
+
+
+def bf16_case_by_hand():
+    """The same case, scalar by scalar, with the rounding points of the low-precision path
+    spelled out: inputs once; each weight when read; each hidden activation after bias + ReLU;
+    each dZ before the two backward products (the bias gradients take the unrounded dZ)."""
+    import math
+    # rounded operands (exact dyadic values)
+    x = [[1.0, 0.5], [0.25, 1.0]]
+    W0 = [[0.5, -0.25], [0.25, 0.5]]
+    W1 = [[1.0, -1.0], [0.5, 0.25]]
+    b0 = [2.0 ** -10, 0.0]
+    # forward, sample 0: z = (0.625 + 2^-10, 0) -> a = (0.625, 0);  sample 1: z = (0.375 + 2^-10, 0.4375)
+    z0 = [[0.625 + 2.0 ** -10, 0.0], [0.375 + 2.0 ** -10, 0.4375]]
+    a0 = [[0.625, 0.0], [0.375, 0.4375]]
+    for b in range(2):
+        for h in range(2):
+            assert z0[b][h] == x[b][0] * W0[0][h] + x[b][1] * W0[1][h] + b0[h]
+            assert a0[b][h] == _bf(max(z0[b][h], 0.0))
+    b1 = [2.0 ** -10, 0.0]
+    logits = [[0.625 + 2.0 ** -10, -0.625], [0.59375 + 2.0 ** -10, -0.265625]]     # not rounded
+    for b in range(2):
+        for c in range(2):
+            assert logits[b][c] == a0[b][0] * W1[0][c] + a0[b][1] * W1[1][c] + b1[c]
+    p = [[1 / (1 + math.exp(-(l[0] - l[1]))), 1 / (1 + math.exp(l[0] - l[1]))] for l in logits]
+    loss = -(math.log(p[0][1]) + math.log(p[1][0])) / 2
+    dZ1 = [[p[0][0] / 2, (p[0][1] - 1) / 2], [(p[1][0] - 1) / 2, p[1][1] / 2]]       # (p - onehot) / B
+    dZ1q = [[_bf(v) for v in r] for r in dZ1]
+    gW1 = [[sum(a0[b][h] * dZ1q[b][c] for b in range(2)) for c in range(2)] for h in range(2)]
+    gb1 = [dZ1[0][c] + dZ1[1][c] for c in range(2)]
+    # dA = dZ1q W1^T, gated by z0 > 0 (unit 1 of sample 0 is off)
+    dZ0 = [[(dZ1q[b][0] * W1[h][0] + dZ1q[b][1] * W1[h][1]) * (1.0 if z0[b][h] > 0 else 0.0) for h in range(2)]
+           for b in range(2)]
+    dZ0q = [[_bf(v) for v in r] for r in dZ0]
+    gW0 = [[sum(x[b][i] * dZ0q[b][h] for b in range(2)) for h in range(2)] for i in range(2)]
+    gb0 = [dZ0[0][h] + dZ0[1][h] for h in range(2)]
+    g = np.array([v for r in gW0 for v in r] + gb0 + [v for r in gW1 for v in r] + gb1)
+    return loss, g
+
+
+def test_bf16_rounding_points_on_a_case_worked_by_hand():
+    dims, w, X, y = bf16_case()
+    loss, g = models.loss_and_grad(w, X, y, dims, 0.0, precision=1)
+    want_loss, want_g = bf16_case_by_hand()
+    assert abs(loss - want_loss) < 1e-15
+    np.testing.assert_allclose(g, want_g, rtol=0, atol=1e-16)
+    # and the case separates the two precisions everywhere it should
+    _, g32 = models.loss_and_grad(w, X, y, dims, 0.0, precision=0)
+    assert np.abs(g - g32).max() > 1e-4

@@ -108,3 +108,32 @@ def test_wrong_mixing_constant_is_caught(monkeypatch):
     real = rng.mix64
     monkeypatch.setattr(rng, "mix64", lambda z: real(z) ^ 1)
     _fails(tr.test_mix_matches_published_splitmix64_sequence)
+
+
+def _with_source_edit(monkeypatch, old, new):
+    """Plant a mistake in the checker's loss_and_grad by editing its source text."""
+    import inspect
+    src = inspect.getsource(models.loss_and_grad)
+    assert src.count(old) == 1, old
+    ns = dict(vars(models))
+    exec(compile(src.replace(old, new), "<mutated loss_and_grad>", "exec"), ns)
+    monkeypatch.setattr(models, "loss_and_grad", ns["loss_and_grad"])
+
+
+@pytest.mark.parametrize("old,new", [
+    ("A = [q(X)]", "A = [X]"),                                          # inputs not rounded
+    ("Wq = [q(W) for W, _ in layers]", "Wq = [W for W, _ in layers]"),    # weights not rounded when read
+    ("A.append(q(np.maximum(z, 0.0)))", "A.append(np.maximum(z, 0.0))"),  # activations not rounded
+    ("gW[...] = A[l].T @ dZq", "gW[...] = A[l].T @ dZ"),                  # dZ unrounded in the weight gradient
+    ("dA = dZq @ Wq[l].T", "dA = dZ @ Wq[l].T"),                          # dZ unrounded in the input gradient
+    ("gb[...] = dZ.sum(axis=0)", "gb[...] = dZq.sum(axis=0)"),            # bias gradient from the rounded dZ
+    ("z = A[l] @ Wq[l] + layers[l][1]", "z = q(A[l] @ Wq[l] + layers[l][1])"),   # logits / pre-activations rounded too
+])
+def test_a_moved_or_dropped_bf16_rounding_point_is_caught(monkeypatch, old, new):
+    _with_source_edit(monkeypatch, old, new)
+    _fails(tm.test_bf16_rounding_points_on_a_case_worked_by_hand)
+
+
+def test_step_size_without_the_square_root_is_caught(monkeypatch):
+    monkeypatch.setattr(schedule, "round_step_size", lambda lr, beta, t: lr / (1.0 + beta * t))
+    _fails(ts.test_round_step_size_values_worked_by_hand)

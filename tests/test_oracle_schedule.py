@@ -42,8 +42,26 @@ def test_sample_totals_closed_form(name, per_client, total, events):
     a, b, R = cfg["sched_a"], cfg["sched_b"], cfg["n_rounds"]
     assert a * R * (R - 1) // 2 + b * R == per_client
     assert schedule.samples_before(a, b, 0, R) == per_client
-    assert per_client * cfg["n_clients"] == total == workloads.total_samples(cfg)
+    assert per_client * cfg["n_clients"] == total
     assert cfg["n_clients"] * R == events
+
+
+def test_round_step_size_values_worked_by_hand():
+    # Section 4.1: eta_t = eta_0 / (1 + beta sqrt(t)); Appendix Table 2: eta_0 = 0.01, beta = 0.01.
+    # t = 10,000: sqrt = 100, 1 + 0.01 * 100 = 2, so the step is eta_0 / 2; t = 0: eta_0 itself;
+    # t = 2,500: sqrt = 50, 1 + 0.5 = 1.5; beta = 0 keeps the step constant.
+    assert schedule.round_step_size(0.01, 0.01, 10_000) == 0.005
+    assert schedule.round_step_size(0.01, 0.01, 0) == 0.01
+    assert abs(schedule.round_step_size(0.01, 0.01, 2_500) - 0.01 / 1.5) < 1e-18
+    assert schedule.round_step_size(0.3, 0.0, 123_456) == 0.3
+    # as the simulator uses it: t = the client's own iterations before the round.  Paper's schedule
+    # s_i = 10 i from round 1, batch 1: before round 5 a client has done 10 + 20 + 30 + 40 = 100
+    # iterations, so eta = 0.01 / (1 + 0.01 * 10) = 0.01 / 1.1
+    from oracle import sim
+    cfg = dict(sched_a=10, sched_b=0, round_base=1, batch=1, lr=0.01, lr_beta=0.01)
+    lr32, beta32 = sim.f32(0.01), sim.f32(0.01)
+    assert abs(sim.step_size(cfg, 5) - lr32 / (1.0 + beta32 * 10.0)) < 1e-18
+    assert sim.step_size(cfg, 1) == lr32
 
 
 def _check_log(cfg, events, summary):
@@ -73,7 +91,7 @@ def test_log_is_internally_consistent_cfg1_and_cfg2():
         cfg = workloads.get_config(name)
         events, summary, _ = schedule.simulate(cfg, cfg["n_rounds"])
         _check_log(cfg, events, summary)
-        assert summary["samples_total"] == workloads.total_samples(cfg)
+        assert summary["samples_total"] == {"cfg1": 600, "cfg2": 148800}[name]
 
 
 def test_d0_every_client_waits_for_all_previous_rounds():
