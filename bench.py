@@ -4,9 +4,12 @@
 One step = one pass of the whole path (schedule -> waves of local-SGD rounds ->
 ordered aggregation) over one workload: `aet_reset` + `aet_run_rounds(R)`.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--impl reference]
 
-Prints one JSON line.  `value` is device-timed with the inputs resident in HBM;
+Prints one JSON line.  The default workload is cfg5 at 1,024 clients; the line also carries the
+other configurations, device-timed for a few passes each, under `per_config`.  A pass of cfg5
+takes under 2 ms, so a step repeats the pass (`config.passes_per_step`) until the timed region
+is long enough for the clock sampler.  `value` is device-timed with the inputs resident in HBM;
 `e2e` goes through the C ABI from pinned host buffers; `roofline` is the
 local-SGD kernel against the measured HBM copy bandwidth; `cpu_baseline` is the
 CPU checker timed on this machine.  With several GPUs every rank runs an independent
@@ -40,7 +43,11 @@ DESCRIBE = {
     "cfg3": "cfg3: 32 clients, MLP 784-128-10 fp32, batch 32, s_i=64i+64, 40 rounds",
     "cfg4": "cfg4: 64 clients, MLP 3072-256-128-10 bf16 operands / fp32 accumulate, batch 64, s_i=128i+128, 30 rounds",
     "cfg5": "cfg5: 1,024 clients, softmax regression 784->10 fp32, 1,024 samples/client, s_i=8i+8, 10 rounds",
+    "cfg6": "cfg6 (the paper's own setting, Appendix Table 2): 5 nodes, softmax regression 784->10 fp32, "
+            "s_i=10i from round 1, 110 rounds, eta_0=0.01 beta=0.01, d=1, uniform delays",
 }
+DEFAULT_WORKLOAD = "cfg5"   # the configuration the HBM-roofline target of the regression kernel is quoted on
+MIN_TIMED_S = 2.0           # short passes are repeated inside a step until the timed region is this long
 
 
 # DRAM bytes (read + write) over algorithmic bytes of one launch of the round kernel, from the
@@ -48,7 +55,7 @@ DESCRIBE = {
 # Set an entry to None when its kernel changes after the counters were taken.
 TRAFFIC_RATIO = {
     "cfg2": (20.505344 / 21.1008, "profiles/lr_block_kernel_cfg2.md"),
-    "cfg5": (45.324544 / 50.41584, "profiles/lr_block_kernel_cfg5_512clients.md"),
+    "cfg5": None,
 }
 
 
@@ -183,6 +190,14 @@ def blas_threads(cfg):
     return 1 if cfg["model"] == 0 and cfg["batch"] == 1 else (os.cpu_count() or 1)
 
 
+def config_block(cfg, samples, n_events):
+    """The `config` object of the JSON line: names the workload, identical for both arms."""
+    return {"workload": DESCRIBE[cfg["name"]], "n_clients": cfg["n_clients"], "rounds": cfg["n_rounds"],
+            "network_delay_mean": cfg["network_delay_mean"],
+            "max_lag_d": "never wait" if cfg["max_lag_d"] == 0xFFFFFFFF else cfg["max_lag_d"],
+            "samples_per_pass": samples, "events_per_pass": n_events}
+
+
 def run_reference(args, cfg):
     """--impl reference: the CPU checker, timed per step on a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -194,6 +209,9 @@ def run_reference(args, cfg):
     w0 = workloads.make_start_model(cfg)
     cores = blas_threads(cfg)
     rates, sample = [], ""
+    from oracle import schedule as _sched
+    _ev, _sum, _ = _sched.simulate(cfg, cfg["n_rounds"])
+    ref_samples, ref_events = _sum["samples_total"], len(_ev)
     with threadpool_limits(limits=cores):
         for step in range(args.warmup + args.steps):
             rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, REF_STEP_LIMIT_S)
@@ -207,7 +225,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": DESCRIBE[cfg["name"]]},
+        "data": "synthetic", "config": config_block(cfg, ref_samples, ref_events),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -215,19 +233,127 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def measure_device(cfg, steps, warmup, passes_per_step=None, clock_index=None):
+    """Device-timed passes of one workload with its inputs resident in HBM.
+    Returns a dict with value (local, before any cross-rank reduction), roofline, stats."""
+    import torch
+    from paper_2112_13935_b200 import api, workloads
+    stream = torch.cuda.current_stream()
+    data = workloads.make_client_data(cfg)
+    w0 = workloads.make_start_model(cfg)
+    R = cfg["n_rounds"]
+    dev = [(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()) for x, y in data]
+    w0_dev = torch.from_numpy(w0).cuda()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > L2 (126 MB)
+    sess = api.Session(cfg, dev, w0_dev)
+    plan_ms = None
+    t_warm = []
+    for _ in range(warmup):
+        sess.reset()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        sess.run(R)
+        b.record(stream)
+        t_warm.append((a, b))
+        if plan_ms is None:   # host time of the integer schedule + launch plan; later runs reuse the cached plan
+            plan_ms = api.aet_get_stats(sess.h)["plan_ms"]
+    torch.cuda.synchronize()
+    events, summary = sess.log()
+    samples = summary["samples_total"]
+    stats = api.aet_get_stats(sess.h)
+    launches_per_pass = sum(stats["launches"])
+    if passes_per_step is None:
+        pass_s = min(a.elapsed_time(b) for a, b in t_warm) / 1e3
+        passes_per_step = max(1, int(np.ceil(MIN_TIMED_S / max(pass_s * steps, 1e-9))))
+    n_pass = steps * passes_per_step
+
+    # ---- timed region: every pass bracketed by events on the launching stream, L2 flushed before it ----
+    from paper_2112_13935_b200 import dist
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(n_pass)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(n_pass)]
+    dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(clock_index) if clock_index is not None else None
+    if sampler:
+        sampler.__enter__()
+    for k in range(n_pass):
+        flush.fill_(k & 0xFF)                      # evict L2 between timed passes
+        sess.reset()
+        starts[k].record(stream)
+        sess.run(R)
+        ends[k].record(stream)
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.__exit__()
+    dist.barrier()
+    seconds = sum(s.elapsed_time(e) for s, e in zip(starts, ends)) / 1e3
+
+    # ---- per-kernel device time: a second set of passes with events around every launch ----
+    api.aet_set_kernel_timing(sess.h, True)
+    k_ms = [0.0, 0.0]
+    k_pass = min(n_pass, 5)
+    for k in range(k_pass):
+        flush.fill_(k & 0xFF)
+        sess.reset()
+        sess.run(R)
+        st = api.aet_get_stats(sess.h)
+        k_ms[0] += st["kernel_ms"][0]
+        k_ms[1] += st["kernel_ms"][1]
+    api.aet_set_kernel_timing(sess.h, False)
+    sess.close()
+    del dev, flush
+
+    n_sgd_launches = stats["launches"][0]
+    alg_bytes = algorithmic_bytes(cfg, events)
+    sgd_ms = k_ms[0] / k_pass
+    achieved = alg_bytes / (sgd_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak_gbs()
+    ratio = TRAFFIC_RATIO.get(cfg["name"])
+    traffic = ratio[0] * alg_bytes / n_sgd_launches if ratio and ratio[0] and not cfg.get("_cut") else None
+    roof = {"bound": "hbm", "kernel": "local-SGD rounds", "achieved": achieved, "peak": peak,
+            "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+            "traffic_source": ratio[1] if traffic else None, "peak_kind": peak_kind,
+            "algorithmic_bytes_per_launch": alg_bytes / n_sgd_launches}
+    if cfg["model"] == 1:
+        tf = algorithmic_flops(cfg, events) / (sgd_ms * 1e-3) / 1e12
+        if cfg["precision"] == 1:     # bf16 operands: the dense contraction runs on the tensor cores
+            tpeak, tkind = measured_peak_tflops()
+            bound = "tensor"
+        else:                         # fp32 model: plain FMAs
+            tpeak, tkind = fp32_fma_peak_tflops()
+            bound = "alu"
+        roof = {"bound": bound, "kernel": "local-SGD rounds (MLP)", "achieved": tf, "peak": tpeak,
+                "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "peak_kind": tkind,
+                "hbm_gbs_algorithmic": achieved}
+    else:
+        # the batch-1 regression kernel sits on the FMA / HBM ridge: its fp32 FMA rate beside the HBM figure
+        apeak, akind = fp32_fma_peak_tflops()
+        atf = regression_flops(cfg, events) / (sgd_ms * 1e-3) / 1e12
+        roof.update(alu_tflops=atf, alu_peak=apeak, alu_frac=atf / apeak, alu_peak_kind=akind)
+    roof.update(launches_per_step=n_sgd_launches, kernel_ms_per_step=sgd_ms,
+                kernel_ms_mode="separate passes with events around every launch: no overlap between a kernel "
+                               "and its neighbours, so the sum can exceed the pass it belongs to",
+                aggregation_ms_per_step=k_ms[1] / k_pass, algorithmic_bytes_per_step=alg_bytes)
+    return dict(samples=samples, seconds=seconds, n_pass=n_pass, passes_per_step=passes_per_step, roof=roof,
+                launches_per_pass=launches_per_pass, events=len(events), waves=stats["waves"], plan_ms=plan_ms,
+                clocks=sampler.summary() if sampler else None, data=data, w0=w0)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg2", choices=sorted(DESCRIBE))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(DESCRIBE))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--clients", type=int, default=0, help="override the workload's client count (cfg5 sweep)")
     ap.add_argument("--rounds", type=int, default=0, help="override the number of rounds (profiling on a smaller case)")
     ap.add_argument("--net-delay", type=float, default=None, help="override the mean network delay (time units)")
     ap.add_argument("--max-lag", type=int, default=None, help="override the checkpoint threshold d (-1 = never wait)")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--passes-per-step", type=int, default=0, help="0 = enough for a 2 s timed region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the device-timed passes of the other configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -241,6 +367,8 @@ def main():
     if args.max_lag is not None:
         over["max_lag_d"] = workloads.NEVER_WAIT if args.max_lag < 0 else args.max_lag
     cfg = workloads.get_config(args.workload, seed=rank, **over)
+    if args.rounds:
+        cfg["_cut"] = True
     if args.impl == "reference":
         run_reference(args, cfg)
         return
@@ -250,91 +378,11 @@ def main():
     rank, world, local = dist.init_from_env()
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
     torch.cuda.set_device(local)
-    stream = torch.cuda.current_stream()
 
-    data = workloads.make_client_data(cfg)
-    w0 = workloads.make_start_model(cfg)
-    R = cfg["n_rounds"]
-    samples = None  # filled from the library's own summary after the first run
-    dev = [(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()) for x, y in data]
-    w0_dev = torch.from_numpy(w0).cuda()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > L2 (126 MB)
-
-    sess = api.Session(cfg, dev, w0_dev)
-    plan_ms = None
-    for _ in range(args.warmup):
-        sess.reset()
-        sess.run(R)
-        if plan_ms is None:   # host time of the integer schedule + launch plan; later runs reuse the cached plan
-            plan_ms = api.aet_get_stats(sess.h)["plan_ms"]
-    torch.cuda.synchronize()
-    events, summary = sess.log()
-    assert summary["samples_total"] == samples
-    stats = api.aet_get_stats(sess.h)
-    launches_per_step = sum(stats["launches"])
-
-    # ---- timed region: K steps, each bracketed by events on the launching stream ----
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    dist.barrier()
-    torch.cuda.synchronize()
-    with ClockSampler(local) as clocks:
-        for k in range(args.steps):
-            flush.fill_(k & 0xFF)                      # evict L2 between timed iterations
-            sess.reset()
-            starts[k].record(stream)
-            sess.run(R)
-            ends[k].record(stream)
-        torch.cuda.synchronize()
-    dist.barrier()
-    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    seconds = sum(step_ms) / 1e3
-    value = dist.job_throughput(samples * args.steps, seconds)
-    slowest = dist.max_over_ranks(seconds)
-
-    # ---- per-kernel device time (same steps again with events around every launch) ----
-    api.aet_set_kernel_timing(sess.h, True)
-    k_ms = [0.0, 0.0]
-    k_steps = min(args.steps, 5)
-    for k in range(k_steps):
-        flush.fill_(k & 0xFF)
-        sess.reset()
-        sess.run(R)
-        st = api.aet_get_stats(sess.h)
-        k_ms[0] += st["kernel_ms"][0]
-        k_ms[1] += st["kernel_ms"][1]
-    api.aet_set_kernel_timing(sess.h, False)
-    n_sgd_launches = stats["launches"][0]
-    alg_bytes = algorithmic_bytes(cfg, events)
-    sgd_ms_per_step = k_ms[0] / k_steps
-    achieved = alg_bytes / (sgd_ms_per_step * 1e-3) / 1e9
-    peak, peak_kind = measured_peak_gbs()
-    ratio = TRAFFIC_RATIO.get(args.workload)
-    traffic = ratio[0] * alg_bytes / n_sgd_launches if ratio and ratio[0] and not args.rounds else None
-    roof = {"bound": "hbm", "kernel": "local-SGD rounds", "achieved": achieved, "peak": peak,
-            "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
-            "traffic_source": ratio[1] if traffic else None, "peak_kind": peak_kind,
-            "algorithmic_bytes_per_launch": alg_bytes / n_sgd_launches}
-    if cfg["model"] == 1:
-        tf = algorithmic_flops(cfg, events) / (sgd_ms_per_step * 1e-3) / 1e12
-        if cfg["precision"] == 1:     # bf16 operands: the dense contraction runs on the tensor cores
-            tpeak, tkind = measured_peak_tflops()
-            bound = "tensor"
-        else:                         # fp32 model: plain FMAs
-            tpeak, tkind = fp32_fma_peak_tflops()
-            bound = "alu"
-        roof = {"bound": bound, "kernel": "local-SGD rounds (MLP)", "achieved": tf, "peak": tpeak,
-                "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "peak_kind": tkind,
-                "hbm_gbs_algorithmic": achieved}
-    else:
-        # the batch-1 regression kernel sits on the FMA / HBM ridge: its fp32 FMA rate beside the HBM figure
-        apeak, akind = fp32_fma_peak_tflops()
-        atf = regression_flops(cfg, events) / (sgd_ms_per_step * 1e-3) / 1e12
-        roof.update(alu_tflops=atf, alu_peak=apeak, alu_frac=atf / apeak, alu_peak_kind=akind)
-    roof.update(launches_per_step=n_sgd_launches, kernel_ms_per_step=sgd_ms_per_step,
-                aggregation_ms_per_step=k_ms[1] / k_steps, algorithmic_bytes_per_step=alg_bytes)
-    sess.close()
-    del dev
+    m = measure_device(cfg, args.steps, args.warmup, args.passes_per_step or None, clock_index=local)
+    data, w0, samples, R = m["data"], m["w0"], m["samples"], cfg["n_rounds"]
+    value = dist.job_throughput(samples * m["n_pass"], m["seconds"])
+    slowest = dist.max_over_ranks(m["seconds"])
 
     # ---- end to end through the C ABI from pinned host buffers ----
     pinned = [(torch.from_numpy(x).pin_memory(), torch.from_numpy(y).pin_memory()) for x, y in data]
@@ -358,7 +406,8 @@ def main():
         api.aet_destroy(h)
         if k > 0:                                      # first one warms allocator and caches
             e2e_s.append(dt)
-    e2e_value = dist.job_throughput(samples * len(e2e_s), sum(e2e_s))
+    e2e_value = dist.job_throughput(samples * len(e2e_s), sum(e2e_s)) if e2e_s else None
+    del pinned
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -368,6 +417,21 @@ def main():
             rate, n_s, n_t, n_e, dt = oracle_bounded(cfg, data, w0, CPU_LIMIT_S)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"schedule + first {n_t} of {n_e} round-tasks in start order ({n_s} samples, {dt:.1f} s)"}
+    del data
+
+    # ---- the other configurations, device-timed for a few passes each (no e2e, no CPU leg) ----
+    per_config = []
+    if rank == 0 and world == 1 and not args.no_per_config and not args.rounds and not args.clients:
+        for name, steps in (("cfg2", 10), ("cfg3", 5), ("cfg4", 3), ("cfg6", 5)):
+            if name == args.workload:
+                continue
+            c2 = workloads.get_config(name, seed=rank)
+            r = measure_device(c2, steps, 3, passes_per_step=1)
+            per_config.append({"workload": DESCRIBE[name], "value": r["samples"] * r["n_pass"] / r["seconds"],
+                               "unit": UNIT, "ms_per_step": 1e3 * r["seconds"] / r["n_pass"], "steps": r["n_pass"],
+                               "dtype": "bf16" if c2["precision"] == 1 else "f32",
+                               "roofline": {k: r["roof"][k] for k in ("bound", "achieved", "peak", "unit", "frac",
+                                                                      "peak_kind", "kernel_ms_per_step")}})
 
     if rank == 0:
         line = {
@@ -375,19 +439,18 @@ def main():
             "warmup": args.warmup, "ms_per_step": 1e3 * slowest / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg["precision"] == 1 else "f32",
             "data": "synthetic",
-            "config": {"workload": DESCRIBE[args.workload], "n_clients": cfg["n_clients"], "rounds": R,
-                       "network_delay_mean": cfg["network_delay_mean"],
-                       "max_lag_d": "never wait" if cfg["max_lag_d"] == workloads.NEVER_WAIT else cfg["max_lag_d"],
-                       "samples_per_step": samples, "events_per_step": len(events),
-                       "waves_per_step": stats["waves"], "l2": "flushed between timed steps (256 MB fill)",
-                       "multi_gpu": "independent replicas, one seed per rank"},
-            "clocks": clocks.summary(),
+            "config": dict(config_block(cfg, samples, m["events"]), l2="flushed before every timed pass (256 MB fill)",
+                           passes_per_step=m["passes_per_step"]),
+            "run": {"waves_per_pass": m["waves"], "ms_per_pass": 1e3 * slowest / m["n_pass"],
+                    "multi_gpu": "independent replicas, one seed per rank"},
+            "clocks": m["clocks"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": len(e2e_s)},
-            "gpu_launches": launches_per_step * args.steps,
-            "roofline": roof,
+                    "steps": len(e2e_s), "note": "one pass per e2e step: create, load from pinned host memory, run, model back"},
+            "gpu_launches": m["launches_per_pass"] * m["n_pass"],
+            "roofline": m["roof"],
             "cpu_baseline": cpu,
-            "schedule_and_plan_ms_first_run": plan_ms,
+            "per_config": per_config,
+            "schedule_and_plan_ms_first_run": m["plan_ms"],
         }
         print(json.dumps(line))
     dist.shutdown()

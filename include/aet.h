@@ -40,7 +40,7 @@ typedef enum {
   AET_ERR_NOMEM = 4,   /* host or device allocation failed                   */
   AET_ERR_CUDA = 5,    /* a CUDA runtime call failed (see aet_last_error)    */
   AET_ERR_TIMEOUT = 6, /* a bounded device-side wait gave up                 */
-  AET_ERR_NUMERIC = 7  /* non-finite value met in a model or update sum      */
+  AET_ERR_NUMERIC = 7  /* non-finite value met in the server model or in data */
 } aet_status;
 
 #define AET_MAX_LAYERS 7
@@ -61,15 +61,35 @@ typedef struct {
   uint32_t max_lag_d;  /* threshold d of Synchronize (Algorithm 3)                */
   float lr, lr_beta;   /* eta_i = lr / (1 + lr_beta * sqrt(t)) (Section 5)        */
   float l2;            /* lambda of (lambda/2)|W|^2 on weight matrices            */
-  uint32_t delay_dist; /* 0 = exponential(mean), 1 = uniform[lo, hi]              */
+  uint32_t delay_dist; /* 0 = exponential(mean), 1 = uniform[lo, hi]: the paper draws
+                          its delays uniformly (Section 5 "System delay", Appendix
+                          "Hyper-parameters selection"); the exponential form and the
+                          lo / hi fields below extend that to other delay models     */
   uint64_t seed;
   double compute_delay_mean, network_delay_mean; /* time units, dist 0           */
   double compute_delay_lo, compute_delay_hi;     /* time units, dist 1           */
   double network_delay_lo, network_delay_hi;
   double straggler_factor; /* scales the compute delay of the stragglers          */
   uint32_t n_stragglers;   /* the last n_stragglers client ids                    */
-  uint32_t flags;          /* reserved, 0                                          */
+  uint32_t flags;          /* AET_FLAG_* bits, 0 for the defaults                  */
 } aet_config;
+
+/* aet_load_client_data keeps the caller's device pointers instead of copying
+ * (precision 0 only; precision 1 always makes its own bf16 copy).  Both arrays
+ * must be device memory, x 16-byte aligned with dims[0] a multiple of 4, and
+ * must stay alive and unchanged until aet_destroy. */
+#define AET_FLAG_BORROW_DATA 1u
+/* Debug checks in place of a memory checker: every label is range-checked and
+ * every pixel checked finite as a data set is loaded, and every round kernel
+ * checks the rows and slots its task names before touching them.  A violation
+ * sets a status word (nothing traps); the next synchronising call returns
+ * AET_ERR_STATE or AET_ERR_NUMERIC and the task concerned was skipped. */
+#define AET_FLAG_DEBUG_CHECKS 2u
+/* Keep every round's update sum U_i until the next aet_run_rounds so that
+ * aet_get_update_sum can read it back.  Without it the rows are recycled as
+ * soon as the server has applied them (memory ~ rounds in flight, not all
+ * rounds of the call). */
+#define AET_FLAG_KEEP_UPDATE_SUMS 4u
 
 /* One round-task = one message (c, U_i, i) of Algorithm 3.  64 bytes.
  * Times are integer ticks (2^20 per time unit). */
@@ -105,12 +125,15 @@ typedef struct {
   double plan_ms;              /* host time spent on schedule + launch plan         */
 } aet_stats;
 
-/* Create a run.  Allocates the global model (zeros) and per-client state on the
- * current CUDA device.  Errors: AET_ERR_ARG (null, bad struct_size),
+/* Create a run: n clients with local data sets and a server holding the global
+ * model (Section 1, client-server form; Algorithm 2 "Setup" fixes the step-size
+ * and sample-size sequences and d, here through cfg).  Allocates the global
+ * model (zeros) and per-client state on the current CUDA device.  Errors: AET_ERR_ARG (null, bad struct_size),
  * AET_ERR_CONFIG (unsupported model/dims/batch), AET_ERR_CUDA, AET_ERR_NOMEM. */
 aet_status aet_create(const aet_config* cfg, aet_handle** out);
 
-/* Free everything the handle owns (synchronises the device first). */
+/* End of the run of Algorithm 3's loop "for round i": free everything the
+ * handle owns (synchronises the device first). */
 aet_status aet_destroy(aet_handle* h);
 
 /* Back to the state right after aet_create + aet_set_global_model + data load:
@@ -138,13 +161,20 @@ aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x,
  * AET_ERR_CONFIG (batch does not divide s_i), AET_ERR_CUDA, AET_ERR_NOMEM. */
 aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream);
 
-/* Copy the server's model out (host or device pointer, n_params floats).
- * Synchronises `cuda_stream`. */
+/* Copy the server's model out: the global model w the server keeps and
+ * broadcasts (Section 1; Algorithm 3, Receive: w = w - eta_k U).  Host or device
+ * pointer, n_params floats.  Synchronises `cuda_stream`.  Errors:
+ * AET_ERR_TIMEOUT, AET_ERR_STATE (debug check), AET_ERR_NUMERIC (a non-finite
+ * value reached the model); `out` is then untouched and the handle stays usable
+ * (aet_reset, reload the offending data, run again). */
 aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params,
                                 void* cuda_stream);
 
-/* The event log of all rounds run so far, ordered by seq within each
- * aet_run_rounds call, and its summary.  `out` is a host array of `capacity`
+/* The event log of all rounds run so far - one record per message (c, U_i, i)
+ * of Algorithm 3 with its start, trigger and apply times, the checkpoint wait
+ * (Synchronize) and the history count behind it - ordered by seq within each
+ * aet_run_rounds call, and its summary (message counts for the communication-
+ * cost comparison of Section 5).  `out` is a host array of `capacity`
  * records (may be null with capacity 0 to query *n_events).  Synchronises the
  * last stream used and cross-checks the trigger/apply records the kernels
  * wrote against the schedule (AET_ERR_STATE on a mismatch). */
@@ -152,7 +182,8 @@ aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity,
                              size_t* n_events, aet_summary* summary);
 
 /* Update sum number `seq` of the most recent aet_run_rounds (host or device
- * pointer, n_params floats).  Synchronises `cuda_stream`. */
+ * pointer, n_params floats).  Needs AET_FLAG_KEEP_UPDATE_SUMS (AET_ERR_STATE
+ * without it).  Synchronises `cuda_stream`. */
 aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params,
                               void* cuda_stream);
 
@@ -193,7 +224,10 @@ const char* aet_last_error(const aet_handle* h);
  * `client` (Algorithm 3, MainComputeNode) from the model w_in, writing the update
  * sum U_out and the end-of-round model w_out.  x [n, dims[0]] fp32, y [n] int32,
  * w_in, U_out, w_out (n_params floats each) are DEVICE pointers owned by the
- * caller.  The kernel's scratch (descriptors, the working model, activations)
+ * caller.  The entry point always runs the library's generic fp32 round kernel
+ * (any layer widths; not the shape-specialised kernels a handle may pick), so
+ * its results agree with aet_debug_run_client_round within fp32 rounding order,
+ * not bit for bit.  The kernel's scratch (descriptors, the working model, activations)
  * is a fixed array inside the library image: every GPU that loads the library
  * holds about 1 MB for it until the process exits.  Limits: precision 0, at most
  * 131,072 parameters and 131,072 floats of activation scratch (about
@@ -227,6 +261,17 @@ uint64_t aet_debug_delay_ticks(uint32_t dist, uint64_t draw, uint64_t p0, uint64
 /* Number of waves (groups of mutually independent round-tasks) the launch
  * plan of a fresh run of n_rounds has; 0 on error. */
 uint32_t aet_debug_plan_waves(const aet_config* cfg, uint32_t n_rounds);
+
+/* The launch plan of a fresh run of n_rounds, for checking it on the host: tasks
+ * in launch order (their seq, wave and the snapshot slot they start from; arrays
+ * of n_clients * n_rounds entries), per seq the row of the update-sum array and
+ * the slot the server model is kept in after that update (-1: none), the number
+ * of updates applied after each wave (first counts[0] entries of an array of
+ * n_clients * n_rounds), and counts = {waves, update-sum rows, snapshot slots}
+ * the run allocates.  cfg->flags decides whether rows are recycled. */
+aet_status aet_debug_plan_layout(const aet_config* cfg, uint32_t n_rounds, uint32_t* task_seq,
+                                 uint32_t* task_wave, uint32_t* task_snap_slot, uint32_t* u_row,
+                                 int32_t* snap_slot_after, uint32_t* apply_upto, uint32_t* counts);
 
 #ifdef __cplusplus
 }

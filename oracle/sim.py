@@ -58,7 +58,8 @@ def run(cfg, data, w0, n_rounds=None, keep=False, state=None):
 
     w0 is the server model the call starts from; state (from a previous call's
     result) continues the simulated clock, histories and round counters.
-    Returns dict(events, summary, w, U (by seq), w_start (by seq, if keep), state).
+    keep: True keeps every round's start model, a collection of seq numbers only those.
+    Returns dict(events, summary, w, U (by seq), w_start (by seq, where kept), state).
     """
     n_rounds = cfg["n_rounds"] if n_rounds is None else n_rounds
     events, summary, state_after = schedule.simulate(cfg, n_rounds, state)
@@ -76,7 +77,7 @@ def run(cfg, data, w0, n_rounds=None, keep=False, state=None):
                 w_start -= step_size(cfg, f["round"]) * U_by_seq[f["seq"]]
             U, _ = run_task(cfg, data[c], c, i, w_start)
             U_by_seq[e["seq"]] = U
-            if keep:
+            if keep is True or (keep and e["seq"] in keep):
                 w_start_by_seq[e["seq"]] = w_start
             in_flight[c].append(e)
         else:

@@ -76,6 +76,7 @@ PROTOTYPES = {
     "aet_debug_draw": (C.c_uint64, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64]),
     "aet_debug_delay_ticks": (C.c_uint64, [C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64]),
     "aet_debug_plan_waves": (C.c_uint32, [C.POINTER(AetConfig), C.c_uint32]),
+    "aet_debug_plan_layout": (C.c_int, [C.POINTER(AetConfig), C.c_uint32] + [C.c_void_p] * 7),
 }
 
 _lib = None

@@ -12,6 +12,8 @@ import numpy as np
 from . import _lib
 from ._lib import AetConfig, AetEvent, AetStats, AetSummary, NEVER_WAIT, STATUS_NAMES  # noqa: F401
 
+FLAG_BORROW_DATA, FLAG_DEBUG_CHECKS, FLAG_KEEP_UPDATE_SUMS = 1, 2, 4   # AET_FLAG_* of include/aet.h
+
 
 class AetError(RuntimeError):
     def __init__(self, status: int, message: str):
@@ -31,6 +33,7 @@ def make_config(cfg: dict) -> AetConfig:
         if name in ("struct_size", "n_layers", "dims", "flags"):
             continue
         setattr(c, name, cfg[name])
+    c.flags = int(cfg.get("flags", 0))
     return c
 
 
@@ -193,6 +196,21 @@ def aet_debug_delay_ticks(dist, draw, p0, p1=0) -> int:
 def aet_debug_plan_waves(cfg, n_rounds) -> int:
     conf = cfg if isinstance(cfg, AetConfig) else make_config(cfg)
     return int(_lib.load().aet_debug_plan_waves(C.byref(conf), n_rounds))
+
+
+def aet_debug_plan_layout(cfg, n_rounds) -> dict:
+    """Host only: the launch plan of a fresh run (see include/aet.h)."""
+    conf = cfg if isinstance(cfg, AetConfig) else make_config(cfg)
+    E = conf.n_clients * n_rounds
+    u32 = lambda: np.zeros(max(E, 1), dtype=np.uint32)
+    out = dict(task_seq=u32(), task_wave=u32(), task_snap_slot=u32(), u_row=u32(),
+               snap_slot_after=np.zeros(max(E, 1), dtype=np.int32), apply_upto=u32())
+    counts = np.zeros(3, dtype=np.uint32)
+    _check(None, _lib.load().aet_debug_plan_layout(C.byref(conf), n_rounds, *[_ptr(v) for v in out.values()], _ptr(counts)))
+    out = {k: v[:E] for k, v in out.items()}
+    out["apply_upto"] = out["apply_upto"][:int(counts[0])]
+    out.update(waves=int(counts[0]), n_u_rows=int(counts[1]), n_snap=int(counts[2]))
+    return out
 
 
 class Session:

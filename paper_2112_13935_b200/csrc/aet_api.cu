@@ -192,10 +192,10 @@ aet_status upload_clients(aet_handle* h, cudaStream_t s) {
 aet_status check_device_status(aet_handle* h) {
   uint32_t st = 0;
   AET_CUDA(h, cudaMemcpy(&st, h->d_status.p, sizeof(st), cudaMemcpyDeviceToHost));
-  if (st & 1u) {
-    cudaMemset(h->d_status.p, 0, sizeof(uint32_t));
-    return fail(h, AET_ERR_TIMEOUT, "a bounded wait for an asynchronous row copy gave up; results are invalid");
-  }
+  if (st) cudaMemset(h->d_status.p, 0, sizeof(uint32_t));
+  if (st & 1u) return fail(h, AET_ERR_TIMEOUT, "a bounded wait for an asynchronous row copy gave up; results are invalid");
+  if (st & 4u) return fail(h, AET_ERR_STATE, "a debug check failed on the device: a label, row number or slot was out of range; results are invalid");
+  if (st & 2u) return fail(h, AET_ERR_NUMERIC, "a non-finite value reached the server model (or, with debug checks, sits in a client's rows); results are invalid");
   return AET_OK;
 }
 
@@ -229,6 +229,8 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   const uint32_t P = count_params(*cfg);
   if (!P) return fail(nullptr, AET_ERR_CONFIG, "model too large");
   if (cfg->dims[cfg->n_layers] > 32) return fail(nullptr, AET_ERR_CONFIG, "at most 32 classes are supported");
+  if (cfg->flags & ~(uint32_t)(AET_FLAG_BORROW_DATA | AET_FLAG_DEBUG_CHECKS | AET_FLAG_KEEP_UPDATE_SUMS))
+    return fail(nullptr, AET_ERR_CONFIG, "unknown bit in flags");
   int dev = 0;
   cudaError_t ce = cudaGetDevice(&dev);
   if (ce != cudaSuccess) { cudaGetLastError(); return fail(nullptr, AET_ERR_CUDA, std::string("no CUDA device: ") + cudaGetErrorString(ce)); }
@@ -318,6 +320,25 @@ aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x, c
   const size_t D = h->cfg.dims[0];
   const size_t elems = (size_t)n * D;
   const bool bf16 = h->cfg.precision == 1;
+  const bool debug = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) != 0;
+  if ((h->cfg.flags & AET_FLAG_BORROW_DATA) && !bf16) {
+    // D_c stays where the caller put it: both arrays must be device memory the kernels can read
+    // with 16-byte row copies, and must stay alive and unchanged until aet_destroy.
+    cudaPointerAttributes ax{}, ay{};
+    const bool okx = cudaPointerGetAttributes(&ax, x) == cudaSuccess &&
+                     (ax.type == cudaMemoryTypeDevice || ax.type == cudaMemoryTypeManaged);
+    const bool oky = cudaPointerGetAttributes(&ay, y) == cudaSuccess &&
+                     (ay.type == cudaMemoryTypeDevice || ay.type == cudaMemoryTypeManaged);
+    cudaGetLastError();
+    if (!okx || !oky) return fail(h, AET_ERR_ARG, "AET_FLAG_BORROW_DATA needs device pointers");
+    if (((uintptr_t)x & 15) || ((D * 4) & 15) || ((uintptr_t)y & 3))
+      return fail(h, AET_ERR_ARG, "AET_FLAG_BORROW_DATA needs 16-byte aligned rows");
+    if (debug) AET_CUDA(h, launch_validate_data((const float*)x, y, n, (uint32_t)D, h->cfg.dims[h->cfg.n_layers], h->d_status.p, s));
+    h->h_clients[client] = ClientData{x, y, n, 0};
+    h->clients_dirty = true;
+    h->last_stream = s;
+    return AET_OK;
+  }
   void* dx = h->arena.alloc(elems * (bf16 ? 2 : 4));
   int32_t* dy = (int32_t*)h->arena.alloc((size_t)n * sizeof(int32_t));
   if (!dx || !dy) return fail(h, AET_ERR_NOMEM, "device allocation failed");
@@ -341,6 +362,10 @@ aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x, c
     }
   }
   AET_CUDA(h, cudaMemcpyAsync(dy, y, (size_t)n * sizeof(int32_t), cudaMemcpyDefault, s));
+  if (debug) {
+    if (!bf16) AET_CUDA(h, launch_validate_data((const float*)dx, dy, n, (uint32_t)D, h->cfg.dims[h->cfg.n_layers], h->d_status.p, s));
+    else AET_CUDA(h, launch_validate_data(nullptr, dy, n, (uint32_t)D, h->cfg.dims[h->cfg.n_layers], h->d_status.p, s));
+  }
   h->h_clients[client] = ClientData{dx, dy, n, 0};
   h->clients_dirty = true;
   h->last_stream = s;
@@ -370,7 +395,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
     std::string err;
     if (!simulate(h->cfg, n_rounds, st, h->delays, cp.sched, err)) return fail(h, AET_ERR_CONFIG, err);
     cp.after = st;
-    build_plan(h->cfg, cp.sched.events, cp.plan);
+    build_plan(h->cfg, cp.sched.events, (h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, cp.plan);
     cp.valid = true;
   }
   const Plan& plan = cp.plan;
@@ -380,7 +405,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   // ---- device buffers ----
   aet_status st_up = upload_clients(h, s);
   if (st_up != AET_OK) return st_up;
-  bool ok = h->snaps.reserve((size_t)plan.n_snap * h->stride) && h->U.reserve(E * h->stride) &&
+  bool ok = h->snaps.reserve((size_t)plan.n_snap * h->stride) && h->U.reserve((size_t)plan.n_u_rows * h->stride) &&
             h->d_tasks.reserve(E) && h->d_inflight.reserve(plan.inflight.size() + 1) &&
             h->d_applies.reserve(E) && h->d_trig.reserve(E) && h->d_alog.reserve(E);
   if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * mlp_act_floats(h->shape));
@@ -401,9 +426,11 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   r.tasks = h->d_tasks.p; r.inflight = h->d_inflight.p; r.clients = h->d_clients.p;
   r.sample_keys = h->d_keys.p; r.snaps = h->snaps.p; r.U = h->U.p; r.w_end = nullptr;
   r.trig = h->d_trig.p; r.status = h->d_status.p; r.stride = h->stride; r.l2 = h->cfg.l2;
+  r.debug_checks = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) ? 1u : 0u;
+  r.n_u_rows = plan.n_u_rows; r.n_snap = plan.n_snap;
   ApplyLaunch a{};
   a.applies = h->d_applies.p; a.U = h->U.p; a.snaps = h->snaps.p; a.totals = h->totals.p;
-  a.H = h->d_H.p; a.log = h->d_alog.p; a.stride = h->stride; a.n_params = h->P;
+  a.H = h->d_H.p; a.log = h->d_alog.p; a.status = h->d_status.p; a.stride = h->stride; a.n_params = h->P;
 
   // ---- waves: a3/a4 local SGD of independent round-tasks, then a6 aggregation ----
   const uint32_t n_waves = (uint32_t)plan.apply_upto.size();
@@ -446,15 +473,19 @@ aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params, void
   if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
   cudaStream_t s = (cudaStream_t)cuda_stream;
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  if (aet_status ds = check_device_status(h)) return ds;   // `out` stays untouched on error
   AET_CUDA(h, cudaMemcpyAsync(out, h->w_cur(), (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   AET_CUDA(h, cudaStreamSynchronize(s));
-  return check_device_status(h);
+  return AET_OK;
 }
 
 aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params, void* cuda_stream) {
   if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
   if (seq >= h->last_n_events) return fail(h, AET_ERR_ARG, "seq is not an event of the most recent run");
+  if (!(h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS))
+    return fail(h, AET_ERR_STATE, "update sums are recycled during a run unless the handle was created with AET_FLAG_KEEP_UPDATE_SUMS");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaMemcpyAsync(out, h->U.p + (size_t)seq * h->stride, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   AET_CUDA(h, cudaStreamSynchronize(s));
@@ -530,6 +561,8 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   r.tasks = dtask; r.inflight = nullptr; r.clients = h->d_clients.p; r.sample_keys = h->d_keys.p;
   r.snaps = snap; r.U = U; r.w_end = wend; r.trig = dtrig; r.status = h->d_status.p; r.stride = h->stride;
   r.task_begin = 0; r.n_tasks = 1; r.l2 = h->cfg.l2;
+  r.debug_checks = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) ? 1u : 0u;
+  r.n_u_rows = 1; r.n_snap = 1;
   const aet_stats keep = h->stats;
   const bool timing = h->timing;
   h->timing = false;
@@ -608,8 +641,39 @@ uint32_t aet_debug_plan_waves(const aet_config* cfg, uint32_t n_rounds) {
   SchedResult res;
   if (!simulate(*cfg, n_rounds, st, cache, res, err)) return 0;
   Plan plan;
-  build_plan(*cfg, res.events, plan);
+  build_plan(*cfg, res.events, (cfg->flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, plan);
   return (uint32_t)plan.apply_upto.size();
+}
+
+aet_status aet_debug_plan_layout(const aet_config* cfg, uint32_t n_rounds, uint32_t* task_seq, uint32_t* task_wave,
+                                 uint32_t* task_snap_slot, uint32_t* u_row, int32_t* snap_slot_after,
+                                 uint32_t* apply_upto, uint32_t* counts) {
+  if (!cfg || !task_seq || !task_wave || !task_snap_slot || !u_row || !snap_slot_after || !apply_upto || !counts)
+    return fail(nullptr, AET_ERR_ARG, "null argument");
+  if (cfg->struct_size != sizeof(aet_config)) return fail(nullptr, AET_ERR_ARG, "struct_size does not match sizeof(aet_config)");
+  std::string err;
+  if (!validate_config(*cfg, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+  SchedState st;
+  DelayCache cache;
+  SchedResult res;
+  if (!simulate(*cfg, n_rounds, st, cache, res, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+  Plan plan;
+  build_plan(*cfg, res.events, (cfg->flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, plan);
+  const uint32_t n_waves = (uint32_t)plan.apply_upto.size();
+  for (uint32_t L = 0; L < n_waves; ++L) {
+    apply_upto[L] = plan.apply_upto[L];
+    for (uint32_t q = plan.wave_off[L]; q < plan.wave_off[L + 1]; ++q) {
+      task_seq[q] = plan.tasks[q].seq;
+      task_wave[q] = L;
+      task_snap_slot[q] = plan.tasks[q].snap_slot;
+    }
+  }
+  for (size_t k = 0; k < res.events.size(); ++k) {
+    u_row[k] = plan.applies[k].u_row;
+    snap_slot_after[k] = plan.applies[k].snap_slot;
+  }
+  counts[0] = n_waves; counts[1] = plan.n_u_rows; counts[2] = plan.n_snap;
+  return AET_OK;
 }
 
 }  // extern "C"

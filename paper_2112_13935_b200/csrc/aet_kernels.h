@@ -29,12 +29,15 @@ struct RoundLaunch {
   const ClientData* clients;     // device, [n_clients]
   const uint64_t* sample_keys;   // device, [n_clients]
   const float* snaps;            // [n_snap, stride] models rounds start from
-  float* U;                      // [n_events, stride] update sums, row = seq
+  float* U;                      // [n_u_rows, stride] update sums, row = TaskDesc::u_row
   float* w_end;                  // optional [n_events, stride] end-of-round models
   TriggerRec* trig;              // [n_events], row = seq
-  uint32_t* status;              // optional: bit 0 set if a bounded device wait gave up
+  uint32_t* status;              // optional: bit 0 set if a bounded device wait gave up,
+                                 // bit 2 if a debug index check failed (see debug_checks)
+  uint32_t debug_checks;         // non-zero: sample indices and row numbers are range-checked before use
   size_t stride;
   uint32_t task_begin, n_tasks;
+  uint32_t n_u_rows, n_snap;     // extents of U and snaps (for the debug checks)
   float l2;
 };
 
@@ -79,12 +82,30 @@ struct ApplyLaunch {
   float* totals;             // scratch [groups, stride], used when groups > 1
   uint32_t* H;               // [n_clients]
   ApplyRec* log;             // [n_events]
+  uint32_t* status;          // optional: bit 1 set if the model after the range is not finite
   size_t stride;
   uint32_t n_params, lo, hi;
   uint32_t groups;           // apply_groups(hi - lo)
 };
 uint32_t apply_groups(uint32_t n_updates);
 cudaError_t launch_apply_updates(const ApplyLaunch& p, cudaStream_t s);
+
+// Debug checks at load time: labels in range (else bit 2 of *status), pixels finite (else bit 1; x may be null).
+cudaError_t launch_validate_data(const float* x, const int32_t* y, uint32_t n, uint32_t dim, uint32_t n_classes,
+                                 uint32_t* status, cudaStream_t s);
+
+#if defined(__CUDACC__)
+// Debug check at the top of every round kernel (all threads of a CTA, and all CTAs of a cluster,
+// take the same decision): are the rows and slots the task names inside the arrays?  If not,
+// bit 2 of *status is set and the caller skips the task without touching memory.
+__device__ __forceinline__ bool debug_task_ok(const RoundLaunch& p, const TaskDesc& t) {
+  if (!p.debug_checks) return true;
+  bool ok = t.u_row < p.n_u_rows && t.snap_slot < p.n_snap;
+  for (uint32_t f = 0; ok && f < t.inflight_cnt; ++f) ok = p.inflight[t.inflight_off + f].row < p.n_u_rows;
+  if (!ok && threadIdx.x == 0 && p.status) atomicOr(p.status, 4u);
+  return ok;
+}
+#endif
 
 // bf16 conversion of a client's rows at load time (precision 1).
 cudaError_t launch_to_bf16(const float* src, void* dst, size_t n, cudaStream_t s);

@@ -221,10 +221,11 @@ bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache
   return true;
 }
 
-void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan& plan) {
+void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool keep_all, Plan& plan) {
   const size_t E = events.size();
   plan = Plan{};
   plan.applies.resize(E);
+  plan.u_row_of.assign(E, 0);
   // Level of a task = 1 + max(level of every update it starts from, level of
   // the client's previous round).  Tasks of one level are mutually independent.
   std::vector<uint32_t> order(E);
@@ -242,17 +243,6 @@ void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan&
     prev_level[e.client] = lv;
     n_waves = std::max(n_waves, lv);
   }
-  // Snapshot slots: one per distinct `seen`; slot 0 is the model at call start.
-  std::vector<int32_t> slot_of(E + 1, -1);
-  slot_of[0] = 0;
-  plan.n_snap = 1;
-  for (const aet_event& e : events) if (slot_of[e.seen] < 0) slot_of[e.seen] = (int32_t)plan.n_snap++;
-  for (size_t k = 0; k < E; ++k) {
-    plan.applies[k].eta = (float)round_step_size(c, events[k].round);
-    plan.applies[k].snap_slot = slot_of[k + 1];
-    plan.applies[k].client = events[k].client;
-    plan.applies[k].round = events[k].round;
-  }
   // Tasks grouped by wave, longest first.
   std::vector<uint32_t> by_wave(E);
   for (size_t k = 0; k < E; ++k) by_wave[k] = (uint32_t)k;
@@ -261,12 +251,93 @@ void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan&
     if (events[a].samples != events[b].samples) return events[a].samples > events[b].samples;
     return a < b;
   });
-  // seq of (client, round) for the in-flight lists
-  std::vector<std::vector<uint32_t>> mine(c.n_clients);
-  for (size_t k = 0; k < E; ++k) mine[events[k].client].push_back((uint32_t)k);
-  plan.tasks.reserve(E);
   plan.wave_off.assign(n_waves + 1, 0);
   plan.apply_upto.assign(n_waves, 0);
+  for (uint32_t k : by_wave) plan.wave_off[level[k]] += 1;   // size of wave level-1, shifted by one
+  for (uint32_t L = 1; L <= n_waves; ++L) plan.wave_off[L] += plan.wave_off[L - 1];
+  for (uint32_t L = 0; L < n_waves; ++L) {
+    plan.max_wave_tasks = std::max(plan.max_wave_tasks, plan.wave_off[L + 1] - plan.wave_off[L]);
+    // the next wave's tasks need every update with seq < their `seen`
+    uint32_t upto = 0;
+    if (L + 1 < n_waves) {
+      for (uint32_t q = plan.wave_off[L + 1]; q < plan.wave_off[L + 2]; ++q)
+        upto = std::max(upto, events[by_wave[q]].seen);
+    } else {
+      upto = (uint32_t)E;
+    }
+    plan.apply_upto[L] = std::max(upto, L ? plan.apply_upto[L - 1] : 0u);
+  }
+  // A client's update sums still in flight when one of its rounds starts.
+  std::vector<std::vector<uint32_t>> mine(c.n_clients);
+  for (size_t k = 0; k < E; ++k) mine[events[k].client].push_back((uint32_t)k);
+  auto for_each_inflight = [&](const aet_event& e, auto&& fn) {
+    for (uint32_t j : mine[e.client])
+      if (events[j].round < e.round && events[j].seq >= e.seen) fn(j);
+  };
+
+  // ---- rows of the update-sum array and snapshot slots ----
+  // Launch order: round kernel of wave 0, aggregation 0, round kernel of wave 1, ...  The row of
+  // update k is written by the round kernel of its wave and last read by the later of the
+  // aggregation that applies it and the round kernels of the tasks that start with it in flight.
+  // The snapshot for start position v is written by the aggregation that applies update v - 1
+  // and last read by the last wave holding a task with seen == v.
+  std::vector<int32_t> slot_of(E + 1, -1);
+  if (keep_all) {
+    for (size_t k = 0; k < E; ++k) plan.u_row_of[k] = (uint32_t)k;
+    plan.n_u_rows = (uint32_t)E;
+    slot_of[0] = 0;
+    plan.n_snap = 1;
+    for (const aet_event& e : events) if (slot_of[e.seen] < 0) slot_of[e.seen] = (int32_t)plan.n_snap++;
+  } else {
+    std::vector<uint32_t> applied_in(E, 0), u_last(E, 0);
+    {
+      uint32_t lo = 0;
+      for (uint32_t L = 0; L < n_waves; ++L) {
+        for (uint32_t k = lo; k < plan.apply_upto[L]; ++k) applied_in[k] = L;
+        lo = plan.apply_upto[L];
+      }
+    }
+    std::vector<int32_t> snap_last(E + 1, -1);   // last wave reading the snapshot of position v
+    for (size_t k = 0; k < E; ++k) {
+      const uint32_t L = level[k] - 1;
+      u_last[k] = std::max(u_last[k], applied_in[k]);
+      snap_last[events[k].seen] = std::max(snap_last[events[k].seen], (int32_t)L);
+      for_each_inflight(events[k], [&](uint32_t j) { u_last[j] = std::max(u_last[j], L); });
+    }
+    std::vector<std::vector<uint32_t>> u_dead_after(n_waves), snap_dead_after(n_waves);
+    for (size_t k = 0; k < E; ++k) u_dead_after[u_last[k]].push_back((uint32_t)k);
+    for (size_t v = 0; v <= E; ++v) if (snap_last[v] >= 0) snap_dead_after[snap_last[v]].push_back((uint32_t)v);
+    std::vector<uint32_t> free_rows, free_slots;
+    slot_of[0] = 0;            // written by the host before the first launch
+    plan.n_snap = 1;
+    uint32_t lo = 0;
+    for (uint32_t L = 0; L < n_waves; ++L) {
+      for (uint32_t q = plan.wave_off[L]; q < plan.wave_off[L + 1]; ++q) {   // round kernel of wave L writes
+        const uint32_t k = by_wave[q];
+        if (free_rows.empty()) { plan.u_row_of[k] = plan.n_u_rows++; }
+        else { plan.u_row_of[k] = free_rows.back(); free_rows.pop_back(); }
+      }
+      // the round kernel of wave L has run when aggregation L writes: its snapshots are free
+      for (uint32_t v : snap_dead_after[L]) free_slots.push_back((uint32_t)slot_of[v]);
+      for (uint32_t k = lo; k < plan.apply_upto[L]; ++k) {                  // aggregation L writes
+        const uint32_t v = k + 1;
+        if (snap_last[v] < 0) continue;
+        if (free_slots.empty()) { slot_of[v] = (int32_t)plan.n_snap++; }
+        else { slot_of[v] = (int32_t)free_slots.back(); free_slots.pop_back(); }
+      }
+      lo = plan.apply_upto[L];
+      for (uint32_t k : u_dead_after[L]) free_rows.push_back(plan.u_row_of[k]);
+    }
+  }
+
+  for (size_t k = 0; k < E; ++k) {
+    plan.applies[k].eta = (float)round_step_size(c, events[k].round);
+    plan.applies[k].snap_slot = slot_of[k + 1];
+    plan.applies[k].client = events[k].client;
+    plan.applies[k].round = events[k].round;
+    plan.applies[k].u_row = plan.u_row_of[k];
+  }
+  plan.tasks.reserve(E);
   for (uint32_t k : by_wave) {
     const aet_event& e = events[k];
     TaskDesc t{};
@@ -275,27 +346,13 @@ void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan&
     t.n_samples = e.samples; t.steps = e.steps;
     t.sample_ctr0 = samples_before(c, e.round);
     t.eta = (float)round_step_size(c, e.round);
+    t.u_row = plan.u_row_of[k];
     t.inflight_off = (uint32_t)plan.inflight.size();
-    for (uint32_t j : mine[e.client])
-      if (events[j].round < e.round && events[j].seq >= e.seen)
-        plan.inflight.push_back({events[j].seq, (float)round_step_size(c, events[j].round)});
+    for_each_inflight(e, [&](uint32_t j) {
+      plan.inflight.push_back({plan.u_row_of[j], (float)round_step_size(c, events[j].round)});
+    });
     t.inflight_cnt = (uint32_t)plan.inflight.size() - t.inflight_off;
-    plan.wave_off[level[k]] += 1;  // size of wave level-1, shifted by one
     plan.tasks.push_back(t);
-  }
-  // wave_off[L] holds the size of wave L-1; a running sum turns it into offsets.
-  for (uint32_t L = 1; L <= n_waves; ++L) plan.wave_off[L] += plan.wave_off[L - 1];
-  for (uint32_t L = 0; L < n_waves; ++L) {
-    plan.max_wave_tasks = std::max(plan.max_wave_tasks, plan.wave_off[L + 1] - plan.wave_off[L]);
-    // the next wave's tasks need every update with seq < their `seen`
-    uint32_t upto = 0;
-    if (L + 1 < n_waves) {
-      for (uint32_t k = plan.wave_off[L + 1]; k < plan.wave_off[L + 2]; ++k)
-        upto = std::max(upto, events[plan.tasks[k].seq].seen);
-    } else {
-      upto = (uint32_t)E;
-    }
-    plan.apply_upto[L] = std::max(upto, L ? plan.apply_upto[L - 1] : 0u);
   }
 }
 

@@ -46,13 +46,14 @@ struct TaskDesc {          // one round-task, read by the local-SGD kernels
   uint32_t inflight_off, inflight_cnt;  // own update sums not yet applied at start
   uint64_t sample_ctr0;    // client's running sample counter at round start
   float eta;               // round step size
-  uint32_t pad;
+  uint32_t u_row;          // row of the update-sum array this round's U_i goes to
 };
-struct InflightRef { uint32_t seq; float eta; };
+struct InflightRef { uint32_t row; float eta; };   // row of the update-sum array, step size of its round
 struct ApplyDesc {         // one server update, in seq order
   float eta;
   int32_t snap_slot;       // where to keep the model after this update (-1: nowhere)
   uint32_t client, round;
+  uint32_t u_row;          // row of the update-sum array that holds U of this update
 };
 struct Plan {
   std::vector<TaskDesc> tasks;       // sorted by wave, longest first inside a wave
@@ -60,9 +61,14 @@ struct Plan {
   std::vector<uint32_t> apply_upto;  // after wave L the server applies seq < apply_upto[L]
   std::vector<InflightRef> inflight;
   std::vector<ApplyDesc> applies;
-  uint32_t n_snap = 0;               // snapshot slots; slot 0 = model at call start
+  std::vector<uint32_t> u_row_of;    // seq -> row of the update-sum array
+  uint32_t n_snap = 0;               // snapshot slots in use at once (slot 0 = model at call start)
+  uint32_t n_u_rows = 0;             // update-sum rows in use at once
   uint32_t max_wave_tasks = 0;
 };
-void build_plan(const aet_config& c, const std::vector<aet_event>& events, Plan& plan);
+// keep_all: one row per event and one slot per distinct start position, never reused
+// (row = seq), so that every update sum can be read back after the run.  Otherwise rows
+// and slots are recycled as soon as nothing later in the launch order reads them.
+void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool keep_all, Plan& plan);
 
 }  // namespace aet

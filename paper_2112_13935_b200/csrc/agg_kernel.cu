@@ -46,11 +46,11 @@ __global__ void __launch_bounds__(kAggThreads) group_totals_kernel(ApplyLaunch p
   for (; k + kAhead <= hi; k += kAhead) {
     float u[kAhead];
 #pragma unroll
-    for (int a = 0; a < kAhead; ++a) u[a] = __ldg(U + (size_t)(k + a) * p.stride);
+    for (int a = 0; a < kAhead; ++a) u[a] = __ldg(U + (size_t)p.applies[k + a].u_row * p.stride);
 #pragma unroll
     for (int a = 0; a < kAhead; ++a) s = fmaf(-p.applies[k + a].eta, u[a], s);
   }
-  for (; k < hi; ++k) s = fmaf(-p.applies[k].eta, __ldg(U + (size_t)k * p.stride), s);
+  for (; k < hi; ++k) s = fmaf(-p.applies[k].eta, __ldg(U + (size_t)p.applies[k].u_row * p.stride), s);
   p.totals[(size_t)blockIdx.y * p.stride + j] = s;
 }
 
@@ -73,20 +73,29 @@ __global__ void __launch_bounds__(kAggThreads) apply_updates_kernel(ApplyLaunch 
     for (; k + kAhead <= hi; k += kAhead) {
       float u[kAhead];
 #pragma unroll
-      for (int a = 0; a < kAhead; ++a) u[a] = __ldcs(U + (size_t)(k + a) * p.stride);
+      ApplyDesc ds[kAhead];
+#pragma unroll
+      for (int a = 0; a < kAhead; ++a) ds[a] = p.applies[k + a];
+#pragma unroll
+      for (int a = 0; a < kAhead; ++a) u[a] = __ldcs(U + (size_t)ds[a].u_row * p.stride);
 #pragma unroll
       for (int a = 0; a < kAhead; ++a) {
-        const ApplyDesc d = p.applies[k + a];
+        const ApplyDesc d = ds[a];
         w = fmaf(-d.eta, u[a], w);
         if (d.snap_slot >= 0) p.snaps[(size_t)d.snap_slot * p.stride + j] = w;
       }
     }
     for (; k < hi; ++k) {
       const ApplyDesc d = p.applies[k];
-      w = fmaf(-d.eta, __ldcs(U + (size_t)k * p.stride), w);
+      w = fmaf(-d.eta, __ldcs(U + (size_t)d.u_row * p.stride), w);
       if (d.snap_slot >= 0) p.snaps[(size_t)d.snap_slot * p.stride + j] = w;
     }
-    if (g + 1 == p.groups) p.w_out[j] = w;
+    if (g + 1 == p.groups) {
+      p.w_out[j] = w;
+      // the server model after this range: a non-finite entry (a NaN or an overflow that came in
+      // through a client's rows or step size) is reported, never trapped on
+      if (p.status && !isfinite(w)) atomicOr(p.status, 2u);
+    }
   }
   // history map and apply log: one thread per update of the group
   if (blockIdx.x == 0)
@@ -105,7 +114,31 @@ __global__ void to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __r
   for (; i < n; i += step) dst[i] = __float2bfloat16_rn(src[i]);
 }
 
+// Debug pass over a client's data set as it is loaded: a label outside [0, n_classes) sets bit 2
+// of *status, a non-finite pixel bit 1.  Nothing is trapped on; the host turns the bits into
+// AET_ERR_STATE / AET_ERR_NUMERIC at its next synchronising call.
+__global__ void validate_data_kernel(const float* __restrict__ x, const int32_t* __restrict__ y, uint32_t n,
+                                     uint32_t dim, uint32_t n_classes, uint32_t* status) {
+  const size_t step = (size_t)gridDim.x * blockDim.x;
+  uint32_t bad = 0;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step)
+    if ((uint32_t)y[i] >= n_classes) bad |= 4u;
+  if (x)
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)n * dim; i += step)
+      if (!isfinite(x[i])) bad |= 2u;
+  if (bad) atomicOr(status, bad);
+}
+
 }  // namespace
+
+cudaError_t launch_validate_data(const float* x, const int32_t* y, uint32_t n, uint32_t dim, uint32_t n_classes,
+                                 uint32_t* status, cudaStream_t s) {
+  if (!n) return cudaSuccess;
+  size_t blocks = ((size_t)n * dim + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  validate_data_kernel<<<(unsigned)blocks, 256, 0, s>>>(x, y, n, dim, n_classes, status);
+  return cudaGetLastError();
+}
 
 uint32_t apply_groups(uint32_t n_updates) {
   uint32_t g = n_updates / 32;

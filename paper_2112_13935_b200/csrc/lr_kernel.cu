@@ -158,6 +158,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
   __shared__ __align__(8) uint64_t full[kStages];
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
+  if (!debug_task_ok(p, t)) return;   // debug checks only: rows and slots in range, else flag and skip
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_raw = warp * kLanes + lane;
   const bool active = lane < kLanes && u_raw < kGroups;
@@ -220,7 +221,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
       }
     for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
       const InflightRef ref = p.inflight[t.inflight_off + f];
-      const float* us = p.U + (size_t)ref.seq * p.stride;
+      const float* us = p.U + (size_t)ref.row * p.stride;
       const float2* u2 = reinterpret_cast<const float2*>(us + (is_bias ? (size_t)kD * kC : (size_t)u * (kPix * kC)));
       const u64 ne = pack2(-ref.eta, -ref.eta);
 #pragma unroll
@@ -390,8 +391,8 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
   // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model) ----
   {
     const size_t off = is_bias ? (size_t)kD * kC : (size_t)u * (kPix * kC);
-    float2* dU = reinterpret_cast<float2*>(p.U + (size_t)t.seq * p.stride + off);
-    float2* dW = p.w_end ? reinterpret_cast<float2*>(p.w_end + (size_t)t.seq * p.stride + off) : nullptr;
+    float2* dU = reinterpret_cast<float2*>(p.U + (size_t)t.u_row * p.stride + off);
+    float2* dW = p.w_end ? reinterpret_cast<float2*>(p.w_end + (size_t)t.u_row * p.stride + off) : nullptr;
 #pragma unroll
     for (int a = 0; a < kPix; ++a)
 #pragma unroll
@@ -544,6 +545,7 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
   constexpr int kGramRanks = kDed ? 2 : kWarps - 1;       // warps sharing the Gram matrix of a block
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
+  if (!debug_task_ok(p, t)) return;   // debug checks only: rows and slots in range, else flag and skip
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool rw = kDed && warp >= kWarps;            // the warps without pixels: R (warp 4), Gram and row copies (warp 5)
   const bool gw = kDed && (warp == kWarps + 1 || warp == kWarps + 2);   // warps 5 and 6
@@ -610,7 +612,7 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
         scale = 1.f;
       } else {
         const InflightRef ref = p.inflight[t.inflight_off + f - 1];
-        row = p.U + (size_t)ref.seq * p.stride;
+        row = p.U + (size_t)ref.row * p.stride;
         scale = -ref.eta;
       }
       if (whole_rows) {
@@ -863,7 +865,7 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model W_start - eta U) ----
   for (int pass = 0; pass < (p.w_end ? 2 : 1); ++pass) {
-    float* dst = (pass == 0 ? p.U : p.w_end) + (size_t)t.seq * p.stride;
+    float* dst = (pass == 0 ? p.U : p.w_end) + (size_t)t.u_row * p.stride;
     float* out = whole_rows ? sm.stage : dst;
     if (whole_rows) {
       if (pass) __syncthreads();   // the previous row has left stage[]

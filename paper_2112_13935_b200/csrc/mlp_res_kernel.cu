@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
 
   const int rank = (int)cluster_rank();
   const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / kCL];
+  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = (int)p.shape.dims[2];
   const ClientData cd = p.r.clients[t.client];
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
     float w = __ldg(snap + j);
     for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
       const InflightRef ref = p.r.inflight[t.inflight_off + f];
-      w = fmaf(-ref.eta, __ldg(p.r.U + (size_t)ref.seq * p.r.stride + j), w);
+      w = fmaf(-ref.eta, __ldg(p.r.U + (size_t)ref.row * p.r.stride + j), w);
     }
     return w;
   };
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
   bool ok = mbar_wait(&sm.wbar, 0);
   for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
     const InflightRef ref = p.r.inflight[t.inflight_off + f];
-    const float4* us = reinterpret_cast<const float4*>(p.r.U + (size_t)ref.seq * p.r.stride + w0_mine);
+    const float4* us = reinterpret_cast<const float4*>(p.r.U + (size_t)ref.row * p.r.stride + w0_mine);
     float4* w4 = reinterpret_cast<float4*>(&sm.W0[0][0]);
     for (int e = tid; e < kR * kH / 4; e += kT) {
       const float4 u = __ldg(us + e);
@@ -385,8 +386,8 @@ __global__ void __launch_bounds__(kT, 1) mlp_res_kernel(MlpLaunch p) {
 
   // ---- event trigger: h reached s_{i,c}; publish U_i (and the end model) ----
   {
-    float* Urow = p.r.U + (size_t)t.seq * p.r.stride;
-    float* Wend = p.r.w_end ? p.r.w_end + (size_t)t.seq * p.r.stride : nullptr;
+    float* Urow = p.r.U + (size_t)t.u_row * p.r.stride;
+    float* Wend = p.r.w_end ? p.r.w_end + (size_t)t.u_row * p.r.stride : nullptr;
     if (warp < kGW) {
 #pragma unroll
       for (int i = 0; i < kRW; ++i) {

@@ -184,6 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
   const bool clustered = C > 1;
   const int rank = clustered ? (int)cluster_rank() : 0;
   const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / C];
+  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int L = (int)S.n_layers, B = (int)S.batch;
   const int D0 = (int)S.dims[0];
@@ -201,7 +202,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
 
   float* act = p.act + (size_t)(blockIdx.x / C) * p.act_stride;
   float* work = p.work + (size_t)t.client * p.r.stride;
-  float* Urow = p.r.U + (size_t)t.seq * p.r.stride;
+  float* Urow = p.r.U + (size_t)t.u_row * p.r.stride;
   const ClientData cd = p.r.clients[t.client];
   const __nv_bfloat16* xdata = reinterpret_cast<const __nv_bfloat16*>(cd.x);
   const uint64_t key = p.r.sample_keys[t.client];
@@ -247,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
         float w = snap[j];
         for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
           const InflightRef ref = p.r.inflight[t.inflight_off + f];
-          w = fmaf(-ref.eta, p.r.U[(size_t)ref.seq * p.r.stride + j], w);
+          w = fmaf(-ref.eta, p.r.U[(size_t)ref.row * p.r.stride + j], w);
         }
         work[j] = w;
         Urow[j] = (kDeriveU0 && l == 0) ? w : 0.f;
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
           float w = snap[boff[l] + j];
           for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
             const InflightRef ref = p.r.inflight[t.inflight_off + f];
-            w = fmaf(-ref.eta, p.r.U[(size_t)ref.seq * p.r.stride + boff[l] + j], w);
+            w = fmaf(-ref.eta, p.r.U[(size_t)ref.row * p.r.stride + boff[l] + j], w);
           }
           work[boff[l] + j] = w;
           Urow[boff[l] + j] = 0.f;
@@ -928,7 +929,7 @@ __global__ void __launch_bounds__(kThreads, 1) mlp_tc_kernel(MlpLaunch p) {
     }
   }
   if (p.r.w_end) {
-    float* dst = p.r.w_end + (size_t)t.seq * p.r.stride;
+    float* dst = p.r.w_end + (size_t)t.u_row * p.r.stride;
     for (int l = 0; l < L; ++l) {
       const int N = (int)S.dims[l + 1];
       const size_t lo = woff[l] + (size_t)r0[l] * N, hi = woff[l] + (size_t)r1[l] * N;
@@ -968,11 +969,11 @@ cudaError_t launch_mlp_tc_rounds(const MlpLaunch& p, cudaStream_t s) {
   // 512-column tensor-memory allocation of one can never wait on a cluster peer.
   size_t smem = (size_t)make_tc_smem(p.shape).total;
   if (smem < 120 * 1024) smem = 120 * 1024;
-  static size_t configured = 0;
-  if (smem > configured) {
+  // The shared-memory opt-in is a per-device attribute of the kernel and cheap to set: set it on
+  // every launch rather than caching it per process (a second device, or two host threads).
+  {
     cudaError_t e = cudaFuncSetAttribute(mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = smem;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(p.r.n_tasks * p.shape.cluster, 1, 1);

@@ -10,6 +10,7 @@
 // that loads the library holds these kMaxScratchBytes until the process exits.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <string>
 
 #include "../../include/aet.h"
@@ -33,7 +34,11 @@ constexpr size_t kMaxScratchBytes = kHeaderBytes + (kMaxParams + kMaxActFloats) 
 // it asks the runtime for the device address once per device (scratch_for).
 static __device__ __align__(256) unsigned char g_scratch[kMaxScratchBytes];
 
-struct Header {  // first kHeaderBytes of the scratch
+// First kHeaderBytes of the scratch.  `status` is where the round kernel would flag a bounded
+// wait that gave up; the generic fp32 kernel this entry point always runs has no such waits, and
+// no call reads the word back.  A kernel with bounded waits must not be routed through here
+// without adding that read.
+struct Header {
   TaskDesc task;
   ClientData client;
   uint64_t key;
@@ -52,7 +57,7 @@ __global__ void fill_header_kernel(TaskDesc t, ClientData c, uint64_t key) {
 }
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_dev_ptr[kMaxDevices] = {};
+std::atomic<unsigned char*> g_dev_ptr[kMaxDevices] = {};   // two host threads may look an address up at once: same value
 
 // Device address of the scratch on the current device; looked up on first use.
 cudaError_t scratch_for_current_device(unsigned char** out) {
@@ -60,13 +65,15 @@ cudaError_t scratch_for_current_device(unsigned char** out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (!g_dev_ptr[dev]) {
+  unsigned char* known = g_dev_ptr[dev].load(std::memory_order_acquire);
+  if (!known) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_scratch);
     if (e != cudaSuccess) return e;
-    g_dev_ptr[dev] = static_cast<unsigned char*>(p);
+    known = static_cast<unsigned char*>(p);
+    g_dev_ptr[dev].store(known, std::memory_order_release);
   }
-  *out = g_dev_ptr[dev];
+  *out = known;
   return cudaSuccess;
 }
 

@@ -65,6 +65,12 @@ CONFIGS = {
     "cfg5": dict(_COMMON, n_clients=1024, model=0, dims=[784, 10], lr=None,
                  sched_a=8, sched_b=8, n_rounds=10,
                  data=dict(kind="per_client", per_client=1024, dim=784)),
+    # The paper's own setting (Appendix Table 2 and A.2): five nodes, s_i = 10 i counted from round 1,
+    # eta_0 = 0.01 diminishing with beta = 0.01, d = 1, uniform delays of 0.1-1 per SGD iteration and
+    # 0.1-1.5 per message; K = 60,000 iterations per node take 110 rounds (61,050 samples).
+    "cfg6": dict(_COMMON, n_clients=5, model=0, dims=[784, 10], lr=0.01, lr_beta=0.01,
+                 sched_a=10, sched_b=0, round_base=1, n_rounds=110, delay_dist=1,
+                 data=dict(kind="iid", total=60000, dim=784)),
 }
 
 

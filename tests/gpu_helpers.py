@@ -25,6 +25,8 @@ def rel_err(got, want):
 
 
 def run_gpu(cfg, data, w0, n_rounds=None, want_U=True):
+    if want_U:   # update sums are recycled during a run unless the handle is told to keep them
+        cfg = dict(cfg, flags=cfg.get("flags", 0) | api.FLAG_KEEP_UPDATE_SUMS)
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
         s.run(n_rounds)
         blob, summary = s.log(raw=True)

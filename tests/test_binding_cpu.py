@@ -111,3 +111,63 @@ def test_create_without_a_gpu_fails_cleanly():
     with pytest.raises(api.AetError) as e:
         api.aet_create(workloads.get_config("cfg1"))
     assert e.value.status == 5
+
+
+def _replay_plan(cfg, n_rounds, events, lay):
+    """Walk the launch order (round kernel of wave 0, aggregation 0, wave 1, ...) keeping track of
+    what every update-sum row and snapshot slot holds, and check that every read finds what it
+    needs: a task its start snapshot and its own sums still in flight, the server every sum it
+    applies."""
+    E = len(events)
+    row_holds = {}            # row -> seq whose update sum it holds
+    slot_holds = {0: 0}       # slot -> start position (number of updates applied) it holds
+    mine = {}
+    for e in events:
+        mine.setdefault(e["client"], []).append(e)
+    lo, q = 0, 0
+    for L in range(lay["waves"]):
+        wave = []
+        while q < E and lay["task_wave"][q] == L:
+            wave.append(q)
+            q += 1
+        assert wave, "empty wave"
+        for t in wave:                                        # reads of the round kernel
+            e = events[int(lay["task_seq"][t])]
+            assert slot_holds.get(int(lay["task_snap_slot"][t])) == e["seen"], (L, e)
+            for f in mine[e["client"]]:
+                if f["round"] < e["round"] and f["seq"] >= e["seen"]:
+                    assert row_holds.get(int(lay["u_row"][f["seq"]])) == f["seq"], (L, e, f)
+        rows = [int(lay["u_row"][int(lay["task_seq"][t])]) for t in wave]
+        assert len(set(rows)) == len(rows), "two tasks of a wave share a row"
+        for t in wave:                                        # its writes
+            row_holds[int(lay["u_row"][int(lay["task_seq"][t])])] = int(lay["task_seq"][t])
+        hi = int(lay["apply_upto"][L])
+        for k in range(lo, hi):                               # the aggregation, in seq order
+            assert row_holds.get(int(lay["u_row"][k])) == k, (L, k)
+            s = int(lay["snap_slot_after"][k])
+            if s >= 0:
+                slot_holds[s] = k + 1
+        lo = hi
+    assert q == E and lo == E
+    assert max(row_holds) < lay["n_u_rows"] and max(slot_holds) < lay["n_snap"]
+
+
+@pytest.mark.parametrize("name,over", [
+    ("cfg1", {}), ("cfg2", {}), ("cfg5", dict(n_clients=128)),
+    ("cfg1", dict(n_clients=3, n_rounds=8, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=500.0)),
+    ("cfg1", dict(n_clients=7, n_rounds=9, max_lag_d=0)),
+    ("cfg2", dict(max_lag_d=3, network_delay_mean=20.0)),
+])
+def test_recycled_rows_and_slots_always_hold_what_is_read(name, over):
+    cfg = workloads.get_config(name, **over)
+    R = cfg["n_rounds"]
+    events, _, _ = schedule.simulate(cfg, R)
+    lay = api.aet_debug_plan_layout(cfg, R)
+    _replay_plan(cfg, R, events, lay)
+    keep = api.aet_debug_plan_layout(dict(cfg, flags=api.FLAG_KEEP_UPDATE_SUMS), R)
+    _replay_plan(cfg, R, events, keep)
+    assert keep["n_u_rows"] == len(events) and list(keep["u_row"]) == list(range(len(events)))
+    assert lay["n_u_rows"] <= keep["n_u_rows"] and lay["n_snap"] <= keep["n_snap"]
+    assert lay["waves"] == keep["waves"] == api.aet_debug_plan_waves(cfg, R)
+    if name == "cfg2" and not over:
+        assert lay["n_u_rows"] < len(events) // 4     # recycling pays: rows ~ rounds in flight

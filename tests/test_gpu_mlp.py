@@ -10,7 +10,10 @@ from gpu_helpers import U_TOL, check_against_oracle, check_round_U, make, rel_er
 
 pytestmark = pytest.mark.gpu
 
-BF16_U_TOL = 2e-3   # precision 1: an fp32-vs-fp64 sum can flip a bf16 rounding (2^-8 relative)
+# precision 1: an fp32-vs-fp64 difference in a sum can flip one bf16 rounding (2^-8 relative on that
+# element), so the fp32 bar cannot hold; the bar is twice the worst per-round error measured over these
+# cases (1.4e-4).  The same shapes with fp32 operands meet the fp32 bar (test below).
+BF16_U_TOL = 3e-4
 
 
 def _small_cfg3(**kw):
@@ -87,24 +90,57 @@ def test_mlp_bf16_tensor_core_path(over):
     print("tensor-core path per-round U errors:", ["%.1e" % v for v in errs])
 
 
-def test_cfg3_full_size_log_invariant_and_sampled_rounds():
+def test_bf16_shapes_with_fp32_operands_meet_the_fp32_bar():
+    # the cut-down cfg4 of the bf16 test above, precision 0: every per-round update sum within 1e-5
+    cfg = workloads.get_config("cfg4", precision=0, n_clients=4, n_rounds=3, dims=[3072, 64, 32, 10],
+                               n_stragglers=1, data=dict(total=800))
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert rel_err(gpu["w"], ref["w"]) <= 2e-5
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for e in ref["events"]:
+            check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], U_TOL)
+
+
+def test_cfg3_full_size_against_the_checker():
     cfg = workloads.get_config("cfg3")
     data, w0 = make(cfg)
-    from oracle import schedule
-    events, summary, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    picks = {0, 500, 1279}
+    ref = sim.run(cfg, data, w0, keep=picks)
     gpu = run_gpu(cfg, data, w0)
-    assert gpu["blob"] == schedule.pack_events(events) and gpu["summary"] == summary
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert rel_err(gpu["w"], ref["w"]) <= 5e-5
     acc = w0.astype(np.float64)
-    for e in events:
+    for e in ref["events"]:
         acc -= sim.step_size(cfg, e["round"]) * gpu["U"][e["seq"]].astype(np.float64)
     assert np.abs(acc - gpu["w"]).max() <= 2e-6 * max(1.0, np.abs(acc).max())
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
-        for c, i in ((0, 0), (31, 7), (13, 39)):
-            check_round_U(cfg, data, s.h, c, i, gpu["w"])
+        for k in picks:
+            e = ref["events"][k]
+            check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][k])
+
+
+def test_cfg4_real_dims_first_rounds_against_the_checker():
+    # 3072-256-128-10, all 64 clients with their stragglers, the launch configuration bench.py times
+    # (clusters of 2, every wide layer on tensor cores); the first 8 rounds = 294,912 samples
+    cfg = workloads.get_config("cfg4", n_rounds=8)
+    data, w0 = make(cfg)
+    picks = {0, 255, 511}
+    ref = sim.run(cfg, data, w0, keep=picks)
+    gpu = run_gpu(cfg, data, w0, want_U=False)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert rel_err(gpu["w"], ref["w"]) <= 1e-3
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        errs = [check_round_U(cfg, data, s.h, ref["events"][k]["client"], ref["events"][k]["round"],
+                              ref["w_start"][k], BF16_U_TOL) for k in picks]
+    print("cfg4 per-round U errors:", ["%.1e" % v for v in errs])
 
 
 def test_cfg4_full_size_log_and_sampled_rounds():
-    # full size, the launch configuration bench.py times: clusters of 2, all layers with 128-row slices on tensor cores
+    # full size: 30 rounds, 3.8 M samples; the checker would need ten minutes for it, so the log is compared
+    # in full and three rounds are restarted on both sides from the GPU's final model
     cfg = workloads.get_config("cfg4")
     data, w0 = make(cfg)
     from oracle import schedule
