@@ -90,6 +90,12 @@ typedef struct {
  * soon as the server has applied them (memory ~ rounds in flight, not all
  * rounds of the call). */
 #define AET_FLAG_KEEP_UPDATE_SUMS 4u
+/* Softmax regression with many clients takes eight steps of the recursion at
+ * once and, where the coupling eta * (x_s . x_t) between them is small, solves
+ * for the eight logit vectors by sweeps that stop when they no longer move
+ * (2e-7).  This flag makes the kernel always walk the eight steps one after
+ * the other instead (same result up to that tolerance; slower). */
+#define AET_FLAG_STEPWISE_RECURRENCE 8u
 
 /* One round-task = one message (c, U_i, i) of Algorithm 3.  64 bytes.
  * Times are integer ticks (2^20 per time unit). */

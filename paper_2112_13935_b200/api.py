@@ -12,7 +12,7 @@ import numpy as np
 from . import _lib
 from ._lib import AetConfig, AetEvent, AetStats, AetSummary, NEVER_WAIT, STATUS_NAMES  # noqa: F401
 
-FLAG_BORROW_DATA, FLAG_DEBUG_CHECKS, FLAG_KEEP_UPDATE_SUMS = 1, 2, 4   # AET_FLAG_* of include/aet.h
+FLAG_BORROW_DATA, FLAG_DEBUG_CHECKS, FLAG_KEEP_UPDATE_SUMS, FLAG_STEPWISE_RECURRENCE = 1, 2, 4, 8   # AET_FLAG_*
 
 
 class AetError(RuntimeError):

@@ -229,7 +229,7 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   const uint32_t P = count_params(*cfg);
   if (!P) return fail(nullptr, AET_ERR_CONFIG, "model too large");
   if (cfg->dims[cfg->n_layers] > 32) return fail(nullptr, AET_ERR_CONFIG, "at most 32 classes are supported");
-  if (cfg->flags & ~(uint32_t)(AET_FLAG_BORROW_DATA | AET_FLAG_DEBUG_CHECKS | AET_FLAG_KEEP_UPDATE_SUMS))
+  if (cfg->flags & ~(uint32_t)(AET_FLAG_BORROW_DATA | AET_FLAG_DEBUG_CHECKS | AET_FLAG_KEEP_UPDATE_SUMS | AET_FLAG_STEPWISE_RECURRENCE))
     return fail(nullptr, AET_ERR_CONFIG, "unknown bit in flags");
   int dev = 0;
   cudaError_t ce = cudaGetDevice(&dev);
@@ -427,6 +427,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   r.sample_keys = h->d_keys.p; r.snaps = h->snaps.p; r.U = h->U.p; r.w_end = nullptr;
   r.trig = h->d_trig.p; r.status = h->d_status.p; r.stride = h->stride; r.l2 = h->cfg.l2;
   r.debug_checks = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) ? 1u : 0u;
+  r.step_by_step = (h->cfg.flags & AET_FLAG_STEPWISE_RECURRENCE) ? 1u : 0u;
   r.n_u_rows = plan.n_u_rows; r.n_snap = plan.n_snap;
   ApplyLaunch a{};
   a.applies = h->d_applies.p; a.U = h->U.p; a.snaps = h->snaps.p; a.totals = h->totals.p;
@@ -562,7 +563,15 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   r.snaps = snap; r.U = U; r.w_end = wend; r.trig = dtrig; r.status = h->d_status.p; r.stride = h->stride;
   r.task_begin = 0; r.n_tasks = 1; r.l2 = h->cfg.l2;
   r.debug_checks = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) ? 1u : 0u;
+  r.step_by_step = (h->cfg.flags & AET_FLAG_STEPWISE_RECURRENCE) ? 1u : 0u;
   r.n_u_rows = 1; r.n_snap = 1;
+  // the kernel a full wave of this handle's clients would run, so that this parity aid checks it
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
+      r.crowded_hint = h->cfg.n_clients > (uint32_t)sms ? 1u : 0u;
+    cudaGetLastError();
+  }
   const aet_stats keep = h->stats;
   const bool timing = h->timing;
   h->timing = false;

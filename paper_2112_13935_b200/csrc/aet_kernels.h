@@ -38,6 +38,9 @@ struct RoundLaunch {
   size_t stride;
   uint32_t task_begin, n_tasks;
   uint32_t n_u_rows, n_snap;     // extents of U and snaps (for the debug checks)
+  uint32_t crowded_hint;         // non-zero: pick the kernel a full wave of this run's clients would get,
+                                 // however few tasks this launch holds (single-task parity runs)
+  uint32_t step_by_step;         // non-zero: the recurrence of a block is always walked step by step
   float l2;
 };
 
@@ -48,6 +51,9 @@ cudaError_t launch_wait_probe(uint32_t* status, uint32_t max_polls, cudaStream_t
 // how many round-tasks the launch holds.  Asynchronous on s; may start under the tail of the previous kernel in s
 // (programmatic stream serialisation) and waits on the device before reading that kernel's output.
 cudaError_t launch_lr_rounds(const RoundLaunch& p, cudaStream_t s);
+// lambda = 0, more round-tasks than SMs: update sum in tensor memory, accumulated by tcgen05.mma (tf32 x 3)
+bool lr_tc_eligible(const RoundLaunch& p);
+cudaError_t launch_lr_tc_rounds(const RoundLaunch& p, cudaStream_t s);
 
 struct MlpShape {
   uint32_t n_layers, dims[8], batch, precision;

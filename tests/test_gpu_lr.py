@@ -133,6 +133,32 @@ def test_many_clients_take_the_kernel_variant_for_crowded_waves(n_clients, l2):
 
 
 @pytest.mark.parametrize("over", [
+    dict(),                                                    # cfg5's step size: weak coupling, a few sweeps per block
+    dict(flags=api.FLAG_STEPWISE_RECURRENCE),                  # the same walked step by step
+    dict(lr=0.002),                                            # stronger coupling: more sweeps
+    dict(lr=0.05),                                             # coupling too strong for the sweeps: the kernel walks
+    dict(sched_a=3, sched_b=1, n_rounds=9),                    # rounds of 1, 4, 7, ... samples: every tail length
+    dict(max_lag_d=workloads.NEVER_WAIT, network_delay_mean=50.0, n_rounds=4),   # own sums in flight at round start
+])
+def test_tensor_memory_kernel_every_sampled_round_from_the_checkers_start_model(over):
+    # more clients than SMs: the kernel that keeps U in tensor memory (tcgen05.mma, tf32 x 3); the single-round
+    # parity call of such a handle runs that kernel too
+    over = dict(dict(n_clients=200, n_rounds=6, data=dict(per_client=96)), **over)
+    cfg = workloads.get_config("cfg5", **over)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 2e-5
+    for k in range(0, len(ref["events"]), 23):
+        assert rel_err(gpu["U"][k], ref["U"][k]) <= 1e-4, k
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
+                for e in ref["events"][::41]]
+    print("tensor-memory kernel per-round U errors: max %.1e" % max(errs))
+
+
+@pytest.mark.parametrize("over", [
     dict(max_lag_d=0), dict(max_lag_d=workloads.NEVER_WAIT, network_delay_mean=20.0),
     dict(n_clients=1), dict(lr_beta=0.05, l2=0.0), dict(delay_dist=1, n_stragglers=1, straggler_factor=30.0),
     dict(sched_a=3, sched_b=1, n_rounds=7),   # ragged: rounds of 1, 4, 7, ... samples
