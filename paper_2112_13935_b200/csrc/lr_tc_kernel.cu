@@ -64,7 +64,8 @@ struct __align__(128) TcSmem {
   int ys[kRing][kM];
   uint64_t full[kRing];
   uint64_t staged;
-  uint64_t mma_done;
+  uint64_t delta_ready;            // R has written the block's delta operand
+  uint64_t mma_done;               // the seven tiles' products of a block have completed
   uint32_t tmem_base;
 };
 static_assert(sizeof(float) * 2 * kTiles * 2 * 128 * 4 >= sizeof(float) * kStageFloats, "staging area fits the operand tiles");
@@ -94,10 +95,12 @@ __device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, uint32_t (&v)[8])
                : "r"(taddr));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Nearest tf32 (10 stored mantissa bits) of a finite fp32, as fp32: exactly representable in the
-// tensor cores' input format whatever they do with the low 13 bits.
+// Nearest tf32 (10 stored mantissa bits, low 13 bits of the word zero) of a finite fp32, as fp32:
+// exactly representable in the tensor cores' input format whatever they do with the low bits.
 __device__ __forceinline__ float tf32_head(float v) {
-  return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+  return __uint_as_float(r);
 }
 
 template <bool kSweep>
@@ -125,7 +128,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
 #pragma unroll
     for (int s = 0; s < kRing; ++s) mbar_init(&sm.full[s], 1);
     mbar_init(&sm.staged, 1);
-    mbar_init(&sm.mma_done, 1);
+    mbar_init(&sm.delta_ready, 1);
+    mbar_init(&sm.mma_done, kTiles);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (threadIdx.x < 8) sm.consts[threadIdx.x] = threadIdx.x == 0 ? 1.f : 0.f;
@@ -151,6 +155,9 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
       bulk_load_row(sm.rows[sb][lane], xrows + (size_t)idx * kD, &sm.full[sb]);
       sm.ys[sb][lane] = __ldg(cd.y + idx);
     }
+    // a short last block: the rows nobody copies are zeroed, so that they add nothing anywhere
+    for (uint32_t r = nvb; r < (uint32_t)kM; ++r)
+      for (int i = lane; i < kD; i += 32) sm.rows[sb][r][i] = 0.f;
   };
 
   // ---- start model: server snapshot minus own update sums still in flight ----
@@ -282,19 +289,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
         const int rs = j < kTiles - 1 ? kD : rs6;
         float x[kM];
 #pragma unroll
-        for (int s = 0; s < kM; ++s) {
-          const float v = xp[s * rs];
-          x[s] = (uint32_t)s < nv ? v : 0.f;     // a short last block: rows nobody copied stay out
-        }
+        for (int s = 0; s < kM; ++s) x[s] = xp[s * rs];   // rows of a short last block were zeroed by the producer
 #pragma unroll
         for (int s = 0; s < kM; ++s)
 #pragma unroll
           for (int c = 0; c < kCh; ++c) acc[s][c] = fmaf(x[s], W[c], acc[s][c]);
         float o8[kM];
+        if (ch == 0) {   // warp-uniform: the heads
 #pragma unroll
-        for (int s = 0; s < kM; ++s) {
-          const float hi = tf32_head(x[s]);
-          o8[s] = ch == 0 ? hi : x[s] - hi;
+          for (int s = 0; s < kM; ++s) o8[s] = tf32_head(x[s]);
+        } else {         // the remainders
+#pragma unroll
+          for (int s = 0; s < kM; ++s) o8[s] = x[s] - tf32_head(x[s]);
         }
         *reinterpret_cast<float4*>(&sm.A[ch][j][0][row][0]) = make_float4(o8[0], o8[1], o8[2], o8[3]);
         *reinterpret_cast<float4*>(&sm.A[ch][j][1][row][0]) = make_float4(o8[4], o8[5], o8[6], o8[7]);
@@ -434,22 +440,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) {
-        // ---- U: U^T += X^T delta on the tensor cores, hi.hi + lo.hi + hi.lo ----
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t bhi = umma_desc(smem_addr(&sm.B[0][0][0][0]), 256, 128);
-        const uint64_t blo = umma_desc(smem_addr(&sm.B[1][0][0][0]), 256, 128);
-#pragma unroll
-        for (int jt = 0; jt < kTiles; ++jt) {
-          const uint64_t ahi = umma_desc(smem_addr(&sm.A[0][jt][0][0][0]), 2048, 128);
-          const uint64_t alo = umma_desc(smem_addr(&sm.A[1][jt][0][0][0]), 2048, 128);
-          const uint32_t d = tmem + 16u * jt;
-          umma_tf32(d, ahi, bhi, k ? 1u : 0u);
-          umma_tf32(d, alo, bhi, 1u);
-          umma_tf32(d, ahi, blo, 1u);
-        }
-        umma_commit(&sm.mma_done);
-      }
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&sm.delta_ready)) : "memory");
     } else if (rel <= kGramRanks) {
       if (k + 1 < nblk) {
         ok = mbar_wait(&sm.full[(k + 1) % kRing], ((k + 1) / kRing) & 1) && ok;
@@ -458,6 +449,26 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
     } else if (rel == kGramRanks + 1) {
       // block k+2 takes the slot of block k: free since barrier A
       if (k + 2 < nblk) produce(k + 2);
+    }
+    if (rel != 0) {
+      // ---- U: U^T += X^T delta on the tensor cores, hi.hi + lo.hi + hi.lo.  Each of the seven warps
+      // other than R issues the three products of one 128-pixel tile (an instruction keeps its
+      // issuing thread for some 80 cycles, whatever its size) and commits them to mma_done.
+      ok = mbar_wait(&sm.delta_ready, k & 1) && ok;
+      if (lane == 0 && ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int jt = rel - 1;
+        const uint64_t bhi = umma_desc(smem_addr(&sm.B[0][0][0][0]), 256, 128);
+        const uint64_t blo = umma_desc(smem_addr(&sm.B[1][0][0][0]), 256, 128);
+        const uint64_t ahi = umma_desc(smem_addr(&sm.A[0][jt][0][0][0]), 2048, 128);
+        const uint64_t alo = umma_desc(smem_addr(&sm.A[1][jt][0][0][0]), 2048, 128);
+        const uint32_t d = tmem + 16u * jt;
+        umma_tf32(d, ahi, bhi, k ? 1u : 0u);
+        umma_tf32(d, alo, bhi, 1u);
+        umma_tf32(d, ahi, blo, 1u);
+        umma_commit(&sm.mma_done);
+      }
+      __syncwarp();
     }
   }
 
