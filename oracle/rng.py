@@ -19,7 +19,7 @@ Section 5 "System delay").  The convention used here:
 
 MASK64 = (1 << 64) - 1
 GAMMA = 0x9E3779B97F4A7C15
-STREAM_SAMPLE, STREAM_COMPUTE, STREAM_NETWORK = 0, 1, 2
+STREAM_SAMPLE, STREAM_COMPUTE, STREAM_NETWORK, STREAM_SETUP = 0, 1, 2, 3
 TICKS_PER_UNIT = 1 << 20
 LN2_Q32 = 2977044471  # floor(ln(2) * 2^32)
 

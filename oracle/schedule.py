@@ -63,6 +63,65 @@ def round_step_size(lr: float, beta: float, t: int) -> float:
     return lr / (1.0 + beta * math.sqrt(t))
 
 
+# ---- Algorithm 2, "Setup": the coin-flip split of a global round size among the nodes ----
+# With cfg["split_mode"] == 1 the sequence s_i = a*i + b is the GLOBAL number of SGD iterations
+# of round i; each of its iterations t is assigned to node c with probability p_c
+# (a(i, t) = c) and s_{i,c} = |{t : a(i, t) = c}|, so E[s_{i,c}] = p_c s_i.  p_c is given by
+# integer shares (p_c = shares[c] / sum(shares); all equal when absent: the paper's p_c = 1/n).
+# The coin of iteration t of round i is draw number (iterations of all earlier rounds) + t of
+# the stream (seed, SETUP, client 0); node = first c whose cumulative share exceeds
+# floor(hi32(draw) * sum(shares) / 2^32).  A node may get no iteration in a round: it then
+# sends U = 0 at once (Algorithm 3 sends after the inner loop, however short).
+def split_mode(cfg) -> int:
+    return cfg.get("split_mode", 0)
+
+
+def client_shares(cfg):
+    sh = cfg.get("client_shares")
+    return list(sh) if sh else [1] * cfg["n_clients"]
+
+
+def assign_node(r: int, shares) -> int:
+    """Node a coin (one 64-bit draw) falls to."""
+    v = ((r >> 32) * sum(shares)) >> 32
+    acc = 0
+    for c, w in enumerate(shares):
+        acc += w
+        if v < acc:
+            return c
+    raise AssertionError("coin outside the shares")
+
+
+def split_round(cfg, i: int):
+    """[s_{i,c} for every node c] of global round i (split_mode 1)."""
+    a, b, base = cfg["sched_a"], cfg["sched_b"], cfg["round_base"]
+    key = rng.stream_key(cfg["seed"], rng.STREAM_SETUP, 0)
+    g0 = samples_before(a, b, base, i)
+    shares = client_shares(cfg)
+    out = [0] * cfg["n_clients"]
+    for t in range(sample_size(a, b, i)):
+        out[assign_node(rng.draw(key, g0 + t), shares)] += 1
+    return out
+
+
+def node_sample_size(cfg, c: int, i: int, _cache={}) -> int:
+    """s_{i,c}: the node's own sequence (split_mode 0) or its share of the global round (1)."""
+    if not split_mode(cfg):
+        return sample_size(cfg["sched_a"], cfg["sched_b"], i)
+    k = (cfg["seed"], cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["n_clients"],
+         tuple(client_shares(cfg)), i)
+    if k not in _cache:
+        _cache[k] = split_round(cfg, i)
+    return _cache[k][c]
+
+
+def node_samples_before(cfg, c: int, i: int) -> int:
+    """Samples node c has consumed before round i."""
+    if not split_mode(cfg):
+        return samples_before(cfg["sched_a"], cfg["sched_b"], cfg["round_base"], i)
+    return sum(node_sample_size(cfg, c, j) for j in range(cfg["round_base"], i))
+
+
 def new_state(cfg):
     return dict(clock=0, H=[0] * cfg["n_clients"], rounds_done=0)
 
@@ -126,11 +185,11 @@ def simulate(cfg, n_rounds, state=None):
         if d != NEVER_WAIT and lag > d:
             blocked[c] = i
             continue
-        s = sample_size(a, b, i)
+        s = node_sample_size(cfg, c, i)
         if s % B:
             raise ValueError("batch must divide every s_i")
         steps = s // B
-        it0 = samples_before(a, b, base, i) // B
+        it0 = node_samples_before(cfg, c, i) // B
         straggler = c >= n - cfg["n_stragglers"]
         busy = 0
         for j in range(steps):
@@ -153,6 +212,8 @@ def simulate(cfg, n_rounds, state=None):
     events.sort(key=lambda e: e["seq"])
     samples_total = sum(e["samples"] for e in events)
     s_first = sample_size(a, b, base)
+    if split_mode(cfg):
+        s_first = max(1, s_first // n)     # a node's expected share of the first global round
     per_client = samples_total // n if n else 0
     summary = dict(
         messages_up=len(events), model_pulls=len(events), samples_total=samples_total,

@@ -22,18 +22,19 @@ def f32(v) -> float:
     return float(np.float32(v))
 
 
-def step_size(cfg, i):
-    a, b, base, B = cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["batch"]
-    t = schedule.samples_before(a, b, base, i) // B
+def step_size(cfg, i, c=0):
+    """Round step size of node c's round i: t = the node's own iterations before the round
+    (every node has the same count unless the Setup split of Algorithm 2 is on)."""
+    t = schedule.node_samples_before(cfg, c, i) // cfg["batch"]
     return schedule.round_step_size(f32(cfg["lr"]), f32(cfg["lr_beta"]), t)
 
 
 def task_indices(cfg, c, i, n_c):
     """Sample indices of round-task (c, i), shape [steps, B] (with replacement,
     keyed by the client's running sample counter)."""
-    a, b, base, B = cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["batch"]
-    k0 = schedule.samples_before(a, b, base, i)
-    s = schedule.sample_size(a, b, i)
+    B = cfg["batch"]
+    k0 = schedule.node_samples_before(cfg, c, i)
+    s = schedule.node_sample_size(cfg, c, i)
     key = rng.stream_key(cfg["seed"], rng.STREAM_SAMPLE, c)
     idx = [rng.sample_index(rng.draw(key, k0 + k), n_c) for k in range(s)]
     return np.asarray(idx, dtype=np.int64).reshape(s // B, B)
@@ -43,7 +44,7 @@ def run_task(cfg, client_data, c, i, w_start):
     """One round of client c from model w_start: returns (U_i, w_end)."""
     X, y = client_data
     dims, l2, prec = cfg["dims"], f32(cfg["l2"]), cfg["precision"]
-    eta = step_size(cfg, i)
+    eta = step_size(cfg, i, c)
     w = np.array(w_start, dtype=np.float64)
     U = np.zeros_like(w)
     for idx in task_indices(cfg, c, i, len(y)):
@@ -74,14 +75,14 @@ def run(cfg, data, w0, n_rounds=None, keep=False, state=None):
         if kind == schedule.START:
             w_start = w_g.copy()
             for f in in_flight[c]:
-                w_start -= step_size(cfg, f["round"]) * U_by_seq[f["seq"]]
+                w_start -= step_size(cfg, f["round"], c) * U_by_seq[f["seq"]]
             U, _ = run_task(cfg, data[c], c, i, w_start)
             U_by_seq[e["seq"]] = U
             if keep is True or (keep and e["seq"] in keep):
                 w_start_by_seq[e["seq"]] = w_start
             in_flight[c].append(e)
         else:
-            w_g -= step_size(cfg, i) * U_by_seq[e["seq"]]
+            w_g -= step_size(cfg, i, c) * U_by_seq[e["seq"]]
             in_flight[c].remove(e)
     assert all(not v for v in in_flight.values())
     return dict(events=events, summary=summary, w=w_g, U=U_by_seq, w_start=w_start_by_seq,

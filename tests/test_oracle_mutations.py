@@ -137,3 +137,27 @@ def test_a_moved_or_dropped_bf16_rounding_point_is_caught(monkeypatch, old, new)
 def test_step_size_without_the_square_root_is_caught(monkeypatch):
     monkeypatch.setattr(schedule, "round_step_size", lambda lr, beta, t: lr / (1.0 + beta * t))
     _fails(ts.test_round_step_size_values_worked_by_hand)
+
+
+def test_setup_split_that_reuses_the_coins_of_every_round_is_caught(monkeypatch):
+    real = schedule.samples_before
+    # coins keyed by the position inside the round only: every round replays the same coins
+    monkeypatch.setattr(schedule, "split_round", lambda cfg, i: (
+        lambda key, sh: [sum(1 for t in range(schedule.sample_size(cfg["sched_a"], cfg["sched_b"], i))
+                             if schedule.assign_node(rng.draw(key, t), sh) == c) for c in range(cfg["n_clients"])])(
+        rng.stream_key(cfg["seed"], rng.STREAM_SETUP, 0), schedule.client_shares(cfg)))
+    _fails(ts.test_setup_split_uses_a_fresh_coin_for_every_iteration_of_every_round)
+
+
+def test_setup_split_by_independent_draws_per_node_is_caught(monkeypatch):
+    # each node flips its own coins: the expectation is right, the round total is not conserved
+    def independent(cfg, i):
+        n, sh = cfg["n_clients"], schedule.client_shares(cfg)
+        s_i = schedule.sample_size(cfg["sched_a"], cfg["sched_b"], i)
+        out = []
+        for c in range(n):
+            key = rng.stream_key(cfg["seed"], rng.STREAM_SETUP, c)
+            out.append(sum(1 for t in range(s_i) if ((rng.draw(key, 1000 * i + t) >> 32) * sum(sh)) >> 32 < sh[c]))
+        return out
+    monkeypatch.setattr(schedule, "split_round", independent)
+    _fails(ts.test_setup_split_conserves_every_round_and_reduces_to_one_node)

@@ -5,7 +5,7 @@ import os
 
 import pytest
 
-from oracle import schedule
+from oracle import rng, schedule
 from paper_2112_13935_b200 import workloads
 
 HERE = os.path.dirname(os.path.abspath(__file__))
@@ -210,3 +210,66 @@ def test_packed_log_layout():
     assert len(blob) == 64 * 6
     first = schedule.EVENT_STRUCT.unpack_from(blob, 0)
     assert first == (0, 4, 9, 0, 0, 0, 1, 1, 0, 0, 0, 0)
+
+
+# ---- Algorithm 2 "Setup": the coin-flip split of the global round size ----
+def _split_cfg(**kw):
+    return workloads.get_config("cfg1", split_mode=1, l2=0.0, **kw)
+
+
+def test_setup_split_conserves_every_round_and_reduces_to_one_node():
+    # s_{i,c} = |{t : a(i,t) = c}|: every iteration of a round goes to exactly one node
+    cfg = _split_cfg(n_clients=7, sched_a=10, sched_b=3)
+    for i in range(12):
+        per_node = schedule.split_round(cfg, i)
+        assert sum(per_node) == 10 * i + 3 and len(per_node) == 7 and min(per_node) >= 0
+        assert per_node == [schedule.node_sample_size(cfg, c, i) for c in range(7)]
+    one = _split_cfg(n_clients=1, sched_a=10, sched_b=3)
+    assert [schedule.node_sample_size(one, 0, i) for i in range(6)] == [10 * i + 3 for i in range(6)]
+    assert schedule.node_samples_before(one, 0, 4) == 3 + 13 + 23 + 33
+
+
+def test_setup_split_expectation_is_p_c_times_s_i():
+    # E[s_{i,c}] = p_c s_i (the remark after Algorithm 2); shares 1 : 3 : 4 over 8,000 coins
+    cfg = _split_cfg(n_clients=3, sched_a=0, sched_b=8000, client_shares=[1, 3, 4])
+    got = schedule.split_round(cfg, 0)
+    for c, p in enumerate((1 / 8, 3 / 8, 4 / 8)):
+        sd = (8000 * p * (1 - p)) ** 0.5
+        assert abs(got[c] - 8000 * p) < 4.5 * sd, (c, got)
+    # equal shares: p_c = 1/n, chi-square over 5 nodes (4 degrees of freedom, 0.999 quantile 18.5)
+    uni = schedule.split_round(_split_cfg(n_clients=5, sched_a=0, sched_b=10000), 0)
+    assert sum((g - 2000) ** 2 / 2000 for g in uni) < 18.5
+
+
+def test_setup_split_uses_a_fresh_coin_for_every_iteration_of_every_round():
+    # rounds do not repeat one another's coins, and a round's split does not depend on how far the run goes
+    cfg = _split_cfg(n_clients=4, sched_a=0, sched_b=64)
+    rounds = [schedule.split_round(cfg, i) for i in range(6)]
+    assert len({tuple(r) for r in rounds}) > 1
+    seq = []
+    key = rng.stream_key(cfg["seed"], rng.STREAM_SETUP, 0)
+    for g in range(6 * 64):
+        seq.append(schedule.assign_node(rng.draw(key, g), [1, 1, 1, 1]))
+    assert len(set(zip(seq[:64], seq[64:128]))) > 4          # consecutive rounds are not copies of each other
+    for i in range(6):
+        assert rounds[i] == [seq[64 * i:64 * i + 64].count(c) for c in range(4)]
+    # assign_node on the extremes of the coin: first and last node
+    assert schedule.assign_node(0, [2, 1, 1]) == 0 and schedule.assign_node((1 << 64) - 1, [2, 1, 1]) == 2
+    assert schedule.assign_node(1 << 63, [2, 1, 1]) == 1      # v = floor(2^31 * 4 / 2^32) = 2: past node 0's two shares
+
+
+def test_setup_split_log_counts_and_step_sizes_follow_each_nodes_own_sequence():
+    from oracle import sim
+    cfg = _split_cfg(n_clients=3, sched_a=6, sched_b=3, n_rounds=6, lr_beta=0.05, client_shares=[1, 2, 3])
+    events, summary, _ = schedule.simulate(cfg, 6)
+    assert len(events) == 18 and summary["samples_total"] == sum(6 * i + 3 for i in range(6))
+    for e in events:
+        assert e["samples"] == schedule.node_sample_size(cfg, e["client"], e["round"]) == e["steps"]
+        assert e["t_start"] <= e["t_trigger"] < e["t_apply"]
+        if e["samples"] == 0:
+            assert e["t_trigger"] == e["t_start"]             # nothing to compute: the (zero) sum goes out at once
+    # node 2 runs about three times node 0's iterations, so its step size has diminished further by round 5
+    assert schedule.node_samples_before(cfg, 2, 5) > schedule.node_samples_before(cfg, 0, 5)
+    assert sim.step_size(cfg, 5, 2) < sim.step_size(cfg, 5, 0) < sim.f32(cfg["lr"])
+    t0 = schedule.node_samples_before(cfg, 0, 5)
+    assert abs(sim.step_size(cfg, 5, 0) - sim.f32(cfg["lr"]) / (1 + sim.f32(0.05) * t0 ** 0.5)) < 1e-15
