@@ -72,6 +72,15 @@ typedef struct {
   double straggler_factor; /* scales the compute delay of the stragglers          */
   uint32_t n_stragglers;   /* the last n_stragglers client ids                    */
   uint32_t flags;          /* AET_FLAG_* bits, 0 for the defaults                  */
+  uint32_t split_mode;     /* 0: every node runs its own sequence s_{i,c} = a*i + b (the
+                              paper's experiments, Appendix A.2).  1: Algorithm 2, Setup:
+                              s_i = a*i + b is the global size of round i and each of its
+                              iterations goes to node c with probability p_c, so that
+                              s_{i,c} = |{t : a(i,t) = c}| and E[s_{i,c}] = p_c s_i; needs
+                              batch 1; a node that gets no iteration sends U = 0          */
+  uint32_t reserved0;      /* 0                                                     */
+  const uint32_t* client_shares; /* split_mode 1: host array of n_clients integer weights,
+                              p_c = shares[c] / sum (copied by aet_create); NULL: p_c = 1/n */
 } aet_config;
 
 /* aet_load_client_data keeps the caller's device pointers instead of copying

@@ -27,6 +27,7 @@ class AetConfig(C.Structure):
         ("compute_delay_lo", C.c_double), ("compute_delay_hi", C.c_double),
         ("network_delay_lo", C.c_double), ("network_delay_hi", C.c_double),
         ("straggler_factor", C.c_double), ("n_stragglers", C.c_uint32), ("flags", C.c_uint32),
+        ("split_mode", C.c_uint32), ("reserved0", C.c_uint32), ("client_shares", C.POINTER(C.c_uint32)),
     ]
 
 

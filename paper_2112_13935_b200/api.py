@@ -30,10 +30,16 @@ def make_config(cfg: dict) -> AetConfig:
     for i, d in enumerate(dims):
         c.dims[i] = d
     for name, _ in AetConfig._fields_:
-        if name in ("struct_size", "n_layers", "dims", "flags"):
+        if name in ("struct_size", "n_layers", "dims", "flags", "split_mode", "reserved0", "client_shares"):
             continue
         setattr(c, name, cfg[name])
     c.flags = int(cfg.get("flags", 0))
+    c.split_mode = int(cfg.get("split_mode", 0))
+    shares = cfg.get("client_shares")
+    if shares:
+        arr = (C.c_uint32 * len(shares))(*[int(v) for v in shares])
+        c.client_shares = C.cast(arr, C.POINTER(C.c_uint32))
+        c._shares_keepalive = arr      # the library copies them in aet_create; until then they live here
     return c
 
 

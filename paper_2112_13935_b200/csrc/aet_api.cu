@@ -83,6 +83,7 @@ void set_thread_error(const std::string& msg) { g_create_error = msg; }
 
 struct aet_handle {
   aet_config cfg{};
+  std::vector<uint32_t> shares;   // copy of cfg.client_shares (cfg.client_shares points here)
   uint32_t P = 0;
   size_t stride = 0;
   bool lr_fast = false;  // 784 -> 10, batch 1, fp32: the specialised kernel
@@ -237,6 +238,10 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   aet_handle* h = new (std::nothrow) aet_handle();
   if (!h) return fail(nullptr, AET_ERR_NOMEM, "out of host memory");
   h->cfg = *cfg;
+  if (cfg->client_shares) {
+    h->shares.assign(cfg->client_shares, cfg->client_shares + cfg->n_clients);
+    h->cfg.client_shares = h->shares.data();
+  }
   h->P = P;
   h->stride = ((size_t)P + 31) & ~(size_t)31;
   h->lr_fast = cfg->model == 0 && cfg->dims[0] == 784 && cfg->dims[1] == 10 && cfg->batch == 1 && cfg->precision == 0;
@@ -395,7 +400,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
     std::string err;
     if (!simulate(h->cfg, n_rounds, st, h->delays, cp.sched, err)) return fail(h, AET_ERR_CONFIG, err);
     cp.after = st;
-    build_plan(h->cfg, cp.sched.events, (h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, cp.plan);
+    build_plan(h->cfg, h->delays, cp.sched.events, (h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, cp.plan);
     cp.valid = true;
   }
   const Plan& plan = cp.plan;
@@ -535,8 +540,10 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   if (client >= h->cfg.n_clients) return fail(h, AET_ERR_ARG, "client index out of range");
   if (round < h->cfg.round_base) return fail(h, AET_ERR_ARG, "round is before round_base");
   if (!h->h_clients[client].x) return fail(h, AET_ERR_STATE, "client has no data");
-  const uint32_t s_i = sample_size(h->cfg, round);
-  if (s_i == 0 || s_i % h->cfg.batch) return fail(h, AET_ERR_CONFIG, "batch must divide the round's sample count");
+  ensure_split(h->cfg, round + 1, h->delays);
+  const uint32_t s_i = node_sample_size(h->cfg, h->delays, client, round);
+  if (s_i % h->cfg.batch || (s_i == 0 && !h->cfg.split_mode))
+    return fail(h, AET_ERR_CONFIG, "batch must divide the round's sample count");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   aet_status up = upload_clients(h, s);
   if (up != AET_OK) return up;
@@ -553,8 +560,8 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   t.client = client; t.round = round; t.seq = 0; t.snap_slot = 0;
   t.n_samples = s_i; t.steps = s_i / h->cfg.batch;
   t.inflight_off = 0; t.inflight_cnt = 0;
-  t.sample_ctr0 = samples_before(h->cfg, round);
-  t.eta = (float)round_step_size(h->cfg, round);
+  t.sample_ctr0 = node_samples_before(h->cfg, h->delays, client, round);
+  t.eta = (float)round_step_size(h->cfg, h->delays, client, round);
   AET_CUDA(h, cudaMemcpyAsync(snap, w_in, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   AET_CUDA(h, cudaMemcpyAsync(dtask, &t, sizeof(t), cudaMemcpyHostToDevice, s));
   AET_CUDA(h, cudaStreamSynchronize(s));
@@ -650,7 +657,7 @@ uint32_t aet_debug_plan_waves(const aet_config* cfg, uint32_t n_rounds) {
   SchedResult res;
   if (!simulate(*cfg, n_rounds, st, cache, res, err)) return 0;
   Plan plan;
-  build_plan(*cfg, res.events, (cfg->flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, plan);
+  build_plan(*cfg, cache, res.events, (cfg->flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, plan);
   return (uint32_t)plan.apply_upto.size();
 }
 
@@ -667,7 +674,7 @@ aet_status aet_debug_plan_layout(const aet_config* cfg, uint32_t n_rounds, uint3
   SchedResult res;
   if (!simulate(*cfg, n_rounds, st, cache, res, err)) return fail(nullptr, AET_ERR_CONFIG, err);
   Plan plan;
-  build_plan(*cfg, res.events, (cfg->flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, plan);
+  build_plan(*cfg, cache, res.events, (cfg->flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, plan);
   const uint32_t n_waves = (uint32_t)plan.apply_upto.size();
   for (uint32_t L = 0; L < n_waves; ++L) {
     apply_upto[L] = plan.apply_upto[L];

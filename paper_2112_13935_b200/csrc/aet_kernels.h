@@ -111,6 +111,29 @@ __device__ __forceinline__ bool debug_task_ok(const RoundLaunch& p, const TaskDe
   if (!ok && threadIdx.x == 0 && p.status) atomicOr(p.status, 4u);
   return ok;
 }
+// A round without a single iteration (a node the Setup split of Algorithm 2 gave nothing in this
+// round): Algorithm 3 still sends (c, U_i, i) after the empty inner loop, with U_i = 0.  One CTA
+// writes the zero update sum, the unchanged model where the caller wants it, and the trigger record.
+__device__ __forceinline__ void publish_empty_round(const RoundLaunch& p, const TaskDesc& t, uint32_t n_params) {
+  float* U = p.U + (size_t)t.u_row * p.stride;
+  const float* snap = p.snaps + (size_t)t.snap_slot * p.stride;
+  for (uint32_t i = threadIdx.x; i < n_params; i += blockDim.x) {
+    U[i] = 0.f;
+    if (p.w_end) {
+      float w = snap[i];
+      for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+        const InflightRef ref = p.inflight[t.inflight_off + f];
+        w = fmaf(-ref.eta, p.U[(size_t)ref.row * p.stride + i], w);
+      }
+      p.w_end[(size_t)t.u_row * p.stride + i] = w;
+    }
+  }
+  if (threadIdx.x == 0) {
+    TriggerRec rec;
+    rec.client = t.client; rec.round = t.round; rec.samples_done = 0; rec.flags = 1;
+    p.trig[t.seq] = rec;
+  }
+}
 #endif
 
 // bf16 conversion of a client's rows at load time (precision 1).

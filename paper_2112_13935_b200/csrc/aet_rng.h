@@ -19,7 +19,7 @@ namespace aet {
 
 constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
 constexpr uint64_t kLn2Q32 = 2977044471ull;  // floor(ln 2 * 2^32)
-enum Stream : uint32_t { kStreamSample = 0, kStreamCompute = 1, kStreamNetwork = 2 };
+enum Stream : uint32_t { kStreamSample = 0, kStreamCompute = 1, kStreamNetwork = 2, kStreamSetup = 3 };
 
 AET_HD uint64_t mix64(uint64_t z) {
   z ^= z >> 30;

@@ -28,8 +28,49 @@ uint64_t samples_before(const aet_config& c, uint32_t round) {
   return (uint64_t)c.sched_a * sum_j + (uint64_t)c.sched_b * n;
 }
 
-double round_step_size(const aet_config& c, uint32_t round) {
-  double t = (double)(samples_before(c, round) / c.batch);
+// Algorithm 2, Setup: iteration t of global round i goes to node a(i, t) = c with probability
+// p_c = shares[c] / sum(shares) (all equal without shares); s_{i,c} counts the node's iterations.
+// The coin of an iteration is draw number (iterations of all earlier rounds) + t of the stream
+// (seed, setup, client 0); node = first c whose cumulative share exceeds hi32(draw) * sum >> 32.
+void ensure_split(const aet_config& c, uint32_t last_round, DelayCache& cache) {
+  if (!c.split_mode) return;
+  const uint32_t n = c.n_clients;
+  if (cache.split.size() != n) { cache.split.assign(n, {}); cache.split_before.assign(n, {}); }
+  const uint32_t need = last_round - c.round_base;
+  uint32_t have = (uint32_t)cache.split[0].size();
+  if (have >= need) return;
+  std::vector<uint64_t> cum(n);
+  uint64_t total = 0;
+  for (uint32_t cl = 0; cl < n; ++cl) { total += c.client_shares ? c.client_shares[cl] : 1u; cum[cl] = total; }
+  const uint64_t key = stream_key(c.seed, kStreamSetup, 0);
+  for (uint32_t rel = have; rel < need; ++rel) {
+    const uint32_t round = c.round_base + rel;
+    const uint64_t g0 = samples_before(c, round);
+    const uint32_t s_i = sample_size(c, round);
+    std::vector<uint32_t> cnt(n, 0);
+    for (uint32_t t = 0; t < s_i; ++t) {
+      const uint64_t v = ((draw(key, g0 + t) >> 32) * total) >> 32;
+      const uint32_t cl = (uint32_t)(std::upper_bound(cum.begin(), cum.end(), v) - cum.begin());
+      cnt[cl] += 1;
+    }
+    for (uint32_t cl = 0; cl < n; ++cl) {
+      const uint64_t before = rel ? cache.split_before[cl][rel - 1] + cache.split[cl][rel - 1] : 0;
+      cache.split[cl].push_back(cnt[cl]);
+      cache.split_before[cl].push_back(before);
+    }
+  }
+}
+
+uint32_t node_sample_size(const aet_config& c, const DelayCache& cache, uint32_t client, uint32_t round) {
+  return c.split_mode ? cache.split[client][round - c.round_base] : sample_size(c, round);
+}
+
+uint64_t node_samples_before(const aet_config& c, const DelayCache& cache, uint32_t client, uint32_t round) {
+  return c.split_mode ? cache.split_before[client][round - c.round_base] : samples_before(c, round);
+}
+
+double round_step_size(const aet_config& c, const DelayCache& cache, uint32_t client, uint32_t round) {
+  double t = (double)(node_samples_before(c, cache, client, round) / c.batch);
   return (double)c.lr / (1.0 + (double)c.lr_beta * sqrt(t));
 }
 
@@ -51,6 +92,13 @@ bool validate_config(const aet_config& c, std::string& err) {
   if (c.delay_dist == 1 && (c.compute_delay_hi < c.compute_delay_lo || c.network_delay_hi < c.network_delay_lo ||
                             c.compute_delay_lo < 0 || c.network_delay_lo < 0)) { err = "uniform delay range is empty"; return false; }
   if (!(c.straggler_factor >= 0) || c.straggler_factor > 65535.0) { err = "straggler_factor out of range"; return false; }
+  if (c.split_mode > 1) { err = "split_mode must be 0 or 1"; return false; }
+  if (c.split_mode && c.batch != 1) { err = "the Setup split assigns single SGD iterations: batch must be 1"; return false; }
+  if (c.client_shares) {
+    uint64_t total = 0;
+    for (uint32_t cl = 0; cl < c.n_clients; ++cl) total += c.client_shares[cl];
+    if (total == 0 || total > 0xFFFFFFFFull) { err = "client_shares must sum to 1 .. 2^32 - 1"; return false; }
+  }
   return true;
 }
 
@@ -95,8 +143,8 @@ void fill_delays(const aet_config& c, uint32_t first, uint32_t last, DelayCache&
     std::vector<uint64_t>& net = cache.net[cl];
     for (uint32_t rel = (uint32_t)busy.size(); rel < need; ++rel) {
       const uint32_t round = c.round_base + rel;
-      const uint64_t it0 = samples_before(c, round) / c.batch;
-      const uint32_t steps = sample_size(c, round) / c.batch;
+      const uint64_t it0 = node_samples_before(c, cache, cl, round) / c.batch;
+      const uint32_t steps = node_sample_size(c, cache, cl, round) / c.batch;
       uint64_t sum = 0;
       for (uint32_t j = 0; j < steps; ++j) {
         uint64_t dt = dm.compute(draw(kc, it0 + j));
@@ -136,6 +184,7 @@ bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache
       err = "batch must divide every round's sample count, and rounds may not be empty";
       return false;
     }
+  ensure_split(c, last, cache);
   fill_delays(c, first, last, cache);
 
   out.events.clear();
@@ -194,7 +243,7 @@ bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache
     e.t_apply = e.t_trigger + cache.net[cl][round - c.round_base];
     e.wait_ticks = it.t - ready[cl];
     e.client = cl; e.round = round;
-    e.samples = sample_size(c, round);
+    e.samples = node_sample_size(c, cache, cl, round);
     e.steps = e.samples / c.batch;
     e.seq = 0; e.seen = seq; e.lag = lag; e.pad = 0;
     ev_of[(size_t)cl * n_rounds + (round - first)] = (uint32_t)out.events.size();
@@ -212,7 +261,8 @@ bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache
   s.messages_up = s.model_pulls = out.events.size();
   for (const aet_event& e : out.events) s.samples_total += e.samples;
   s.messages_if_per_sample = s.samples_total / c.batch;
-  const uint64_t s_first = sample_size(c, c.round_base);
+  uint64_t s_first = sample_size(c, c.round_base);
+  if (c.split_mode) s_first = std::max<uint64_t>(1, s_first / n);   // a node's expected share of the first global round
   const uint64_t per_client = n ? s.samples_total / n : 0;
   s.messages_if_constant_b = s_first ? n * ((per_client + s_first - 1) / s_first) : 0;
   s.t_end_ticks = out.events.empty() ? st.clock : out.events.back().t_apply;
@@ -221,7 +271,7 @@ bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache
   return true;
 }
 
-void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool keep_all, Plan& plan) {
+void build_plan(const aet_config& c, const DelayCache& cache, const std::vector<aet_event>& events, bool keep_all, Plan& plan) {
   const size_t E = events.size();
   plan = Plan{};
   plan.applies.resize(E);
@@ -231,7 +281,9 @@ void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool 
   std::vector<uint32_t> order(E);
   for (size_t k = 0; k < E; ++k) order[k] = (uint32_t)k;
   std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
-    return std::tie(events[a].t_start, events[a].client) < std::tie(events[b].t_start, events[b].client);
+    // an empty round starts and ends on the same tick as the client's next one: keep round order
+    return std::tie(events[a].t_start, events[a].client, events[a].round) <
+           std::tie(events[b].t_start, events[b].client, events[b].round);
   });
   std::vector<uint32_t> level(E, 0), prev_level(c.n_clients, 0);
   uint32_t pref = 0, pref_max = 0, n_waves = 0;
@@ -331,7 +383,7 @@ void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool 
   }
 
   for (size_t k = 0; k < E; ++k) {
-    plan.applies[k].eta = (float)round_step_size(c, events[k].round);
+    plan.applies[k].eta = (float)round_step_size(c, cache, events[k].client, events[k].round);
     plan.applies[k].snap_slot = slot_of[k + 1];
     plan.applies[k].client = events[k].client;
     plan.applies[k].round = events[k].round;
@@ -344,12 +396,12 @@ void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool 
     t.client = e.client; t.round = e.round; t.seq = e.seq;
     t.snap_slot = (uint32_t)slot_of[e.seen];
     t.n_samples = e.samples; t.steps = e.steps;
-    t.sample_ctr0 = samples_before(c, e.round);
-    t.eta = (float)round_step_size(c, e.round);
+    t.sample_ctr0 = node_samples_before(c, cache, e.client, e.round);
+    t.eta = (float)round_step_size(c, cache, e.client, e.round);
     t.u_row = plan.u_row_of[k];
     t.inflight_off = (uint32_t)plan.inflight.size();
     for_each_inflight(e, [&](uint32_t j) {
-      plan.inflight.push_back({plan.u_row_of[j], (float)round_step_size(c, events[j].round)});
+      plan.inflight.push_back({plan.u_row_of[j], (float)round_step_size(c, cache, events[j].client, events[j].round)});
     });
     t.inflight_cnt = (uint32_t)plan.inflight.size() - t.inflight_off;
     plan.tasks.push_back(t);

@@ -22,6 +22,9 @@ struct SchedState {
 // only on (client, round); cached so a repeated run does not redraw them.
 struct DelayCache {
   std::vector<std::vector<uint64_t>> busy, net;  // [client][round - round_base]
+  // Setup split (Algorithm 2), split_mode 1 only: s_{i,c} and its running sum per node
+  std::vector<std::vector<uint32_t>> split;      // [client][round - round_base]
+  std::vector<std::vector<uint64_t>> split_before;  // [client][round - round_base]: samples before that round
 };
 
 struct SchedResult {
@@ -29,9 +32,15 @@ struct SchedResult {
   aet_summary summary;
 };
 
-uint32_t sample_size(const aet_config& c, uint32_t round);
+uint32_t sample_size(const aet_config& c, uint32_t round);      // s_i = a i + b
 uint64_t samples_before(const aet_config& c, uint32_t round);  // rounds round_base .. round-1
-double round_step_size(const aet_config& c, uint32_t round);
+// The same per node: the node's own sequence, or (split_mode 1) its coin-flip share of the global
+// round (Algorithm 2, Setup), which the cache must hold (ensure_split) for every round asked for.
+void ensure_split(const aet_config& c, uint32_t last_round, DelayCache& cache);
+uint32_t node_sample_size(const aet_config& c, const DelayCache& cache, uint32_t client, uint32_t round);
+uint64_t node_samples_before(const aet_config& c, const DelayCache& cache, uint32_t client, uint32_t round);
+// eta_0 / (1 + beta sqrt(t)), t = the node's own SGD iterations before the round (Section 4.1)
+double round_step_size(const aet_config& c, const DelayCache& cache, uint32_t client, uint32_t round);
 
 // Returns false and fills err on an invalid configuration.
 bool validate_config(const aet_config& c, std::string& err);
@@ -69,6 +78,6 @@ struct Plan {
 // keep_all: one row per event and one slot per distinct start position, never reused
 // (row = seq), so that every update sum can be read back after the run.  Otherwise rows
 // and slots are recycled as soon as nothing later in the launch order reads them.
-void build_plan(const aet_config& c, const std::vector<aet_event>& events, bool keep_all, Plan& plan);
+void build_plan(const aet_config& c, const DelayCache& cache, const std::vector<aet_event>& events, bool keep_all, Plan& plan);
 
 }  // namespace aet

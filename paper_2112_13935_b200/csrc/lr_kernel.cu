@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(kThreads, 2) lr_round_kernel(RoundLaunch p) {
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
   if (!debug_task_ok(p, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  if (t.n_samples == 0) { publish_empty_round(p, t, kD * kC + kC); return; }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_raw = warp * kLanes + lane;
   const bool active = lane < kLanes && u_raw < kGroups;
@@ -369,6 +370,11 @@ __global__ void __launch_bounds__(kDed ? 2 * kThreads : kThreads, kDed ? 1 : 2) 
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
   if (!debug_task_ok(p, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  if (t.n_samples == 0) {   // this grid may run under the tail of the aggregation before it: wait before writing
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    publish_empty_round(p, t, kParams);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool rw = kDed && warp >= kWarps;            // the warps without pixels: R (warp 4), Gram and row copies (warp 5)
   const bool gw = kDed && (warp == kWarps + 1 || warp == kWarps + 2);   // warps 5 and 6

@@ -111,6 +111,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
 
   const TaskDesc t = p.tasks[p.task_begin + blockIdx.x];
   if (!debug_task_ok(p, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  if (t.n_samples == 0) {   // this grid may run under the tail of the aggregation before it: wait before writing
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    publish_empty_round(p, t, kParams);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = warp & 3, ch = warp >> 2;
   const int row = 32 * q + lane;                        // this thread's row of every 128-row tile

@@ -64,6 +64,14 @@ __global__ void __launch_bounds__(kThreads) mlp_round_kernel(MlpLaunch p) {
   const int rank = clustered ? (int)cluster_rank() : 0;
   const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / C];
   if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  if (t.n_samples == 0) {   // an empty round (every CTA of the cluster takes this branch)
+    if (rank == 0) {
+      uint32_t P = 0;
+      for (uint32_t l = 0; l < S.n_layers; ++l) P += S.dims[l] * S.dims[l + 1] + S.dims[l + 1];
+      publish_empty_round(p.r, t, P);
+    }
+    return;
+  }
   const int tid = threadIdx.x;
   const int L = (int)S.n_layers, B = (int)S.batch, Bp = up4(B);
   const bool bf = S.precision == 1;

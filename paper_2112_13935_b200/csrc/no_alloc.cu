@@ -93,6 +93,7 @@ extern "C" aet_status aet_round_no_alloc(const aet_config* cfg, uint32_t client,
   std::string err;
   if (!validate_config(*cfg, err)) return fail(AET_ERR_CONFIG, err);
   if (cfg->precision != 0) return fail(AET_ERR_CONFIG, "aet_round_no_alloc runs fp32 models only");
+  if (cfg->split_mode != 0) return fail(AET_ERR_CONFIG, "aet_round_no_alloc runs a node's own sequence s_i = a*i + b only (split_mode 0)");
   if (client >= cfg->n_clients) return fail(AET_ERR_ARG, "client index out of range");
   if (round < cfg->round_base) return fail(AET_ERR_ARG, "round is before round_base");
   if (n == 0 || n < cfg->batch) return fail(AET_ERR_ARG, "a client needs at least max(1, batch) samples");
@@ -130,7 +131,7 @@ extern "C" aet_status aet_round_no_alloc(const aet_config* cfg, uint32_t client,
   t.n_samples = s_i; t.steps = s_i / cfg->batch;
   t.inflight_off = 0; t.inflight_cnt = 0;
   t.sample_ctr0 = samples_before(*cfg, round);
-  t.eta = (float)round_step_size(*cfg, round);
+  t.eta = (float)round_step_size(*cfg, DelayCache{}, client, round);
   const ClientData cd{x, y, n, 0};
   fill_header_kernel<<<1, 1, 0, s>>>(t, cd, stream_key(cfg->seed, kStreamSample, client));
   e = cudaGetLastError();

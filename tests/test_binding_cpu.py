@@ -79,6 +79,11 @@ def test_schedule_is_bit_identical_to_the_checker(name):
          network_delay_lo=5 / 2 ** 20, network_delay_hi=5 / 2 ** 20, max_lag_d=workloads.NEVER_WAIT),
     dict(n_clients=3, sched_a=0, sched_b=2, delay_dist=1, compute_delay_lo=4 / 2 ** 20, compute_delay_hi=4 / 2 ** 20,
          network_delay_lo=8 / 2 ** 20, network_delay_hi=8 / 2 ** 20, max_lag_d=1),
+    # Algorithm 2, Setup: the global round size split among the nodes by coin flips (some rounds are empty)
+    dict(split_mode=1, n_clients=5, sched_a=6, sched_b=2),
+    dict(split_mode=1, n_clients=3, sched_a=10, sched_b=5, client_shares=[1, 2, 5], lr_beta=0.02, max_lag_d=2),
+    dict(split_mode=1, n_clients=1, sched_a=3, sched_b=1),
+    dict(split_mode=1, n_clients=12, sched_a=1, sched_b=1, max_lag_d=0),
 ])
 def test_schedule_variants_match_the_checker(over):
     cfg = workloads.get_config("cfg1", **over)
@@ -89,7 +94,9 @@ def test_schedule_variants_match_the_checker(over):
 
 def test_schedule_rejects_bad_configs():
     for over, status in [(dict(batch=3), 2), (dict(n_clients=0), 2), (dict(precision=5), 2),
-                         (dict(n_stragglers=9), 2), (dict(lr=0.0), 2), (dict(sched_b=0), 2)]:
+                         (dict(n_stragglers=9), 2), (dict(lr=0.0), 2), (dict(sched_b=0), 2),
+                         (dict(split_mode=2), 2), (dict(split_mode=1, client_shares=[0, 0, 0, 0]), 2),
+                         (dict(split_mode=1, model=1, dims=[784, 16, 10], batch=2, sched_a=2, sched_b=2), 2)]:
         with pytest.raises(api.AetError) as e:
             api.aet_schedule_only(workloads.get_config("cfg1", **over), 3)
         assert e.value.status == status, over
@@ -157,6 +164,7 @@ def _replay_plan(cfg, n_rounds, events, lay):
     ("cfg1", dict(n_clients=3, n_rounds=8, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=500.0)),
     ("cfg1", dict(n_clients=7, n_rounds=9, max_lag_d=0)),
     ("cfg2", dict(max_lag_d=3, network_delay_mean=20.0)),
+    ("cfg1", dict(split_mode=1, n_clients=9, sched_a=4, sched_b=2, n_rounds=8)),
 ])
 def test_recycled_rows_and_slots_always_hold_what_is_read(name, over):
     cfg = workloads.get_config(name, **over)

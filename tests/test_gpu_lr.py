@@ -347,3 +347,36 @@ def test_errors_are_reported_not_raised_by_the_device():
     with pytest.raises(api.AetError) as e:
         api.aet_create(workloads.get_config("cfg1", dims=[784, 64]))   # too many classes
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("over", [
+    dict(n_clients=5, sched_a=6, sched_b=2, l2=0.0),                                   # blocked kernel; some rounds are empty
+    dict(n_clients=3, sched_a=10, sched_b=5, client_shares=[1, 2, 5], lr_beta=0.02, l2=1e-4),   # unequal p_c, step-by-step kernel
+    dict(n_clients=200, sched_a=300, sched_b=200, l2=0.0, lr=1e-4, n_rounds=4, data=dict(per_client=64)),   # tensor-memory kernel
+    dict(model=0, dims=[784, 10], batch=1, n_clients=4, sched_a=5, sched_b=3, l2=0.0, flags=0, precision=0,
+         data=dict(per_client=100), generic=True),                                     # the generic kernel (see below)
+])
+def test_setup_split_of_a_global_round_size_end_to_end(over):
+    # Algorithm 2: s_i = a i + b is the global size of round i, split among the nodes by coin flips
+    over = dict(over)
+    generic = over.pop("generic", False)
+    base = dict(split_mode=1, n_rounds=7, data=dict(per_client=300))
+    base.update(over)
+    if generic:
+        base["dims"] = [784, 10]
+    cfg = workloads.get_config("cfg1", **base)
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    sizes = [e["samples"] for e in ref["events"]]
+    assert len(set(sizes)) > 3 and ref["summary"]["samples_total"] == sum(
+        cfg["sched_a"] * i + cfg["sched_b"] for i in range(cfg["n_rounds"]))
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert np.abs(gpu["w"] - ref["w"]).max() <= 1e-5
+    for k, e in enumerate(ref["events"]):
+        if e["samples"] == 0:
+            assert not gpu["U"][k].any()                # an empty round sends a zero sum
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for e in ref["events"][::max(1, len(ref["events"]) // 25)]:
+            if e["samples"]:
+                check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]])
