@@ -224,6 +224,148 @@ def simulate(cfg, n_rounds, state=None):
     return events, summary, after
 
 
+# ---- peer-to-peer ring (Section 1, Fig. 1b; the topology of the paper's experiments) ----
+# Every node keeps its own model and history map.  A round's sum (c, U_i, i) goes to the node's
+# ring neighbours only (Algorithm 3: "Send a tuple (c, U_i, i) to the other c's neighbors") and is
+# not forwarded (Algorithm 3 has no relay step).  Receive bumps H_v[c] when the message arrives;
+# Synchronize(H, d, i) looks at the node's neighbours only.  One network delay per message and
+# destination: draw number 2 * round + side of the sender's network stream (side 0 = node c - 1,
+# side 1 = node c + 1; a node with a single neighbour uses side 0).  Ties: (tick, RECEIVE before
+# START, node, then sender and round).  A log record is one delivery (sender, round, destination);
+# a node without neighbours logs its rounds with destination NO_DEST.
+RECEIVE = 0
+NO_DEST = 0xFFFFFFFF
+
+
+def ring_neighbours(n: int, c: int):
+    """Neighbours of node c with the side each one sits on: [(side, node)]."""
+    out = []
+    for side, v in ((0, (c - 1) % n), (1, (c + 1) % n)):
+        if v != c and v not in [w for _, w in out]:
+            out.append((side, v))
+    return out
+
+
+def new_ring_state(cfg):
+    n = cfg["n_clients"]
+    return dict(clock=0, H=[{v: 0 for _, v in ring_neighbours(n, c)} for c in range(n)], rounds_done=0)
+
+
+def simulate_ring(cfg, n_rounds, state=None):
+    """Event schedule of the ring for n_rounds more rounds per node, to quiescence.
+
+    Returns (tasks, deliveries, summary, state_after).  tasks: one dict per round-task in
+    (t_trigger, client, round) order with `task` = its position there and `applied` = the
+    deliveries (indices into deliveries) that reached the node before the round started and
+    after its previous start.  deliveries: one dict per (sender, round, destination) in
+    processing order = (t_apply, dest, client, round), `seq` = its position."""
+    n = cfg["n_clients"]
+    a, b, base, B = cfg["sched_a"], cfg["sched_b"], cfg["round_base"], cfg["batch"]
+    d, seed = cfg["max_lag_d"], cfg["seed"]
+    st = new_ring_state(cfg) if state is None else state
+    H = [dict(h) for h in st["H"]]
+    t0 = st["clock"]
+    first = base + st["rounds_done"]
+    last = first + n_rounds
+    straggler_q16 = rng.to_q16(cfg["straggler_factor"])
+    key_c = [rng.stream_key(seed, rng.STREAM_COMPUTE, c) for c in range(n)]
+    key_n = [rng.stream_key(seed, rng.STREAM_NETWORK, c) for c in range(n)]
+    nbrs = [ring_neighbours(n, c) for c in range(n)]
+    ready = [t0] * n
+    blocked = {}
+    pending = [[] for _ in range(n)]          # deliveries that reached a node since its last start
+    n_received = [0] * n
+    heap = [(t0, START, c, first, 0) for c in range(n)] if n_rounds > 0 else []
+    heapq.heapify(heap)
+    tasks, deliveries = [], []
+
+    def lag_of(c, i):
+        if not H[c]:
+            return 0
+        return max(0, (i - base) - min(H[c].values()))
+
+    while heap:
+        t, kind, node, x, y = heapq.heappop(heap)
+        if kind == RECEIVE:
+            sender, rnd = x, y
+            H[node][sender] += 1
+            dl = next(q for q in deliveries if q["seq"] is None and q["dest"] == node and q["client"] == sender
+                      and q["round"] == rnd)
+            dl["seq"] = sum(1 for q in deliveries if q["seq"] is not None)
+            pending[node].append(dl)
+            n_received[node] += 1
+            if node in blocked and (d == NEVER_WAIT or lag_of(node, blocked[node]) <= d):
+                heapq.heappush(heap, (t, START, node, blocked.pop(node), 0))
+            continue
+        c, i = node, x
+        lag = lag_of(c, i)
+        if d != NEVER_WAIT and lag > d:
+            blocked[c] = i
+            continue
+        s = node_sample_size(cfg, c, i)
+        if s % B:
+            raise ValueError("batch must divide every s_i")
+        steps = s // B
+        it0 = node_samples_before(cfg, c, i) // B
+        straggler = c >= n - cfg["n_stragglers"]
+        busy = 0
+        for j in range(steps):
+            dt = _delay(cfg, "compute", rng.draw(key_c[c], it0 + j))
+            if straggler:
+                dt = max(1, (dt * straggler_q16) >> 16)
+            busy += dt
+        t_trigger = t + busy
+        task = dict(t_start=t, t_trigger=t_trigger, wait_ticks=t - ready[c], client=c, round=i, samples=s,
+                    steps=steps, seen=n_received[c], lag=lag, applied=[q for q in pending[c]], task=None)
+        pending[c] = []
+        tasks.append(task)
+        for side, v in nbrs[c]:
+            t_arr = t_trigger + _delay(cfg, "network", rng.draw(key_n[c], 2 * i + side))
+            deliveries.append(dict(task, t_apply=t_arr, dest=v, seq=None, of_task=task))
+            heapq.heappush(heap, (t_arr, RECEIVE, v, c, i))
+        if not nbrs[c]:
+            deliveries.append(dict(task, t_apply=t_trigger, dest=NO_DEST, seq=None, of_task=task))
+        ready[c] = t_trigger
+        if i + 1 < last:
+            heapq.heappush(heap, (t_trigger, START, c, i + 1, 0))
+
+    assert not blocked
+    # a node without neighbours: its records take the places the trigger times give them
+    lone = sorted((q for q in deliveries if q["dest"] == NO_DEST), key=lambda q: (q["t_apply"], q["client"], q["round"]))
+    for k, q in enumerate(lone):
+        q["seq"] = k
+    assert all(q["seq"] is not None for q in deliveries)
+    deliveries.sort(key=lambda q: q["seq"])
+    tasks.sort(key=lambda e: (e["t_trigger"], e["client"], e["round"]))
+    for k, e in enumerate(tasks):
+        e["task"] = k
+    for q in deliveries:
+        q["task"] = q["of_task"]["task"]
+    samples_total = sum(e["samples"] for e in tasks)
+    s_first = sample_size(a, b, base)
+    if split_mode(cfg):
+        s_first = max(1, s_first // n)
+    per_client = samples_total // n if n else 0
+    n_links = sum(len(v) for v in nbrs)
+    summary = dict(
+        messages_up=sum(1 for q in deliveries if q["dest"] != NO_DEST), model_pulls=0, samples_total=samples_total,
+        messages_if_per_sample=(samples_total // B) * (n_links // n if n else 0),
+        messages_if_constant_b=(n_links * -(-per_client // s_first)) if s_first else 0,
+        t_end_ticks=max([q["t_apply"] for q in deliveries] + [t0]))
+    after = dict(clock=summary["t_end_ticks"], H=H, rounds_done=st["rounds_done"] + n_rounds)
+    return tasks, deliveries, summary, after
+
+
+def pack_ring_events(deliveries) -> bytes:
+    """The ring's log as the library lays it out: one 64-byte record per delivery."""
+    out = bytearray()
+    for q in deliveries:
+        out += EVENT_STRUCT.pack(q["t_start"], q["t_trigger"], q["t_apply"], q["wait_ticks"],
+                                 q["client"], q["round"], q["samples"], q["steps"],
+                                 q["seq"], q["seen"], q["lag"], q["dest"])
+    return bytes(out)
+
+
 def pack_events(events) -> bytes:
     """The event log as the library lays it out (64 bytes per record)."""
     out = bytearray()

@@ -87,3 +87,36 @@ def run(cfg, data, w0, n_rounds=None, keep=False, state=None):
     assert all(not v for v in in_flight.values())
     return dict(events=events, summary=summary, w=w_g, U=U_by_seq, w_start=w_start_by_seq,
                 state=state_after)
+
+
+def run_ring(cfg, data, w0, n_rounds=None, keep=False, state=None, node_models=None):
+    """The peer-to-peer ring (Section 1, Fig. 1b): every node keeps its own model.
+
+    A node's round starts from its own model after the update sums that reached it since its
+    previous start have been applied (Receive: w_c -= eta_k * U, in arrival order); its own sum
+    is applied when the round ends (w_c -= eta_i * U_i, the net effect of the inner loop); sums are
+    not forwarded.  Returns dict(tasks, deliveries, summary, W (node models at quiescence),
+    U (by task), w_start (by task, where kept), state)."""
+    n = cfg["n_clients"]
+    n_rounds = cfg["n_rounds"] if n_rounds is None else n_rounds
+    tasks, deliveries, summary, state_after = schedule.simulate_ring(cfg, n_rounds, state)
+    W = [np.array(w0 if node_models is None else node_models[c], dtype=np.float64) for c in range(n)]
+    U_by_task = [None] * len(tasks)
+    w_start_by_task = [None] * len(tasks)
+    applied = set()
+    for e in sorted(tasks, key=lambda e: (e["t_start"], e["client"], e["round"])):
+        c = e["client"]
+        for q in e["applied"]:
+            W[c] -= step_size(cfg, q["round"], q["client"]) * U_by_task[q["task"]]
+            applied.add(q["seq"])
+        w_start = W[c].copy()
+        U, _ = run_task(cfg, data[c], c, e["round"], w_start)
+        U_by_task[e["task"]] = U
+        if keep is True or (keep and e["task"] in keep):
+            w_start_by_task[e["task"]] = w_start
+        W[c] -= step_size(cfg, e["round"], c) * U
+    for q in deliveries:                       # quiescence: what is still on its way arrives
+        if q["dest"] != schedule.NO_DEST and q["seq"] not in applied:
+            W[q["dest"]] -= step_size(cfg, q["round"], q["client"]) * U_by_task[q["task"]]
+    return dict(tasks=tasks, deliveries=deliveries, summary=summary, W=W, U=U_by_task,
+                w_start=w_start_by_task, state=state_after)

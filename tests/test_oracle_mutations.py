@@ -11,7 +11,7 @@ from oracle import models, rng, schedule, sim
 
 
 def _fails(fn, *args):
-    with pytest.raises((AssertionError, IndexError, ValueError)):
+    with pytest.raises((AssertionError, IndexError, ValueError, KeyError)):
         fn(*args)
 
 
@@ -161,3 +161,38 @@ def test_setup_split_by_independent_draws_per_node_is_caught(monkeypatch):
         return out
     monkeypatch.setattr(schedule, "split_round", independent)
     _fails(ts.test_setup_split_conserves_every_round_and_reduces_to_one_node)
+
+
+def test_ring_that_sends_to_every_node_is_caught(monkeypatch):
+    import test_oracle_ring as tring
+    monkeypatch.setattr(schedule, "ring_neighbours",
+                        lambda n, c: [(k, v) for k, v in enumerate(w for w in range(n) if w != c)][:2] if n <= 3
+                        else [(0, (c - 1) % n), (1, (c + 2) % n)])       # right-hand link skips a node
+    _fails(tring.test_four_node_timeline_worked_by_hand)
+    _fails(tring.test_node_model_is_w0_minus_own_and_neighbours_sums)
+
+
+def test_ring_receive_with_the_receivers_step_size_is_caught(monkeypatch):
+    import inspect
+    import test_oracle_ring as tring
+    src = inspect.getsource(sim.run_ring)
+    old = 'W[c] -= step_size(cfg, q["round"], q["client"]) * U_by_task[q["task"]]'
+    assert src.count(old) == 1
+    ns = dict(vars(sim))
+    exec(compile(src.replace(old, 'W[c] -= step_size(cfg, e["round"], c) * U_by_task[q["task"]]'), "<mutated run_ring>", "exec"), ns)
+    monkeypatch.setattr(sim, "run_ring", ns["run_ring"])
+    _fails(tring.test_node_model_is_w0_minus_own_and_neighbours_sums)
+
+
+def test_ring_history_that_counts_at_round_start_instead_of_arrival_is_caught(monkeypatch):
+    # Synchronize must see a message as soon as it arrives (the wait loop keeps tracking H); a history that only
+    # moves when the node starts a round would leave the blocked node of the hand-worked timeline waiting for ever
+    import inspect
+    import test_oracle_ring as tring
+    src = inspect.getsource(schedule.simulate_ring)
+    old = "            H[node][sender] += 1\n"
+    assert src.count(old) == 1
+    ns = dict(vars(schedule))
+    exec(compile(src.replace(old, "            H[node][sender] += 0\n"), "<mutated simulate_ring>", "exec"), ns)
+    monkeypatch.setattr(schedule, "simulate_ring", ns["simulate_ring"])
+    _fails(tring.test_four_node_timeline_worked_by_hand)
