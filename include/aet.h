@@ -78,7 +78,11 @@ typedef struct {
                               iterations goes to node c with probability p_c, so that
                               s_{i,c} = |{t : a(i,t) = c}| and E[s_{i,c}] = p_c s_i; needs
                               batch 1; a node that gets no iteration sends U = 0          */
-  uint32_t reserved0;      /* 0                                                     */
+  uint32_t topology;       /* 0: client-server (Section 1, Fig. 1a): a server applies the
+                              sums and clients pull its model.  1: peer-to-peer ring (Fig. 1b,
+                              the paper's experiments): every node keeps its own model and
+                              history map, sends its sums to its two ring neighbours only
+                              (no forwarding) and Synchronize looks at those neighbours     */
   const uint32_t* client_shares; /* split_mode 1: host array of n_clients integer weights,
                               p_c = shares[c] / sum (copied by aet_create); NULL: p_c = 1/n */
 } aet_config;
@@ -107,7 +111,10 @@ typedef struct {
 #define AET_FLAG_STEPWISE_RECURRENCE 8u
 
 /* One round-task = one message (c, U_i, i) of Algorithm 3.  64 bytes.
- * Times are integer ticks (2^20 per time unit). */
+ * Times are integer ticks (2^20 per time unit).  In the ring topology a record
+ * is one delivery (sender, round, destination): t_apply is its arrival, seq its
+ * place among all deliveries ordered by (arrival, destination, sender, round),
+ * seen the messages the SENDER had received when that round started. */
 typedef struct {
   uint64_t t_start;    /* round began (after any checkpoint wait)                  */
   uint64_t t_trigger;  /* h reached s_{i,c}: the update sum was sent               */
@@ -119,7 +126,8 @@ typedef struct {
   uint32_t seq;        /* position in the server's apply order                      */
   uint32_t seen;       /* updates already in the server model the round started from */
   uint32_t lag;        /* max(0, rounds done - min over other clients of H) at start */
-  uint32_t pad;
+  uint32_t dest;       /* ring: the node this delivery went to (0xFFFFFFFF: the node has
+                          no neighbour); client-server: 0, the server                  */
 } aet_event;
 
 typedef struct {
@@ -185,6 +193,14 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream);
 aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params,
                                 void* cuda_stream);
 
+/* The model node `node` holds (host or device pointer, n_params floats): its
+ * own model in the ring topology (Section 1, Fig. 1b: every compute node keeps
+ * a model; at quiescence it is w_0 minus the applied sums of the node and of its
+ * two neighbours); in the client-server topology the model every client would
+ * pull, i.e. the server's.  Synchronises `cuda_stream`. */
+aet_status aet_get_node_model(aet_handle* h, uint32_t node, float* out, size_t n_params,
+                              void* cuda_stream);
+
 /* The event log of all rounds run so far - one record per message (c, U_i, i)
  * of Algorithm 3 with its start, trigger and apply times, the checkpoint wait
  * (Synchronize) and the history count behind it - ordered by seq within each
@@ -198,7 +214,8 @@ aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity,
 
 /* Update sum number `seq` of the most recent aet_run_rounds (host or device
  * pointer, n_params floats).  Needs AET_FLAG_KEEP_UPDATE_SUMS (AET_ERR_STATE
- * without it).  Synchronises `cuda_stream`. */
+ * without it).  In the ring topology `seq` counts round-tasks in (trigger time,
+ * node, round) order and the flag is not needed.  Synchronises `cuda_stream`. */
 aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params,
                               void* cuda_stream);
 

@@ -27,7 +27,7 @@ class AetConfig(C.Structure):
         ("compute_delay_lo", C.c_double), ("compute_delay_hi", C.c_double),
         ("network_delay_lo", C.c_double), ("network_delay_hi", C.c_double),
         ("straggler_factor", C.c_double), ("n_stragglers", C.c_uint32), ("flags", C.c_uint32),
-        ("split_mode", C.c_uint32), ("reserved0", C.c_uint32), ("client_shares", C.POINTER(C.c_uint32)),
+        ("split_mode", C.c_uint32), ("topology", C.c_uint32), ("client_shares", C.POINTER(C.c_uint32)),
     ]
 
 
@@ -36,7 +36,7 @@ class AetEvent(C.Structure):
         ("t_start", C.c_uint64), ("t_trigger", C.c_uint64), ("t_apply", C.c_uint64),
         ("wait_ticks", C.c_uint64), ("client", C.c_uint32), ("round", C.c_uint32),
         ("samples", C.c_uint32), ("steps", C.c_uint32), ("seq", C.c_uint32),
-        ("seen", C.c_uint32), ("lag", C.c_uint32), ("pad", C.c_uint32),
+        ("seen", C.c_uint32), ("lag", C.c_uint32), ("dest", C.c_uint32),
     ]
 
 
@@ -60,6 +60,7 @@ PROTOTYPES = {
     "aet_load_client_data": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]),
     "aet_run_rounds": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p]),
     "aet_get_global_model": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "aet_get_node_model": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]),
     "aet_get_event_log": (C.c_int, [C.c_void_p, C.POINTER(AetEvent), C.c_size_t, C.POINTER(C.c_size_t),
                                     C.POINTER(AetSummary)]),
     "aet_get_update_sum": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]),

@@ -30,11 +30,12 @@ def make_config(cfg: dict) -> AetConfig:
     for i, d in enumerate(dims):
         c.dims[i] = d
     for name, _ in AetConfig._fields_:
-        if name in ("struct_size", "n_layers", "dims", "flags", "split_mode", "reserved0", "client_shares"):
+        if name in ("struct_size", "n_layers", "dims", "flags", "split_mode", "topology", "client_shares"):
             continue
         setattr(c, name, cfg[name])
     c.flags = int(cfg.get("flags", 0))
     c.split_mode = int(cfg.get("split_mode", 0))
+    c.topology = int(cfg.get("topology", 0))
     shares = cfg.get("client_shares")
     if shares:
         arr = (C.c_uint32 * len(shares))(*[int(v) for v in shares])
@@ -110,6 +111,14 @@ def aet_get_global_model(h, out=None, stream=None):
     return out
 
 
+def aet_get_node_model(h, node: int, out=None, stream=None):
+    if out is None:
+        out = np.empty(aet_n_params(h), dtype=np.float32)
+    n = out.size if isinstance(out, np.ndarray) else out.numel()
+    _check(h, _lib.load().aet_get_node_model(h, node, _ptr(out), n, _stream(stream)))
+    return out
+
+
 def aet_get_update_sum(h, seq: int, out=None, stream=None):
     if out is None:
         out = np.empty(aet_n_params(h), dtype=np.float32)
@@ -119,7 +128,7 @@ def aet_get_update_sum(h, seq: int, out=None, stream=None):
 
 
 def _events_from(arr, n):
-    names = [f for f, _ in AetEvent._fields_ if f != "pad"]
+    names = [f for f, _ in AetEvent._fields_]
     return [{f: int(getattr(arr[k], f)) for f in names} for k in range(n)]
 
 

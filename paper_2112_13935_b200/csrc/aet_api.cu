@@ -66,6 +66,14 @@ struct DevBuf {  // grow-only device array
   void release() { if (p) cudaFree(p); p = nullptr; cap = 0; }
 };
 
+struct CachedRingPlan {
+  bool valid = false, uploaded = false;
+  uint32_t rounds_before = 0, n_rounds = 0;
+  RingState before, after;
+  RingResult sched;
+  RingPlan plan;
+};
+
 struct CachedPlan {
   bool valid = false, uploaded = false;
   uint32_t rounds_before = 0, n_rounds = 0;
@@ -91,8 +99,11 @@ struct aet_handle {
   std::string err;
 
   SchedState st;
+  RingState rst;                  // topology 1
   DelayCache delays;
   CachedPlan cached;
+  CachedRingPlan ring_cached;
+  std::vector<RingTask> last_ring_tasks;
   std::vector<aet_event> log;
   aet_summary total{};
 
@@ -102,6 +113,9 @@ struct aet_handle {
   DevBuf<uint64_t> d_keys;
   DevBuf<uint32_t> d_H;
   DevBuf<float> w_buf[2], w0, snaps, U, work, act, dbg, totals;
+  DevBuf<float> node_w;           // topology 1: [n_clients, stride], every node's own model
+  DevBuf<RingApplyDesc> d_ring_applies;
+  DevBuf<RingOp> d_ring_ops;
   int w_sel = 0;  // which of w_buf holds the server model
   float* w_cur() { return w_buf[w_sel].p; }
   DevBuf<uint32_t> d_status;
@@ -218,6 +232,87 @@ aet_status launch_rounds(aet_handle* h, const RoundLaunch& r, cudaStream_t s) {
   return AET_OK;
 }
 
+// Peer-to-peer ring: waves of round-tasks (each from its node's own model), and before every wave
+// the Receive step of the nodes about to start; after the last wave every node takes what is left.
+aet_status run_ring_rounds(aet_handle* h, uint32_t n_rounds, cudaStream_t s) {
+  auto t0 = std::chrono::steady_clock::now();
+  CachedRingPlan& cp = h->ring_cached;
+  if (!(cp.valid && cp.rounds_before == h->rst.rounds_done && cp.n_rounds == n_rounds &&
+        cp.before.clock == h->rst.clock && cp.before.H == h->rst.H)) {
+    cp.valid = false;
+    cp.uploaded = false;
+    cp.before = h->rst;
+    cp.rounds_before = h->rst.rounds_done;
+    cp.n_rounds = n_rounds;
+    RingState st = h->rst;
+    std::string err;
+    if (!simulate_ring(h->cfg, n_rounds, st, h->delays, cp.sched, err)) return fail(h, AET_ERR_CONFIG, err);
+    cp.after = st;
+    build_ring_plan(h->cfg, h->delays, cp.sched, cp.plan);
+    cp.valid = true;
+  }
+  const RingPlan& plan = cp.plan;
+  const size_t T = cp.sched.tasks.size();
+  h->stats.plan_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+
+  aet_status st_up = upload_clients(h, s);
+  if (st_up != AET_OK) return st_up;
+  bool ok = h->U.reserve(T * h->stride) && h->d_tasks.reserve(T) && h->d_trig.reserve(T) &&
+            h->d_ring_applies.reserve(plan.applies.size() + 1) && h->d_ring_ops.reserve(plan.ops.size() + 1);
+  if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * mlp_act_floats(h->shape));
+  if (!ok) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  if (!cp.uploaded) {
+    AET_CUDA(h, cudaMemcpyAsync(h->d_tasks.p, plan.tasks.data(), T * sizeof(TaskDesc), cudaMemcpyHostToDevice, s));
+    if (!plan.applies.empty())
+      AET_CUDA(h, cudaMemcpyAsync(h->d_ring_applies.p, plan.applies.data(), plan.applies.size() * sizeof(RingApplyDesc), cudaMemcpyHostToDevice, s));
+    if (!plan.ops.empty())
+      AET_CUDA(h, cudaMemcpyAsync(h->d_ring_ops.p, plan.ops.data(), plan.ops.size() * sizeof(RingOp), cudaMemcpyHostToDevice, s));
+    AET_CUDA(h, cudaStreamSynchronize(s));
+    cp.uploaded = true;
+  }
+  AET_CUDA(h, cudaMemsetAsync(h->d_trig.p, 0, T * sizeof(TriggerRec), s));
+
+  RoundLaunch r{};
+  r.tasks = h->d_tasks.p; r.inflight = nullptr; r.clients = h->d_clients.p;
+  r.sample_keys = h->d_keys.p; r.snaps = h->node_w.p; r.U = h->U.p; r.w_end = nullptr;
+  r.trig = h->d_trig.p; r.status = h->d_status.p; r.stride = h->stride; r.l2 = h->cfg.l2;
+  r.debug_checks = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) ? 1u : 0u;
+  r.step_by_step = (h->cfg.flags & AET_FLAG_STEPWISE_RECURRENCE) ? 1u : 0u;
+  r.n_u_rows = (uint32_t)T; r.n_snap = h->cfg.n_clients;
+  RingApplyLaunch a{};
+  a.applies = h->d_ring_applies.p; a.ops = h->d_ring_ops.p; a.U = h->U.p; a.node_w = h->node_w.p;
+  a.status = h->d_status.p; a.stride = h->stride; a.n_params = h->P;
+
+  const uint32_t n_waves = (uint32_t)plan.wave_off.size() - 1;
+  for (uint32_t L = 0; L <= n_waves; ++L) {
+    a.lo = plan.apply_off[L]; a.hi = plan.apply_off[L + 1];
+    if (a.hi > a.lo) {
+      KernelTimer kt(h, s, 1);
+      cudaError_t e = launch_ring_apply(a, s);
+      if (e != cudaSuccess) return cuda_fail(h, e, "ring receive kernel launch");
+    }
+    if (L == n_waves) break;
+    r.task_begin = plan.wave_off[L];
+    r.n_tasks = plan.wave_off[L + 1] - plan.wave_off[L];
+    aet_status rs = launch_rounds(h, r, s);
+    if (rs != AET_OK) return rs;
+  }
+  h->stats.waves = n_waves;
+
+  h->last_first_event = h->log.size();
+  h->last_n_events = T;                 // update sums are indexed by round-task here
+  h->last_ring_tasks = cp.sched.tasks;
+  h->last_checked = false;
+  h->last_stream = s;
+  h->log.insert(h->log.end(), cp.sched.events.begin(), cp.sched.events.end());
+  const aet_summary& q = cp.sched.summary;
+  h->total.messages_up += q.messages_up; h->total.model_pulls += q.model_pulls;
+  h->total.samples_total += q.samples_total; h->total.messages_if_per_sample += q.messages_if_per_sample;
+  h->total.messages_if_constant_b += q.messages_if_constant_b; h->total.t_end_ticks = q.t_end_ticks;
+  h->rst = cp.after;
+  return AET_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -258,7 +353,13 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   bool ok = h->w_buf[0].reserve(h->stride) && h->w_buf[1].reserve(h->stride) && h->w0.reserve(h->stride) &&
             h->d_H.reserve(cfg->n_clients) && h->d_status.reserve(1) && h->totals.reserve(32 * h->stride);
   if (ok && !h->lr_fast) ok = h->work.reserve((size_t)cfg->n_clients * h->stride);
+  if (ok && cfg->topology == 1) ok = h->node_w.reserve((size_t)cfg->n_clients * h->stride);
   if (!ok) { aet_destroy(h); return fail(nullptr, AET_ERR_NOMEM, "device allocation failed"); }
+  if (cfg->topology == 1 && cudaMemset(h->node_w.p, 0, (size_t)cfg->n_clients * h->stride * sizeof(float)) != cudaSuccess) {
+    cudaError_t e = cudaGetLastError();
+    aet_destroy(h);
+    return fail(nullptr, AET_ERR_CUDA, std::string("cudaMemset: ") + cudaGetErrorString(e));
+  }
   if (cudaMemset(h->w_buf[0].p, 0, h->stride * sizeof(float)) != cudaSuccess ||
       cudaMemset(h->w_buf[1].p, 0, h->stride * sizeof(float)) != cudaSuccess ||
       cudaMemset(h->d_status.p, 0, sizeof(uint32_t)) != cudaSuccess ||
@@ -281,6 +382,7 @@ aet_status aet_destroy(aet_handle* h) {
   h->d_clients.release(); h->d_keys.release(); h->d_H.release();
   h->w_buf[0].release(); h->w_buf[1].release(); h->totals.release(); h->d_status.release(); h->w0.release(); h->snaps.release(); h->U.release();
   h->work.release(); h->act.release(); h->dbg.release();
+  h->node_w.release(); h->d_ring_applies.release(); h->d_ring_ops.release();
   h->d_tasks.release(); h->d_inflight.release(); h->d_applies.release();
   h->d_trig.release(); h->d_alog.release();
   cudaGetLastError();
@@ -293,6 +395,10 @@ aet_status aet_reset(aet_handle* h, void* cuda_stream) {
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaMemcpyAsync(h->w_cur(), h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
   AET_CUDA(h, cudaMemsetAsync(h->d_H.p, 0, h->cfg.n_clients * sizeof(uint32_t), s));
+  if (h->cfg.topology == 1)
+    for (uint32_t c = 0; c < h->cfg.n_clients; ++c)
+      AET_CUDA(h, cudaMemcpyAsync(h->node_w.p + (size_t)c * h->stride, h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  h->rst = RingState{};
   h->st = SchedState{};
   h->st.H.assign(h->cfg.n_clients, 0);
   h->log.clear();
@@ -309,6 +415,9 @@ aet_status aet_set_global_model(aet_handle* h, const float* w0, size_t n_params,
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaMemcpyAsync(h->w_cur(), w0, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
   AET_CUDA(h, cudaMemcpyAsync(h->w0.p, h->w_cur(), (size_t)h->P * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  if (h->cfg.topology == 1)   // every node starts from it (Algorithm 2: the same initial model for all compute nodes)
+    for (uint32_t c = 0; c < h->cfg.n_clients; ++c)
+      AET_CUDA(h, cudaMemcpyAsync(h->node_w.p + (size_t)c * h->stride, h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
   AET_CUDA(h, cudaStreamSynchronize(s));
   h->have_w0 = true;
   h->last_stream = s;
@@ -385,6 +494,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   if (n_rounds == 0) return AET_OK;
   collect_timings(h);
   h->stats = aet_stats{};
+  if (h->cfg.topology == 1) return run_ring_rounds(h, n_rounds, s);
 
   // ---- a0: integer schedule and launch plan (cached for repeated runs) ----
   auto t0 = std::chrono::steady_clock::now();
@@ -478,6 +588,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
 aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params, void* cuda_stream) {
   if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
+  if (h->cfg.topology == 1) return fail(h, AET_ERR_STATE, "the peer-to-peer topology has no server model: use aet_get_node_model");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaStreamSynchronize(s));
   if (aet_status ds = check_device_status(h)) return ds;   // `out` stays untouched on error
@@ -486,11 +597,25 @@ aet_status aet_get_global_model(aet_handle* h, float* out, size_t n_params, void
   return AET_OK;
 }
 
+aet_status aet_get_node_model(aet_handle* h, uint32_t node, float* out, size_t n_params, void* cuda_stream) {
+  if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
+  if (node >= h->cfg.n_clients) return fail(h, AET_ERR_ARG, "node index out of range");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  if (aet_status ds = check_device_status(h)) return ds;
+  // client-server: at quiescence every client slot equals the server model
+  const float* src = h->cfg.topology == 1 ? h->node_w.p + (size_t)node * h->stride : h->w_cur();
+  AET_CUDA(h, cudaMemcpyAsync(out, src, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
+  AET_CUDA(h, cudaStreamSynchronize(s));
+  return AET_OK;
+}
+
 aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params, void* cuda_stream) {
   if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
   if (seq >= h->last_n_events) return fail(h, AET_ERR_ARG, "seq is not an event of the most recent run");
-  if (!(h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS))
+  if (h->cfg.topology == 0 && !(h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS))
     return fail(h, AET_ERR_STATE, "update sums are recycled during a run unless the handle was created with AET_FLAG_KEEP_UPDATE_SUMS");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaMemcpyAsync(out, h->U.p + (size_t)seq * h->stride, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));
@@ -500,6 +625,20 @@ aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_
 
 aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity, size_t* n_events, aet_summary* summary) {
   if (!h || !n_events) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
+  if (!h->last_checked && h->last_n_events && h->cfg.topology == 1) {
+    // the trigger record every round kernel left behind, against the schedule it was launched from
+    const size_t T = h->last_n_events;
+    std::vector<TriggerRec> trig(T);
+    AET_CUDA(h, cudaStreamSynchronize(h->last_stream));
+    AET_CUDA(h, cudaMemcpy(trig.data(), h->d_trig.p, T * sizeof(TriggerRec), cudaMemcpyDeviceToHost));
+    if (aet_status ds = check_device_status(h)) return ds;
+    for (size_t k = 0; k < T; ++k) {
+      const RingTask& t = h->last_ring_tasks[k];
+      if (trig[k].flags != 1 || trig[k].client != t.client || trig[k].round != t.round || trig[k].samples_done != t.samples)
+        return fail(h, AET_ERR_STATE, "device trigger record " + std::to_string(k) + " does not match the schedule");
+    }
+    h->last_checked = true;
+  }
   if (!h->last_checked && h->last_n_events) {
     // Compare what the kernels recorded (trigger per round-task, apply order and
     // history counts) with the schedule they were launched from.
@@ -627,16 +766,28 @@ aet_status aet_schedule_only(const aet_config* cfg, uint32_t n_rounds, aet_event
   std::string err;
   if (cfg->struct_size != sizeof(aet_config)) return fail(nullptr, AET_ERR_ARG, "struct_size does not match sizeof(aet_config)");
   if (!validate_config(*cfg, err)) return fail(nullptr, AET_ERR_CONFIG, err);
-  SchedState st;
   DelayCache cache;
-  SchedResult res;
-  if (!simulate(*cfg, n_rounds, st, cache, res, err)) return fail(nullptr, AET_ERR_CONFIG, err);
-  if (out) {
-    if (capacity < res.events.size()) return fail(nullptr, AET_ERR_ARG, "capacity is smaller than the log");
-    memcpy(out, res.events.data(), res.events.size() * sizeof(aet_event));
+  std::vector<aet_event> events;
+  aet_summary sum{};
+  if (cfg->topology == 1) {
+    RingState rst;
+    RingResult rres;
+    if (!simulate_ring(*cfg, n_rounds, rst, cache, rres, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+    events.swap(rres.events);
+    sum = rres.summary;
+  } else {
+    SchedState st;
+    SchedResult res;
+    if (!simulate(*cfg, n_rounds, st, cache, res, err)) return fail(nullptr, AET_ERR_CONFIG, err);
+    events.swap(res.events);
+    sum = res.summary;
   }
-  *n_events = res.events.size();
-  if (summary) *summary = res.summary;
+  if (out) {
+    if (capacity < events.size()) return fail(nullptr, AET_ERR_ARG, "capacity is smaller than the log");
+    memcpy(out, events.data(), events.size() * sizeof(aet_event));
+  }
+  *n_events = events.size();
+  if (summary) *summary = sum;
   return AET_OK;
 }
 

@@ -96,6 +96,18 @@ struct ApplyLaunch {
 uint32_t apply_groups(uint32_t n_updates);
 cudaError_t launch_apply_updates(const ApplyLaunch& p, cudaStream_t s);
 
+// Peer-to-peer ring: the models of the nodes listed in applies[lo, hi) take their operations.
+struct RingApplyLaunch {
+  const RingApplyDesc* applies;  // device
+  const RingOp* ops;             // device
+  const float* U;                // [n_tasks, stride]
+  float* node_w;                 // [n_nodes, stride]
+  uint32_t* status;              // optional: bit 1 set if a model is not finite afterwards
+  size_t stride;
+  uint32_t n_params, lo, hi;
+};
+cudaError_t launch_ring_apply(const RingApplyLaunch& p, cudaStream_t s);
+
 // Debug checks at load time: labels in range (else bit 2 of *status), pixels finite (else bit 1; x may be null).
 cudaError_t launch_validate_data(const float* x, const int32_t* y, uint32_t n, uint32_t dim, uint32_t n_classes,
                                  uint32_t* status, cudaStream_t s);

@@ -93,6 +93,7 @@ bool validate_config(const aet_config& c, std::string& err) {
                             c.compute_delay_lo < 0 || c.network_delay_lo < 0)) { err = "uniform delay range is empty"; return false; }
   if (!(c.straggler_factor >= 0) || c.straggler_factor > 65535.0) { err = "straggler_factor out of range"; return false; }
   if (c.split_mode > 1) { err = "split_mode must be 0 or 1"; return false; }
+  if (c.topology > 1) { err = "topology must be 0 (client-server) or 1 (ring)"; return false; }
   if (c.split_mode && c.batch != 1) { err = "the Setup split assigns single SGD iterations: batch must be 1"; return false; }
   if (c.client_shares) {
     uint64_t total = 0;
@@ -245,7 +246,7 @@ bool simulate(const aet_config& c, uint32_t n_rounds, SchedState& st, DelayCache
     e.client = cl; e.round = round;
     e.samples = node_sample_size(c, cache, cl, round);
     e.steps = e.samples / c.batch;
-    e.seq = 0; e.seen = seq; e.lag = lag; e.pad = 0;
+    e.seq = 0; e.seen = seq; e.lag = lag; e.dest = 0;
     ev_of[(size_t)cl * n_rounds + (round - first)] = (uint32_t)out.events.size();
     out.events.push_back(e);
     q.push({e.t_apply, kApply, cl, round});
@@ -406,6 +407,275 @@ void build_plan(const aet_config& c, const DelayCache& cache, const std::vector<
     t.inflight_cnt = (uint32_t)plan.inflight.size() - t.inflight_off;
     plan.tasks.push_back(t);
   }
+}
+
+// ---------------------------------------------------------------------------
+// Peer-to-peer ring.  Algorithm 3 read per node: Receive bumps H_v[sender] when the message
+// arrives, Synchronize(H, d, i) looks at the node's own neighbours, "Send a tuple (c, U_i, i) to
+// the other c's neighbors" goes to the two ring neighbours with a network delay each (draw
+// 2 * round + side of the sender's network stream; side 0 = node c - 1, side 1 = node c + 1).
+// Ties: (tick, receive before start, node, then sender and round).
+namespace {
+
+struct RingQItem {
+  uint64_t t; uint32_t kind, node, x, y;   // receive: node = destination, x = sender, y = round; start: x = round
+  bool operator>(const RingQItem& o) const {
+    return std::tie(t, kind, node, x, y) > std::tie(o.t, o.kind, o.node, o.x, o.y);
+  }
+};
+enum RingKind : uint32_t { kReceive = 0, kRingStart = 1 };
+
+// Neighbours of node c: up to two (side, node) pairs, no duplicates, never c itself.
+int ring_neighbours(uint32_t n, uint32_t c, uint32_t (&side)[2], uint32_t (&node)[2]) {
+  int cnt = 0;
+  const uint32_t cand[2] = {(c + n - 1) % n, (c + 1) % n};
+  for (uint32_t sd = 0; sd < 2; ++sd) {
+    if (cand[sd] == c) continue;
+    if (cnt == 1 && node[0] == cand[sd]) continue;
+    side[cnt] = sd; node[cnt] = cand[sd]; ++cnt;
+  }
+  return cnt;
+}
+
+}  // namespace
+
+bool simulate_ring(const aet_config& c, uint32_t n_rounds, RingState& st, DelayCache& cache,
+                   RingResult& out, std::string& err) {
+  const uint32_t n = c.n_clients;
+  if (st.H.size() != 2 * (size_t)n) st.H.assign(2 * (size_t)n, 0);
+  const uint32_t first = c.round_base + st.rounds_done, last = first + n_rounds;
+  for (uint32_t r = first; r < last; ++r)
+    if (sample_size(c, r) == 0 || sample_size(c, r) % c.batch) {
+      err = "batch must divide every round's sample count, and rounds may not be empty";
+      return false;
+    }
+  ensure_split(c, last, cache);
+  fill_delays(c, first, last, cache);
+  const DelayModel dm = make_delay_model(c);
+  std::vector<uint64_t> key_n(n);
+  for (uint32_t cl = 0; cl < n; ++cl) key_n[cl] = stream_key(c.seed, kStreamNetwork, cl);
+
+  out = RingResult{};
+  std::vector<uint32_t>& H = st.H;
+  std::vector<uint64_t> ready(n, st.clock);
+  std::vector<int64_t> blocked(n, -1);
+  std::vector<std::vector<uint32_t>> pending(n);   // deliveries (creation index) that reached a node since its last start
+  std::vector<uint32_t> n_received(n, 0);
+  struct Made { aet_event e; uint32_t task_creation; bool sequenced; };
+  std::vector<Made> made;                          // deliveries in creation order
+  struct TaskTmp { RingTask t; std::vector<uint32_t> applied; };
+  std::vector<TaskTmp> tmp;                        // tasks in start order
+  std::priority_queue<RingQItem, std::vector<RingQItem>, std::greater<RingQItem>> q;
+  for (uint32_t cl = 0; cl < n && n_rounds; ++cl) q.push({st.clock, kRingStart, cl, first, 0});
+  const bool never_wait = c.max_lag_d == AET_NEVER_WAIT;
+  uint32_t seq = 0, n_blocked = 0;
+  // (destination, sender, round) -> creation index of the delivery
+  std::vector<std::vector<uint32_t>> made_of((size_t)n * n_rounds);   // per sender task: its deliveries
+
+  auto lag_of = [&](uint32_t cl, uint32_t round) -> uint32_t {
+    uint32_t sd[2], nd[2];
+    const int k = ring_neighbours(n, cl, sd, nd);
+    if (!k) return 0;
+    uint32_t m = UINT32_MAX;
+    for (int j = 0; j < k; ++j) m = std::min(m, H[2 * cl + sd[j]]);
+    const uint32_t rel = round - c.round_base;
+    return rel > m ? rel - m : 0;
+  };
+
+  while (!q.empty()) {
+    const RingQItem it = q.top();
+    q.pop();
+    if (it.kind == kReceive) {
+      const uint32_t dest = it.node, sender = it.x, round = it.y;
+      // which side of dest the sender sits on
+      uint32_t sd[2], nd[2];
+      const int k = ring_neighbours(n, dest, sd, nd);
+      for (int j = 0; j < k; ++j) if (nd[j] == sender) H[2 * dest + sd[j]] += 1;
+      for (uint32_t m : made_of[(size_t)sender * n_rounds + (round - first)])
+        if (made[m].e.dest == dest && !made[m].sequenced) {
+          made[m].e.seq = seq++;
+          made[m].sequenced = true;
+          pending[dest].push_back(m);
+          break;
+        }
+      n_received[dest] += 1;
+      if (blocked[dest] >= 0 && (never_wait || lag_of(dest, (uint32_t)blocked[dest]) <= c.max_lag_d)) {
+        q.push({it.t, kRingStart, dest, (uint32_t)blocked[dest], 0});
+        blocked[dest] = -1;
+        --n_blocked;
+      }
+      continue;
+    }
+    const uint32_t cl = it.node, round = it.x;
+    const uint32_t lag = lag_of(cl, round);
+    if (!never_wait && lag > c.max_lag_d) { blocked[cl] = round; ++n_blocked; continue; }
+    TaskTmp tt;
+    tt.t.t_start = it.t;
+    tt.t.t_trigger = it.t + cache.busy[cl][round - c.round_base];
+    tt.t.client = cl; tt.t.round = round;
+    tt.t.samples = node_sample_size(c, cache, cl, round);
+    tt.t.steps = tt.t.samples / c.batch;
+    tt.t.applied_off = tt.t.applied_cnt = 0;
+    tt.applied.swap(pending[cl]);
+    aet_event e{};
+    e.t_start = it.t; e.t_trigger = tt.t.t_trigger; e.wait_ticks = it.t - ready[cl];
+    e.client = cl; e.round = round; e.samples = tt.t.samples; e.steps = tt.t.steps;
+    e.seen = n_received[cl]; e.lag = lag;
+    uint32_t sd[2], nd[2];
+    const int k = ring_neighbours(n, cl, sd, nd);
+    const uint32_t task_creation = (uint32_t)tmp.size();
+    for (int j = 0; j < k; ++j) {
+      e.t_apply = tt.t.t_trigger + dm.network(draw(key_n[cl], 2ull * round + sd[j]));
+      e.dest = nd[j];
+      made_of[(size_t)cl * n_rounds + (round - first)].push_back((uint32_t)made.size());
+      made.push_back({e, task_creation, false});
+      q.push({e.t_apply, kReceive, nd[j], cl, round});
+    }
+    if (!k) {
+      e.t_apply = tt.t.t_trigger;
+      e.dest = kNoDest;
+      made.push_back({e, task_creation, false});
+    }
+    tmp.push_back(std::move(tt));
+    ready[cl] = e.t_trigger;
+    if (round + 1 < last) q.push({e.t_trigger, kRingStart, cl, round + 1, 0});
+  }
+  if (n_blocked) { err = "schedule did not reach quiescence"; return false; }
+  // records of a node without neighbours take their places by trigger time
+  {
+    std::vector<uint32_t> lone;
+    for (uint32_t m = 0; m < made.size(); ++m) if (made[m].e.dest == kNoDest) lone.push_back(m);
+    std::sort(lone.begin(), lone.end(), [&](uint32_t a, uint32_t b) {
+      return std::tie(made[a].e.t_apply, made[a].e.client, made[a].e.round) <
+             std::tie(made[b].e.t_apply, made[b].e.client, made[b].e.round);
+    });
+    for (uint32_t m : lone) { made[m].e.seq = seq++; made[m].sequenced = true; }
+  }
+  if (seq != made.size()) { err = "schedule did not deliver every message"; return false; }
+  // tasks in (t_trigger, client, round) order; deliveries in seq order
+  std::vector<uint32_t> torder(tmp.size());
+  for (uint32_t k = 0; k < tmp.size(); ++k) torder[k] = k;
+  std::sort(torder.begin(), torder.end(), [&](uint32_t a, uint32_t b) {
+    return std::tie(tmp[a].t.t_trigger, tmp[a].t.client, tmp[a].t.round) <
+           std::tie(tmp[b].t.t_trigger, tmp[b].t.client, tmp[b].t.round);
+  });
+  std::vector<uint32_t> task_index(tmp.size());
+  for (uint32_t k = 0; k < torder.size(); ++k) task_index[torder[k]] = k;
+  out.events.resize(made.size());
+  out.event_task.resize(made.size());
+  for (const Made& m : made) {
+    out.events[m.e.seq] = m.e;
+    out.event_task[m.e.seq] = task_index[m.task_creation];
+  }
+  out.tasks.resize(tmp.size());
+  for (uint32_t k = 0; k < torder.size(); ++k) {
+    TaskTmp& tt = tmp[torder[k]];
+    tt.t.applied_off = (uint32_t)out.applied.size();
+    tt.t.applied_cnt = (uint32_t)tt.applied.size();
+    for (uint32_t m : tt.applied) out.applied.push_back(made[m].e.seq);
+    out.tasks[k] = tt.t;
+  }
+  aet_summary& s = out.summary;
+  s = aet_summary{};
+  uint64_t links = 0;
+  for (uint32_t cl = 0; cl < n; ++cl) { uint32_t sd[2], nd[2]; links += ring_neighbours(n, cl, sd, nd); }
+  for (const aet_event& e : out.events) if (e.dest != kNoDest) s.messages_up += 1;
+  for (const RingTask& t : out.tasks) s.samples_total += t.samples;
+  s.model_pulls = 0;
+  s.messages_if_per_sample = (s.samples_total / c.batch) * (n ? links / n : 0);
+  uint64_t s_first = sample_size(c, c.round_base);
+  if (c.split_mode) s_first = std::max<uint64_t>(1, s_first / n);
+  const uint64_t per_client = n ? s.samples_total / n : 0;
+  s.messages_if_constant_b = s_first ? links * ((per_client + s_first - 1) / s_first) : 0;
+  s.t_end_ticks = st.clock;
+  for (const aet_event& e : out.events) s.t_end_ticks = std::max(s.t_end_ticks, e.t_apply);
+  st.clock = s.t_end_ticks;
+  st.rounds_done += n_rounds;
+  return true;
+}
+
+// Waves and per-node operation lists of a ring run.  A round-task's level is one more than the
+// levels of its node's previous round and of every round whose sum reached the node before it
+// started.  Before wave L the model of every node with a task in L takes, in this order, the
+// node's own previous sum (the net effect of that round's inner loop) and the sums that arrived
+// since its previous start; after the last wave every node takes what is still outstanding.
+void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingResult& r, RingPlan& plan) {
+  plan = RingPlan{};
+  const uint32_t n = c.n_clients;
+  const size_t T = r.tasks.size();
+  std::vector<uint32_t> order(T);
+  for (size_t k = 0; k < T; ++k) order[k] = (uint32_t)k;
+  std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+    return std::tie(r.tasks[a].t_start, r.tasks[a].client, r.tasks[a].round) <
+           std::tie(r.tasks[b].t_start, r.tasks[b].client, r.tasks[b].round);
+  });
+  std::vector<uint32_t> level(T, 0), prev_level(n, 0);
+  std::vector<int64_t> prev_task(T, -1), last_task(n, -1);
+  uint32_t n_waves = 0;
+  for (uint32_t k : order) {
+    const RingTask& t = r.tasks[k];
+    uint32_t lv = prev_level[t.client];
+    for (uint32_t a = 0; a < t.applied_cnt; ++a) lv = std::max(lv, level[r.event_task[r.applied[t.applied_off + a]]]);
+    level[k] = lv + 1;
+    prev_level[t.client] = lv + 1;
+    prev_task[k] = last_task[t.client];
+    last_task[t.client] = k;
+    n_waves = std::max(n_waves, lv + 1);
+  }
+  std::vector<uint32_t> by_wave(T);
+  for (size_t k = 0; k < T; ++k) by_wave[k] = (uint32_t)k;
+  std::sort(by_wave.begin(), by_wave.end(), [&](uint32_t a, uint32_t b) {
+    if (level[a] != level[b]) return level[a] < level[b];
+    if (r.tasks[a].samples != r.tasks[b].samples) return r.tasks[a].samples > r.tasks[b].samples;
+    return a < b;
+  });
+  plan.wave_off.assign(n_waves + 1, 0);
+  for (uint32_t k : by_wave) plan.wave_off[level[k]] += 1;
+  for (uint32_t L = 1; L <= n_waves; ++L) plan.wave_off[L] += plan.wave_off[L - 1];
+  plan.apply_off.assign(n_waves + 2, 0);
+  std::vector<char> delivered(r.events.size(), 0);
+  auto eta_of_task = [&](uint32_t k) { return (float)round_step_size(c, cache, r.tasks[k].client, r.tasks[k].round); };
+  for (uint32_t L = 0; L < n_waves; ++L) {
+    plan.max_wave_tasks = std::max(plan.max_wave_tasks, plan.wave_off[L + 1] - plan.wave_off[L]);
+    for (uint32_t q = plan.wave_off[L]; q < plan.wave_off[L + 1]; ++q) {
+      const uint32_t k = by_wave[q];
+      const RingTask& t = r.tasks[k];
+      TaskDesc d{};
+      d.client = t.client; d.round = t.round; d.seq = k; d.snap_slot = t.client;
+      d.n_samples = t.samples; d.steps = t.steps;
+      d.inflight_off = 0; d.inflight_cnt = 0;
+      d.sample_ctr0 = node_samples_before(c, cache, t.client, t.round);
+      d.eta = eta_of_task(k);
+      d.u_row = k;
+      plan.tasks.push_back(d);
+      RingApplyDesc a{t.client, (uint32_t)plan.ops.size(), 0, 0};
+      if (prev_task[k] >= 0) plan.ops.push_back({(uint32_t)prev_task[k], eta_of_task((uint32_t)prev_task[k])});
+      for (uint32_t j = 0; j < t.applied_cnt; ++j) {
+        const uint32_t ev = r.applied[t.applied_off + j];
+        plan.ops.push_back({r.event_task[ev], eta_of_task(r.event_task[ev])});
+        delivered[ev] = 1;
+      }
+      a.op_cnt = (uint32_t)plan.ops.size() - a.op_off;
+      if (a.op_cnt) plan.applies.push_back(a);
+    }
+    plan.apply_off[L + 1] = (uint32_t)plan.applies.size();
+  }
+  // Shift: the operations collected for wave L run before it, i.e. they belong to slot L.
+  // apply_off[L] .. apply_off[L + 1] already has that meaning (slot 0 = before wave 0).
+  // After the last wave: every node's last own sum and the deliveries nobody has taken yet, in seq order.
+  std::vector<std::vector<RingOp>> tail(n);
+  for (uint32_t cl = 0; cl < n; ++cl)
+    if (last_task[cl] >= 0) tail[cl].push_back({(uint32_t)last_task[cl], eta_of_task((uint32_t)last_task[cl])});
+  for (size_t ev = 0; ev < r.events.size(); ++ev)
+    if (!delivered[ev] && r.events[ev].dest != kNoDest)
+      tail[r.events[ev].dest].push_back({r.event_task[ev], eta_of_task(r.event_task[ev])});
+  for (uint32_t cl = 0; cl < n; ++cl) {
+    if (tail[cl].empty()) continue;
+    RingApplyDesc a{cl, (uint32_t)plan.ops.size(), (uint32_t)tail[cl].size(), 0};
+    plan.ops.insert(plan.ops.end(), tail[cl].begin(), tail[cl].end());
+    plan.applies.push_back(a);
+  }
+  plan.apply_off[n_waves + 1] = (uint32_t)plan.applies.size();
 }
 
 }  // namespace aet

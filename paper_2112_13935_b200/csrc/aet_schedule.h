@@ -80,4 +80,42 @@ struct Plan {
 // and slots are recycled as soon as nothing later in the launch order reads them.
 void build_plan(const aet_config& c, const DelayCache& cache, const std::vector<aet_event>& events, bool keep_all, Plan& plan);
 
+// ---- peer-to-peer ring (Section 1, Fig. 1b) ------------------------------
+// Every node keeps its own model and history map; a round's sum goes to the two ring neighbours
+// only and is not forwarded.  One log record per delivery (sender, round, destination).
+constexpr uint32_t kNoDest = 0xFFFFFFFFu;   // destination of the records of a node without neighbours
+struct RingState {
+  uint64_t clock = 0;
+  std::vector<uint32_t> H;     // [2 * node + side]: messages node has received from that side's neighbour
+  uint32_t rounds_done = 0;
+};
+struct RingTask {              // one round-task, in (t_trigger, client, round) order
+  uint64_t t_start, t_trigger;
+  uint32_t client, round, samples, steps;
+  uint32_t applied_off, applied_cnt;   // deliveries (indices into RingResult::events) that reached the node
+                                       // since its previous start, in arrival order
+};
+struct RingResult {
+  std::vector<aet_event> events;       // deliveries ordered by seq; pad holds the destination
+  std::vector<uint32_t> event_task;    // task index of the round each delivery carries
+  std::vector<RingTask> tasks;
+  std::vector<uint32_t> applied;       // flat lists referenced by RingTask
+  aet_summary summary;
+};
+bool simulate_ring(const aet_config& c, uint32_t n_rounds, RingState& st, DelayCache& cache,
+                   RingResult& out, std::string& err);
+
+struct RingOp { uint32_t u_row; float eta; };   // w_node -= eta * U[u_row]
+struct RingApplyDesc { uint32_t node, op_off, op_cnt, pad; };
+struct RingPlan {
+  std::vector<TaskDesc> tasks;          // sorted by wave; snap_slot = node, u_row = task index, no sums in flight
+  std::vector<uint32_t> wave_off;
+  // before wave L (and once more after the last wave): the nodes whose models move and their operations
+  std::vector<RingApplyDesc> applies;   // grouped by wave: [apply_off[L], apply_off[L + 1])
+  std::vector<uint32_t> apply_off;      // n_waves + 2 entries
+  std::vector<RingOp> ops;
+  uint32_t max_wave_tasks = 0;
+};
+void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingResult& r, RingPlan& plan);
+
 }  // namespace aet

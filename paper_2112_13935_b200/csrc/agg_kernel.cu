@@ -114,6 +114,23 @@ __global__ void to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __r
   for (; i < n; i += step) dst[i] = __float2bfloat16_rn(src[i]);
 }
 
+// Peer-to-peer ring: Receive at every node (Algorithm 3: w_c = w_c - eta_k * U) for the sums that
+// reached it, preceded by the node's own sum of the round it has just finished.  One y-block per node
+// whose model moves; a thread keeps its parameter in a register and walks the node's short list.
+__global__ void __launch_bounds__(kAggThreads) ring_apply_kernel(RingApplyLaunch p) {
+  const uint32_t j = blockIdx.x * kAggThreads + threadIdx.x;
+  if (j >= p.n_params) return;
+  const RingApplyDesc a = p.applies[p.lo + blockIdx.y];
+  float* wp = p.node_w + (size_t)a.node * p.stride + j;
+  float w = *wp;
+  for (uint32_t k = 0; k < a.op_cnt; ++k) {
+    const RingOp op = p.ops[a.op_off + k];
+    w = fmaf(-op.eta, __ldg(p.U + (size_t)op.u_row * p.stride + j), w);
+  }
+  *wp = w;
+  if (p.status && !isfinite(w)) atomicOr(p.status, 2u);
+}
+
 // Debug pass over a client's data set as it is loaded: a label outside [0, n_classes) sets bit 2
 // of *status, a non-finite pixel bit 1.  Nothing is trapped on; the host turns the bits into
 // AET_ERR_STATE / AET_ERR_NUMERIC at its next synchronising call.
@@ -137,6 +154,13 @@ cudaError_t launch_validate_data(const float* x, const int32_t* y, uint32_t n, u
   size_t blocks = ((size_t)n * dim + 255) / 256;
   if (blocks > 148 * 8) blocks = 148 * 8;
   validate_data_kernel<<<(unsigned)blocks, 256, 0, s>>>(x, y, n, dim, n_classes, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ring_apply(const RingApplyLaunch& p, cudaStream_t s) {
+  if (p.hi <= p.lo) return cudaSuccess;
+  const uint32_t blocks = (p.n_params + kAggThreads - 1) / kAggThreads;
+  ring_apply_kernel<<<dim3(blocks, p.hi - p.lo, 1), kAggThreads, 0, s>>>(p);
   return cudaGetLastError();
 }
 

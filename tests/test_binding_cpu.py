@@ -179,3 +179,22 @@ def test_recycled_rows_and_slots_always_hold_what_is_read(name, over):
     assert lay["waves"] == keep["waves"] == api.aet_debug_plan_waves(cfg, R)
     if name == "cfg2" and not over:
         assert lay["n_u_rows"] < len(events) // 4     # recycling pays: rows ~ rounds in flight
+
+
+@pytest.mark.parametrize("over", [
+    dict(n_clients=5), dict(n_clients=5, max_lag_d=0), dict(n_clients=5, max_lag_d=2), dict(n_clients=8, max_lag_d=5),
+    dict(n_clients=1), dict(n_clients=2), dict(n_clients=3, network_delay_mean=30.0),
+    dict(n_clients=6, n_stragglers=2, straggler_factor=25.0, max_lag_d=1),
+    dict(n_clients=7, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=40.0),
+    dict(n_clients=5, delay_dist=1, round_base=1, sched_b=0, lr_beta=0.01),              # the paper's own ring setting
+    dict(n_clients=4, split_mode=1, sched_a=9, sched_b=4, client_shares=[3, 1, 1, 2]),    # with the Setup split
+    # constant, equal delays: many simultaneous arrivals (tie rule: by destination, then sender)
+    dict(n_clients=4, sched_a=0, sched_b=1, delay_dist=1, compute_delay_lo=10 / 2 ** 20, compute_delay_hi=10 / 2 ** 20,
+         network_delay_lo=25 / 2 ** 20, network_delay_hi=25 / 2 ** 20, max_lag_d=1),
+])
+def test_ring_schedule_is_bit_identical_to_the_checker(over):
+    cfg = workloads.get_config("cfg1", topology=1, **over)
+    blob, summary = api.aet_schedule_only(cfg, 7, raw=True)
+    tasks, deliveries, want, _ = schedule.simulate_ring(cfg, 7)
+    assert blob == schedule.pack_ring_events(deliveries)
+    assert summary == want

@@ -353,17 +353,13 @@ def test_errors_are_reported_not_raised_by_the_device():
     dict(n_clients=5, sched_a=6, sched_b=2, l2=0.0),                                   # blocked kernel; some rounds are empty
     dict(n_clients=3, sched_a=10, sched_b=5, client_shares=[1, 2, 5], lr_beta=0.02, l2=1e-4),   # unequal p_c, step-by-step kernel
     dict(n_clients=200, sched_a=300, sched_b=200, l2=0.0, lr=1e-4, n_rounds=4, data=dict(per_client=64)),   # tensor-memory kernel
-    dict(model=0, dims=[784, 10], batch=1, n_clients=4, sched_a=5, sched_b=3, l2=0.0, flags=0, precision=0,
-         data=dict(per_client=100), generic=True),                                     # the generic kernel (see below)
+    dict(model=0, dims=[50, 10], n_clients=4, sched_a=5, sched_b=3, l2=0.0,
+         data=dict(per_client=100, dim=50)),                                           # another width: the generic round kernel
 ])
 def test_setup_split_of_a_global_round_size_end_to_end(over):
     # Algorithm 2: s_i = a i + b is the global size of round i, split among the nodes by coin flips
-    over = dict(over)
-    generic = over.pop("generic", False)
     base = dict(split_mode=1, n_rounds=7, data=dict(per_client=300))
     base.update(over)
-    if generic:
-        base["dims"] = [784, 10]
     cfg = workloads.get_config("cfg1", **base)
     data, w0 = make(cfg)
     ref = sim.run(cfg, data, w0, keep=True)
