@@ -99,6 +99,136 @@ def loss_and_grad(w, X, y, dims, l2=0.0, precision=0):
     return loss, g
 
 
+# ---- a small convolutional classifier (the paper trains LeNet on its 28x28 sets; Appendix,
+# "Objective function") ----
+# The paper names the network and no more; this is the classical LeNet shape with the details
+# fixed here: dims = [side, c_in, c1, c2, f1, f2, classes];
+#   conv 5x5 valid (c_in -> c1) + bias, ReLU, 2x2 average pooling,
+#   conv 5x5 valid (c1 -> c2) + bias, ReLU, 2x2 average pooling, flatten [c2][y][x],
+#   dense f1, ReLU, dense f2, ReLU, dense classes, softmax cross-entropy (mean over the batch).
+# "conv" is the cross-correlation z[c, y, x] = sum W[c, ci, dy, dx] * in[ci, y + dy, x + dx] + b[c].
+# Parameters are flattened in layer order: W1 [c1, c_in, 5, 5], b1, W2 [c2, c1, 5, 5], b2, then the
+# dense layers as in the MLP (W row-major [in, out], then b).  The l2 term covers every weight
+# tensor (conv and dense), no bias.  Inputs are rows of side*side*c_in values, plane by plane.
+KS = 5   # kernel side of both convolutions
+
+
+def cnn_shapes(dims):
+    side, c_in, c1, c2, f1, f2, ncls = dims
+    s1 = side - KS + 1
+    p1 = s1 // 2
+    s2 = p1 - KS + 1
+    p2 = s2 // 2
+    assert s1 > 0 and s1 % 2 == 0 and s2 > 0 and s2 % 2 == 0, "sides must stay even through both stages"
+    return dict(side=side, c_in=c_in, c1=c1, c2=c2, s1=s1, p1=p1, s2=s2, p2=p2, flat=c2 * p2 * p2,
+                dense=[c2 * p2 * p2, f1, f2, ncls])
+
+
+def cnn_n_params(dims) -> int:
+    sh = cnn_shapes(dims)
+    n = sh["c1"] * sh["c_in"] * KS * KS + sh["c1"] + sh["c2"] * sh["c1"] * KS * KS + sh["c2"]
+    d = sh["dense"]
+    return n + sum(d[l] * d[l + 1] + d[l + 1] for l in range(3))
+
+
+def cnn_unpack(w, dims):
+    sh = cnn_shapes(dims)
+    o = 0
+    def take(shape):
+        nonlocal o
+        n = int(np.prod(shape))
+        v = w[o:o + n].reshape(shape)
+        o += n
+        return v
+    W1 = take((sh["c1"], sh["c_in"], KS, KS)); b1 = take((sh["c1"],))
+    W2 = take((sh["c2"], sh["c1"], KS, KS)); b2 = take((sh["c2"],))
+    dense = []
+    d = sh["dense"]
+    for l in range(3):
+        Wl = take((d[l], d[l + 1])); bl = take((d[l + 1],))
+        dense.append((Wl, bl))
+    assert o == w.size
+    return W1, b1, W2, b2, dense
+
+
+def _windows(a):
+    """All 5x5 windows of a [B, C, H, W] array: [B, C, H-4, W-4, 5, 5] (a view)."""
+    return np.lib.stride_tricks.sliding_window_view(a, (KS, KS), axis=(2, 3))
+
+
+def _pool(a):
+    B, C, H, W = a.shape
+    return a.reshape(B, C, H // 2, 2, W // 2, 2).mean(axis=(3, 5))
+
+
+def _unpool(g):
+    return np.repeat(np.repeat(g, 2, axis=2), 2, axis=3) / 4.0
+
+
+def cnn_loss_and_grad(w, X, y, dims, l2=0.0):
+    """Mean loss over the rows of X (plus the l2 term) and its gradient (flat), fp64."""
+    w = np.asarray(w, dtype=np.float64)
+    sh = cnn_shapes(dims)
+    B = X.shape[0]
+    x0 = np.asarray(X, dtype=np.float64).reshape(B, sh["c_in"], sh["side"], sh["side"])
+    W1, b1, W2, b2, dense = cnn_unpack(w, dims)
+    z1 = np.einsum("bcyxij,kcij->bkyx", _windows(x0), W1) + b1[None, :, None, None]
+    a1 = np.maximum(z1, 0.0)
+    q1 = _pool(a1)
+    z2 = np.einsum("bcyxij,kcij->bkyx", _windows(q1), W2) + b2[None, :, None, None]
+    a2 = np.maximum(z2, 0.0)
+    q2 = _pool(a2)
+    A = [q2.reshape(B, -1)]
+    Z = []
+    for l in range(3):
+        z = A[l] @ dense[l][0] + dense[l][1]
+        Z.append(z)
+        if l < 2:
+            A.append(np.maximum(z, 0.0))
+    P = softmax_rows(Z[-1])
+    reg = (W1 * W1).sum() + (W2 * W2).sum() + sum((Wl * Wl).sum() for Wl, _ in dense)
+    loss = _ce(P, y).mean() + 0.5 * l2 * reg
+    g = np.empty_like(w)
+    gW1, gb1, gW2, gb2, gdense = cnn_unpack(g, dims)
+    dZ = P.copy()
+    dZ[np.arange(B), y] -= 1.0
+    dZ *= 1.0 / B
+    for l in range(2, -1, -1):
+        gdense[l][0][...] = A[l].T @ dZ + l2 * dense[l][0]
+        gdense[l][1][...] = dZ.sum(axis=0)
+        dA = dZ @ dense[l][0].T
+        if l > 0:
+            dZ = dA * (Z[l - 1] > 0.0)
+    dz2 = _unpool(dA.reshape(q2.shape)) * (z2 > 0.0)
+    gW2[...] = np.einsum("bkyx,bcyxij->kcij", dz2, _windows(q1)) + l2 * W2
+    gb2[...] = dz2.sum(axis=(0, 2, 3))
+    # gradient with respect to the pooled first-stage maps: every output position hands its dz2 back
+    # through the window it read
+    dq1 = np.zeros_like(q1)
+    for i in range(KS):
+        for j in range(KS):
+            dq1[:, :, i:i + sh["s2"], j:j + sh["s2"]] += np.einsum("bkyx,kc->bcyx", dz2, W2[:, :, i, j])
+    dz1 = _unpool(dq1) * (z1 > 0.0)
+    gW1[...] = np.einsum("bkyx,bcyxij->kcij", dz1, _windows(x0)) + l2 * W1
+    gb1[...] = dz1.sum(axis=(0, 2, 3))
+    return loss, g
+
+
+def cnn_full_loss(w, data, dims, l2=0.0, chunk=2048):
+    """F(w) over the union of all clients' data for the convolutional classifier."""
+    tot, cnt = 0.0, 0
+    for X, y in data:
+        for s in range(0, len(y), chunk):
+            n = len(y[s:s + chunk])
+            l, _ = cnn_loss_and_grad(w, X[s:s + chunk], y[s:s + chunk], dims, 0.0)
+            tot += l * n
+            cnt += n
+    w = np.asarray(w, dtype=np.float64)
+    W1, _, W2, _, dense = cnn_unpack(w, dims)
+    reg = (W1 * W1).sum() + (W2 * W2).sum() + sum((Wl * Wl).sum() for Wl, _ in dense)
+    return tot / cnt + 0.5 * l2 * reg
+
+
 def full_loss(w, data, dims, l2=0.0, precision=0, chunk=8192):
     """F(w): mean loss over the union of all clients' data plus the l2 term."""
     w = np.asarray(w, dtype=np.float64)

@@ -48,7 +48,10 @@ def run_task(cfg, client_data, c, i, w_start):
     w = np.array(w_start, dtype=np.float64)
     U = np.zeros_like(w)
     for idx in task_indices(cfg, c, i, len(y)):
-        _, g = models.loss_and_grad(w, X[idx], y[idx], dims, l2, prec)
+        if cfg["model"] == 2:      # the small convolutional classifier
+            _, g = models.cnn_loss_and_grad(w, X[idx], y[idx], dims, l2)
+        else:
+            _, g = models.loss_and_grad(w, X[idx], y[idx], dims, l2, prec)
         w -= eta * g
         U += g
     return U, w

@@ -71,6 +71,11 @@ CONFIGS = {
     "cfg6": dict(_COMMON, n_clients=5, model=0, dims=[784, 10], lr=0.01, lr_beta=0.01,
                  sched_a=10, sched_b=0, round_base=1, n_rounds=110, delay_dist=1,
                  data=dict(kind="iid", total=60000, dim=784)),
+    # A LeNet-shaped convolutional classifier on the 28x28 set (the paper's model for those sets; Appendix,
+    # "Objective function"): 16 clients, minibatch 16, s_i = 32 i + 32 for 12 rounds.
+    "cfg7": dict(_COMMON, n_clients=16, model=2, dims=[28, 1, 6, 16, 120, 84, 10], lr=0.005, batch=16,
+                 sched_a=32, sched_b=32, n_rounds=12, network_delay_mean=1.0,
+                 data=dict(kind="iid", total=60000, dim=784)),
 }
 
 
@@ -89,6 +94,27 @@ def get_config(name: str, **overrides) -> dict:
 
 def n_params(dims) -> int:
     return sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+
+
+CONV_K = 5   # kernel side of the convolutional classifier's two convolutions
+
+
+def cnn_layer_shapes(dims):
+    """(fan_in, number of weights, number of biases) of the five layers of the convolutional classifier
+    dims = [side, c_in, c1, c2, f1, f2, classes] (two 5x5 valid convolutions, each followed by 2x2 average
+    pooling, then three dense layers)."""
+    side, c_in, c1, c2, f1, f2, ncls = dims
+    p2 = ((side - CONV_K + 1) // 2 - CONV_K + 1) // 2
+    flat = c2 * p2 * p2
+    k2 = CONV_K * CONV_K
+    return [(c_in * k2, c1 * c_in * k2, c1), (c1 * k2, c2 * c1 * k2, c2),
+            (flat, flat * f1, f1), (f1, f1 * f2, f2), (f2, f2 * ncls, ncls)]
+
+
+def model_n_params(cfg) -> int:
+    if cfg["model"] == 2:
+        return sum(nw + nb for _, nw, nb in cnn_layer_shapes(cfg["dims"]))
+    return n_params(cfg["dims"])
 
 
 def make_pool(n: int, dim: int, seed: int):
@@ -144,7 +170,7 @@ def make_client_data(cfg: dict):
     n = cfg["n_clients"]
     seed = int(cfg["seed"])
     dim = d["dim"]
-    assert dim == cfg["dims"][0]
+    assert dim == (cfg["dims"][0] * cfg["dims"][0] * cfg["dims"][1] if cfg["model"] == 2 else cfg["dims"][0])
     if d["kind"] == "per_client":
         x, y = make_pool(n * d["per_client"], dim, seed)
         m = d["per_client"]
@@ -163,6 +189,14 @@ def make_start_model(cfg: dict) -> np.ndarray:
     """Start model w_0 as a flat float32 vector (layers in order, W_l row-major
     [in, out] then b_l).  Softmax regression starts at zero; MLPs are seeded."""
     dims = cfg["dims"]
+    if cfg["model"] == 2:      # every tensor ~ U(-1/sqrt(fan_in), 1/sqrt(fan_in)), weights then biases, layer by layer
+        rng = np.random.default_rng(int(cfg["seed"]) + 2000)
+        out = []
+        for fan_in, nw, nb in cnn_layer_shapes(dims):
+            bound = 1.0 / math.sqrt(fan_in)
+            out.append(rng.uniform(-bound, bound, size=nw).astype(np.float32))
+            out.append(rng.uniform(-bound, bound, size=nb).astype(np.float32))
+        return np.concatenate(out)
     P = n_params(dims)
     if cfg["model"] == 0:
         return np.zeros(P, dtype=np.float32)

@@ -41,8 +41,12 @@ def check_against_oracle(cfg, data, w0, gpu, ref, u_tol=U_TOL, loss_tol=LOSS_TOL
     assert gpu["blob"] == schedule.pack_events(ref["events"]), "event log differs"
     assert gpu["summary"] == ref["summary"]
     dims, l2, prec = cfg["dims"], sim.f32(cfg["l2"]), cfg["precision"]
-    f_gpu = models.full_loss(gpu["w"], data, dims, l2, prec)
-    f_ref = models.full_loss(ref["w"], data, dims, l2, prec)
+    if cfg["model"] == 2:
+        f_gpu = models.cnn_full_loss(gpu["w"], data, dims, l2)
+        f_ref = models.cnn_full_loss(ref["w"], data, dims, l2)
+    else:
+        f_gpu = models.full_loss(gpu["w"], data, dims, l2, prec)
+        f_ref = models.full_loss(ref["w"], data, dims, l2, prec)
     assert abs(f_gpu - f_ref) <= loss_tol, (f_gpu, f_ref)
     return f_gpu, f_ref
 

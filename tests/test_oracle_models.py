@@ -169,3 +169,94 @@ def test_bf16_rounding_points_on_a_case_worked_by_hand():
     # and the case separates the two precisions everywhere it should
     _, g32 = models.loss_and_grad(w, X, y, dims, 0.0, precision=0)
     assert np.abs(g - g32).max() > 1e-4
+
+
+# ---- the small convolutional classifier ----
+def _cnn_problem(dims, B, seed):
+    g = np.random.default_rng(seed)
+    w = g.normal(0, 0.2, size=models.cnn_n_params(dims))
+    X = g.uniform(0, 1, size=(B, dims[0] * dims[0] * dims[1]))
+    y = g.integers(0, dims[-1], size=B)
+    return w, X, y
+
+
+def test_cnn_parameter_count_of_the_lenet_shape():
+    # 28x28x1 -> conv 6 -> pool -> conv 16 -> pool -> 256 -> 120 -> 84 -> 10
+    dims = [28, 1, 6, 16, 120, 84, 10]
+    sh = models.cnn_shapes(dims)
+    assert (sh["s1"], sh["p1"], sh["s2"], sh["p2"], sh["flat"]) == (24, 12, 8, 4, 256)
+    assert models.cnn_n_params(dims) == 156 + 2416 + 30840 + 10164 + 850 == 44426
+
+
+@pytest.mark.parametrize("l2", [0.0, 0.05])
+def test_cnn_gradient_matches_central_differences(l2):
+    dims = [16, 2, 3, 4, 7, 6, 5]
+    w, X, y = _cnn_problem(dims, 3, 21)
+    _, g = models.cnn_loss_and_grad(w, X, y, dims, l2)
+    h = 1e-6
+    for j in np.random.default_rng(5).choice(w.size, size=80, replace=False):
+        e = np.zeros_like(w)
+        e[j] = h
+        fp, _ = models.cnn_loss_and_grad(w + e, X, y, dims, l2)
+        fm, _ = models.cnn_loss_and_grad(w - e, X, y, dims, l2)
+        assert abs((fp - fm) / (2 * h) - g[j]) < 2e-7, j
+
+
+def test_cnn_matches_torch_conv_pool_autograd():
+    # a library's convolution, pooling and reverse-mode derivative of the same network, written independently
+    import torch.nn.functional as F
+    dims = [16, 2, 3, 4, 7, 6, 5]
+    w, X, y = _cnn_problem(dims, 4, 8)
+    loss, g = models.cnn_loss_and_grad(w, X, y, dims, 0.01)
+    wt = torch.tensor(w, dtype=torch.float64, requires_grad=True)
+    o = 0
+    def take(*shape):
+        nonlocal o
+        n = int(np.prod(shape))
+        v = wt[o:o + n].reshape(*shape)
+        o += n
+        return v
+    W1, b1, W2, b2 = take(3, 2, 5, 5), take(3), take(4, 3, 5, 5), take(4)
+    a = torch.tensor(X).reshape(4, 2, 16, 16)
+    a = F.avg_pool2d(torch.relu(F.conv2d(a, W1, b1)), 2)
+    a = F.avg_pool2d(torch.relu(F.conv2d(a, W2, b2)), 2).reshape(4, -1)
+    reg = (W1 * W1).sum() + (W2 * W2).sum()
+    for l, (i, j) in enumerate([(4, 7), (7, 6), (6, 5)]):
+        Wl, bl = take(i, j), take(j)
+        reg = reg + (Wl * Wl).sum()
+        a = a @ Wl + bl
+        if l < 2:
+            a = torch.relu(a)
+    lt = F.cross_entropy(a, torch.tensor(y)) + 0.5 * 0.01 * reg
+    lt.backward()
+    assert abs(loss - float(lt)) < 1e-12
+    np.testing.assert_allclose(g, wt.grad.numpy(), rtol=1e-9, atol=1e-12)
+
+
+def test_cnn_one_bright_pixel_by_hand():
+    # one sample, one input plane, every conv weight 0 except W1[0,0,0,0] = 1 and b1 = 0: z1 = the image cropped to
+    # its top-left 12x12; the image is zero except pixel (2, 3) = 0.8, so z1 has one non-zero, a1 the same, and the
+    # pooled map one entry 0.8 / 4 at (1, 1).  With W2 = 0 and b2 = 0.5 every second-stage output is 0.5 (ReLU keeps
+    # it, pooling keeps it), the dense layers are zero with zero bias: logits 0, loss ln(classes).
+    dims = [16, 1, 1, 1, 2, 2, 3]
+    w = np.zeros(models.cnn_n_params(dims))
+    W1, b1, W2, b2, dense = models.cnn_unpack(w, dims)
+    W1[0, 0, 0, 0] = 1.0
+    b2[0] = 0.5
+    x = np.zeros((1, 256))
+    x[0, 2 * 16 + 3] = 0.8
+    loss, g = models.cnn_loss_and_grad(w, x, np.array([1]), dims)
+    assert np.isclose(loss, np.log(3.0))
+    gW1, gb1, gW2, gb2, gd = models.cnn_unpack(g, dims)
+    # only the last dense layer's bias sees a gradient (its input is relu(0) = 0): p - onehot = (1/3, -2/3, 1/3)
+    np.testing.assert_allclose(gd[2][1], [1 / 3, -2 / 3, 1 / 3], atol=1e-15)
+    assert not gd[2][0].any() and not gW1.any() and not gW2.any() and not gd[0][0].any()
+    # now let the second stage read the pooled first-stage map: W2[0,0,1,1] = 4 reads q1[y+1, x+1], which is 0.2 at
+    # (1, 1), so z2[0, 0] = 4 * 0.2 + 0.5 = 1.3 and the other three entries stay 0.5; pooled: (1.3 + 1.5) / 4 = 0.7.
+    # Dense chain: f1 unit 0 = 2 * 0.7 = 1.4, f2 unit 1 = 3 * 1.4 = 4.2, logit 2 = 4.2.
+    W2[0, 0, 1, 1] = 4.0
+    dense[0][0][0, 0] = 2.0
+    dense[1][0][0, 1] = 3.0
+    dense[2][0][1, 2] = 1.0
+    loss2, _ = models.cnn_loss_and_grad(w, x, np.array([2]), dims)
+    assert np.isclose(loss2, -np.log(np.exp(4.2) / (np.exp(4.2) + 2.0)), rtol=0, atol=1e-14)

@@ -196,3 +196,16 @@ def test_ring_history_that_counts_at_round_start_instead_of_arrival_is_caught(mo
     exec(compile(src.replace(old, "            H[node][sender] += 0\n"), "<mutated simulate_ring>", "exec"), ns)
     monkeypatch.setattr(schedule, "simulate_ring", ns["simulate_ring"])
     _fails(tring.test_four_node_timeline_worked_by_hand)
+
+
+def test_cnn_pooling_gradient_without_the_quarter_is_caught(monkeypatch):
+    monkeypatch.setattr(models, "_unpool", lambda g: np.repeat(np.repeat(g, 2, axis=2), 2, axis=3))
+    _fails(tm.test_cnn_gradient_matches_central_differences, 0.0)
+    _fails(tm.test_cnn_matches_torch_conv_pool_autograd)
+
+
+def test_cnn_true_convolution_instead_of_correlation_is_caught(monkeypatch):
+    real = models._windows
+    monkeypatch.setattr(models, "_windows", lambda a: real(a)[..., ::-1, ::-1])
+    _fails(tm.test_cnn_matches_torch_conv_pool_autograd)
+    _fails(tm.test_cnn_one_bright_pixel_by_hand)
