@@ -51,9 +51,16 @@ typedef enum {
 typedef struct {
   uint32_t struct_size;
   uint32_t n_clients;
-  uint32_t model;      /* 0 = softmax regression, 1 = ReLU MLP (Eq. 1: f(w; xi)) */
-  uint32_t n_layers;   /* weight layers = entries of dims - 1                     */
-  uint32_t dims[8];    /* {784,10}, {784,128,10}, {3072,256,128,10}               */
+  uint32_t model;      /* 0 = softmax regression, 1 = ReLU MLP (Eq. 1: f(w; xi)), 2 = a
+                          small convolutional classifier of the LeNet shape (the paper's
+                          model for its 28x28 sets): 5x5 valid convolution + ReLU + 2x2
+                          average pooling, twice, then three dense layers           */
+  uint32_t n_layers;   /* entries of dims - 1                                      */
+  uint32_t dims[8];    /* {784,10}, {784,128,10}, {3072,256,128,10}; model 2:
+                          {side, c_in, c1, c2, f1, f2, classes} = {28,1,6,16,120,84,10};
+                          rows of a data set are then side*side*c_in values, plane by
+                          plane, and parameters run W1[c1][c_in][5][5], b1,
+                          W2[c2][c1][5][5], b2, then the dense layers as below      */
   uint32_t precision;  /* 0 = fp32; 1 = bf16 operands, fp32 accumulate and master */
   uint32_t batch;      /* samples per SGD iteration; must divide every s_i        */
   uint32_t sched_a, sched_b; /* s_i = a*i + b (Section 5; Table 2)                */

@@ -95,7 +95,10 @@ struct aet_handle {
   uint32_t P = 0;
   size_t stride = 0;
   bool lr_fast = false;  // 784 -> 10, batch 1, fp32: the specialised kernel
+  bool cnn = false;      // model 2: the small convolutional classifier
   MlpShape shape{};
+  CnnShape cshape{};
+  size_t act_floats() const { return cnn ? cnn_act_floats(cshape) : mlp_act_floats(shape); }
   std::string err;
 
   SchedState st;
@@ -219,6 +222,13 @@ aet_status launch_rounds(aet_handle* h, const RoundLaunch& r, cudaStream_t s) {
   cudaError_t e;
   if (h->lr_fast) {
     e = launch_lr_rounds(r, s);
+  } else if (h->cnn) {
+    CnnLaunch m;
+    m.r = r;
+    m.shape = h->cshape;
+    m.act = h->act.p;
+    m.act_stride = cnn_act_floats(h->cshape);
+    e = launch_cnn_rounds(m, s);
   } else {
     MlpLaunch m;
     m.r = r;
@@ -259,7 +269,7 @@ aet_status run_ring_rounds(aet_handle* h, uint32_t n_rounds, cudaStream_t s) {
   if (st_up != AET_OK) return st_up;
   bool ok = h->U.reserve(T * h->stride) && h->d_tasks.reserve(T) && h->d_trig.reserve(T) &&
             h->d_ring_applies.reserve(plan.applies.size() + 1) && h->d_ring_ops.reserve(plan.ops.size() + 1);
-  if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * mlp_act_floats(h->shape));
+  if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * h->act_floats());
   if (!ok) return fail(h, AET_ERR_NOMEM, "device allocation failed");
   if (!cp.uploaded) {
     AET_CUDA(h, cudaMemcpyAsync(h->d_tasks.p, plan.tasks.data(), T * sizeof(TaskDesc), cudaMemcpyHostToDevice, s));
@@ -322,7 +332,12 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   std::string err;
   if (cfg->struct_size != sizeof(aet_config)) return fail(nullptr, AET_ERR_ARG, "struct_size does not match sizeof(aet_config)");
   if (!validate_config(*cfg, err)) return fail(nullptr, AET_ERR_CONFIG, err);
-  const uint32_t P = count_params(*cfg);
+  CnnShape cshape{};
+  for (int i = 0; i < 8; ++i) cshape.dims[i] = cfg->dims[i];
+  cshape.batch = cfg->batch;
+  if (cfg->model == 2)
+    if (const char* why = cnn_check_shape(cshape)) return fail(nullptr, AET_ERR_CONFIG, why);
+  const uint32_t P = cfg->model == 2 ? cnn_n_params(cshape) : count_params(*cfg);
   if (!P) return fail(nullptr, AET_ERR_CONFIG, "model too large");
   if (cfg->dims[cfg->n_layers] > 32) return fail(nullptr, AET_ERR_CONFIG, "at most 32 classes are supported");
   if (cfg->flags & ~(uint32_t)(AET_FLAG_BORROW_DATA | AET_FLAG_DEBUG_CHECKS | AET_FLAG_KEEP_UPDATE_SUMS | AET_FLAG_STEPWISE_RECURRENCE))
@@ -345,14 +360,16 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
   h->shape.batch = cfg->batch;
   h->shape.precision = cfg->precision;
   h->shape.cluster = mlp_pick_cluster(h->shape, cfg->n_clients);
-  if (!h->lr_fast && !mlp_tc_eligible(h->shape)) {
+  h->cnn = cfg->model == 2;
+  h->cshape = cshape;
+  if (!h->lr_fast && !h->cnn && !mlp_tc_eligible(h->shape)) {
     if (const char* why = mlp_check_shape(h->shape)) { delete h; return fail(nullptr, AET_ERR_CONFIG, why); }
   }
   h->h_clients.assign(cfg->n_clients, ClientData{nullptr, nullptr, 0, 0});
   h->st.H.assign(cfg->n_clients, 0);
   bool ok = h->w_buf[0].reserve(h->stride) && h->w_buf[1].reserve(h->stride) && h->w0.reserve(h->stride) &&
             h->d_H.reserve(cfg->n_clients) && h->d_status.reserve(1) && h->totals.reserve(32 * h->stride);
-  if (ok && !h->lr_fast) ok = h->work.reserve((size_t)cfg->n_clients * h->stride);
+  if (ok && !h->lr_fast && !h->cnn) ok = h->work.reserve((size_t)cfg->n_clients * h->stride);
   if (ok && cfg->topology == 1) ok = h->node_w.reserve((size_t)cfg->n_clients * h->stride);
   if (!ok) { aet_destroy(h); return fail(nullptr, AET_ERR_NOMEM, "device allocation failed"); }
   if (cfg->topology == 1 && cudaMemset(h->node_w.p, 0, (size_t)cfg->n_clients * h->stride * sizeof(float)) != cudaSuccess) {
@@ -431,7 +448,8 @@ aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x, c
   if (client >= h->cfg.n_clients) return fail(h, AET_ERR_ARG, "client index out of range");
   if (n == 0 || n < h->cfg.batch) return fail(h, AET_ERR_ARG, "a client needs at least max(1, batch) samples");
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  const size_t D = h->cfg.dims[0];
+  // a row: the input layer's width, or side * side * c_in values for the convolutional classifier
+  const size_t D = h->cfg.model == 2 ? (size_t)h->cfg.dims[0] * h->cfg.dims[0] * h->cfg.dims[1] : h->cfg.dims[0];
   const size_t elems = (size_t)n * D;
   const bool bf16 = h->cfg.precision == 1;
   const bool debug = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) != 0;
@@ -523,7 +541,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   bool ok = h->snaps.reserve((size_t)plan.n_snap * h->stride) && h->U.reserve((size_t)plan.n_u_rows * h->stride) &&
             h->d_tasks.reserve(E) && h->d_inflight.reserve(plan.inflight.size() + 1) &&
             h->d_applies.reserve(E) && h->d_trig.reserve(E) && h->d_alog.reserve(E);
-  if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * mlp_act_floats(h->shape));
+  if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * h->act_floats());
   if (!ok) return fail(h, AET_ERR_NOMEM, "device allocation failed");
   if (!cp.uploaded) {
     AET_CUDA(h, cudaMemcpyAsync(h->d_tasks.p, plan.tasks.data(), E * sizeof(TaskDesc), cudaMemcpyHostToDevice, s));
@@ -689,7 +707,7 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   // private area: [snapshot | U | w_end | task | trigger record]
   const size_t fl = 3 * h->stride + 64;
   if (!h->dbg.reserve(fl)) return fail(h, AET_ERR_NOMEM, "device allocation failed");
-  if (!h->lr_fast && !h->act.reserve(mlp_act_floats(h->shape))) return fail(h, AET_ERR_NOMEM, "device allocation failed");
+  if (!h->lr_fast && !h->act.reserve(h->act_floats())) return fail(h, AET_ERR_NOMEM, "device allocation failed");
   float* snap = h->dbg.p;
   float* U = snap + h->stride;
   float* wend = U + h->stride;

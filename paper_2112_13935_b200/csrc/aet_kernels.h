@@ -77,6 +77,20 @@ cudaError_t launch_mlp_res_rounds(const MlpLaunch& p, cudaStream_t s);
 bool mlp_tc_eligible(const MlpShape& shape);
 cudaError_t launch_mlp_tc_rounds(const MlpLaunch& p, cudaStream_t s);
 
+// Small convolutional classifier (two 5x5 convolutions with average pooling, three dense layers):
+// dims = {side, c_in, c1, c2, f1, f2, classes}; the whole model stays in shared memory for the round.
+struct CnnShape { uint32_t dims[8], batch; };
+struct CnnLaunch {
+  RoundLaunch r;
+  CnnShape shape;
+  float* act;                    // per-task activation scratch
+  size_t act_stride;             // floats per task
+};
+uint32_t cnn_n_params(const CnnShape& s);
+size_t cnn_act_floats(const CnnShape& s);
+const char* cnn_check_shape(const CnnShape& s);   // null if the kernel can run it
+cudaError_t launch_cnn_rounds(const CnnLaunch& p, cudaStream_t s);
+
 // Ordered aggregation: for seq in [lo, hi): w -= eta_seq * U[seq]; keep a copy
 // where a later round starts from it; bump H and log the apply.
 struct ApplyLaunch {

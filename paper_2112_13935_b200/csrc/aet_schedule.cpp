@@ -82,7 +82,8 @@ bool validate_config(const aet_config& c, std::string& err) {
   if (c.n_layers < 1 || c.n_layers > AET_MAX_LAYERS) { err = "n_layers out of range"; return false; }
   for (uint32_t l = 0; l <= c.n_layers; ++l)
     if (c.dims[l] == 0) { err = "a layer dimension is zero"; return false; }
-  if (c.model > 1 || (c.model == 0 && c.n_layers != 1)) { err = "model 0 has exactly one weight layer"; return false; }
+  if (c.model > 2 || (c.model == 0 && c.n_layers != 1)) { err = "model 0 has exactly one weight layer"; return false; }
+  if (c.model == 2 && (c.n_layers != 6 || c.precision != 0)) { err = "model 2 takes dims {side, c_in, c1, c2, f1, f2, classes} and precision 0"; return false; }
   if (c.precision > 1) { err = "precision must be 0 or 1"; return false; }
   if (c.batch == 0) { err = "batch must be at least 1"; return false; }
   if (c.delay_dist > 1) { err = "delay_dist must be 0 or 1"; return false; }

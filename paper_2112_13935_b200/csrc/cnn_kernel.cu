@@ -1,0 +1,387 @@
+// Local-SGD round of one client for a small convolutional classifier (the LeNet shape the paper
+// trains on its 28x28 sets; Appendix, "Objective function"):
+//   conv 5x5 valid (c_in -> c1) + bias, ReLU, 2x2 average pooling,
+//   conv 5x5 valid (c1 -> c2) + bias, ReLU, 2x2 average pooling, flatten [c2][y][x],
+//   dense f1, ReLU, dense f2, ReLU, dense classes, softmax cross-entropy.
+// Algorithm 3, MainComputeNode, inner loop with xi a minibatch: g = mean gradient (+ lambda W on
+// weight tensors), w_c -= eta_i g, U_i += g, repeated s_{i,c} / B times; then (c, U_i, i) is sent.
+//
+// One CTA of 512 threads per round-task.  The client's whole model (44,426 parameters for the
+// 28x28 shape, 174 KB) stays in shared memory from the start of the round to its trigger; only the
+// minibatch rows, the activations of the minibatch (global scratch, L2-resident) and the running
+// update sum (one read-modify-write per parameter and iteration) move.  A parameter's gradient is
+// summed over the minibatch by the thread that owns the parameter and applied on the spot, so no
+// gradient buffer exists and nothing needs an atomic.  Weight updates of layer l share a phase
+// with the input-gradient product of layer l - 1 (which reads other weights), so the backward pass
+// costs one block barrier per layer.
+#include <cuda_runtime.h>
+
+#include "aet_kernels.h"
+#include "aet_rng.h"
+
+namespace aet {
+namespace {
+
+constexpr int kCnnThreads = 512;
+constexpr int kK = 5;   // kernel side of both convolutions
+
+struct CnnDims {
+  int side, cin, c1, c2, f1, f2, ncls, s1, p1, s2, p2, flat;
+  int oW1, ob1, oW2, ob2, oF1, obF1, oF2, obF2, oF3, obF3, P;
+  // per-minibatch activation scratch (floats), offsets for batch size B
+  int a1, q1, a2, q2, h1, h2, z3, dz3, dh2, dh1, dq2, dq1, total;
+};
+
+__host__ __device__ inline CnnDims make_cnn_dims(const CnnShape& s) {
+  CnnDims d{};
+  d.side = (int)s.dims[0]; d.cin = (int)s.dims[1]; d.c1 = (int)s.dims[2]; d.c2 = (int)s.dims[3];
+  d.f1 = (int)s.dims[4]; d.f2 = (int)s.dims[5]; d.ncls = (int)s.dims[6];
+  d.s1 = d.side - kK + 1; d.p1 = d.s1 / 2; d.s2 = d.p1 - kK + 1; d.p2 = d.s2 / 2;
+  d.flat = d.c2 * d.p2 * d.p2;
+  int o = 0;
+  d.oW1 = o; o += d.c1 * d.cin * kK * kK; d.ob1 = o; o += d.c1;
+  d.oW2 = o; o += d.c2 * d.c1 * kK * kK; d.ob2 = o; o += d.c2;
+  d.oF1 = o; o += d.flat * d.f1; d.obF1 = o; o += d.f1;
+  d.oF2 = o; o += d.f1 * d.f2; d.obF2 = o; o += d.f2;
+  d.oF3 = o; o += d.f2 * d.ncls; d.obF3 = o; o += d.ncls;
+  d.P = o;
+  const int B = (int)s.batch;
+  int a = 0;
+  d.a1 = a; a += B * d.c1 * d.s1 * d.s1;
+  d.q1 = a; a += B * d.c1 * d.p1 * d.p1;
+  d.a2 = a; a += B * d.c2 * d.s2 * d.s2;
+  d.q2 = a; a += B * d.flat;
+  d.h1 = a; a += B * d.f1;
+  d.h2 = a; a += B * d.f2;
+  d.z3 = a; a += B * d.ncls;
+  d.dz3 = a; a += B * d.ncls;
+  d.dh2 = a; a += B * d.f2;
+  d.dh1 = a; a += B * d.f1;
+  d.dq2 = a; a += B * d.flat;
+  d.dq1 = a; a += B * d.c1 * d.p1 * d.p1;
+  d.total = (a + 31) & ~31;
+  return d;
+}
+
+// Valid 5x5 correlation + bias + ReLU + 2x2 average pooling of one stage, for the whole minibatch.
+// One work item = one pooled output: its four pre-pooling outputs share a 6x6 input patch per plane.
+template <class InAt>
+__device__ __forceinline__ void conv_stage(int B, int cin, int cout, int sin, int sout, const float* W, const float* bias,
+                                           InAt in_at, float* a_out, float* q_out, int tid) {
+  const int pout = sout / 2;
+  const int items = B * cout * pout * pout;
+  for (int e = tid; e < items; e += kCnnThreads) {
+    const int px = e % pout, py = (e / pout) % pout, c = (e / (pout * pout)) % cout, b = e / (pout * pout * cout);
+    float z00 = bias[c], z01 = z00, z10 = z00, z11 = z00;
+    for (int ci = 0; ci < cin; ++ci) {
+      float patch[6][6];
+#pragma unroll
+      for (int r = 0; r < 6; ++r)
+#pragma unroll
+        for (int q = 0; q < 6; ++q) patch[r][q] = in_at(b, ci, 2 * py + r, 2 * px + q);
+      const float* wk = W + (c * cin + ci) * (kK * kK);
+#pragma unroll
+      for (int dy = 0; dy < kK; ++dy)
+#pragma unroll
+        for (int dx = 0; dx < kK; ++dx) {
+          const float wv = wk[dy * kK + dx];
+          z00 = fmaf(wv, patch[dy][dx], z00);
+          z01 = fmaf(wv, patch[dy][dx + 1], z01);
+          z10 = fmaf(wv, patch[dy + 1][dx], z10);
+          z11 = fmaf(wv, patch[dy + 1][dx + 1], z11);
+        }
+    }
+    z00 = fmaxf(z00, 0.f); z01 = fmaxf(z01, 0.f); z10 = fmaxf(z10, 0.f); z11 = fmaxf(z11, 0.f);
+    float* ao = a_out + ((size_t)(b * cout + c) * sout + 2 * py) * sout + 2 * px;
+    ao[0] = z00; ao[1] = z01; ao[sout] = z10; ao[sout + 1] = z11;
+    q_out[((size_t)(b * cout + c) * pout + py) * pout + px] = 0.25f * ((z00 + z01) + (z10 + z11));
+  }
+}
+
+__global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) {
+  extern __shared__ __align__(16) float smem[];
+  const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x];
+  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  const CnnDims D = make_cnn_dims(p.shape);
+  const int B = (int)p.shape.batch;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  float* w = smem;                                     // the client's model, whole round
+  int* idx = reinterpret_cast<int*>(smem + ((D.P + 3) & ~3));
+  int* ylab = idx + B;
+
+  const ClientData cd = p.r.clients[t.client];
+  const float* xrows = reinterpret_cast<const float*>(cd.x);
+  const uint64_t key = p.r.sample_keys[t.client];
+  const float eta = t.eta, lambda = p.r.l2, invB = 1.f / (float)B;
+  const int rowlen = D.cin * D.side * D.side;
+  float* act = p.act + (size_t)blockIdx.x * p.act_stride;
+  float* Urow = p.r.U + (size_t)t.u_row * p.r.stride;
+
+  // ---- start model: snapshot minus own update sums still in flight; U_i = 0 ----
+  {
+    const float* snap = p.r.snaps + (size_t)t.snap_slot * p.r.stride;
+    for (int k = tid; k < D.P; k += kCnnThreads) {
+      float v = snap[k];
+      for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+        const InflightRef ref = p.r.inflight[t.inflight_off + f];
+        v = fmaf(-ref.eta, p.r.U[(size_t)ref.row * p.r.stride + k], v);
+      }
+      w[k] = v;
+      Urow[k] = 0.f;
+    }
+  }
+  __syncthreads();
+
+  // w -= eta (g + lambda w), U += g + lambda w for one parameter; biases take no l2 term
+  auto apply = [&](int k, float g, bool decay) {
+    const float wk = w[k];
+    const float gt = decay ? fmaf(lambda, wk, g) : g;
+    w[k] = fmaf(-eta, gt, wk);
+    Urow[k] += gt;
+  };
+
+  for (uint32_t it = 0; it < t.steps; ++it) {
+    if (tid < B) {
+      const int id = (int)sample_index(draw(key, t.sample_ctr0 + (uint64_t)it * B + tid), cd.n);
+      idx[tid] = id;
+      ylab[tid] = __ldg(cd.y + id);
+    }
+    __syncthreads();
+
+    // ================= forward =================
+    conv_stage(B, D.cin, D.c1, D.side, D.s1, w + D.oW1, w + D.ob1,
+               [&](int b, int ci, int y, int x) { return __ldg(xrows + (size_t)idx[b] * rowlen + (ci * D.side + y) * D.side + x); },
+               act + D.a1, act + D.q1, tid);
+    __syncthreads();
+    {
+      const float* q1 = act + D.q1;
+      conv_stage(B, D.c1, D.c2, D.p1, D.s2, w + D.oW2, w + D.ob2,
+                 [&](int b, int ci, int y, int x) { return q1[((size_t)(b * D.c1 + ci) * D.p1 + y) * D.p1 + x]; },
+                 act + D.a2, act + D.q2, tid);
+    }
+    __syncthreads();
+    auto dense_fwd = [&](const float* in, int K, int N, const float* Wl, const float* bl, float* out, bool relu) {
+      for (int e = tid; e < B * N; e += kCnnThreads) {
+        const int j = e % N, b = e / N;
+        float z = bl[j];
+        const float* a = in + (size_t)b * K;
+        for (int k = 0; k < K; ++k) z = fmaf(a[k], Wl[k * N + j], z);
+        out[e] = relu ? fmaxf(z, 0.f) : z;
+      }
+    };
+    dense_fwd(act + D.q2, D.flat, D.f1, w + D.oF1, w + D.obF1, act + D.h1, true);
+    __syncthreads();
+    dense_fwd(act + D.h1, D.f1, D.f2, w + D.oF2, w + D.obF2, act + D.h2, true);
+    __syncthreads();
+    dense_fwd(act + D.h2, D.f2, D.ncls, w + D.oF3, w + D.obF3, act + D.z3, false);
+    __syncthreads();
+    if (tid < B) {   // softmax cross-entropy: dZ = (p - onehot) / B
+      const float* z = act + D.z3 + tid * D.ncls;
+      float m = -INFINITY;
+      for (int j = 0; j < D.ncls; ++j) m = fmaxf(m, z[j]);
+      float sum = 0.f;
+      for (int j = 0; j < D.ncls; ++j) sum += __expf(z[j] - m);
+      const float inv = 1.f / sum;
+      const int y = ylab[tid];
+      for (int j = 0; j < D.ncls; ++j)
+        act[D.dz3 + tid * D.ncls + j] = (__expf(z[j] - m) * inv - (j == y ? 1.f : 0.f)) * invB;
+    }
+    __syncthreads();
+
+    // ================= backward =================
+    // input gradient of a dense layer, gated by the ReLU of the layer below: dIn[b, i] = [in > 0] sum_j dOut[b, j] W[i, j]
+    auto dense_din = [&](int e, const float* dout, int K, int N, const float* Wl, const float* in, float* din, bool gate) {
+      const int i = e % K, b = e / K;
+      float s = 0.f;
+      const float* dz = dout + (size_t)b * N;
+      const float* wr = Wl + (size_t)i * N;
+      for (int j = 0; j < N; ++j) s = fmaf(dz[j], wr[j], s);
+      din[e] = (!gate || in[e] > 0.f) ? s : 0.f;
+    };
+    // gradient and update of one dense parameter: item < K * N a weight, else a bias
+    auto dense_upd = [&](int e, const float* in, const float* dout, int K, int N, int oW, int ob) {
+      if (e < K * N) {
+        const int j = e % N, i = e / N;
+        float g = 0.f;
+        for (int b = 0; b < B; ++b) g = fmaf(in[(size_t)b * K + i], dout[(size_t)b * N + j], g);
+        apply(oW + e, g, true);
+      } else {
+        const int j = e - K * N;
+        float g = 0.f;
+        for (int b = 0; b < B; ++b) g += dout[(size_t)b * N + j];
+        apply(ob + j, g, false);
+      }
+    };
+    // dh2 from the class layer (its weights are still the old ones)
+    for (int e = tid; e < B * D.f2; e += kCnnThreads)
+      dense_din(e, act + D.dz3, D.f2, D.ncls, w + D.oF3, act + D.h2, act + D.dh2, true);
+    __syncthreads();
+    // class layer update | dh1 through dense layer 2
+    {
+      const int nu = D.f2 * D.ncls + D.ncls, nd = B * D.f1;
+      for (int e = tid; e < nu + nd; e += kCnnThreads) {
+        if (e < nu) dense_upd(e, act + D.h2, act + D.dz3, D.f2, D.ncls, D.oF3, D.obF3);
+        else dense_din(e - nu, act + D.dh2, D.f1, D.f2, w + D.oF2, act + D.h1, act + D.dh1, true);
+      }
+    }
+    __syncthreads();
+    // dense layer 2 update | dq2 through dense layer 1 (the pooled maps carry no ReLU of their own)
+    {
+      const int nu = D.f1 * D.f2 + D.f2, nd = B * D.flat;
+      for (int e = tid; e < nu + nd; e += kCnnThreads) {
+        if (e < nu) dense_upd(e, act + D.h1, act + D.dh2, D.f1, D.f2, D.oF2, D.obF2);
+        else dense_din(e - nu, act + D.dh1, D.flat, D.f1, w + D.oF1, act + D.q2, act + D.dq2, false);
+      }
+    }
+    __syncthreads();
+    // dense layer 1 update | dz2 = [a2 > 0] * dq2 / 4, in place over a2
+    {
+      const int nu = D.flat * D.f1 + D.f1, nd = B * D.c2 * D.s2 * D.s2;
+      for (int e = tid; e < nu + nd; e += kCnnThreads) {
+        if (e < nu) {
+          dense_upd(e, act + D.q2, act + D.dh1, D.flat, D.f1, D.oF1, D.obF1);
+        } else {
+          const int k = e - nu;
+          const int x = k % D.s2, y = (k / D.s2) % D.s2, bc = k / (D.s2 * D.s2);
+          const float g = act[D.dq2 + ((size_t)bc * D.p2 + (y >> 1)) * D.p2 + (x >> 1)];
+          act[D.a2 + k] = act[D.a2 + k] > 0.f ? 0.25f * g : 0.f;
+        }
+      }
+    }
+    __syncthreads();
+    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx] (second convolution's old weights)
+    {
+      const float* dz2 = act + D.a2;
+      const float* W2 = w + D.oW2;
+      for (int e = tid; e < B * D.c1 * D.p1 * D.p1; e += kCnnThreads) {
+        const int x = e % D.p1, y = (e / D.p1) % D.p1, c = (e / (D.p1 * D.p1)) % D.c1, b = e / (D.p1 * D.p1 * D.c1);
+        float s = 0.f;
+        for (int c2 = 0; c2 < D.c2; ++c2) {
+          const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
+          const float* wk = W2 + (c2 * D.c1 + c) * (kK * kK);
+#pragma unroll
+          for (int dy = 0; dy < kK; ++dy) {
+            const int yy = y - dy;
+            if (yy < 0 || yy >= D.s2) continue;
+#pragma unroll
+            for (int dx = 0; dx < kK; ++dx) {
+              const int xx = x - dx;
+              if (xx >= 0 && xx < D.s2) s = fmaf(dzp[yy * D.s2 + xx], wk[dy * kK + dx], s);
+            }
+          }
+        }
+        act[D.dq1 + e] = s;
+      }
+    }
+    __syncthreads();
+    // second convolution's update | dz1 = [a1 > 0] * dq1 / 4, in place over a1
+    {
+      const int nw = D.c2 * D.c1 * kK * kK, nu = nw + D.c2, nd = B * D.c1 * D.s1 * D.s1;
+      const float* dz2 = act + D.a2;
+      const float* q1 = act + D.q1;
+      for (int e = tid; e < nu + nd; e += kCnnThreads) {
+        if (e < nw) {
+          const int dx = e % kK, dy = (e / kK) % kK, c = (e / (kK * kK)) % D.c1, c2 = e / (kK * kK * D.c1);
+          float g = 0.f;
+          for (int b = 0; b < B; ++b) {
+            const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
+            const float* qp = q1 + ((size_t)(b * D.c1 + c) * D.p1 + dy) * D.p1 + dx;
+            for (int y = 0; y < D.s2; ++y)
+              for (int x = 0; x < D.s2; ++x) g = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g);
+          }
+          apply(D.oW2 + e, g, true);
+        } else if (e < nu) {
+          const int c2 = e - nw;
+          float g = 0.f;
+          for (int b = 0; b < B; ++b) {
+            const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
+            for (int k = 0; k < D.s2 * D.s2; ++k) g += dzp[k];
+          }
+          apply(D.ob2 + c2, g, false);
+        } else {
+          const int k = e - nu;
+          const int x = k % D.s1, y = (k / D.s1) % D.s1, bc = k / (D.s1 * D.s1);
+          const float g = act[D.dq1 + ((size_t)bc * D.p1 + (y >> 1)) * D.p1 + (x >> 1)];
+          act[D.a1 + k] = act[D.a1 + k] > 0.f ? 0.25f * g : 0.f;
+        }
+      }
+    }
+    __syncthreads();
+    // first convolution's update: few parameters, long sums (B * s1 * s1 terms each): a warp per parameter,
+    // lanes take the terms in turn, shuffle tree at the end
+    {
+      const int nw = D.c1 * D.cin * kK * kK, nu = nw + D.c1;
+      const float* dz1 = act + D.a1;
+      const int terms = B * D.s1 * D.s1;
+      for (int e = warp; e < nu; e += kCnnThreads / 32) {
+        float g = 0.f;
+        if (e < nw) {
+          const int dx = e % kK, dy = (e / kK) % kK, ci = (e / (kK * kK)) % D.cin, c = e / (kK * kK * D.cin);
+          for (int k = lane; k < terms; k += 32) {
+            const int x = k % D.s1, y = (k / D.s1) % D.s1, b = k / (D.s1 * D.s1);
+            const float xv = __ldg(xrows + (size_t)idx[b] * rowlen + (ci * D.side + y + dy) * D.side + x + dx);
+            g = fmaf(dz1[((size_t)(b * D.c1 + c) * D.s1 + y) * D.s1 + x], xv, g);
+          }
+        } else {
+          const int c = e - nw;
+          for (int k = lane; k < terms; k += 32) {
+            const int r = k % (D.s1 * D.s1), b = k / (D.s1 * D.s1);
+            g += dz1[(size_t)(b * D.c1 + c) * D.s1 * D.s1 + r];
+          }
+        }
+#pragma unroll
+        for (int m = 16; m; m >>= 1) g += __shfl_xor_sync(0xffffffffu, g, m);
+        if (lane == 0) {
+          if (e < nw) apply(D.oW1 + e, g, true);
+          else apply(D.ob1 + (e - nw), g, false);
+        }
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- event trigger: h reached s_{i,c}; U_i is complete in its row; the end model on request ----
+  if (p.r.w_end) {
+    float* dst = p.r.w_end + (size_t)t.u_row * p.r.stride;
+    for (int k = tid; k < D.P; k += kCnnThreads) dst[k] = w[k];
+  }
+  if (tid == 0) {
+    TriggerRec rec;
+    rec.client = t.client; rec.round = t.round; rec.samples_done = t.steps * (uint32_t)B; rec.flags = 1;
+    p.r.trig[t.seq] = rec;
+  }
+}
+
+size_t cnn_smem_bytes(const CnnShape& s) {
+  const CnnDims d = make_cnn_dims(s);
+  return ((size_t)((d.P + 3) & ~3) + 2 * s.batch) * sizeof(float);
+}
+
+}  // namespace
+
+uint32_t cnn_n_params(const CnnShape& s) { return (uint32_t)make_cnn_dims(s).P; }
+size_t cnn_act_floats(const CnnShape& s) { return (size_t)make_cnn_dims(s).total; }
+
+const char* cnn_check_shape(const CnnShape& s) {
+  const int side = (int)s.dims[0];
+  const int s1 = side - kK + 1;
+  if (side < 2 * kK || s1 <= 0 || (s1 & 1)) return "convolutional model: (side - 4) must be even and positive";
+  const int s2 = s1 / 2 - kK + 1;
+  if (s2 <= 0 || (s2 & 1)) return "convolutional model: ((side - 4) / 2 - 4) must be even and positive";
+  for (int i = 1; i < 7; ++i) if (s.dims[i] == 0) return "convolutional model: a width is zero";
+  if (s.dims[6] > 32) return "at most 32 classes are supported";
+  if (s.batch == 0 || s.batch > 64) return "convolutional model: batch must be 1 .. 64";
+  if (cnn_smem_bytes(s) > 220 * 1024) return "convolutional model: the parameters do not fit in shared memory (about 55,000)";
+  return nullptr;
+}
+
+cudaError_t launch_cnn_rounds(const CnnLaunch& p, cudaStream_t s) {
+  if (p.r.n_tasks == 0) return cudaSuccess;
+  const size_t smem = cnn_smem_bytes(p.shape);
+  cudaError_t e = cudaFuncSetAttribute(cnn_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cnn_round_kernel<<<p.r.n_tasks, kCnnThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace aet

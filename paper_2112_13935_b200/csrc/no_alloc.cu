@@ -93,6 +93,7 @@ extern "C" aet_status aet_round_no_alloc(const aet_config* cfg, uint32_t client,
   std::string err;
   if (!validate_config(*cfg, err)) return fail(AET_ERR_CONFIG, err);
   if (cfg->precision != 0) return fail(AET_ERR_CONFIG, "aet_round_no_alloc runs fp32 models only");
+  if (cfg->model > 1) return fail(AET_ERR_CONFIG, "aet_round_no_alloc runs softmax regression and ReLU MLPs only");
   if (cfg->split_mode != 0) return fail(AET_ERR_CONFIG, "aet_round_no_alloc runs a node's own sequence s_i = a*i + b only (split_mode 0)");
   if (client >= cfg->n_clients) return fail(AET_ERR_ARG, "client index out of range");
   if (round < cfg->round_base) return fail(AET_ERR_ARG, "round is before round_base");
