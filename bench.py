@@ -46,6 +46,8 @@ DESCRIBE = {
     "cfg6": "cfg6 (the paper's own setting, Appendix Table 2): 5 nodes, softmax regression 784->10 fp32, "
             "s_i=10i from round 1, 110 rounds, eta_0=0.01 beta=0.01, d=1, uniform delays",
 }
+DESCRIBE["cfg7"] = ("cfg7: 16 clients, convolutional classifier of the LeNet shape (28x28x1 -> conv 6 -> conv 16 -> "
+                    "120 -> 84 -> 10) fp32, batch 16, s_i=32i+32, 12 rounds")
 DEFAULT_WORKLOAD = "cfg5"   # the configuration the HBM-roofline target of the regression kernel is quoted on
 MIN_TIMED_S = 2.0           # short passes are repeated inside a step until the timed region is this long
 
@@ -68,24 +70,39 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
-def algorithmic_bytes(cfg, events):
+def row_values(cfg):
+    return cfg["dims"][0] * cfg["dims"][0] * cfg["dims"][1] if cfg["model"] == 2 else cfg["dims"][0]
+
+
+def algorithmic_bytes(cfg, samples, n_tasks):
     """Bytes the local-SGD kernel must move: per sample one row and its label,
     per round-task the start model in and the update sum out."""
     from paper_2112_13935_b200 import workloads
-    P = workloads.n_params(cfg["dims"])
+    P = workloads.model_n_params(cfg)
     elem = 2 if cfg["precision"] == 1 else 4
-    per_sample = elem * cfg["dims"][0] + 4
-    samples = sum(e["samples"] for e in events)
-    return samples * per_sample + len(events) * 8 * P
+    per_sample = elem * row_values(cfg) + 4
+    return samples * per_sample + n_tasks * 8 * P
 
 
-def algorithmic_flops(cfg, events):
-    """Dense-contraction flops of the MLP path: forward and weight-gradient
-    products of every layer, input-gradient products of all but the first."""
+def algorithmic_flops(cfg, samples):
+    """Contraction flops per sample: forward and weight-gradient products of every layer, input-gradient
+    products of all but the first (dense layers: 2 flops per weight each; convolutions: per weight and
+    output position)."""
     d = cfg["dims"]
+    if cfg["model"] == 2:
+        side, c_in, c1, c2, f1, f2, ncls = d
+        s1 = side - 4
+        p1 = s1 // 2
+        s2 = p1 - 4
+        flat = c2 * (s2 // 2) ** 2
+        conv1 = c1 * c_in * 25 * s1 * s1
+        conv2 = c2 * c1 * 25 * s2 * s2
+        dense = [flat * f1, f1 * f2, f2 * ncls]
+        macs = 2 * conv1 + 3 * conv2 + 3 * sum(dense)          # no input gradient for the first convolution
+        return 2 * macs * samples
     per_sample = sum(4 * d[l] * d[l + 1] for l in range(len(d) - 1)) + \
         sum(2 * d[l] * d[l + 1] for l in range(1, len(d) - 1))
-    return per_sample * sum(e["samples"] for e in events)
+    return per_sample * samples
 
 
 def fp32_fma_peak_tflops():
@@ -101,13 +118,13 @@ def fp32_fma_peak_tflops():
     return 148 * 128 * 2 * mhz * 1e6 / 1e12, f"derived: 148 SMs x 128 fp32 lanes x 2 x {mhz:.0f} MHz"
 
 
-def regression_flops(cfg, events):
+def regression_flops(cfg, samples):
     """Softmax regression, batch 1: logits, model update and update sum are one FMA per
     parameter and sample each (the l2 term adds two more per weight)."""
     from paper_2112_13935_b200 import workloads
     P = workloads.n_params(cfg["dims"])
     per_sample = 2 * (3 + (2 if cfg["l2"] else 0)) * P
-    return per_sample * sum(e["samples"] for e in events)
+    return per_sample * samples
 
 
 def measured_peak_tflops():
@@ -171,7 +188,10 @@ def oracle_bounded(cfg, data, w0, limit_s):
     schedule, then round-tasks in start order until the time limit is reached."""
     from oracle import schedule, sim
     t0 = time.perf_counter()
-    events, _, _ = schedule.simulate(cfg, cfg["n_rounds"])
+    if cfg.get("topology"):
+        events = schedule.simulate_ring(cfg, cfg["n_rounds"])[0]
+    else:
+        events, _, _ = schedule.simulate(cfg, cfg["n_rounds"])
     order = sorted(events, key=lambda e: (e["t_start"], e["client"]))
     w = np.asarray(w0, dtype=np.float64)
     done_samples, done_tasks = 0, 0
@@ -192,7 +212,8 @@ def blas_threads(cfg):
 
 def config_block(cfg, samples, n_events):
     """The `config` object of the JSON line: names the workload, identical for both arms."""
-    return {"workload": DESCRIBE[cfg["name"]], "n_clients": cfg["n_clients"], "rounds": cfg["n_rounds"],
+    return {"workload": DESCRIBE[cfg["name"]] + (" [peer-to-peer ring]" if cfg.get("topology") else ""),
+            "n_clients": cfg["n_clients"], "rounds": cfg["n_rounds"],
             "network_delay_mean": cfg["network_delay_mean"],
             "max_lag_d": "never wait" if cfg["max_lag_d"] == 0xFFFFFFFF else cfg["max_lag_d"],
             "samples_per_pass": samples, "events_per_pass": n_events}
@@ -210,7 +231,10 @@ def run_reference(args, cfg):
     cores = blas_threads(cfg)
     rates, sample = [], ""
     from oracle import schedule as _sched
-    _ev, _sum, _ = _sched.simulate(cfg, cfg["n_rounds"])
+    if cfg.get("topology"):
+        _ev, _, _sum, _ = _sched.simulate_ring(cfg, cfg["n_rounds"])
+    else:
+        _ev, _sum, _ = _sched.simulate(cfg, cfg["n_rounds"])
     ref_samples, ref_events = _sum["samples_total"], len(_ev)
     with threadpool_limits(limits=cores):
         for step in range(args.warmup + args.steps):
@@ -304,7 +328,8 @@ def measure_device(cfg, steps, warmup, passes_per_step=None, clock_index=None):
     del dev, flush
 
     n_sgd_launches = stats["launches"][0]
-    alg_bytes = algorithmic_bytes(cfg, events)
+    n_tasks = cfg["n_clients"] * R
+    alg_bytes = algorithmic_bytes(cfg, samples, n_tasks)
     sgd_ms = k_ms[0] / k_pass
     achieved = alg_bytes / (sgd_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak_gbs()
@@ -314,28 +339,28 @@ def measure_device(cfg, steps, warmup, passes_per_step=None, clock_index=None):
             "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
             "traffic_source": ratio[1] if traffic else None, "peak_kind": peak_kind,
             "algorithmic_bytes_per_launch": alg_bytes / n_sgd_launches}
-    if cfg["model"] == 1:
-        tf = algorithmic_flops(cfg, events) / (sgd_ms * 1e-3) / 1e12
+    if cfg["model"] >= 1:
+        tf = algorithmic_flops(cfg, samples) / (sgd_ms * 1e-3) / 1e12
         if cfg["precision"] == 1:     # bf16 operands: the dense contraction runs on the tensor cores
             tpeak, tkind = measured_peak_tflops()
             bound = "tensor"
         else:                         # fp32 model: plain FMAs
             tpeak, tkind = fp32_fma_peak_tflops()
             bound = "alu"
-        roof = {"bound": bound, "kernel": "local-SGD rounds (MLP)", "achieved": tf, "peak": tpeak,
+        roof = {"bound": bound, "kernel": "local-SGD rounds (MLP)" if cfg["model"] == 1 else "local-SGD rounds (conv)", "achieved": tf, "peak": tpeak,
                 "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "peak_kind": tkind,
                 "hbm_gbs_algorithmic": achieved}
     else:
         # the batch-1 regression kernel sits on the FMA / HBM ridge: its fp32 FMA rate beside the HBM figure
         apeak, akind = fp32_fma_peak_tflops()
-        atf = regression_flops(cfg, events) / (sgd_ms * 1e-3) / 1e12
+        atf = regression_flops(cfg, samples) / (sgd_ms * 1e-3) / 1e12
         roof.update(alu_tflops=atf, alu_peak=apeak, alu_frac=atf / apeak, alu_peak_kind=akind)
     roof.update(launches_per_step=n_sgd_launches, kernel_ms_per_step=sgd_ms,
                 kernel_ms_mode="separate passes with events around every launch: no overlap between a kernel "
                                "and its neighbours, so the sum can exceed the pass it belongs to",
                 aggregation_ms_per_step=k_ms[1] / k_pass, algorithmic_bytes_per_step=alg_bytes)
     return dict(samples=samples, seconds=seconds, n_pass=n_pass, passes_per_step=passes_per_step, roof=roof,
-                launches_per_pass=launches_per_pass, events=len(events), waves=stats["waves"], plan_ms=plan_ms,
+                launches_per_pass=launches_per_pass, events=n_tasks, waves=stats["waves"], plan_ms=plan_ms,
                 clocks=sampler.summary() if sampler else None, data=data, w0=w0)
 
 
@@ -350,6 +375,7 @@ def main():
     ap.add_argument("--rounds", type=int, default=0, help="override the number of rounds (profiling on a smaller case)")
     ap.add_argument("--net-delay", type=float, default=None, help="override the mean network delay (time units)")
     ap.add_argument("--max-lag", type=int, default=None, help="override the checkpoint threshold d (-1 = never wait)")
+    ap.add_argument("--topology", default=None, choices=["server", "ring"], help="override the topology of the workload")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--passes-per-step", type=int, default=0, help="0 = enough for a 2 s timed region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -366,6 +392,8 @@ def main():
         over["network_delay_mean"] = args.net_delay
     if args.max_lag is not None:
         over["max_lag_d"] = workloads.NEVER_WAIT if args.max_lag < 0 else args.max_lag
+    if args.topology:
+        over["topology"] = 1 if args.topology == "ring" else 0
     cfg = workloads.get_config(args.workload, seed=rank, **over)
     if args.rounds:
         cfg["_cut"] = True
@@ -422,12 +450,13 @@ def main():
     # ---- the other configurations, device-timed for a few passes each (no e2e, no CPU leg) ----
     per_config = []
     if rank == 0 and world == 1 and not args.no_per_config and not args.rounds and not args.clients:
-        for name, steps in (("cfg2", 10), ("cfg3", 5), ("cfg4", 3), ("cfg6", 5)):
-            if name == args.workload:
+        for name, steps, extra in (("cfg2", 10, {}), ("cfg3", 5, {}), ("cfg4", 3, {}), ("cfg6", 5, {}),
+                                   ("cfg6", 5, dict(topology=1)), ("cfg7", 5, {})):
+            if name == args.workload and not extra:
                 continue
-            c2 = workloads.get_config(name, seed=rank)
+            c2 = workloads.get_config(name, seed=rank, **extra)
             r = measure_device(c2, steps, 3, passes_per_step=1)
-            per_config.append({"workload": DESCRIBE[name], "value": r["samples"] * r["n_pass"] / r["seconds"],
+            per_config.append({"workload": DESCRIBE[name] + (" [peer-to-peer ring]" if extra.get("topology") else ""), "value": r["samples"] * r["n_pass"] / r["seconds"],
                                "unit": UNIT, "ms_per_step": 1e3 * r["seconds"] / r["n_pass"], "steps": r["n_pass"],
                                "dtype": "bf16" if c2["precision"] == 1 else "f32",
                                "roofline": {k: r["roof"][k] for k in ("bound", "achieved", "peak", "unit", "frac",
