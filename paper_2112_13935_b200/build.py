@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaet_b200.so")
-SOURCES = ["aet_api.cu", "aet_schedule.cpp", "lr_kernel.cu", "lr_tc_kernel.cu", "mlp_kernel.cu", "mlp_tc_kernel.cu", "mlp_res_kernel.cu", "cnn_kernel.cu", "agg_kernel.cu", "no_alloc.cu"]
+SOURCES = ["aet_api.cu", "aet_schedule.cpp", "lr_kernel.cu", "lr_tc_kernel.cu", "mlp_kernel.cu", "mlp_tc_kernel.cu", "mlp_stream_kernel.cu", "mlp_res_kernel.cu", "cnn_kernel.cu", "agg_kernel.cu", "no_alloc.cu"]
 
 
 def _newest(paths):

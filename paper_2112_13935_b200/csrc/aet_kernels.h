@@ -73,6 +73,10 @@ const char* mlp_check_shape(const MlpShape& shape);  // null if the kernel can r
 // fp32 784-128-C models, batch 32: the model stays on-chip for the whole round (4-CTA cluster)
 bool mlp_res_eligible(const MlpLaunch& p);
 cudaError_t launch_mlp_res_rounds(const MlpLaunch& p, cudaStream_t s);
+// bf16 D0-256-128-C models, batch 64: one CTA per round-task streams the first layer through a
+// warp-specialised tcgen05 pipeline (see mlp_stream_kernel.cu)
+bool mlp_stream_eligible(const MlpShape& shape);
+cudaError_t launch_mlp_stream_rounds(const MlpLaunch& p, cudaStream_t s);
 // bf16 models whose first layer fits the tensor-core kernel (tcgen05 + TMEM)
 bool mlp_tc_eligible(const MlpShape& shape);
 cudaError_t launch_mlp_tc_rounds(const MlpLaunch& p, cudaStream_t s);

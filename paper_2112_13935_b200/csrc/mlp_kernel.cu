@@ -411,6 +411,7 @@ uint32_t mlp_pick_cluster(const MlpShape& shape, uint32_t n_clients) {
 
 cudaError_t launch_mlp_rounds(const MlpLaunch& p, cudaStream_t s) {
   if (p.r.n_tasks == 0) return cudaSuccess;
+  if (mlp_stream_eligible(p.shape)) return launch_mlp_stream_rounds(p, s);
   if (mlp_tc_eligible(p.shape)) return launch_mlp_tc_rounds(p, s);
   if (mlp_res_eligible(p)) return launch_mlp_res_rounds(p, s);
   const Smem m = make_smem(p.shape);
