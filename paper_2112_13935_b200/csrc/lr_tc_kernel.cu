@@ -49,6 +49,7 @@ using namespace lr;
 constexpr int kTcWarps = 8, kTcThreads = kTcWarps * 32;
 constexpr int kTiles = 7;          // 128-row tiles of the 785 inputs (784 pixels + the bias input)
 constexpr int kRing = 2;           // blocks of rows in shared memory
+constexpr int kLabelRing = 4;      // blocks of labels: the labels of block k + 2 are written while R still reads those of block k
 constexpr int kGramRanks = 3;      // warps sharing the Gram matrix of a block
 constexpr uint32_t kTmemCols = 128;
 constexpr float kSweepTol = 2e-7f;
@@ -61,7 +62,7 @@ struct __align__(128) TcSmem {
   float partZ[4][kM * kC];         // Z0 partial sums per quarter, index t * 10 + c
   float partG[2][kGramRanks][32];  // Gram pair partial sums, double-buffered by block parity
   float consts[8];                 // [0] = 1 (the bias input), [4] = 0 (rows no pixel maps to)
-  int ys[kRing][kM];
+  int ys[kLabelRing][kM];
   uint64_t full[kRing];
   uint64_t staged;
   uint64_t delta_ready;            // R has written the block's delta operand
@@ -153,16 +154,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
   auto produce = [&](uint32_t kb) {
     const int sb = kb % kRing;
     const uint32_t nvb = min((uint32_t)kM, n - kb * kM);
+    // a short last block: the rows nobody copies are zeroed, so that they add nothing anywhere; the
+    // warp barrier puts these stores ahead of lane 0's arrival, which is what the readers wait for
+    for (uint32_t r = nvb; r < (uint32_t)kM; ++r)
+      for (int i = lane; i < kD; i += 32) sm.rows[sb][r][i] = 0.f;
+    __syncwarp();
     if (lane == 0) mbar_expect_tx(&sm.full[sb], nvb * kRowBytes);
     __syncwarp();
     if ((uint32_t)lane < nvb) {
       const uint32_t idx = sample_index(draw(key, t.sample_ctr0 + kb * kM + lane), cd.n);
       bulk_load_row(sm.rows[sb][lane], xrows + (size_t)idx * kD, &sm.full[sb]);
-      sm.ys[sb][lane] = __ldg(cd.y + idx);
+      sm.ys[kb % kLabelRing][lane] = __ldg(cd.y + idx);
     }
-    // a short last block: the rows nobody copies are zeroed, so that they add nothing anywhere
-    for (uint32_t r = nvb; r < (uint32_t)kM; ++r)
-      for (int i = lane; i < kD; i += 32) sm.rows[sb][r][i] = 0.f;
   };
 
   // ---- start model: server snapshot minus own update sums still in flight ----
@@ -359,7 +362,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
         const float gsum = (1.f + g0[idx]) + (g1[idx] + g2[idx]);   // 1 = the bias input
         return s < j && (uint32_t)j < nv ? gsum * neta : 0.f;
       };
-      const int y = sm.ys[slot][j];
+      const int y = sm.ys[k % kLabelRing][j];
       float oh[kC];
 #pragma unroll
       for (int c = 0; c < kC; ++c) oh[c] = c == y ? -1.f : 0.f;

@@ -38,6 +38,13 @@
 // contiguous bytes per instruction (row by row a warp instruction would touch 32 different lines, half
 // a sector each, and the load/store unit, not HBM, would set the pace: measured 14 K cycles per unit).
 // The start of the round writes that order from the snapshot, the trigger reads it back.
+// When the launch has SMs to spare (two per round-task), a round-task runs on a cluster of two CTAs:
+// each takes one half of the hidden units of layer 0 - its half of every chunk of W0 (so each streams
+// half of the master), its rows of W1 - and everything narrower is computed by both.  What crosses
+// between them goes through distributed shared memory: the bf16 activations A0^T of the own hidden
+// units into the peer's copy after the forward epilogue, the updated bf16 rows of W1 into the peer's W1
+// tile; two hardware cluster barriers per iteration order these pushes against the products that read
+// them (and a last one keeps a CTA alive until its peer has stopped writing to it).
 // The update sums of the two wide layers are not accumulated entry by entry: their rows of U hold
 // w_start during the round and become (w_start - w_end) / eta at the trigger (w -= eta g and U += g
 // in the same step, eta constant within the round); W2 and the biases accumulate theirs explicitly.
@@ -59,9 +66,11 @@ constexpr uint32_t kWaitLimit = 1u << 22;
 
 // shared memory map (bytes)
 constexpr int kOffW1 = 0;                          // W1 tile, rows h0 (256), cols h1 (128), bf16: 64 KB
-constexpr int kOffdZ0 = kOffW1 + kH0 * kH1 * 2;    // dZ0^T tile, rows h0 (256), cols b (64): 32 KB
+constexpr int kOffdZ0 = kOffW1 + kH0 * kH1 * 2;    // dZ0^T tile, rows h0 (256), cols b (64): 32 KB; a CTA of a pair keeps its own
+constexpr int kOffA0peer = kOffdZ0 + 128 * kB * 2; //   128 rows there and, behind them, the peer's half of A0^T (16 KB)
 constexpr int kOffX = kOffdZ0 + kH0 * kB * 2;      // 4 minibatch-row tiles, rows b (64), cols i (128): cur[2], next[2], 16 KB each;
-                                                   // outside the layer-0 pipeline the first 32 KB hold the A0^T tile
+                                                   // outside the layer-0 pipeline the first 32 KB hold the A0^T tile (two halves of
+                                                   // 128 rows; a CTA of a pair keeps only its own half here)
 constexpr int kOffA0 = kOffX;
 constexpr int kOffWn = kOffX + 4 * kB * kCh * 2;   // unit tile, rows i (128), cols h0 (128), bf16: 32 KB; outside the pipeline:
 constexpr int kOffA1 = kOffWn;                     //   A1^T as plain bf16 [h1][b] (16 KB)
@@ -75,6 +84,7 @@ struct Small {
   float W2[kH1 * kMaxC], UW2[kH1 * kMaxC];
   float b0[kH0], Ub0[kH0], b1[kH1], Ub1[kH1], b2[kMaxC], Ub2[kMaxC];
   float logits[kB * kMaxC], dz2[kB * kMaxC], dz2q[kB * kMaxC];   // [b][c]
+  float gb0[2][128];                                               // bias gradient of layer 0, per half of the batch (pairs only)
   int idx[2][kB], ylab[kB];
   uint64_t bar_mma, g_full[2], g_free[2], wn_ready, wn_free, x_ready[2];
   uint32_t tmem_base, failed;
@@ -147,6 +157,24 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
 }
 
+// distributed shared memory of the CTA pair
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t peer_addr(uint32_t saddr, uint32_t peer) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(peer));
+  return r;
+}
+__device__ __forceinline__ void st_peer16(uint32_t addr, const uint4 v) {
+  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // Bounded wait for the completion number `count` (0-based) of an mbarrier.  After a timeout nothing polls any more.
 __device__ __forceinline__ void mbar_wait_n(uint64_t* bar, uint32_t count, bool& failed) {
   const uint32_t parity = count & 1u;
@@ -160,15 +188,20 @@ __device__ __forceinline__ void mbar_wait_n(uint64_t* bar, uint32_t count, bool&
   if (!ok) failed = true;
 }
 
+// NR = CTAs per round-task (1, or 2 as a cluster that splits the hidden units of layer 0)
+template <int NR>
 __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
   extern __shared__ __align__(1024) unsigned char sm[];
   Small& S = *reinterpret_cast<Small*>(sm + kOffSmall);
-  const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x];
-  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  constexpr int UPC = 2 / NR;   // units of a chunk this CTA works through
+  const int rank = NR == 2 ? (int)cluster_rank() : 0;
+  const uint32_t peer = (uint32_t)(rank ^ 1);
+  const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x / NR];
+  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip (both CTAs of a pair alike)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool ewarp = warp < kEWarps;
   const int D0 = (int)p.shape.dims[0], C = (int)p.shape.dims[3];
-  const int nch = D0 / kCh, NU = 2 * nch;   // chunks of 128 input rows; units = chunk x half of the hidden columns
+  const int nch = D0 / kCh, NU = UPC * nch;   // chunks of 128 input rows; units = chunk x half of the hidden columns
   const size_t oW0 = 0, ob0 = (size_t)D0 * kH0, oW1 = ob0 + kH0, ob1 = oW1 + (size_t)kH0 * kH1, oW2 = ob1 + kH1,
                ob2 = oW2 + (size_t)kH1 * C;
   float* work = p.work + (size_t)t.client * p.r.stride;
@@ -177,8 +210,11 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
   const __nv_bfloat16* xdata = reinterpret_cast<const __nv_bfloat16*>(cd.x);
   const uint64_t key = p.r.sample_keys[t.client];
   const float eta = t.eta, lambda = p.r.l2;
-  const uint32_t sW1 = smem_u32(sm + kOffW1), sdZ0 = smem_u32(sm + kOffdZ0), sA0 = smem_u32(sm + kOffA0),
-                 sWn = smem_u32(sm + kOffWn), sdZ1 = smem_u32(sm + kOffdZ1), sX = smem_u32(sm + kOffX);
+  const uint32_t sW1 = smem_u32(sm + kOffW1), sdZ0 = smem_u32(sm + kOffdZ0), sWn = smem_u32(sm + kOffWn),
+                 sdZ1 = smem_u32(sm + kOffdZ1), sX = smem_u32(sm + kOffX);
+  // A0^T, rows [128 tl, 128 tl + 128): a pair keeps the own half where a single CTA keeps its first, the peer's apart
+  auto a0_half = [&](int tl) { return NR == 1 ? kOffA0 + tl * 128 * kB * 2 : (tl == rank ? kOffA0 : kOffA0peer); };
+  auto unit_hh = [&](int u) { return NR == 1 ? (u & 1) : rank; };
 
   // ---- barriers and tensor memory ----
   if (tid == 0) {
@@ -216,24 +252,27 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       }
       return w;
     };
-    // W0 and W1 in work-row order (destination pieces in turn: contiguous stores, strided 16-byte loads)
-    for (size_t d4 = tid; d4 < (size_t)D0 * kH0 / 4; d4 += kSThreads) {
-      const int r = (int)(d4 & 127), k = (int)((d4 >> 7) & 15), blk = (int)(d4 >> 11);
-      const int half = blk & 1, hh = (blk >> 1) & 1, c = blk >> 2;
+    // W0 and W1 in work-row order (destination pieces in turn: contiguous stores, strided 16-byte loads); of a pair,
+    // each CTA the blocks it will own
+    for (size_t e4 = tid; e4 < (size_t)D0 * kH0 / 4 / NR; e4 += kSThreads) {
+      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 15), own = (int)(e4 >> 11);
+      const int half = own & 1, hh = NR == 1 ? (own >> 1) & 1 : rank, c = NR == 1 ? own >> 2 : own >> 1;
+      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + (e4 & 2047);
       const size_t j = oW0 + (size_t)(c * kCh + r) * kH0 + hh * 128 + half * 64 + 4 * k;
       const float4 w = start4(j);
       *reinterpret_cast<float4*>(work + oW0 + 4 * d4) = w;
       *reinterpret_cast<float4*>(Urow + j) = w;
     }
-    for (size_t d4 = tid; d4 < (size_t)kH0 * kH1 / 4; d4 += kSThreads) {
-      const int r = (int)(d4 & 127), k = (int)((d4 >> 7) & 7), blk = (int)(d4 >> 10);
-      const int g32 = blk & 3, tl = blk >> 2;
+    for (size_t e4 = tid; e4 < (size_t)kH0 * kH1 / 4 / NR; e4 += kSThreads) {
+      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 7), own = (int)(e4 >> 10);
+      const int g32 = own & 3, tl = NR == 1 ? own >> 2 : rank;
+      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + (e4 & 1023);
       const size_t j = oW1 + (size_t)(tl * 128 + r) * kH1 + g32 * 32 + 4 * k;
       const float4 w = start4(j);
       *reinterpret_cast<float4*>(work + oW1 + 4 * d4) = w;
       *reinterpret_cast<float4*>(Urow + j) = w;
     }
-    // the narrow rest stays in shared memory for the round
+    // the narrow rest stays in shared memory for the round (in both CTAs of a pair)
     for (int j = tid; j < kH0 + kH1 + kH1 * C + C; j += kSThreads) {
       const size_t g = j < kH0 ? ob0 + j : (j < kH0 + kH1 ? ob1 + (j - kH0) : oW2 + (j - kH0 - kH1));
       float w = snap[g];
@@ -247,7 +286,7 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       else { S.b2[g - ob2] = w; S.Ub2[g - ob2] = 0.f; }
     }
   }
-  __syncthreads();
+  if (NR == 2) cluster_sync(); else __syncthreads();   // the peer's half of the W1 master is in place too
   // W1 tile from the master (rows h0, cols h1)
   for (int e = tid; e < kH0 * (kH1 / 8); e += kSThreads) {
     const int r = e / (kH1 / 8), cg = e % (kH1 / 8);
@@ -283,9 +322,9 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
     // ===== first iteration of a round only: the forward product of layer 0 as a pass of its own =====
     if (it == 0) {
       for (int u = 0; u < NU; ++u) {
-        const int c = u >> 1, hh = u & 1;
+        const int c = u / UPC, hh = unit_hh(u);
         if (ewarp) {
-          if (hh == 0) load_x_tile(sm + kOffX + 2 * kB * kCh * 2, idx, c);     // into next[0]
+          if (u % UPC == 0) load_x_tile(sm + kOffX + 2 * kB * kCh * 2, idx, c);     // into next[0]
           const int q = warp & 3, half = warp >> 2;
           const int r = 32 * q + lane;
           const float* src = work + oW0 + w0_block(c, hh, half) + r * 4;
@@ -304,7 +343,7 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t id = idesc_bf16(128, kB, 1, 0);
           for (int ks = 0; ks < kCh / 16; ++ks)
-            umma_bf16(tmem + kColZ0 + 64 * hh, view_mn(sWn, 128, 0, ks * 16), view_k(sX + 2 * kB * kCh * 2, kCh, 0, ks * 16), id,
+            umma_bf16(tmem + kColZ0 + (NR == 1 ? 64 * hh : 0), view_mn(sWn, 128, 0, ks * 16), view_k(sX + 2 * kB * kCh * 2, kCh, 0, ks * 16), id,
                       (c > 0 || ks > 0) ? 1u : 0u);
           umma_commit(&S.bar_mma);
         }
@@ -314,15 +353,19 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     }
 
-    // ===== Z0 epilogue: A0^T = bf16(relu(Z0^T + b0)) =====
+    // ===== Z0 epilogue: A0^T = bf16(relu(Z0^T + b0)); a pair: own hidden units, each warp half of the batch, and a copy to the peer =====
     if (ewarp) {
-      const int q = warp & 3, tl = warp >> 2;
-      const int h0 = 128 * tl + 32 * q + lane;
-      const float bias = S.b0[h0];
+      const int q = warp & 3, wh = warp >> 2;
+      const int tl = NR == 1 ? wh : rank;
+      const int lr = 32 * q + lane;
+      const float bias = S.b0[128 * tl + lr];
+      const int a0off = a0_half(tl);
+      const uint32_t remote = NR == 2 ? peer_addr(smem_u32(sm + kOffA0peer), peer) : 0u;
 #pragma unroll
-      for (int hb = 0; hb < 2; ++hb) {
+      for (int hq = 0; hq < UPC; ++hq) {
+        const int hb = NR == 1 ? hq : wh;   // which 32 columns of the batch
         uint32_t v[32];
-        tmem_ld32(tq + kColZ0 + 64 * tl + 32 * hb, v);
+        tmem_ld32(tq + kColZ0 + (NR == 1 ? 64 * tl : 0) + 32 * hb, v);
 #pragma unroll
         for (int g8 = 0; g8 < 4; ++g8) {
           uint4 o;
@@ -330,20 +373,23 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
 #pragma unroll
           for (int k = 0; k < 8; ++k) a[k] = fmaxf(__uint_as_float(v[g8 * 8 + k]) + bias, 0.f);
           o.x = pack_bf16(a[0], a[1]); o.y = pack_bf16(a[2], a[3]); o.z = pack_bf16(a[4], a[5]); o.w = pack_bf16(a[6], a[7]);
-          *reinterpret_cast<uint4*>(sm + kOffA0 + tile_off(h0, 32 * hb + g8 * 8, kB)) = o;
+          const int off = tile_off(lr, 32 * hb + g8 * 8, kB);
+          *reinterpret_cast<uint4*>(sm + a0off + off) = o;
+          if (NR == 2) st_peer16(remote + (uint32_t)off, o);
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("fence.proxy.async;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    if (NR == 2) cluster_sync(); else __syncthreads();   // pair: both halves of A0^T are in both CTAs
 
     // ===== layer 1 forward: Z1^T[h1, b] = W1^T A0^T =====
     if (tid == kEThreads) {
+      asm volatile("fence.proxy.async;" ::: "memory");
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t id = idesc_bf16(128, kB, 1, 1);
       for (int ks = 0; ks < kH0 / 16; ++ks)
-        umma_bf16(tmem + kColZ1, view_mn(sW1, kH1, 0, ks * 16), view_mn(sA0, kB, 0, ks * 16), id, ks > 0 ? 1u : 0u);
+        umma_bf16(tmem + kColZ1, view_mn(sW1, kH1, 0, ks * 16), view_mn(smem_u32(sm + a0_half(ks >> 3)), kB, 0, (ks & 7) * 16), id, ks > 0 ? 1u : 0u);
       umma_commit(&S.bar_mma);
     }
     mbar_wait_n(&S.bar_mma, n_mma++, failed);
@@ -430,17 +476,19 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       if (bc == 0) { S.b1[h] = fmaf(-eta, part, S.b1[h]); S.Ub1[h] += part; }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncthreads();
-    // ===== layer 1 backward on tensor cores (old W1): dA0^T first, then dW1 =====
+    // pair: from here on the peer may overwrite its rows of this CTA's W1 tile and, in the next iteration, its half
+    // of A0^T; both were last read by the forward product of layer 1 above, which both CTAs have seen complete
+    if (NR == 2) cluster_sync(); else __syncthreads();
+    // ===== layer 1 backward on tensor cores (old W1): dA0^T first, then dW1; a pair: the own 128 hidden units only =====
     if (tid == kEThreads) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t ida = idesc_bf16(128, kB, 0, 1), idw = idesc_bf16(128, kH1, 0, 0);
-      for (int tl = 0; tl < 2; ++tl)
+      for (int tl = NR == 1 ? 0 : rank; tl < (NR == 1 ? 2 : rank + 1); ++tl)
         for (int ks = 0; ks < kH1 / 16; ++ks)
-          umma_bf16(tmem + kColdA0 + 64 * tl, view_k(sW1, kH1, 128 * tl, ks * 16), view_mn(sdZ1, kB, 0, ks * 16), ida, ks > 0 ? 1u : 0u);
-      for (int tl = 0; tl < 2; ++tl)
+          umma_bf16(tmem + kColdA0 + (NR == 1 ? 64 * tl : 0), view_k(sW1, kH1, 128 * tl, ks * 16), view_mn(sdZ1, kB, 0, ks * 16), ida, ks > 0 ? 1u : 0u);
+      for (int tl = NR == 1 ? 0 : rank; tl < (NR == 1 ? 2 : rank + 1); ++tl)
         for (int ks = 0; ks < kB / 16; ++ks)
-          umma_bf16(tmem + kColdW1 + 128 * tl, view_k(sA0, kB, 128 * tl, ks * 16), view_k(sdZ1, kB, 0, ks * 16), idw, ks > 0 ? 1u : 0u);
+          umma_bf16(tmem + kColdW1 + (NR == 1 ? 128 * tl : 0), view_k(smem_u32(sm + a0_half(tl)), kB, 0, ks * 16), view_k(sdZ1, kB, 0, ks * 16), idw, ks > 0 ? 1u : 0u);
       umma_commit(&S.bar_mma);
     }
     // meanwhile: the class layer's own update (its products above used the old values)
@@ -471,17 +519,20 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
     mbar_wait_n(&S.bar_mma, n_mma++, failed);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ewarp) {
-      const int q = warp & 3, tl = warp >> 2;
-      const int h0 = 128 * tl + 32 * q + lane;
-      // dZ0^T = relu'(A0^T) * dA0^T; bias gradient of layer 0 in fp32 (a thread sees its unit's whole batch)
+      const int q = warp & 3, wh = warp >> 2;
+      const int tl = NR == 1 ? wh : rank;
+      const int lr = 32 * q + lane, h0 = 128 * tl + lr;
+      const int a0off = a0_half(tl), dz0row = NR == 1 ? h0 : lr;
+      // dZ0^T = relu'(A0^T) * dA0^T; bias gradient of layer 0 in fp32 (a thread sees its unit's whole batch, in a pair half of it)
       float gb = 0.f;
 #pragma unroll
-      for (int hb = 0; hb < 2; ++hb) {
+      for (int hq = 0; hq < UPC; ++hq) {
+        const int hb = NR == 1 ? hq : wh;
         uint32_t v[32];
-        tmem_ld32(tq + kColdA0 + 64 * tl + 32 * hb, v);
+        tmem_ld32(tq + kColdA0 + (NR == 1 ? 64 * tl : 0) + 32 * hb, v);
 #pragma unroll
         for (int g8 = 0; g8 < 4; ++g8) {
-          const uint4 a = *reinterpret_cast<const uint4*>(sm + kOffA0 + tile_off(h0, 32 * hb + g8 * 8, kB));
+          const uint4 a = *reinterpret_cast<const uint4*>(sm + a0off + tile_off(lr, 32 * hb + g8 * 8, kB));
           const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
           float d[8];
 #pragma unroll
@@ -492,17 +543,23 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
           }
           uint4 o;
           o.x = pack_bf16(d[0], d[1]); o.y = pack_bf16(d[2], d[3]); o.z = pack_bf16(d[4], d[5]); o.w = pack_bf16(d[6], d[7]);
-          *reinterpret_cast<uint4*>(sm + kOffdZ0 + tile_off(h0, 32 * hb + g8 * 8, kB)) = o;
+          *reinterpret_cast<uint4*>(sm + kOffdZ0 + tile_off(dz0row, 32 * hb + g8 * 8, kB)) = o;
         }
       }
-      S.b0[h0] = fmaf(-eta, gb, S.b0[h0]);
-      S.Ub0[h0] += gb;
-      // dW1 epilogue: row h0 of the master, new bf16 values into the W1 tile
+      if (NR == 1) {
+        S.b0[h0] = fmaf(-eta, gb, S.b0[h0]);
+        S.Ub0[h0] += gb;
+      } else {
+        S.gb0[wh][lr] = gb;   // summed over the two halves of the batch behind the barrier below
+      }
+      // dW1 epilogue: row h0 of the master, new bf16 values into the W1 tile (a pair: and into the peer's)
+      const uint32_t remote = NR == 2 ? peer_addr(sW1, peer) : 0u;
 #pragma unroll 1
-      for (int g32 = 0; g32 < 4; ++g32) {
-        float* wrow = work + oW1 + w1_block(tl, g32) + (32 * q + lane) * 4;
+      for (int gq = 0; gq < 2 * UPC; ++gq) {
+        const int g32 = NR == 1 ? gq : 2 * wh + gq;
+        float* wrow = work + oW1 + w1_block(tl, g32) + lr * 4;
         uint32_t v[32];
-        tmem_ld32(tq + kColdW1 + 128 * tl + 32 * g32, v);
+        tmem_ld32(tq + kColdW1 + (NR == 1 ? 128 * tl : 0) + 32 * g32, v);
         float4 w[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) w[k] = *reinterpret_cast<const float4*>(wrow + k * 512);
@@ -519,13 +576,20 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
           uint4 o;
           o.x = pack_bf16(w[2 * k].x, w[2 * k].y); o.y = pack_bf16(w[2 * k].z, w[2 * k].w);
           o.z = pack_bf16(w[2 * k + 1].x, w[2 * k + 1].y); o.w = pack_bf16(w[2 * k + 1].z, w[2 * k + 1].w);
-          *reinterpret_cast<uint4*>(sm + kOffW1 + tile_off(h0, 32 * g32 + 8 * k, kH1)) = o;
+          const int off = tile_off(h0, 32 * g32 + 8 * k, kH1);
+          *reinterpret_cast<uint4*>(sm + kOffW1 + off) = o;
+          if (NR == 2) st_peer16(remote + (uint32_t)off, o);
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("fence.proxy.async;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();   // dZ0^T and the new W1 tile are complete; the A0^T area becomes minibatch-row tiles
+    if (NR == 2 && tid < 128) {
+      const float gb = S.gb0[0][tid] + S.gb0[1][tid];
+      S.b0[128 * rank + tid] = fmaf(-eta, gb, S.b0[128 * rank + tid]);
+      S.Ub0[128 * rank + tid] += gb;
+    }
 
     // ===== layer 0: gradient, master update and the next iteration's forward product, unit by unit =====
     if (ewarp) {
@@ -540,21 +604,27 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       if (lane == 0) mbar_arrive(&S.x_ready[0]);
       float4 wn[16];
       {
-        const float* src = work + oW0 + w0_block(0, 0, half) + r * 4;
+        const float* src = work + oW0 + w0_block(0, unit_hh(0), half) + r * 4;
 #pragma unroll
         for (int k = 0; k < 16; ++k) wn[k] = *reinterpret_cast<const float4*>(src + k * 512);
       }
       for (int u = 0; u < NU; ++u) {
-        const int c = u >> 1, hh = u & 1, sl = u & 1;
+        const int c = u / UPC, hh = unit_hh(u), sl = u & 1;
+        const bool first = u % UPC == 0, last = u % UPC == UPC - 1, more = c + 1 < nch;
         float4 w[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) w[k] = wn[k];
         float* dst = work + oW0 + w0_block(c, hh, half) + r * 4;
         if (u + 1 < NU) {   // the master rows of the next unit: on their way during this unit's work
-          const int c1 = (u + 1) >> 1, h1 = (u + 1) & 1;
-          const float* src = work + oW0 + w0_block(c1, h1, half) + r * 4;
+          const float* src = work + oW0 + w0_block((u + 1) / UPC, unit_hh(u + 1), half) + r * 4;
 #pragma unroll
           for (int k = 0; k < 16; ++k) wn[k] = *reinterpret_cast<const float4*>(src + k * 512);
+        }
+        // Rows of the next chunk for the gradient product: their buffer was last read by the gradient
+        // products of chunk c - 1, which this thread has already seen complete.
+        if (first && more) {
+          load_x_tile(sm + kOffX + ((c + 1) & 1) * kB * kCh * 2, idx, c + 1);
+          asm volatile("cp.async.commit_group;" ::: "memory");
         }
         mbar_wait_n(&S.g_full[sl], n_gfull[sl]++, failed);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -577,11 +647,11 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
         // Shared-memory work first, the master's stores last: the proxy fence below would otherwise
         // wait for sixteen global stores per thread on every unit.
         if (fuse && u >= 1) mbar_wait_n(&S.wn_free, n_wnfree++, failed);   // the forward product of unit u - 1 has read the unit tile
-        if (hh == 0 && c + 1 < nch) {
-          // rows of the next chunk.  Their buffers were last read by the products of chunk c - 1: its
-          // gradients were waited for above, its forward products just now.
-          load_x_tile(sm + kOffX + ((c + 1) & 1) * kB * kCh * 2, idx, c + 1);
+        if (first && more) {
+          // rows of the next chunk for the forward product: their buffer was last read by the forward
+          // products of chunk c - 1, the last of which was waited for just now
           if (fuse) load_x_tile(sm + kOffX + (2 + ((c + 1) & 1)) * kB * kCh * 2, idxn, c + 1);
+          asm volatile("cp.async.commit_group;" ::: "memory");
         }
         if (fuse) {
 #pragma unroll
@@ -592,8 +662,17 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
             *reinterpret_cast<uint4*>(sm + kOffWn + tile_off(r, 64 * half + 8 * k, 128)) = o;
           }
         }
-        const bool rows_due = hh == 1 && c + 1 < nch;
-        if (rows_due) asm volatile("cp.async.wait_all;" ::: "memory");
+        // What must have landed before the arrivals below: the gradient rows of chunk c + 1 (for the
+        // issuer), the forward rows of chunk c (read by the product that takes this unit tile).  A
+        // single CTA has a whole unit between issue and use; in a pair the forward rows of chunk c + 1,
+        // the group committed last, may stay in flight until the next unit.
+        const bool rows_due = last && more;
+        if (NR == 1) {
+          if (rows_due) asm volatile("cp.async.wait_group 0;" ::: "memory");
+        } else {
+          if (more) asm volatile("cp.async.wait_group 1;" ::: "memory");
+          else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
         if (fuse || rows_due) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
@@ -610,26 +689,26 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       // ---- the issuing warp ----
       const uint32_t idg = idesc_bf16(128, 128, 1, 0), idf = idesc_bf16(128, kB, 1, 0);
       auto issue_fwd = [&](int u) {
-        const int c = u >> 1, hh = u & 1;
+        const int c = u / UPC, hh = unit_hh(u);
         mbar_wait_n(&S.wn_ready, n_wnready++, failed);
         if (lane == 0 && !failed) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t xs = sX + (2 + (c & 1)) * kB * kCh * 2;
           for (int ks = 0; ks < kCh / 16; ++ks)
-            umma_bf16(tmem + kColZ0 + 64 * hh, view_mn(sWn, 128, 0, ks * 16), view_k(xs, kCh, 0, ks * 16), idf, (c > 0 || ks > 0) ? 1u : 0u);
+            umma_bf16(tmem + kColZ0 + (NR == 1 ? 64 * hh : 0), view_mn(sWn, 128, 0, ks * 16), view_k(xs, kCh, 0, ks * 16), idf, (c > 0 || ks > 0) ? 1u : 0u);
         }
         if (lane == 0) umma_commit(&S.wn_free);
         __syncwarp();
       };
       for (int u = 0; u < NU; ++u) {
-        const int c = u >> 1, hh = u & 1, sl = u & 1;
-        if (hh == 0) { mbar_wait_n(&S.x_ready[c & 1], n_xready[c & 1]++, failed); }
+        const int c = u / UPC, hh = unit_hh(u), sl = u & 1;
+        if (u % UPC == 0) { mbar_wait_n(&S.x_ready[c & 1], n_xready[c & 1]++, failed); }
         if (u >= 2) mbar_wait_n(&S.g_free[sl], n_gfree[sl]++, failed);
         if (lane == 0 && !failed) {
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t xs = sX + (c & 1) * kB * kCh * 2;
           for (int ks = 0; ks < kB / 16; ++ks)
-            umma_bf16(tmem + kColG + 128 * sl, view_mn(xs, kCh, 0, ks * 16), view_k(sdZ0, kB, 128 * hh, ks * 16), idg, ks > 0 ? 1u : 0u);
+            umma_bf16(tmem + kColG + 128 * sl, view_mn(xs, kCh, 0, ks * 16), view_k(sdZ0, kB, NR == 1 ? 128 * hh : 0, ks * 16), idg, ks > 0 ? 1u : 0u);
         }
         if (lane == 0) umma_commit(&S.g_full[sl]);
         __syncwarp();
@@ -653,7 +732,7 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
 
-  // ---- event trigger: publish (c, U_i, i) ----
+  // ---- event trigger: publish (c, U_i, i); of a pair, each CTA the blocks it owns ----
   __syncthreads();
   {
     const float inv_eta = 1.f / eta;
@@ -663,18 +742,22 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       *reinterpret_cast<float4*>(Urow + j) = make_float4((a.x - w.x) * inv_eta, (a.y - w.y) * inv_eta, (a.z - w.z) * inv_eta, (a.w - w.w) * inv_eta);
       if (wend) *reinterpret_cast<float4*>(wend + j) = w;
     };
-    for (size_t d4 = tid; d4 < (size_t)D0 * kH0 / 4; d4 += kSThreads) {
-      const int r = (int)(d4 & 127), k = (int)((d4 >> 7) & 15), blk = (int)(d4 >> 11);
-      const int half = blk & 1, hh = (blk >> 1) & 1, c = blk >> 2;
+    for (size_t e4 = tid; e4 < (size_t)D0 * kH0 / 4 / NR; e4 += kSThreads) {
+      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 15), own = (int)(e4 >> 11);
+      const int half = own & 1, hh = NR == 1 ? (own >> 1) & 1 : rank, c = NR == 1 ? own >> 2 : own >> 1;
+      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + (e4 & 2047);
       finish4(oW0 + (size_t)(c * kCh + r) * kH0 + hh * 128 + half * 64 + 4 * k, *reinterpret_cast<const float4*>(work + oW0 + 4 * d4));
     }
-    for (size_t d4 = tid; d4 < (size_t)kH0 * kH1 / 4; d4 += kSThreads) {
-      const int r = (int)(d4 & 127), k = (int)((d4 >> 7) & 7), blk = (int)(d4 >> 10);
-      const int g32 = blk & 3, tl = blk >> 2;
+    for (size_t e4 = tid; e4 < (size_t)kH0 * kH1 / 4 / NR; e4 += kSThreads) {
+      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 7), own = (int)(e4 >> 10);
+      const int g32 = own & 3, tl = NR == 1 ? own >> 2 : rank;
+      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + (e4 & 1023);
       finish4(oW1 + (size_t)(tl * 128 + r) * kH1 + g32 * 32 + 4 * k, *reinterpret_cast<const float4*>(work + oW1 + 4 * d4));
     }
+    // the narrow parameters: identical in both CTAs of a pair except the first bias, of which each holds its half
     for (int j = tid; j < kH0 + kH1 + kH1 * C + C; j += kSThreads) {
       const size_t g = j < kH0 ? ob0 + j : (j < kH0 + kH1 ? ob1 + (j - kH0) : oW2 + (j - kH0 - kH1));
+      if (NR == 2 && (j < kH0 ? (j >> 7) != rank : rank != 0)) continue;
       float u, w;
       if (g < oW1) { u = S.Ub0[g - ob0]; w = S.b0[g - ob0]; }
       else if (g < oW2) { u = S.Ub1[g - ob1]; w = S.b1[g - ob1]; }
@@ -688,12 +771,14 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
   __syncthreads();
   if (tid == 0) {
     if (S.failed && p.r.status) atomicOr(p.r.status, 1u);
-    TriggerRec rec;
-    rec.client = t.client; rec.round = t.round; rec.samples_done = t.steps * (uint32_t)kB; rec.flags = 1;
-    p.r.trig[t.seq] = rec;
+    if (rank == 0) {
+      TriggerRec rec;
+      rec.client = t.client; rec.round = t.round; rec.samples_done = t.steps * (uint32_t)kB; rec.flags = 1;
+      p.r.trig[t.seq] = rec;
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (NR == 2) cluster_sync(); else __syncthreads();   // pair: the peer has stopped writing into this CTA's shared memory
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
@@ -706,10 +791,35 @@ bool mlp_stream_eligible(const MlpShape& s) {
 
 cudaError_t launch_mlp_stream_rounds(const MlpLaunch& p, cudaStream_t s) {
   if (p.r.n_tasks == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(mlp_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, n = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    sms = n;
+  }
+  // two SMs per round-task while the launch leaves that many free; a fuller launch runs one CTA per round-task
+  const bool pair = 2 * (int)p.r.n_tasks <= sms;
+  cudaError_t e = cudaFuncSetAttribute(pair ? mlp_stream_kernel<2> : mlp_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  mlp_stream_kernel<<<p.r.n_tasks, kSThreads, kSmemBytes, s>>>(p);
-  return cudaGetLastError();
+  if (!pair) {
+    mlp_stream_kernel<1><<<p.r.n_tasks, kSThreads, kSmemBytes, s>>>(p);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(p.r.n_tasks * 2, 1, 1);
+  cfg.blockDim = dim3(kSThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, mlp_stream_kernel<2>, p);
 }
 
 }  // namespace aet

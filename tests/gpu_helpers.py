@@ -51,12 +51,22 @@ def check_against_oracle(cfg, data, w0, gpu, ref, u_tol=U_TOL, loss_tol=LOSS_TOL
     return f_gpu, f_ref
 
 
-def check_round_U(cfg, data, h, c, i, w_start, u_tol=U_TOL):
-    """Round-task (c, i) restarted on both sides from the same fp32 model."""
+def check_round_U(cfg, data, h, c, i, w_start, u_tol=U_TOL, flip_frac=0.0, flip_tol=None):
+    """Round-task (c, i) restarted on both sides from the same fp32 model.
+
+    Entry by entry |U_gpu - U_or| / max|U_or| must stay within ``u_tol``.  Where the arithmetic takes discrete
+    decisions whose inputs differ by accumulation order (a bf16 rounding, a ReLU mask), ``flip_tol`` admits a
+    share ``flip_frac`` of the entries above ``u_tol``, none of them above ``flip_tol``."""
     w32 = np.ascontiguousarray(w_start, dtype=np.float32)
     U_gpu, w_gpu = api.aet_debug_run_client_round(h, c, i, w32)
     U_ref, w_ref = sim.run_task(cfg, data[c], c, i, w32.astype(np.float64))
-    eu, ew = rel_err(U_gpu, U_ref), rel_err(w_gpu, w_ref)
-    assert eu <= u_tol, (c, i, eu)
+    d = np.abs(U_gpu - U_ref) / np.abs(U_ref).max()
+    eu, ew = float(d.max()), rel_err(w_gpu, w_ref)
+    if flip_tol is None:
+        assert eu <= u_tol, (c, i, eu)
+    else:
+        share = float((d > u_tol).mean())
+        assert share <= flip_frac, (c, i, share, eu)
+        assert eu <= flip_tol, (c, i, eu)
     assert ew <= u_tol, (c, i, ew)
     return eu

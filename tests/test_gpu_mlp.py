@@ -13,7 +13,15 @@ pytestmark = pytest.mark.gpu
 # precision 1: an fp32-vs-fp64 difference in a sum can flip one bf16 rounding (2^-8 relative on that
 # element), so the fp32 bar cannot hold; the bar is twice the worst per-round error measured over these
 # cases (1.4e-4).  The same shapes with fp32 operands meet the fp32 bar (test below).
+# bf16 operands: entry by entry 3e-4 of max|U|, except where a discrete decision fell the other way.  The kernel
+# accumulates pre-activations in fp32 on the tensor cores, the checker in fp64; where the two sums straddle a bf16
+# rounding boundary or zero, a rounded activation moves by one bf16 step or a ReLU mask flips.  One flipped mask at
+# (sample b, unit h) of layer l adds or removes that sample's whole term dA_l[b, h] <= (2 / B) max|W_{l+1}| (~1e-2 of
+# max|U| at B = 64) in the bias entry h, and its product with the layer's input in row h of the weights: at most
+# 1 + fan-in entries, 0.4 % of this model per flip.  So: at most 1 % of the entries above 3e-4, none above 3e-2.
+# A dropped term, a wrong index or operand order moves most entries by far more than 3e-4.
 BF16_U_TOL = 3e-4
+BF16_FLIPS = dict(flip_frac=1e-2, flip_tol=3e-2)
 
 
 def _small_cfg3(**kw):
@@ -66,7 +74,7 @@ def test_mlp_bf16_small_end_to_end_and_round_U():
     gpu = run_gpu(cfg, data, w0)
     check_against_oracle(cfg, data, w0, gpu, ref)
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
-        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], BF16_U_TOL)
+        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], BF16_U_TOL, **BF16_FLIPS)
                 for e in ref["events"][::3]]
     print("bf16 per-round U errors:", ["%.1e" % v for v in errs])
 
@@ -85,7 +93,7 @@ def test_mlp_bf16_tensor_core_path(over):
     check_against_oracle(cfg, data, w0, gpu, ref)
     assert rel_err(gpu["w"], ref["w"]) <= 1e-3
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
-        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], BF16_U_TOL)
+        errs = [check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][e["seq"]], BF16_U_TOL, **BF16_FLIPS)
                 for e in ref["events"][::max(1, len(ref["events"]) // 6)]]
     print("tensor-core path per-round U errors:", ["%.1e" % v for v in errs])
 
@@ -136,7 +144,7 @@ def test_cfg4_real_dims_first_rounds_against_the_checker():
     assert rel_err(gpu["w"], ref["w"]) <= 1e-3
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
         errs = [check_round_U(cfg, data, s.h, ref["events"][k]["client"], ref["events"][k]["round"],
-                              ref["w_start"][k], BF16_U_TOL) for k in picks]
+                              ref["w_start"][k], BF16_U_TOL, **BF16_FLIPS) for k in picks]
     print("cfg4 per-round U errors:", ["%.1e" % v for v in errs])
 
 
@@ -153,4 +161,4 @@ def test_cfg4_full_size_log_and_sampled_rounds():
     assert np.isfinite(gpu["w"]).all()
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
         for c, i in ((0, 0), (63, 3), (17, 29)):
-            check_round_U(cfg, data, s.h, c, i, gpu["w"], BF16_U_TOL)
+            check_round_U(cfg, data, s.h, c, i, gpu["w"], BF16_U_TOL, **BF16_FLIPS)
