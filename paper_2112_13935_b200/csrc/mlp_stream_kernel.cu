@@ -595,13 +595,17 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
     if (ewarp) {
       const int q = warp & 3, half = warp >> 2;
       const int r = 32 * q + lane;                       // row of the unit this thread owns
-      // rows of chunk 0 (this minibatch, and the next one for the forward product)
+      // rows of chunks 0 and 1 of this minibatch (gradient products), of chunk 0 of the next one (forward product)
       load_x_tile(sm + kOffX, idx, 0);
+      if (nch > 1) load_x_tile(sm + kOffX + kB * kCh * 2, idx, 1);
       if (fuse) load_x_tile(sm + kOffX + 2 * kB * kCh * 2, idxn, 0);
       asm volatile("cp.async.wait_all;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(&S.x_ready[0]);
+      if (lane == 0) {
+        mbar_arrive(&S.x_ready[0]);
+        if (nch > 1) mbar_arrive(&S.x_ready[1]);
+      }
       float4 wn[16];
       {
         const float* src = work + oW0 + w0_block(0, unit_hh(0), half) + r * 4;
@@ -615,19 +619,21 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
 #pragma unroll
         for (int k = 0; k < 16; ++k) w[k] = wn[k];
         float* dst = work + oW0 + w0_block(c, hh, half) + r * 4;
+        // The gradient of this unit was issued a unit ago; taking its barrier first keeps the poll out of
+        // the queue behind the sixteen loads below.
+        mbar_wait_n(&S.g_full[sl], n_gfull[sl]++, failed);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // The chunk's last gradient product has completed: its rows make room for those of the chunk after
+        // the next, so that the issuer always has the next chunk's rows when a slot falls free.
+        if (last) {
+          if (c + 2 < nch) load_x_tile(sm + kOffX + (c & 1) * kB * kCh * 2, idx, c + 2);
+          asm volatile("cp.async.commit_group;" ::: "memory");
+        }
         if (u + 1 < NU) {   // the master rows of the next unit: on their way during this unit's work
           const float* src = work + oW0 + w0_block((u + 1) / UPC, unit_hh(u + 1), half) + r * 4;
 #pragma unroll
           for (int k = 0; k < 16; ++k) wn[k] = *reinterpret_cast<const float4*>(src + k * 512);
         }
-        // Rows of the next chunk for the gradient product: their buffer was last read by the gradient
-        // products of chunk c - 1, which this thread has already seen complete.
-        if (first && more) {
-          load_x_tile(sm + kOffX + ((c + 1) & 1) * kB * kCh * 2, idx, c + 1);
-          asm volatile("cp.async.commit_group;" ::: "memory");
-        }
-        mbar_wait_n(&S.g_full[sl], n_gfull[sl]++, failed);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
         for (int hb = 0; hb < 2; ++hb) {
           uint32_t v[32];
@@ -662,15 +668,13 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
             *reinterpret_cast<uint4*>(sm + kOffWn + tile_off(r, 64 * half + 8 * k, 128)) = o;
           }
         }
-        // What must have landed before the arrivals below: the gradient rows of chunk c + 1 (for the
-        // issuer), the forward rows of chunk c (read by the product that takes this unit tile).  A
-        // single CTA has a whole unit between issue and use; in a pair the forward rows of chunk c + 1,
-        // the group committed last, may stay in flight until the next unit.
-        const bool rows_due = last && more;
-        if (NR == 1) {
-          if (rows_due) asm volatile("cp.async.wait_group 0;" ::: "memory");
-        } else {
-          if (more) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        // What must have landed before the arrivals below: the gradient rows of chunk c + 2 (for the
+        // issuer), the forward rows of chunk c (read by the product that takes this unit tile), and
+        // for a single CTA those of chunk c + 1, whose first unit has no wait of its own.  In a pair the
+        // forward rows of chunk c + 1, the group committed last, may stay in flight until the next unit.
+        const bool rows_due = last && c + 2 < nch;
+        if (last) {
+          if (NR == 2 && more) asm volatile("cp.async.wait_group 1;" ::: "memory");
           else asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
         if (fuse || rows_due) {
@@ -678,7 +682,7 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
           __syncwarp();
           if (lane == 0) {
             if (fuse) mbar_arrive(&S.wn_ready);
-            if (rows_due) mbar_arrive(&S.x_ready[(c + 1) & 1]);
+            if (rows_due) mbar_arrive(&S.x_ready[c & 1]);
           }
         }
 #pragma unroll
