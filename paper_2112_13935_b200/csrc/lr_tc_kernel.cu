@@ -337,20 +337,18 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
     const int rwarp = (int)(k & (kTcWarps - 1));
     const int rel = (warp - rwarp) & (kTcWarps - 1);
     if (rel == 0) {
-      // ---- R: the block's kM dependent softmax steps, lane j owns sample j ----
-      const int j = lane & (kM - 1);
-      float z[kC];
-      {
-        const float2* z0 = reinterpret_cast<const float2*>(&sm.partZ[0][j * kC]);
-        const float2* z1 = reinterpret_cast<const float2*>(&sm.partZ[1][j * kC]);
-        const float2* z2 = reinterpret_cast<const float2*>(&sm.partZ[2][j * kC]);
-        const float2* z3 = reinterpret_cast<const float2*>(&sm.partZ[3][j * kC]);
+      // ---- R: the block's kM dependent softmax steps.  Four lanes share a sample: lane 4 j + g owns
+      // classes g, g + 4 and (g < 2) g + 8 of sample j, so that a sweep costs 21 shuffles instead of 70.
+      const int j = lane >> 2, g = lane & 3;
+      constexpr int kOwn = 3;
+      constexpr float kNoClass = -1e30f;   // stands in for the third class of g >= 2: exp gives 0, nothing moves
+      float z[kOwn];
 #pragma unroll
-        for (int c = 0; c < kC / 2; ++c) {
-          const float2 a0 = z0[c], a1 = z1[c], a2 = z2[c], a3 = z3[c];
-          z[2 * c] = (a0.x + a1.x) + (a2.x + a3.x);
-          z[2 * c + 1] = (a0.y + a1.y) + (a2.y + a3.y);
-        }
+      for (int i = 0; i < kOwn; ++i) {
+        const int c = g + 4 * i;
+        const int at = j * kC + (c < kC ? c : 0);
+        const float v = (sm.partZ[0][at] + sm.partZ[1][at]) + (sm.partZ[2][at] + sm.partZ[3][at]);
+        z[i] = c < kC ? v : kNoClass;
       }
       const float* g0 = sm.partG[k & 1][0];
       const float* g1 = sm.partG[k & 1][1];
@@ -363,24 +361,27 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
         return s < j && (uint32_t)j < nv ? gsum * neta : 0.f;
       };
       const int y = sm.ys[k % kLabelRing][j];
-      float oh[kC];
+      float oh[kOwn];
 #pragma unroll
-      for (int c = 0; c < kC; ++c) oh[c] = c == y ? -1.f : 0.f;
-      auto softmax_delta = [&](const float (&zz)[kC], float (&d)[kC]) {
-        const float m = fmaxf(fmaxf(fmaxf(fmaxf(zz[0], zz[1]), fmaxf(zz[2], zz[3])), fmaxf(fmaxf(zz[4], zz[5]), fmaxf(zz[6], zz[7]))),
-                              fmaxf(zz[8], zz[9]));
+      for (int i = 0; i < kOwn; ++i) oh[i] = g + 4 * i == y ? -1.f : 0.f;
+      auto softmax_delta = [&](const float (&zz)[kOwn], float (&d)[kOwn]) {
+        float m = fmaxf(fmaxf(zz[0], zz[1]), zz[2]);
+        m = fmaxf(m, shx(m, 1));
+        m = fmaxf(m, shx(m, 2));
         const float nms = -m * kLog2e;
-        float e[kC];
+        float e[kOwn];
 #pragma unroll
-        for (int c = 0; c < kC; ++c) e[c] = ex2(fmaf(zz[c], kLog2e, nms));
-        const float sum = (((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]))) + (e[8] + e[9]);
+        for (int i = 0; i < kOwn; ++i) e[i] = ex2(fmaf(zz[i], kLog2e, nms));
+        float sum = (e[0] + e[1]) + e[2];
+        sum += shx(sum, 1);
+        sum += shx(sum, 2);
         const float inv = rcp(sum);
 #pragma unroll
-        for (int c = 0; c < kC; ++c) d[c] = fmaf(e[c], inv, oh[c]);
+        for (int i = 0; i < kOwn; ++i) d[i] = fmaf(e[i], inv, oh[i]);
       };
-      float dk[kC];   // delta of this lane's own sample
+      float dk[kOwn];   // delta of this lane's own sample and classes
 #pragma unroll
-      for (int c = 0; c < kC; ++c) dk[c] = 0.f;
+      for (int i = 0; i < kOwn; ++i) dk[i] = 0.f;
 
       bool swept = false;
       if (kSweep) {
@@ -390,28 +391,28 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
 #pragma unroll
         for (int s = 0; s < kM - 1; ++s) { Lr[s] = corr(s); rowsum += fabsf(Lr[s]); }
         float rho = rowsum;
-        rho = fmaxf(rho, shx(rho, 4)); rho = fmaxf(rho, shx(rho, 2)); rho = fmaxf(rho, shx(rho, 1));
+        rho = fmaxf(rho, shx(rho, 16)); rho = fmaxf(rho, shx(rho, 8)); rho = fmaxf(rho, shx(rho, 4));
         rho *= 0.5f;
         if (rho <= 0.25f) {
           swept = true;
           const float gain = rho / (1.f - rho);
-          float z0[kC];
+          float z0[kOwn];
 #pragma unroll
-          for (int c = 0; c < kC; ++c) z0[c] = z[c];
+          for (int i = 0; i < kOwn; ++i) z0[i] = z[i];
           // at most nv sweeps are ever needed: sweep i makes the first i samples exact
           for (uint32_t sweep = 0; sweep < nv; ++sweep) {
-            float d[kC];
+            float d[kOwn];
             softmax_delta(z, d);
-            float zn[kC];
+            float zn[kOwn];
 #pragma unroll
-            for (int c = 0; c < kC; ++c) zn[c] = z0[c];
+            for (int i = 0; i < kOwn; ++i) zn[i] = z0[i];
 #pragma unroll
             for (int s = 0; s < kM - 1; ++s)
 #pragma unroll
-              for (int c = 0; c < kC; ++c) zn[c] = fmaf(__shfl_sync(0xffffffffu, d[c], s), Lr[s], zn[c]);
+              for (int i = 0; i < kOwn; ++i) zn[i] = fmaf(__shfl_sync(0xffffffffu, d[i], 4 * s + g), Lr[s], zn[i]);
             float change = 0.f;
 #pragma unroll
-            for (int c = 0; c < kC; ++c) { change = fmaxf(change, fabsf(zn[c] - z[c])); z[c] = zn[c]; }
+            for (int i = 0; i < kOwn; ++i) { change = fmaxf(change, fabsf(zn[i] - z[i])); z[i] = zn[i]; }
             if (!__any_sync(0xffffffffu, change * gain > kSweepTol)) break;
           }
           softmax_delta(z, dk);
@@ -423,27 +424,30 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
 #pragma unroll 1
         for (int s = 0; s < (int)nv; ++s) {
           const float gnext = corr(s + 1);
-          float d[kC];
+          float d[kOwn];
           softmax_delta(z, d);
           const bool mine = j == s;
 #pragma unroll
-          for (int c = 0; c < kC; ++c) {
-            dk[c] = mine ? d[c] : dk[c];
-            z[c] = fmaf(__shfl_sync(0xffffffffu, d[c], s), gs, z[c]);
+          for (int i = 0; i < kOwn; ++i) {
+            dk[i] = mine ? d[i] : dk[i];
+            z[i] = fmaf(__shfl_sync(0xffffffffu, d[i], 4 * s + g), gs, z[i]);
           }
           gs = gnext;
         }
       }
       // delta as the tensor cores' second operand: tf32 head and remainder, zero for missing samples
-      if (lane < kM) {
-        const bool live = (uint32_t)lane < nv;
+      {
+        const bool live = (uint32_t)j < nv;
 #pragma unroll
-        for (int c = 0; c < kC; ++c) {
-          const float d = live ? dk[c] : 0.f;
-          const float hi = tf32_head(d);
-          const int col = c < kCh ? c : c + 3;
-          sm.B[0][lane >> 2][col][lane & 3] = hi;
-          sm.B[1][lane >> 2][col][lane & 3] = d - hi;
+        for (int i = 0; i < kOwn; ++i) {
+          const int c = g + 4 * i;
+          if (c < kC) {
+            const float d = live ? dk[i] : 0.f;
+            const float hi = tf32_head(d);
+            const int col = c < kCh ? c : c + 3;
+            sm.B[0][j >> 2][col][j & 3] = hi;
+            sm.B[1][j >> 2][col][j & 3] = d - hi;
+          }
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
