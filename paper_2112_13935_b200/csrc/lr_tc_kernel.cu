@@ -180,26 +180,45 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
     // Everything above reads only what earlier, finished grids and the host wrote.  The snapshot is
     // written by the aggregation kernel launched just before this grid, which may still be running
     // when this grid was launched with programmatic stream serialisation.
-    if (warp == 0) {
-      produce(0);
-      if (nblk > 1) produce(1);
-    }
+    if (warp == 0) produce(0);
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (uint32_t f = 0; f <= t.inflight_cnt; ++f) {   // f = 0: the snapshot, then the sums in flight
-      const float* src;
-      float scale;
-      if (f == 0) {
-        src = p.snaps + (size_t)t.snap_slot * p.stride;
-        scale = 1.f;
-      } else {
-        const InflightRef ref = p.inflight[t.inflight_off + f - 1];
-        src = p.U + (size_t)ref.row * p.stride;
-        scale = -ref.eta;
+    // The snapshot and the first update sum in flight (nine round-tasks in ten have exactly one) come in
+    // side by side: the snapshot into the staging area, the sum behind it in what is left of the operand
+    // tiles, its last 5.6 KB in the second block of rows, whose copies are issued only afterwards.
+    constexpr int kHeadFloats = 2 * kTiles * 2 * 128 * 4 - kStageFloats, kTailFloats = kStageFloats - kHeadFloats;
+    static_assert(kHeadFloats > 0 && kHeadFloats % 4 == 0 && kTailFloats % 4 == 0 && kTailFloats <= kM * kD, "second staging area");
+    const float* head2 = stage + kStageFloats;
+    const float* tail2 = &sm.rows[1][0][0];
+    const uint32_t nfl = t.inflight_cnt;
+    float scale2 = 0.f;
+    if (nfl) scale2 = -p.inflight[t.inflight_off].eta;
+    if (threadIdx.x == 0) {
+      mbar_expect_tx(&sm.staged, (nfl ? 2u : 1u) * kStageFloats * sizeof(float));
+      bulk_load(stage, p.snaps + (size_t)t.snap_slot * p.stride, kStageFloats * sizeof(float), &sm.staged);
+      if (nfl) {
+        const float* src = p.U + (size_t)p.inflight[t.inflight_off].row * p.stride;
+        bulk_load(const_cast<float*>(head2), src, kHeadFloats * sizeof(float), &sm.staged);
+        bulk_load(const_cast<float*>(tail2), src + kHeadFloats, kTailFloats * sizeof(float), &sm.staged);
       }
-      if (f) __syncthreads();   // everybody has taken the previous row out of the staging area
+    }
+    ok = mbar_wait(&sm.staged, 0) && ok;
+#pragma unroll
+    for (int j = 0; j < kTiles; ++j) {
+      const bool live = j < kTiles - 1 || pix6 || bias6;
+#pragma unroll
+      for (int c = 0; c < kCh; ++c) {
+        const int e = (128 * j + row) * kC + kCh * ch + c;
+        float v = live ? stage[e] : 0.f;
+        if (nfl && live) v = fmaf(scale2, e < kHeadFloats ? head2[e] : tail2[e - kHeadFloats], v);
+        ws[j][c] = v;
+      }
+    }
+    for (uint32_t f = 1; f < nfl; ++f) {   // further sums in flight, one after the other
+      const InflightRef ref = p.inflight[t.inflight_off + f];
+      __syncthreads();   // everybody has taken the previous row out of the staging area
       if (threadIdx.x == 0) {
         mbar_expect_tx(&sm.staged, kStageFloats * sizeof(float));
-        bulk_load(stage, src, kStageFloats * sizeof(float), &sm.staged);
+        bulk_load(stage, p.U + (size_t)ref.row * p.stride, kStageFloats * sizeof(float), &sm.staged);
       }
       ok = mbar_wait(&sm.staged, f & 1) && ok;
 #pragma unroll
@@ -208,11 +227,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
 #pragma unroll
         for (int c = 0; c < kCh; ++c) {
           const float v = live ? stage[(128 * j + row) * kC + kCh * ch + c] : 0.f;
-          ws[j][c] = fmaf(scale, v, ws[j][c]);
+          ws[j][c] = fmaf(-ref.eta, v, ws[j][c]);
         }
       }
     }
-    __syncthreads();   // the staging area becomes the operand tiles
+    __syncthreads();   // the staging areas become the operand tiles and the second block of rows
+    if (warp == 0 && nblk > 1) produce(1);
   }
 
   // Where this thread reads its input of sample s for tiles 0..5 and for tile 6.
@@ -497,7 +517,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) lr_tc_kernel(RoundLaunch p) {
     if (threadIdx.x == 0) {
       if (p.status) atomicOr(p.status, 1u);
       for (uint32_t j = timeout_at; j < nblk && j < timeout_at + 2; ++j) mbar_wait(&sm.full[j % kRing], (j / kRing) & 1);
-      mbar_wait(&sm.staged, t.inflight_cnt & 1);   // the last row staged at the start
+      mbar_wait(&sm.staged, (t.inflight_cnt > 1 ? t.inflight_cnt - 1 : 0) & 1);   // the last rows staged at the start
     }
   } else {
     // The aggregation kernel behind this grid in the stream may become resident from here on (it

@@ -98,6 +98,24 @@ def test_mlp_bf16_tensor_core_path(over):
     print("tensor-core path per-round U errors:", ["%.1e" % v for v in errs])
 
 
+def test_stream_kernel_one_cta_and_pair_instances_agree():
+    # 80 round-tasks in the first wave: more than half the SMs, so the run takes the one-CTA instance of the
+    # streaming kernel; a round restarted on its own takes the pair.  Round 0 starts from w0 on both paths.
+    cfg = workloads.get_config("cfg4", n_clients=80, n_rounds=2, dims=[512, 256, 128, 10], n_stragglers=2,
+                               data=dict(kind="iid", total=8000, dim=512))
+    data, w0 = make(cfg)
+    ref = sim.run(cfg, data, w0, keep=True)
+    gpu = run_gpu(cfg, data, w0)
+    check_against_oracle(cfg, data, w0, gpu, ref)
+    assert rel_err(gpu["w"], ref["w"]) <= 1e-3
+    first = [e for e in ref["events"] if e["round"] == 0][::16]
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        for e in first:
+            U_pair, _ = api.aet_debug_run_client_round(s.h, e["client"], 0, w0)
+            assert rel_err(U_pair, gpu["U"][e["seq"]]) <= 2e-6   # same arithmetic; only the first bias gradient is summed in another order
+            check_round_U(cfg, data, s.h, e["client"], 0, w0, BF16_U_TOL, **BF16_FLIPS)
+
+
 def test_bf16_shapes_with_fp32_operands_meet_the_fp32_bar():
     # the cut-down cfg4 of the bf16 test above, precision 0: every per-round update sum within 1e-5
     cfg = workloads.get_config("cfg4", precision=0, n_clients=4, n_rounds=3, dims=[3072, 64, 32, 10],
