@@ -6,14 +6,16 @@
 // Algorithm 3, MainComputeNode, inner loop with xi a minibatch: g = mean gradient (+ lambda W on
 // weight tensors), w_c -= eta_i g, U_i += g, repeated s_{i,c} / B times; then (c, U_i, i) is sent.
 //
-// One CTA of 512 threads per round-task.  The client's whole model (44,426 parameters for the
-// 28x28 shape, 174 KB) stays in shared memory from the start of the round to its trigger; only the
-// minibatch rows, the activations of the minibatch (global scratch, L2-resident) and the running
-// update sum (one read-modify-write per parameter and iteration) move.  A parameter's gradient is
-// summed over the minibatch by the thread that owns the parameter and applied on the spot, so no
-// gradient buffer exists and nothing needs an atomic.  Weight updates of layer l share a phase
-// with the input-gradient product of layer l - 1 (which reads other weights), so the backward pass
-// costs one block barrier per layer.
+// A cluster of up to 8 CTAs of 512 threads per round-task, the minibatch split over the CTAs.  Every
+// CTA keeps the client's whole model (44,426 parameters for the 28x28 shape, 174 KB) in shared memory
+// from the start of the round to its trigger and runs the forward and backward pass of its own
+// samples (activations in global scratch, L2-resident) against the same, old weights; each
+// parameter's gradient over the CTA's samples goes to a per-CTA row of global scratch.  After a
+// cluster barrier every CTA owns a slice of the parameters: it adds the slice over the CTAs' rows in
+// rank order (no atomics, identical from run to run), applies w -= eta g and U += g, and writes the
+// new weights into all the CTAs' copies through distributed shared memory; a second barrier ends the
+// iteration.  With one CTA (a launch too full for clusters, or a minibatch of one) the same code runs
+// with a cluster of one.
 #include <cuda_runtime.h>
 
 #include "aet_kernels.h"
@@ -24,10 +26,11 @@ namespace {
 
 constexpr int kCnnThreads = 512;
 constexpr int kK = 5;   // kernel side of both convolutions
+constexpr int kMaxCl = 8;   // CTAs per round-task at most
 
 struct CnnDims {
   int side, cin, c1, c2, f1, f2, ncls, s1, p1, s2, p2, flat;
-  int oW1, ob1, oW2, ob2, oF1, obF1, oF2, obF2, oF3, obF3, P;
+  int oW1, ob1, oW2, ob2, oF1, obF1, oF2, obF2, oF3, obF3, P, Ppad;
   // per-minibatch activation scratch (floats), offsets for batch size B
   int a1, q1, a2, q2, h1, h2, z3, dz3, dh2, dh1, dq2, dq1, total;
 };
@@ -45,6 +48,7 @@ __host__ __device__ inline CnnDims make_cnn_dims(const CnnShape& s) {
   d.oF2 = o; o += d.f1 * d.f2; d.obF2 = o; o += d.f2;
   d.oF3 = o; o += d.f2 * d.ncls; d.obF3 = o; o += d.ncls;
   d.P = o;
+  d.Ppad = (o + 31) & ~31;
   const int B = (int)s.batch;
   int a = 0;
   d.a1 = a; a += B * d.c1 * d.s1 * d.s1;
@@ -63,15 +67,15 @@ __host__ __device__ inline CnnDims make_cnn_dims(const CnnShape& s) {
   return d;
 }
 
-// Valid 5x5 correlation + bias + ReLU + 2x2 average pooling of one stage, for the whole minibatch.
+// Valid 5x5 correlation + bias + ReLU + 2x2 average pooling of one stage, for samples [b0, b0 + nb).
 // One work item = one pooled output: its four pre-pooling outputs share a 6x6 input patch per plane.
 template <class InAt>
-__device__ __forceinline__ void conv_stage(int B, int cin, int cout, int sin, int sout, const float* W, const float* bias,
+__device__ __forceinline__ void conv_stage(int b0, int nb, int cin, int cout, int sin, int sout, const float* W, const float* bias,
                                            InAt in_at, float* a_out, float* q_out, int tid) {
   const int pout = sout / 2;
-  const int items = B * cout * pout * pout;
+  const int items = nb * cout * pout * pout;
   for (int e = tid; e < items; e += kCnnThreads) {
-    const int px = e % pout, py = (e / pout) % pout, c = (e / (pout * pout)) % cout, b = e / (pout * pout * cout);
+    const int px = e % pout, py = (e / pout) % pout, c = (e / (pout * pout)) % cout, b = b0 + e / (pout * pout * cout);
     float z00 = bias[c], z01 = z00, z10 = z00, z11 = z00;
     for (int ci = 0; ci < cin; ++ci) {
       float patch[6][6];
@@ -98,14 +102,27 @@ __device__ __forceinline__ void conv_stage(int B, int cin, int cout, int sin, in
   }
 }
 
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster(const float* local, uint32_t rank, float v) {
+  uint32_t a;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
+
 __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) {
   extern __shared__ __align__(16) float smem[];
-  const TaskDesc t = p.r.tasks[p.r.task_begin + blockIdx.x];
-  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip
+  const int CL = (int)cluster_size(), rank = (int)cluster_rank();
+  const int task = blockIdx.x / CL;
+  const TaskDesc t = p.r.tasks[p.r.task_begin + task];
+  if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip (the whole cluster alike)
   const CnnDims D = make_cnn_dims(p.shape);
   const int B = (int)p.shape.batch;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  float* w = smem;                                     // the client's model, whole round
+  float* w = smem;                                     // the client's model, whole round, one copy per CTA
   int* idx = reinterpret_cast<int*>(smem + ((D.P + 3) & ~3));
   int* ylab = idx + B;
 
@@ -114,8 +131,13 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
   const uint64_t key = p.r.sample_keys[t.client];
   const float eta = t.eta, lambda = p.r.l2, invB = 1.f / (float)B;
   const int rowlen = D.cin * D.side * D.side;
-  float* act = p.act + (size_t)blockIdx.x * p.act_stride;
+  float* act = p.act + (size_t)task * p.act_stride;
   float* Urow = p.r.U + (size_t)t.u_row * p.r.stride;
+  // this CTA's samples of the minibatch, its row of gradient partials, its slice of the parameters
+  const int per = (B + CL - 1) / CL, nact = (B + per - 1) / per;
+  const int b0 = min(B, rank * per), nb = min(B, b0 + per) - b0;
+  float* G = act + D.total + (size_t)rank * D.Ppad;
+  const int slice = (D.P + CL - 1) / CL, k_lo = min(D.P, rank * slice), k_hi = min(D.P, k_lo + slice);
 
   // ---- start model: snapshot minus own update sums still in flight; U_i = 0 ----
   {
@@ -127,18 +149,10 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
         v = fmaf(-ref.eta, p.r.U[(size_t)ref.row * p.r.stride + k], v);
       }
       w[k] = v;
-      Urow[k] = 0.f;
+      if (k >= k_lo && k < k_hi) Urow[k] = 0.f;
     }
   }
   __syncthreads();
-
-  // w -= eta (g + lambda w), U += g + lambda w for one parameter; biases take no l2 term
-  auto apply = [&](int k, float g, bool decay) {
-    const float wk = w[k];
-    const float gt = decay ? fmaf(lambda, wk, g) : g;
-    w[k] = fmaf(-eta, gt, wk);
-    Urow[k] += gt;
-  };
 
   for (uint32_t it = 0; it < t.steps; ++it) {
     if (tid < B) {
@@ -148,25 +162,25 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     }
     __syncthreads();
 
-    // ================= forward =================
-    conv_stage(B, D.cin, D.c1, D.side, D.s1, w + D.oW1, w + D.ob1,
+    // ================= forward (own samples) =================
+    conv_stage(b0, nb, D.cin, D.c1, D.side, D.s1, w + D.oW1, w + D.ob1,
                [&](int b, int ci, int y, int x) { return __ldg(xrows + (size_t)idx[b] * rowlen + (ci * D.side + y) * D.side + x); },
                act + D.a1, act + D.q1, tid);
     __syncthreads();
     {
       const float* q1 = act + D.q1;
-      conv_stage(B, D.c1, D.c2, D.p1, D.s2, w + D.oW2, w + D.ob2,
+      conv_stage(b0, nb, D.c1, D.c2, D.p1, D.s2, w + D.oW2, w + D.ob2,
                  [&](int b, int ci, int y, int x) { return q1[((size_t)(b * D.c1 + ci) * D.p1 + y) * D.p1 + x]; },
                  act + D.a2, act + D.q2, tid);
     }
     __syncthreads();
     auto dense_fwd = [&](const float* in, int K, int N, const float* Wl, const float* bl, float* out, bool relu) {
-      for (int e = tid; e < B * N; e += kCnnThreads) {
-        const int j = e % N, b = e / N;
+      for (int e = tid; e < nb * N; e += kCnnThreads) {
+        const int j = e % N, b = b0 + e / N;
         float z = bl[j];
         const float* a = in + (size_t)b * K;
         for (int k = 0; k < K; ++k) z = fmaf(a[k], Wl[k * N + j], z);
-        out[e] = relu ? fmaxf(z, 0.f) : z;
+        out[(size_t)b * N + j] = relu ? fmaxf(z, 0.f) : z;
       }
     };
     dense_fwd(act + D.q2, D.flat, D.f1, w + D.oF1, w + D.obF1, act + D.h1, true);
@@ -175,73 +189,75 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     __syncthreads();
     dense_fwd(act + D.h2, D.f2, D.ncls, w + D.oF3, w + D.obF3, act + D.z3, false);
     __syncthreads();
-    if (tid < B) {   // softmax cross-entropy: dZ = (p - onehot) / B
-      const float* z = act + D.z3 + tid * D.ncls;
+    if (tid < nb) {   // softmax cross-entropy: dZ = (p - onehot) / B
+      const int b = b0 + tid;
+      const float* z = act + D.z3 + b * D.ncls;
       float m = -INFINITY;
       for (int j = 0; j < D.ncls; ++j) m = fmaxf(m, z[j]);
       float sum = 0.f;
       for (int j = 0; j < D.ncls; ++j) sum += __expf(z[j] - m);
       const float inv = 1.f / sum;
-      const int y = ylab[tid];
+      const int y = ylab[b];
       for (int j = 0; j < D.ncls; ++j)
-        act[D.dz3 + tid * D.ncls + j] = (__expf(z[j] - m) * inv - (j == y ? 1.f : 0.f)) * invB;
+        act[D.dz3 + b * D.ncls + j] = (__expf(z[j] - m) * inv - (j == y ? 1.f : 0.f)) * invB;
     }
     __syncthreads();
 
-    // ================= backward =================
+    // ================= backward (own samples, old weights throughout) =================
     // input gradient of a dense layer, gated by the ReLU of the layer below: dIn[b, i] = [in > 0] sum_j dOut[b, j] W[i, j]
     auto dense_din = [&](int e, const float* dout, int K, int N, const float* Wl, const float* in, float* din, bool gate) {
-      const int i = e % K, b = e / K;
+      const int i = e % K, b = b0 + e / K;
       float s = 0.f;
       const float* dz = dout + (size_t)b * N;
       const float* wr = Wl + (size_t)i * N;
       for (int j = 0; j < N; ++j) s = fmaf(dz[j], wr[j], s);
-      din[e] = (!gate || in[e] > 0.f) ? s : 0.f;
+      const size_t at = (size_t)b * K + i;
+      din[at] = (!gate || in[at] > 0.f) ? s : 0.f;
     };
-    // gradient and update of one dense parameter: item < K * N a weight, else a bias
-    auto dense_upd = [&](int e, const float* in, const float* dout, int K, int N, int oW, int ob) {
+    // this CTA's share of the gradient of one dense parameter: item < K * N a weight, else a bias
+    auto dense_grad = [&](int e, const float* in, const float* dout, int K, int N, int oW, int ob) {
       if (e < K * N) {
         const int j = e % N, i = e / N;
         float g = 0.f;
-        for (int b = 0; b < B; ++b) g = fmaf(in[(size_t)b * K + i], dout[(size_t)b * N + j], g);
-        apply(oW + e, g, true);
+        for (int b = b0; b < b0 + nb; ++b) g = fmaf(in[(size_t)b * K + i], dout[(size_t)b * N + j], g);
+        G[oW + e] = g;
       } else {
         const int j = e - K * N;
         float g = 0.f;
-        for (int b = 0; b < B; ++b) g += dout[(size_t)b * N + j];
-        apply(ob + j, g, false);
+        for (int b = b0; b < b0 + nb; ++b) g += dout[(size_t)b * N + j];
+        G[ob + j] = g;
       }
     };
-    // dh2 from the class layer (its weights are still the old ones)
-    for (int e = tid; e < B * D.f2; e += kCnnThreads)
+    // dh2 from the class layer
+    for (int e = tid; e < nb * D.f2; e += kCnnThreads)
       dense_din(e, act + D.dz3, D.f2, D.ncls, w + D.oF3, act + D.h2, act + D.dh2, true);
     __syncthreads();
-    // class layer update | dh1 through dense layer 2
+    // class layer gradient | dh1 through dense layer 2
     {
-      const int nu = D.f2 * D.ncls + D.ncls, nd = B * D.f1;
+      const int nu = D.f2 * D.ncls + D.ncls, nd = nb * D.f1;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) dense_upd(e, act + D.h2, act + D.dz3, D.f2, D.ncls, D.oF3, D.obF3);
+        if (e < nu) dense_grad(e, act + D.h2, act + D.dz3, D.f2, D.ncls, D.oF3, D.obF3);
         else dense_din(e - nu, act + D.dh2, D.f1, D.f2, w + D.oF2, act + D.h1, act + D.dh1, true);
       }
     }
     __syncthreads();
-    // dense layer 2 update | dq2 through dense layer 1 (the pooled maps carry no ReLU of their own)
+    // dense layer 2 gradient | dq2 through dense layer 1 (the pooled maps carry no ReLU of their own)
     {
-      const int nu = D.f1 * D.f2 + D.f2, nd = B * D.flat;
+      const int nu = D.f1 * D.f2 + D.f2, nd = nb * D.flat;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) dense_upd(e, act + D.h1, act + D.dh2, D.f1, D.f2, D.oF2, D.obF2);
+        if (e < nu) dense_grad(e, act + D.h1, act + D.dh2, D.f1, D.f2, D.oF2, D.obF2);
         else dense_din(e - nu, act + D.dh1, D.flat, D.f1, w + D.oF1, act + D.q2, act + D.dq2, false);
       }
     }
     __syncthreads();
-    // dense layer 1 update | dz2 = [a2 > 0] * dq2 / 4, in place over a2
+    // dense layer 1 gradient | dz2 = [a2 > 0] * dq2 / 4, in place over a2
     {
-      const int nu = D.flat * D.f1 + D.f1, nd = B * D.c2 * D.s2 * D.s2;
+      const int nu = D.flat * D.f1 + D.f1, per2 = D.c2 * D.s2 * D.s2, nd = nb * per2;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
         if (e < nu) {
-          dense_upd(e, act + D.q2, act + D.dh1, D.flat, D.f1, D.oF1, D.obF1);
+          dense_grad(e, act + D.q2, act + D.dh1, D.flat, D.f1, D.oF1, D.obF1);
         } else {
-          const int k = e - nu;
+          const int k = b0 * per2 + (e - nu);
           const int x = k % D.s2, y = (k / D.s2) % D.s2, bc = k / (D.s2 * D.s2);
           const float g = act[D.dq2 + ((size_t)bc * D.p2 + (y >> 1)) * D.p2 + (x >> 1)];
           act[D.a2 + k] = act[D.a2 + k] > 0.f ? 0.25f * g : 0.f;
@@ -249,12 +265,13 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
       }
     }
     __syncthreads();
-    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx] (second convolution's old weights)
+    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx]
     {
       const float* dz2 = act + D.a2;
       const float* W2 = w + D.oW2;
-      for (int e = tid; e < B * D.c1 * D.p1 * D.p1; e += kCnnThreads) {
-        const int x = e % D.p1, y = (e / D.p1) % D.p1, c = (e / (D.p1 * D.p1)) % D.c1, b = e / (D.p1 * D.p1 * D.c1);
+      const int per1 = D.c1 * D.p1 * D.p1;
+      for (int e = tid; e < nb * per1; e += kCnnThreads) {
+        const int x = e % D.p1, y = (e / D.p1) % D.p1, c = (e / (D.p1 * D.p1)) % D.c1, b = b0 + e / per1;
         float s = 0.f;
         for (int c2 = 0; c2 < D.c2; ++c2) {
           const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
@@ -270,36 +287,36 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
             }
           }
         }
-        act[D.dq1 + e] = s;
+        act[D.dq1 + (size_t)b0 * per1 + e] = s;
       }
     }
     __syncthreads();
-    // second convolution's update | dz1 = [a1 > 0] * dq1 / 4, in place over a1
+    // second convolution's gradient | dz1 = [a1 > 0] * dq1 / 4, in place over a1
     {
-      const int nw = D.c2 * D.c1 * kK * kK, nu = nw + D.c2, nd = B * D.c1 * D.s1 * D.s1;
+      const int nw = D.c2 * D.c1 * kK * kK, nu = nw + D.c2, per1 = D.c1 * D.s1 * D.s1, nd = nb * per1;
       const float* dz2 = act + D.a2;
       const float* q1 = act + D.q1;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
         if (e < nw) {
           const int dx = e % kK, dy = (e / kK) % kK, c = (e / (kK * kK)) % D.c1, c2 = e / (kK * kK * D.c1);
           float g = 0.f;
-          for (int b = 0; b < B; ++b) {
+          for (int b = b0; b < b0 + nb; ++b) {
             const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
             const float* qp = q1 + ((size_t)(b * D.c1 + c) * D.p1 + dy) * D.p1 + dx;
             for (int y = 0; y < D.s2; ++y)
               for (int x = 0; x < D.s2; ++x) g = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g);
           }
-          apply(D.oW2 + e, g, true);
+          G[D.oW2 + e] = g;
         } else if (e < nu) {
           const int c2 = e - nw;
           float g = 0.f;
-          for (int b = 0; b < B; ++b) {
+          for (int b = b0; b < b0 + nb; ++b) {
             const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
             for (int k = 0; k < D.s2 * D.s2; ++k) g += dzp[k];
           }
-          apply(D.ob2 + c2, g, false);
+          G[D.ob2 + c2] = g;
         } else {
-          const int k = e - nu;
+          const int k = b0 * per1 + (e - nu);
           const int x = k % D.s1, y = (k / D.s1) % D.s1, bc = k / (D.s1 * D.s1);
           const float g = act[D.dq1 + ((size_t)bc * D.p1 + (y >> 1)) * D.p1 + (x >> 1)];
           act[D.a1 + k] = act[D.a1 + k] > 0.f ? 0.25f * g : 0.f;
@@ -307,45 +324,59 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
       }
     }
     __syncthreads();
-    // first convolution's update: few parameters, long sums (B * s1 * s1 terms each): a warp per parameter,
+    // first convolution's gradient: few parameters, long sums (nb * s1 * s1 terms each): a warp per parameter,
     // lanes take the terms in turn, shuffle tree at the end
     {
       const int nw = D.c1 * D.cin * kK * kK, nu = nw + D.c1;
       const float* dz1 = act + D.a1;
-      const int terms = B * D.s1 * D.s1;
+      const int terms = nb * D.s1 * D.s1;
       for (int e = warp; e < nu; e += kCnnThreads / 32) {
         float g = 0.f;
         if (e < nw) {
           const int dx = e % kK, dy = (e / kK) % kK, ci = (e / (kK * kK)) % D.cin, c = e / (kK * kK * D.cin);
           for (int k = lane; k < terms; k += 32) {
-            const int x = k % D.s1, y = (k / D.s1) % D.s1, b = k / (D.s1 * D.s1);
+            const int x = k % D.s1, y = (k / D.s1) % D.s1, b = b0 + k / (D.s1 * D.s1);
             const float xv = __ldg(xrows + (size_t)idx[b] * rowlen + (ci * D.side + y + dy) * D.side + x + dx);
             g = fmaf(dz1[((size_t)(b * D.c1 + c) * D.s1 + y) * D.s1 + x], xv, g);
           }
         } else {
           const int c = e - nw;
           for (int k = lane; k < terms; k += 32) {
-            const int r = k % (D.s1 * D.s1), b = k / (D.s1 * D.s1);
+            const int r = k % (D.s1 * D.s1), b = b0 + k / (D.s1 * D.s1);
             g += dz1[(size_t)(b * D.c1 + c) * D.s1 * D.s1 + r];
           }
         }
 #pragma unroll
         for (int m = 16; m; m >>= 1) g += __shfl_xor_sync(0xffffffffu, g, m);
-        if (lane == 0) {
-          if (e < nw) apply(D.oW1 + e, g, true);
-          else apply(D.ob1 + (e - nw), g, false);
-        }
+        if (lane == 0) G[e < nw ? D.oW1 + e : D.ob1 + (e - nw)] = g;
       }
     }
-    __syncthreads();
+    cluster_sync();   // every CTA's partial gradients are in global scratch; nobody reads the old weights any more
+
+    // ================= this CTA's slice: g = sum over the CTAs in rank order; w -= eta (g + lambda w), U += g + lambda w =================
+    {
+      const float* G0 = act + D.total;
+      for (int k = k_lo + tid; k < k_hi; k += kCnnThreads) {
+        float g = 0.f;
+        for (int q = 0; q < nact; ++q) g += G0[(size_t)q * D.Ppad + k];
+        const bool bias = (k >= D.ob1 && k < D.oW2) || (k >= D.ob2 && k < D.oF1) || (k >= D.obF1 && k < D.oF2) ||
+                          (k >= D.obF2 && k < D.oF3) || k >= D.obF3;   // biases take no l2 term
+        const float wk = w[k];
+        const float gt = bias ? g : fmaf(lambda, wk, g);
+        const float wn = fmaf(-eta, gt, wk);
+        Urow[k] += gt;
+        for (int q = 0; q < CL; ++q) st_cluster(w + k, (uint32_t)q, wn);
+      }
+    }
+    cluster_sync();   // the new weights are in every CTA's copy
   }
 
   // ---- event trigger: h reached s_{i,c}; U_i is complete in its row; the end model on request ----
   if (p.r.w_end) {
     float* dst = p.r.w_end + (size_t)t.u_row * p.r.stride;
-    for (int k = tid; k < D.P; k += kCnnThreads) dst[k] = w[k];
+    for (int k = k_lo + tid; k < k_hi; k += kCnnThreads) dst[k] = w[k];
   }
-  if (tid == 0) {
+  if (tid == 0 && rank == 0) {
     TriggerRec rec;
     rec.client = t.client; rec.round = t.round; rec.samples_done = t.steps * (uint32_t)B; rec.flags = 1;
     p.r.trig[t.seq] = rec;
@@ -360,7 +391,11 @@ size_t cnn_smem_bytes(const CnnShape& s) {
 }  // namespace
 
 uint32_t cnn_n_params(const CnnShape& s) { return (uint32_t)make_cnn_dims(s).P; }
-size_t cnn_act_floats(const CnnShape& s) { return (size_t)make_cnn_dims(s).total; }
+// activations of a minibatch, then one row of gradient partials per CTA of the cluster
+size_t cnn_act_floats(const CnnShape& s) {
+  const CnnDims d = make_cnn_dims(s);
+  return (size_t)d.total + (size_t)kMaxCl * d.Ppad;
+}
 
 const char* cnn_check_shape(const CnnShape& s) {
   const int side = (int)s.dims[0];
@@ -377,11 +412,33 @@ const char* cnn_check_shape(const CnnShape& s) {
 
 cudaError_t launch_cnn_rounds(const CnnLaunch& p, cudaStream_t s) {
   if (p.r.n_tasks == 0) return cudaSuccess;
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, n = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    sms = n;
+  }
   const size_t smem = cnn_smem_bytes(p.shape);
   cudaError_t e = cudaFuncSetAttribute(cnn_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  cnn_round_kernel<<<p.r.n_tasks, kCnnThreads, smem, s>>>(p);
-  return cudaGetLastError();
+  // CTAs per round-task: as many as the minibatch has samples and the launch leaves SMs for
+  uint32_t cl = kMaxCl;
+  while (cl > 1 && (cl > p.shape.batch || p.r.n_tasks * cl > (uint32_t)sms)) cl >>= 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(p.r.n_tasks * cl, 1, 1);
+  cfg.blockDim = dim3(kCnnThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cl;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, cnn_round_kernel, p);
 }
 
 }  // namespace aet
