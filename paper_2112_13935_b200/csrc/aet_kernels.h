@@ -89,6 +89,8 @@ struct CnnLaunch {
   CnnShape shape;
   float* act;                    // per-task activation scratch
   size_t act_stride;             // floats per task
+  uint32_t stage_rows = 0;       // set by the launcher: the CTA's minibatch rows fit in shared memory beside the model,
+  uint32_t stage_acts = 0;       //   and so do its activations other than the first convolution's maps
 };
 uint32_t cnn_n_params(const CnnShape& s);
 size_t cnn_act_floats(const CnnShape& s);

@@ -113,6 +113,11 @@ __device__ __forceinline__ void st_cluster(const float* local, uint32_t rank, fl
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
 }
 
+// floats of per-sample activations that may live in shared memory (everything but the first convolution's maps)
+__host__ __device__ inline int cnn_small_acts(const CnnDims& d) {
+  return 2 * d.c1 * d.p1 * d.p1 + d.c2 * d.s2 * d.s2 + 2 * d.flat + 2 * d.f1 + 2 * d.f2 + 2 * d.ncls;
+}
+
 __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) {
   extern __shared__ __align__(16) float smem[];
   const int CL = (int)cluster_size(), rank = (int)cluster_rank();
@@ -138,6 +143,31 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
   const int b0 = min(B, rank * per), nb = min(B, b0 + per) - b0;
   float* G = act + D.total + (size_t)rank * D.Ppad;
   const int slice = (D.P + CL - 1) / CL, k_lo = min(D.P, rank * slice), k_hi = min(D.P, k_lo + slice);
+  // Where the launch found room, the CTA's minibatch rows and all its activations except the first convolution's
+  // maps sit in shared memory behind the model (indexed by the sample's place in the minibatch all the same);
+  // otherwise they stay in global scratch.
+  const bool rows_staged = p.stage_rows != 0, acts_staged = p.stage_acts != 0;
+  float* xs = reinterpret_cast<float*>(ylab + B);
+  float* sa = xs + (rows_staged ? per * rowlen : 0);
+  auto place = [&](int per_sample, int global_off) -> float* {
+    if (!acts_staged) return act + global_off;
+    float* r = sa - (ptrdiff_t)b0 * per_sample;
+    sa += per * per_sample;
+    return r;
+  };
+  const int n_q1 = D.c1 * D.p1 * D.p1, n_a2 = D.c2 * D.s2 * D.s2, n_a1 = D.c1 * D.s1 * D.s1;
+  float* a1 = act + D.a1;
+  float* q1 = place(n_q1, D.q1);
+  float* a2 = place(n_a2, D.a2);
+  float* q2 = place(D.flat, D.q2);
+  float* h1 = place(D.f1, D.h1);
+  float* h2 = place(D.f2, D.h2);
+  float* z3 = place(D.ncls, D.z3);
+  float* dz3 = place(D.ncls, D.dz3);
+  float* dh2 = place(D.f2, D.dh2);
+  float* dh1 = place(D.f1, D.dh1);
+  float* dq2 = place(D.flat, D.dq2);
+  float* dq1 = place(n_q1, D.dq1);
 
   // ---- start model: snapshot minus own update sums still in flight; U_i = 0 ----
   {
@@ -161,45 +191,55 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
       ylab[tid] = __ldg(cd.y + id);
     }
     __syncthreads();
+    if (rows_staged) {   // the rows are read 25 times over by the first convolution and its gradient: one coalesced copy first
+      for (int e = tid; e < nb * rowlen; e += kCnnThreads) xs[e] = __ldg(xrows + (size_t)idx[b0 + e / rowlen] * rowlen + e % rowlen);
+      __syncthreads();
+    }
+    // pixel (ci, y, x) of minibatch sample b (one of this CTA's)
+    auto x_at = [&](int b, int ci, int y, int x) {
+      const int at = (ci * D.side + y) * D.side + x;
+      return rows_staged ? xs[(b - b0) * rowlen + at] : __ldg(xrows + (size_t)idx[b] * rowlen + at);
+    };
 
     // ================= forward (own samples) =================
-    conv_stage(b0, nb, D.cin, D.c1, D.side, D.s1, w + D.oW1, w + D.ob1,
-               [&](int b, int ci, int y, int x) { return __ldg(xrows + (size_t)idx[b] * rowlen + (ci * D.side + y) * D.side + x); },
-               act + D.a1, act + D.q1, tid);
+    conv_stage(b0, nb, D.cin, D.c1, D.side, D.s1, w + D.oW1, w + D.ob1, x_at, a1, q1, tid);
     __syncthreads();
-    {
-      const float* q1 = act + D.q1;
-      conv_stage(b0, nb, D.c1, D.c2, D.p1, D.s2, w + D.oW2, w + D.ob2,
-                 [&](int b, int ci, int y, int x) { return q1[((size_t)(b * D.c1 + ci) * D.p1 + y) * D.p1 + x]; },
-                 act + D.a2, act + D.q2, tid);
-    }
+    conv_stage(b0, nb, D.c1, D.c2, D.p1, D.s2, w + D.oW2, w + D.ob2,
+               [&](int b, int ci, int y, int x) { return q1[((size_t)(b * D.c1 + ci) * D.p1 + y) * D.p1 + x]; }, a2, q2, tid);
     __syncthreads();
     auto dense_fwd = [&](const float* in, int K, int N, const float* Wl, const float* bl, float* out, bool relu) {
       for (int e = tid; e < nb * N; e += kCnnThreads) {
         const int j = e % N, b = b0 + e / N;
-        float z = bl[j];
+        float z0 = bl[j], z1 = 0.f, z2 = 0.f, z3v = 0.f;   // four chains: the operands come from shared memory with latency
         const float* a = in + (size_t)b * K;
-        for (int k = 0; k < K; ++k) z = fmaf(a[k], Wl[k * N + j], z);
+        int k = 0;
+        for (; k + 4 <= K; k += 4) {
+          z0 = fmaf(a[k], Wl[k * N + j], z0);
+          z1 = fmaf(a[k + 1], Wl[(k + 1) * N + j], z1);
+          z2 = fmaf(a[k + 2], Wl[(k + 2) * N + j], z2);
+          z3v = fmaf(a[k + 3], Wl[(k + 3) * N + j], z3v);
+        }
+        for (; k < K; ++k) z0 = fmaf(a[k], Wl[k * N + j], z0);
+        const float z = (z0 + z1) + (z2 + z3v);
         out[(size_t)b * N + j] = relu ? fmaxf(z, 0.f) : z;
       }
     };
-    dense_fwd(act + D.q2, D.flat, D.f1, w + D.oF1, w + D.obF1, act + D.h1, true);
+    dense_fwd(q2, D.flat, D.f1, w + D.oF1, w + D.obF1, h1, true);
     __syncthreads();
-    dense_fwd(act + D.h1, D.f1, D.f2, w + D.oF2, w + D.obF2, act + D.h2, true);
+    dense_fwd(h1, D.f1, D.f2, w + D.oF2, w + D.obF2, h2, true);
     __syncthreads();
-    dense_fwd(act + D.h2, D.f2, D.ncls, w + D.oF3, w + D.obF3, act + D.z3, false);
+    dense_fwd(h2, D.f2, D.ncls, w + D.oF3, w + D.obF3, z3, false);
     __syncthreads();
     if (tid < nb) {   // softmax cross-entropy: dZ = (p - onehot) / B
       const int b = b0 + tid;
-      const float* z = act + D.z3 + b * D.ncls;
+      const float* z = z3 + b * D.ncls;
       float m = -INFINITY;
       for (int j = 0; j < D.ncls; ++j) m = fmaxf(m, z[j]);
       float sum = 0.f;
       for (int j = 0; j < D.ncls; ++j) sum += __expf(z[j] - m);
       const float inv = 1.f / sum;
       const int y = ylab[b];
-      for (int j = 0; j < D.ncls; ++j)
-        act[D.dz3 + b * D.ncls + j] = (__expf(z[j] - m) * inv - (j == y ? 1.f : 0.f)) * invB;
+      for (int j = 0; j < D.ncls; ++j) dz3[b * D.ncls + j] = (__expf(z[j] - m) * inv - (j == y ? 1.f : 0.f)) * invB;
     }
     __syncthreads();
 
@@ -207,12 +247,14 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     // input gradient of a dense layer, gated by the ReLU of the layer below: dIn[b, i] = [in > 0] sum_j dOut[b, j] W[i, j]
     auto dense_din = [&](int e, const float* dout, int K, int N, const float* Wl, const float* in, float* din, bool gate) {
       const int i = e % K, b = b0 + e / K;
-      float s = 0.f;
+      float s0 = 0.f, s1 = 0.f;
       const float* dz = dout + (size_t)b * N;
       const float* wr = Wl + (size_t)i * N;
-      for (int j = 0; j < N; ++j) s = fmaf(dz[j], wr[j], s);
+      int j = 0;
+      for (; j + 2 <= N; j += 2) { s0 = fmaf(dz[j], wr[j], s0); s1 = fmaf(dz[j + 1], wr[j + 1], s1); }
+      if (j < N) s0 = fmaf(dz[j], wr[j], s0);
       const size_t at = (size_t)b * K + i;
-      din[at] = (!gate || in[at] > 0.f) ? s : 0.f;
+      din[at] = (!gate || in[at] > 0.f) ? s0 + s1 : 0.f;
     };
     // this CTA's share of the gradient of one dense parameter: item < K * N a weight, else a bias
     auto dense_grad = [&](int e, const float* in, const float* dout, int K, int N, int oW, int ob) {
@@ -229,15 +271,14 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
       }
     };
     // dh2 from the class layer
-    for (int e = tid; e < nb * D.f2; e += kCnnThreads)
-      dense_din(e, act + D.dz3, D.f2, D.ncls, w + D.oF3, act + D.h2, act + D.dh2, true);
+    for (int e = tid; e < nb * D.f2; e += kCnnThreads) dense_din(e, dz3, D.f2, D.ncls, w + D.oF3, h2, dh2, true);
     __syncthreads();
     // class layer gradient | dh1 through dense layer 2
     {
       const int nu = D.f2 * D.ncls + D.ncls, nd = nb * D.f1;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) dense_grad(e, act + D.h2, act + D.dz3, D.f2, D.ncls, D.oF3, D.obF3);
-        else dense_din(e - nu, act + D.dh2, D.f1, D.f2, w + D.oF2, act + D.h1, act + D.dh1, true);
+        if (e < nu) dense_grad(e, h2, dz3, D.f2, D.ncls, D.oF3, D.obF3);
+        else dense_din(e - nu, dh2, D.f1, D.f2, w + D.oF2, h1, dh1, true);
       }
     }
     __syncthreads();
@@ -245,68 +286,79 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     {
       const int nu = D.f1 * D.f2 + D.f2, nd = nb * D.flat;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) dense_grad(e, act + D.h1, act + D.dh2, D.f1, D.f2, D.oF2, D.obF2);
-        else dense_din(e - nu, act + D.dh1, D.flat, D.f1, w + D.oF1, act + D.q2, act + D.dq2, false);
+        if (e < nu) dense_grad(e, h1, dh2, D.f1, D.f2, D.oF2, D.obF2);
+        else dense_din(e - nu, dh1, D.flat, D.f1, w + D.oF1, q2, dq2, false);
       }
     }
     __syncthreads();
     // dense layer 1 gradient | dz2 = [a2 > 0] * dq2 / 4, in place over a2
     {
-      const int nu = D.flat * D.f1 + D.f1, per2 = D.c2 * D.s2 * D.s2, nd = nb * per2;
+      const int nu = D.flat * D.f1 + D.f1, nd = nb * n_a2;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
         if (e < nu) {
-          dense_grad(e, act + D.q2, act + D.dh1, D.flat, D.f1, D.oF1, D.obF1);
+          dense_grad(e, q2, dh1, D.flat, D.f1, D.oF1, D.obF1);
         } else {
-          const int k = b0 * per2 + (e - nu);
+          const int k = b0 * n_a2 + (e - nu);
           const int x = k % D.s2, y = (k / D.s2) % D.s2, bc = k / (D.s2 * D.s2);
-          const float g = act[D.dq2 + ((size_t)bc * D.p2 + (y >> 1)) * D.p2 + (x >> 1)];
-          act[D.a2 + k] = act[D.a2 + k] > 0.f ? 0.25f * g : 0.f;
+          const float g = dq2[((size_t)bc * D.p2 + (y >> 1)) * D.p2 + (x >> 1)];
+          a2[k] = a2[k] > 0.f ? 0.25f * g : 0.f;
         }
       }
     }
     __syncthreads();
-    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx]
+    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx].  Taps that fall off the map
+    // read a clamped address and count as zero, so that the loads carry no branches and issue together.
     {
-      const float* dz2 = act + D.a2;
+      const float* dz2 = a2;
       const float* W2 = w + D.oW2;
-      const int per1 = D.c1 * D.p1 * D.p1;
-      for (int e = tid; e < nb * per1; e += kCnnThreads) {
-        const int x = e % D.p1, y = (e / D.p1) % D.p1, c = (e / (D.p1 * D.p1)) % D.c1, b = b0 + e / per1;
-        float s = 0.f;
+      for (int e = tid; e < nb * n_q1; e += kCnnThreads) {
+        const int x = e % D.p1, y = (e / D.p1) % D.p1, c = (e / (D.p1 * D.p1)) % D.c1, b = b0 + e / n_q1;
+        int ro[kK], co[kK];
+        bool rok[kK], cok[kK];
+#pragma unroll
+        for (int d = 0; d < kK; ++d) {
+          const int yy = y - d, xx = x - d;
+          rok[d] = yy >= 0 && yy < D.s2; cok[d] = xx >= 0 && xx < D.s2;
+          ro[d] = min(max(yy, 0), D.s2 - 1) * D.s2; co[d] = min(max(xx, 0), D.s2 - 1);
+        }
+        float s0 = 0.f, s1 = 0.f;
         for (int c2 = 0; c2 < D.c2; ++c2) {
           const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
           const float* wk = W2 + (c2 * D.c1 + c) * (kK * kK);
 #pragma unroll
-          for (int dy = 0; dy < kK; ++dy) {
-            const int yy = y - dy;
-            if (yy < 0 || yy >= D.s2) continue;
+          for (int dy = 0; dy < kK; ++dy)
 #pragma unroll
             for (int dx = 0; dx < kK; ++dx) {
-              const int xx = x - dx;
-              if (xx >= 0 && xx < D.s2) s = fmaf(dzp[yy * D.s2 + xx], wk[dy * kK + dx], s);
+              const float v = rok[dy] && cok[dx] ? dzp[ro[dy] + co[dx]] : 0.f;
+              if ((dy * kK + dx) & 1) s1 = fmaf(v, wk[dy * kK + dx], s1);
+              else s0 = fmaf(v, wk[dy * kK + dx], s0);
             }
-          }
         }
-        act[D.dq1 + (size_t)b0 * per1 + e] = s;
+        dq1[(size_t)b0 * n_q1 + e] = s0 + s1;
       }
     }
     __syncthreads();
     // second convolution's gradient | dz1 = [a1 > 0] * dq1 / 4, in place over a1
     {
-      const int nw = D.c2 * D.c1 * kK * kK, nu = nw + D.c2, per1 = D.c1 * D.s1 * D.s1, nd = nb * per1;
-      const float* dz2 = act + D.a2;
-      const float* q1 = act + D.q1;
+      const int nw = D.c2 * D.c1 * kK * kK, nu = nw + D.c2, nd = nb * n_a1;
+      const float* dz2 = a2;
       for (int e = tid; e < nu + nd; e += kCnnThreads) {
         if (e < nw) {
           const int dx = e % kK, dy = (e / kK) % kK, c = (e / (kK * kK)) % D.c1, c2 = e / (kK * kK * D.c1);
-          float g = 0.f;
+          float g0 = 0.f, g1 = 0.f;
           for (int b = b0; b < b0 + nb; ++b) {
             const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
             const float* qp = q1 + ((size_t)(b * D.c1 + c) * D.p1 + dy) * D.p1 + dx;
-            for (int y = 0; y < D.s2; ++y)
-              for (int x = 0; x < D.s2; ++x) g = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g);
+            for (int y = 0; y < D.s2; ++y) {
+              int x = 0;
+              for (; x + 2 <= D.s2; x += 2) {
+                g0 = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g0);
+                g1 = fmaf(dzp[y * D.s2 + x + 1], qp[y * D.p1 + x + 1], g1);
+              }
+              if (x < D.s2) g0 = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g0);
+            }
           }
-          G[D.oW2 + e] = g;
+          G[D.oW2 + e] = g0 + g1;
         } else if (e < nu) {
           const int c2 = e - nw;
           float g = 0.f;
@@ -316,39 +368,51 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
           }
           G[D.ob2 + c2] = g;
         } else {
-          const int k = b0 * per1 + (e - nu);
+          const int k = b0 * n_a1 + (e - nu);
           const int x = k % D.s1, y = (k / D.s1) % D.s1, bc = k / (D.s1 * D.s1);
-          const float g = act[D.dq1 + ((size_t)bc * D.p1 + (y >> 1)) * D.p1 + (x >> 1)];
-          act[D.a1 + k] = act[D.a1 + k] > 0.f ? 0.25f * g : 0.f;
+          const float g = dq1[((size_t)bc * D.p1 + (y >> 1)) * D.p1 + (x >> 1)];
+          a1[k] = a1[k] > 0.f ? 0.25f * g : 0.f;
         }
       }
     }
     __syncthreads();
-    // first convolution's gradient: few parameters, long sums (nb * s1 * s1 terms each): a warp per parameter,
-    // lanes take the terms in turn, shuffle tree at the end
+    // First convolution's gradient: few parameters, long sums.  A warp takes one (output plane, input plane)
+    // pair: lanes across a row of the output map, every lane all 25 taps, so that a value of dz1 (global,
+    // one load per row, the rows independent of one another) meets 25 inputs from shared memory; 26
+    // shuffle trees at the end (the 25 taps and, for the first input plane, the bias).
     {
-      const int nw = D.c1 * D.cin * kK * kK, nu = nw + D.c1;
-      const float* dz1 = act + D.a1;
-      const int terms = nb * D.s1 * D.s1;
-      for (int e = warp; e < nu; e += kCnnThreads / 32) {
-        float g = 0.f;
-        if (e < nw) {
-          const int dx = e % kK, dy = (e / kK) % kK, ci = (e / (kK * kK)) % D.cin, c = e / (kK * kK * D.cin);
-          for (int k = lane; k < terms; k += 32) {
-            const int x = k % D.s1, y = (k / D.s1) % D.s1, b = b0 + k / (D.s1 * D.s1);
-            const float xv = __ldg(xrows + (size_t)idx[b] * rowlen + (ci * D.side + y + dy) * D.side + x + dx);
-            g = fmaf(dz1[((size_t)(b * D.c1 + c) * D.s1 + y) * D.s1 + x], xv, g);
-          }
-        } else {
-          const int c = e - nw;
-          for (int k = lane; k < terms; k += 32) {
-            const int r = k % (D.s1 * D.s1), b = b0 + k / (D.s1 * D.s1);
-            g += dz1[(size_t)(b * D.c1 + c) * D.s1 * D.s1 + r];
+      const float* dz1 = a1;
+      for (int e = warp; e < D.c1 * D.cin; e += kCnnThreads / 32) {
+        const int ci = e % D.cin, c = e / D.cin;
+        float g[kK * kK], gb = 0.f;
+#pragma unroll
+        for (int k = 0; k < kK * kK; ++k) g[k] = 0.f;
+        for (int b = b0; b < b0 + nb; ++b) {
+          const float* dzp = dz1 + (size_t)(b * D.c1 + c) * D.s1 * D.s1;
+          for (int x = lane; x < D.s1; x += 32) {
+#pragma unroll 4
+            for (int y = 0; y < D.s1; ++y) {
+              const float d = dzp[y * D.s1 + x];
+              gb += d;
+#pragma unroll
+              for (int dy = 0; dy < kK; ++dy)
+#pragma unroll
+                for (int dx = 0; dx < kK; ++dx) g[dy * kK + dx] = fmaf(d, x_at(b, ci, y + dy, x + dx), g[dy * kK + dx]);
+            }
           }
         }
 #pragma unroll
-        for (int m = 16; m; m >>= 1) g += __shfl_xor_sync(0xffffffffu, g, m);
-        if (lane == 0) G[e < nw ? D.oW1 + e : D.ob1 + (e - nw)] = g;
+        for (int k = 0; k < kK * kK; ++k) {
+#pragma unroll
+          for (int m = 16; m; m >>= 1) g[k] += __shfl_xor_sync(0xffffffffu, g[k], m);
+        }
+#pragma unroll
+        for (int m = 16; m; m >>= 1) gb += __shfl_xor_sync(0xffffffffu, gb, m);
+        if (lane == 0) {
+#pragma unroll
+          for (int k = 0; k < kK * kK; ++k) G[D.oW1 + (c * D.cin + ci) * (kK * kK) + k] = g[k];
+          if (ci == 0) G[D.ob1 + c] = gb;
+        }
       }
     }
     cluster_sync();   // every CTA's partial gradients are in global scratch; nobody reads the old weights any more
@@ -357,8 +421,12 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     {
       const float* G0 = act + D.total;
       for (int k = k_lo + tid; k < k_hi; k += kCnnThreads) {
+        float part[kMaxCl];
+#pragma unroll
+        for (int q = 0; q < kMaxCl; ++q) part[q] = q < nact ? G0[(size_t)q * D.Ppad + k] : 0.f;
         float g = 0.f;
-        for (int q = 0; q < nact; ++q) g += G0[(size_t)q * D.Ppad + k];
+#pragma unroll
+        for (int q = 0; q < kMaxCl; ++q) g += part[q];
         const bool bias = (k >= D.ob1 && k < D.oW2) || (k >= D.ob2 && k < D.oF1) || (k >= D.obF1 && k < D.oF2) ||
                           (k >= D.obF2 && k < D.oF3) || k >= D.obF3;   // biases take no l2 term
         const float wk = w[k];
@@ -387,6 +455,15 @@ size_t cnn_smem_bytes(const CnnShape& s) {
   const CnnDims d = make_cnn_dims(s);
   return ((size_t)((d.P + 3) & ~3) + 2 * s.batch) * sizeof(float);
 }
+// with room for the minibatch rows of one CTA of a cluster of `cl` and, if `acts`, for its small activations
+// (0 if they do not fit)
+size_t cnn_smem_bytes_staged(const CnnShape& s, uint32_t cl, bool acts) {
+  const CnnDims d = make_cnn_dims(s);
+  const size_t per = (s.batch + cl - 1) / cl;
+  const size_t extra = per * ((size_t)d.cin * d.side * d.side + (acts ? (size_t)cnn_small_acts(d) : 0)) * sizeof(float);
+  const size_t all = cnn_smem_bytes(s) + extra;
+  return all <= 227 * 1024 ? all : 0;
+}
 
 }  // namespace
 
@@ -410,8 +487,8 @@ const char* cnn_check_shape(const CnnShape& s) {
   return nullptr;
 }
 
-cudaError_t launch_cnn_rounds(const CnnLaunch& p, cudaStream_t s) {
-  if (p.r.n_tasks == 0) return cudaSuccess;
+cudaError_t launch_cnn_rounds(const CnnLaunch& p0, cudaStream_t s) {
+  if (p0.r.n_tasks == 0) return cudaSuccess;
   static int sms = 0;
   if (sms == 0) {
     int dev = 0, n = 0;
@@ -420,12 +497,17 @@ cudaError_t launch_cnn_rounds(const CnnLaunch& p, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     sms = n;
   }
-  const size_t smem = cnn_smem_bytes(p.shape);
-  cudaError_t e = cudaFuncSetAttribute(cnn_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   // CTAs per round-task: as many as the minibatch has samples and the launch leaves SMs for
   uint32_t cl = kMaxCl;
-  while (cl > 1 && (cl > p.shape.batch || p.r.n_tasks * cl > (uint32_t)sms)) cl >>= 1;
+  while (cl > 1 && (cl > p0.shape.batch || p0.r.n_tasks * cl > (uint32_t)sms)) cl >>= 1;
+  CnnLaunch p = p0;
+  size_t smem = cnn_smem_bytes_staged(p.shape, cl, true);
+  p.stage_acts = smem != 0;
+  if (!smem) smem = cnn_smem_bytes_staged(p.shape, cl, false);
+  p.stage_rows = smem != 0;
+  if (!smem) smem = cnn_smem_bytes(p.shape);
+  cudaError_t e = cudaFuncSetAttribute(cnn_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(p.r.n_tasks * cl, 1, 1);
   cfg.blockDim = dim3(kCnnThreads, 1, 1);

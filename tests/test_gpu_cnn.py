@@ -17,6 +17,8 @@ pytestmark = pytest.mark.gpu
     dict(n_rounds=4, n_clients=3, max_lag_d=workloads.NEVER_WAIT, network_delay_mean=300.0, batch=8, sched_a=8, sched_b=8,
          data=dict(total=600)),                                                                                    # own sums in flight
     dict(topology=1, n_rounds=3, n_clients=4, data=dict(total=600)),                                               # on the ring
+    dict(n_rounds=2, n_clients=40, data=dict(total=2400)),   # fuller launch: clusters of 2, rows in shared memory, activations in scratch
+    dict(n_rounds=2, n_clients=80, data=dict(total=4000)),   # one CTA per round-task, nothing staged beside the model
 ])
 def test_conv_classifier_end_to_end_and_round_U(over):
     base = dict(n_clients=4, n_rounds=4)
