@@ -107,11 +107,6 @@ __device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("m
 __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void st_cluster(const float* local, uint32_t rank, float v) {
-  uint32_t a;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(rank));
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
-}
 
 // floats of per-sample activations that may live in shared memory (everything but the first convolution's maps)
 __host__ __device__ inline int cnn_small_acts(const CnnDims& d) {
@@ -256,85 +251,82 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
       const size_t at = (size_t)b * K + i;
       din[at] = (!gate || in[at] > 0.f) ? s0 + s1 : 0.f;
     };
-    // this CTA's share of the gradient of one dense parameter: item < K * N a weight, else a bias
-    auto dense_grad = [&](int e, const float* in, const float* dout, int K, int N, int oW, int ob) {
-      if (e < K * N) {
-        const int j = e % N, i = e / N;
-        float g = 0.f;
-        for (int b = b0; b < b0 + nb; ++b) g = fmaf(in[(size_t)b * K + i], dout[(size_t)b * N + j], g);
-        G[oW + e] = g;
-      } else {
-        const int j = e - K * N;
-        float g = 0.f;
-        for (int b = b0; b < b0 + nb; ++b) g += dout[(size_t)b * N + j];
-        G[ob + j] = g;
-      }
+    // This CTA's share of the gradient of a dense layer: warps `wfirst`, `wfirst + wstep`, ... of the CTA take the
+    // input rows in turn (row K is the bias), lanes run across the outputs - no index arithmetic per parameter.
+    auto dense_grad = [&](int wfirst, int wstep, const float* in, const float* dout, int K, int N, int oW, int ob) {
+      for (int i = wfirst; i <= K; i += wstep)
+        for (int j = lane; j < N; j += 32) {
+          float g = 0.f;
+          if (i < K) {
+            for (int b = b0; b < b0 + nb; ++b) g = fmaf(in[(size_t)b * K + i], dout[(size_t)b * N + j], g);
+            G[oW + i * N + j] = g;
+          } else {
+            for (int b = b0; b < b0 + nb; ++b) g += dout[(size_t)b * N + j];
+            G[ob + j] = g;
+          }
+        }
     };
     // dh2 from the class layer
     for (int e = tid; e < nb * D.f2; e += kCnnThreads) dense_din(e, dz3, D.f2, D.ncls, w + D.oF3, h2, dh2, true);
     __syncthreads();
-    // class layer gradient | dh1 through dense layer 2
-    {
-      const int nu = D.f2 * D.ncls + D.ncls, nd = nb * D.f1;
-      for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) dense_grad(e, h2, dz3, D.f2, D.ncls, D.oF3, D.obF3);
-        else dense_din(e - nu, dh2, D.f1, D.f2, w + D.oF2, h1, dh1, true);
-      }
+    // class layer gradient (warps 0-3) | dh1 through dense layer 2 (the other warps)
+    constexpr int kW = kCnnThreads / 32, kGradW = 4;
+    if (warp < kGradW) dense_grad(warp, kGradW, h2, dz3, D.f2, D.ncls, D.oF3, D.obF3);
+    else for (int e = tid - 32 * kGradW; e < nb * D.f1; e += kCnnThreads - 32 * kGradW) dense_din(e, dh2, D.f1, D.f2, w + D.oF2, h1, dh1, true);
+    __syncthreads();
+    // dense layer 2 gradient (first half of the warps) | dq2 through dense layer 1 (the pooled maps carry no ReLU of their own)
+    if (warp < kW / 2) dense_grad(warp, kW / 2, h1, dh2, D.f1, D.f2, D.oF2, D.obF2);
+    else for (int e = tid - kCnnThreads / 2; e < nb * D.flat; e += kCnnThreads / 2) dense_din(e, dh1, D.flat, D.f1, w + D.oF1, q2, dq2, false);
+    __syncthreads();
+    // dense layer 1 gradient (all warps), then dz2 = [a2 > 0] * dq2 / 4, in place over a2
+    dense_grad(warp, kW, q2, dh1, D.flat, D.f1, D.oF1, D.obF1);
+    for (int e = tid; e < nb * n_a2; e += kCnnThreads) {
+      const int k = b0 * n_a2 + e;
+      const int x = k % D.s2, y = (k / D.s2) % D.s2, bc = k / (D.s2 * D.s2);
+      const float g = dq2[((size_t)bc * D.p2 + (y >> 1)) * D.p2 + (x >> 1)];
+      a2[k] = a2[k] > 0.f ? 0.25f * g : 0.f;
     }
     __syncthreads();
-    // dense layer 2 gradient | dq2 through dense layer 1 (the pooled maps carry no ReLU of their own)
-    {
-      const int nu = D.f1 * D.f2 + D.f2, nd = nb * D.flat;
-      for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) dense_grad(e, h1, dh2, D.f1, D.f2, D.oF2, D.obF2);
-        else dense_din(e - nu, dh1, D.flat, D.f1, w + D.oF1, q2, dq2, false);
-      }
-    }
-    __syncthreads();
-    // dense layer 1 gradient | dz2 = [a2 > 0] * dq2 / 4, in place over a2
-    {
-      const int nu = D.flat * D.f1 + D.f1, nd = nb * n_a2;
-      for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nu) {
-          dense_grad(e, q2, dh1, D.flat, D.f1, D.oF1, D.obF1);
-        } else {
-          const int k = b0 * n_a2 + (e - nu);
-          const int x = k % D.s2, y = (k / D.s2) % D.s2, bc = k / (D.s2 * D.s2);
-          const float g = dq2[((size_t)bc * D.p2 + (y >> 1)) * D.p2 + (x >> 1)];
-          a2[k] = a2[k] > 0.f ? 0.25f * g : 0.f;
-        }
-      }
-    }
-    __syncthreads();
-    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx].  Taps that fall off the map
-    // read a clamped address and count as zero, so that the loads carry no branches and issue together.
+    // dq1[b, c1, y, x] = sum_{c2, dy, dx} dz2[b, c2, y - dy, x - dx] W2[c2, c1, dy, dx].  A work item is four
+    // neighbouring outputs of a row: per (c2, dy) it reads the eight values of dz2's row y - dy that they touch
+    // (off the map: a clamped address, counted as zero) and the five weights, and does twenty multiply-adds;
+    // rows off the map are skipped whole.
     {
       const float* dz2 = a2;
       const float* W2 = w + D.oW2;
-      for (int e = tid; e < nb * n_q1; e += kCnnThreads) {
-        const int x = e % D.p1, y = (e / D.p1) % D.p1, c = (e / (D.p1 * D.p1)) % D.c1, b = b0 + e / n_q1;
-        int ro[kK], co[kK];
-        bool rok[kK], cok[kK];
+      const int xq = (D.p1 + 3) / 4, items = nb * D.c1 * D.p1 * xq;
+      for (int e = tid; e < items; e += kCnnThreads) {
+        const int x0 = (e % xq) * 4, y = (e / xq) % D.p1, c = (e / (xq * D.p1)) % D.c1, b = b0 + e / (xq * D.p1 * D.c1);
+        int co[8];
+        bool cok[8];
 #pragma unroll
-        for (int d = 0; d < kK; ++d) {
-          const int yy = y - d, xx = x - d;
-          rok[d] = yy >= 0 && yy < D.s2; cok[d] = xx >= 0 && xx < D.s2;
-          ro[d] = min(max(yy, 0), D.s2 - 1) * D.s2; co[d] = min(max(xx, 0), D.s2 - 1);
+        for (int k = 0; k < 8; ++k) {   // column x0 - 4 + k of dz2
+          const int xx = x0 - 4 + k;
+          cok[k] = xx >= 0 && xx < D.s2;
+          co[k] = min(max(xx, 0), D.s2 - 1);
         }
-        float s0 = 0.f, s1 = 0.f;
+        float o[4] = {0.f, 0.f, 0.f, 0.f};
         for (int c2 = 0; c2 < D.c2; ++c2) {
           const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
           const float* wk = W2 + (c2 * D.c1 + c) * (kK * kK);
 #pragma unroll
-          for (int dy = 0; dy < kK; ++dy)
+          for (int dy = 0; dy < kK; ++dy) {
+            const int yy = y - dy;
+            if (yy < 0 || yy >= D.s2) continue;
+            float v[8], wv[kK];
 #pragma unroll
-            for (int dx = 0; dx < kK; ++dx) {
-              const float v = rok[dy] && cok[dx] ? dzp[ro[dy] + co[dx]] : 0.f;
-              if ((dy * kK + dx) & 1) s1 = fmaf(v, wk[dy * kK + dx], s1);
-              else s0 = fmaf(v, wk[dy * kK + dx], s0);
-            }
+            for (int k = 0; k < 8; ++k) v[k] = cok[k] ? dzp[yy * D.s2 + co[k]] : 0.f;
+#pragma unroll
+            for (int dx = 0; dx < kK; ++dx) wv[dx] = wk[dy * kK + dx];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int dx = 0; dx < kK; ++dx) o[i] = fmaf(v[4 + i - dx], wv[dx], o[i]);   // output x0 + i takes column x0 + i - dx
+          }
         }
-        dq1[(size_t)b0 * n_q1 + e] = s0 + s1;
+        float* out = dq1 + ((size_t)(b * D.c1 + c) * D.p1 + y) * D.p1 + x0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) if (x0 + i < D.p1) out[i] = o[i];
       }
     }
     __syncthreads();
@@ -420,6 +412,10 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     // ================= this CTA's slice: g = sum over the CTAs in rank order; w -= eta (g + lambda w), U += g + lambda w =================
     {
       const float* G0 = act + D.total;
+      uint32_t peer_w[kMaxCl];   // the model's shared-memory address in every CTA of the cluster
+#pragma unroll
+      for (int q = 0; q < kMaxCl; ++q)
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer_w[q]) : "r"((uint32_t)__cvta_generic_to_shared(w)), "r"((uint32_t)(q < CL ? q : 0)));
       for (int k = k_lo + tid; k < k_hi; k += kCnnThreads) {
         float part[kMaxCl];
 #pragma unroll
@@ -433,7 +429,9 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
         const float gt = bias ? g : fmaf(lambda, wk, g);
         const float wn = fmaf(-eta, gt, wk);
         Urow[k] += gt;
-        for (int q = 0; q < CL; ++q) st_cluster(w + k, (uint32_t)q, wn);
+#pragma unroll
+        for (int q = 0; q < kMaxCl; ++q)
+          if (q < CL) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_w[q] + 4u * (uint32_t)k), "f"(wn) : "memory");
       }
     }
     cluster_sync();   // the new weights are in every CTA's copy
