@@ -239,17 +239,22 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     __syncthreads();
 
     // ================= backward (own samples, old weights throughout) =================
-    // input gradient of a dense layer, gated by the ReLU of the layer below: dIn[b, i] = [in > 0] sum_j dOut[b, j] W[i, j]
-    auto dense_din = [&](int e, const float* dout, int K, int N, const float* Wl, const float* in, float* din, bool gate) {
-      const int i = e % K, b = b0 + e / K;
-      float s0 = 0.f, s1 = 0.f;
-      const float* dz = dout + (size_t)b * N;
-      const float* wr = Wl + (size_t)i * N;
-      int j = 0;
-      for (; j + 2 <= N; j += 2) { s0 = fmaf(dz[j], wr[j], s0); s1 = fmaf(dz[j + 1], wr[j + 1], s1); }
-      if (j < N) s0 = fmaf(dz[j], wr[j], s0);
-      const size_t at = (size_t)b * K + i;
-      din[at] = (!gate || in[at] > 0.f) ? s0 + s1 : 0.f;
+    constexpr int kW = kCnnThreads / 32, kGradW = 4;
+    // Input gradient of a dense layer, gated by the ReLU of the layer below: dIn[b, i] = [in > 0] sum_j dOut[b, j] W[i, j].
+    // Warps `wfirst`, `wfirst + wstep`, ... take the (sample, input) pairs in turn; lanes run along row i of W
+    // (contiguous in shared memory) and meet in a shuffle tree.
+    auto dense_din = [&](int wfirst, int wstep, const float* dout, int K, int N, const float* Wl, const float* in, float* din, bool gate) {
+      for (int e = wfirst; e < nb * K; e += wstep) {
+        const int i = e % K, b = b0 + e / K;
+        const float* dz = dout + (size_t)b * N;
+        const float* wr = Wl + (size_t)i * N;
+        float s = 0.f;
+        for (int j = lane; j < N; j += 32) s = fmaf(dz[j], wr[j], s);
+#pragma unroll
+        for (int m = 16; m; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
+        const size_t at = (size_t)b * K + i;
+        if (lane == 0) din[at] = (!gate || in[at] > 0.f) ? s : 0.f;
+      }
     };
     // This CTA's share of the gradient of a dense layer: warps `wfirst`, `wfirst + wstep`, ... of the CTA take the
     // input rows in turn (row K is the bias), lanes run across the outputs - no index arithmetic per parameter.
@@ -267,16 +272,15 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
         }
     };
     // dh2 from the class layer
-    for (int e = tid; e < nb * D.f2; e += kCnnThreads) dense_din(e, dz3, D.f2, D.ncls, w + D.oF3, h2, dh2, true);
+    dense_din(warp, kCnnThreads / 32, dz3, D.f2, D.ncls, w + D.oF3, h2, dh2, true);
     __syncthreads();
     // class layer gradient (warps 0-3) | dh1 through dense layer 2 (the other warps)
-    constexpr int kW = kCnnThreads / 32, kGradW = 4;
     if (warp < kGradW) dense_grad(warp, kGradW, h2, dz3, D.f2, D.ncls, D.oF3, D.obF3);
-    else for (int e = tid - 32 * kGradW; e < nb * D.f1; e += kCnnThreads - 32 * kGradW) dense_din(e, dh2, D.f1, D.f2, w + D.oF2, h1, dh1, true);
+    else dense_din(warp - kGradW, kW - kGradW, dh2, D.f1, D.f2, w + D.oF2, h1, dh1, true);
     __syncthreads();
     // dense layer 2 gradient (first half of the warps) | dq2 through dense layer 1 (the pooled maps carry no ReLU of their own)
     if (warp < kW / 2) dense_grad(warp, kW / 2, h1, dh2, D.f1, D.f2, D.oF2, D.obF2);
-    else for (int e = tid - kCnnThreads / 2; e < nb * D.flat; e += kCnnThreads / 2) dense_din(e, dh1, D.flat, D.f1, w + D.oF1, q2, dq2, false);
+    else dense_din(warp - kW / 2, kW / 2, dh1, D.flat, D.f1, w + D.oF1, q2, dq2, false);
     __syncthreads();
     // dense layer 1 gradient (all warps), then dz2 = [a2 > 0] * dq2 / 4, in place over a2
     dense_grad(warp, kW, q2, dh1, D.flat, D.f1, D.oF1, D.obF1);
@@ -330,29 +334,34 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
       }
     }
     __syncthreads();
-    // second convolution's gradient | dz1 = [a1 > 0] * dq1 / 4, in place over a1
+    // Second convolution's gradient.  A work item is one kernel row (c2, c, dy): its five taps share every value of
+    // dz2 they meet, and the input row slides through a five-register window (two loads per five multiply-adds).
+    // Then the bias gradients, and dz1 = [a1 > 0] * dq1 / 4 in place over a1.
     {
-      const int nw = D.c2 * D.c1 * kK * kK, nu = nw + D.c2, nd = nb * n_a1;
+      const int nrow = D.c2 * D.c1 * kK, nd = nb * n_a1;
       const float* dz2 = a2;
-      for (int e = tid; e < nu + nd; e += kCnnThreads) {
-        if (e < nw) {
-          const int dx = e % kK, dy = (e / kK) % kK, c = (e / (kK * kK)) % D.c1, c2 = e / (kK * kK * D.c1);
-          float g0 = 0.f, g1 = 0.f;
+      for (int e = tid; e < nrow + D.c2 + nd; e += kCnnThreads) {
+        if (e < nrow) {
+          const int dy = e % kK, c = (e / kK) % D.c1, c2 = e / (kK * D.c1);
+          float g[kK] = {0.f, 0.f, 0.f, 0.f, 0.f};
           for (int b = b0; b < b0 + nb; ++b) {
             const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
-            const float* qp = q1 + ((size_t)(b * D.c1 + c) * D.p1 + dy) * D.p1 + dx;
+            const float* qp = q1 + ((size_t)(b * D.c1 + c) * D.p1 + dy) * D.p1;
             for (int y = 0; y < D.s2; ++y) {
-              int x = 0;
-              for (; x + 2 <= D.s2; x += 2) {
-                g0 = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g0);
-                g1 = fmaf(dzp[y * D.s2 + x + 1], qp[y * D.p1 + x + 1], g1);
+              const float* qr = qp + y * D.p1;
+              float q0 = qr[0], q1v = qr[1], q2v = qr[2], q3v = qr[3];
+              for (int x = 0; x < D.s2; ++x) {
+                const float d = dzp[y * D.s2 + x], q4v = qr[x + 4];
+                g[0] = fmaf(d, q0, g[0]); g[1] = fmaf(d, q1v, g[1]); g[2] = fmaf(d, q2v, g[2]);
+                g[3] = fmaf(d, q3v, g[3]); g[4] = fmaf(d, q4v, g[4]);
+                q0 = q1v; q1v = q2v; q2v = q3v; q3v = q4v;
               }
-              if (x < D.s2) g0 = fmaf(dzp[y * D.s2 + x], qp[y * D.p1 + x], g0);
             }
           }
-          G[D.oW2 + e] = g0 + g1;
-        } else if (e < nu) {
-          const int c2 = e - nw;
+#pragma unroll
+          for (int dx = 0; dx < kK; ++dx) G[D.oW2 + e * kK + dx] = g[dx];
+        } else if (e < nrow + D.c2) {
+          const int c2 = e - nrow;
           float g = 0.f;
           for (int b = b0; b < b0 + nb; ++b) {
             const float* dzp = dz2 + (size_t)(b * D.c2 + c2) * D.s2 * D.s2;
@@ -360,7 +369,7 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
           }
           G[D.ob2 + c2] = g;
         } else {
-          const int k = b0 * n_a1 + (e - nu);
+          const int k = b0 * n_a1 + (e - nrow - D.c2);
           const int x = k % D.s1, y = (k / D.s1) % D.s1, bc = k / (D.s1 * D.s1);
           const float g = dq1[((size_t)bc * D.p1 + (y >> 1)) * D.p1 + (x >> 1)];
           a1[k] = a1[k] > 0.f ? 0.25f * g : 0.f;
@@ -381,15 +390,18 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
         for (int k = 0; k < kK * kK; ++k) g[k] = 0.f;
         for (int b = b0; b < b0 + nb; ++b) {
           const float* dzp = dz1 + (size_t)(b * D.c1 + c) * D.s1 * D.s1;
+          // input plane ci of sample b: shared memory if the rows were staged, else the client's data
+          const float* xp = (rows_staged ? xs + (b - b0) * rowlen : xrows + (size_t)idx[b] * rowlen) + ci * D.side * D.side;
           for (int x = lane; x < D.s1; x += 32) {
-#pragma unroll 4
+#pragma unroll 2
             for (int y = 0; y < D.s1; ++y) {
               const float d = dzp[y * D.s1 + x];
+              const float* xr = xp + y * D.side + x;
               gb += d;
 #pragma unroll
               for (int dy = 0; dy < kK; ++dy)
 #pragma unroll
-                for (int dx = 0; dx < kK; ++dx) g[dy * kK + dx] = fmaf(d, x_at(b, ci, y + dy, x + dx), g[dy * kK + dx]);
+                for (int dx = 0; dx < kK; ++dx) g[dy * kK + dx] = fmaf(d, xr[dy * D.side + dx], g[dy * kK + dx]);
             }
           }
         }
