@@ -35,7 +35,7 @@ struct CnnDims {
   int a1, q1, a2, q2, h1, h2, z3, dz3, dh2, dh1, dq2, dq1, total;
 };
 
-__host__ __device__ inline CnnDims make_cnn_dims(const CnnShape& s) {
+__host__ __device__ constexpr CnnDims make_cnn_dims(const CnnShape& s) {
   CnnDims d{};
   d.side = (int)s.dims[0]; d.cin = (int)s.dims[1]; d.c1 = (int)s.dims[2]; d.c2 = (int)s.dims[3];
   d.f1 = (int)s.dims[4]; d.f2 = (int)s.dims[5]; d.ncls = (int)s.dims[6];
@@ -109,18 +109,26 @@ __device__ __forceinline__ void cluster_sync() {
 }
 
 // floats of per-sample activations that may live in shared memory (everything but the first convolution's maps)
-__host__ __device__ inline int cnn_small_acts(const CnnDims& d) {
+__host__ __device__ constexpr int cnn_small_acts(const CnnDims& d) {
   return 2 * d.c1 * d.p1 * d.p1 + d.c2 * d.s2 * d.s2 + 2 * d.flat + 2 * d.f1 + 2 * d.f2 + 2 * d.ncls;
 }
 
+// The shape the paper trains on its 28x28 sets, minibatch 16 on a cluster of 8: with every extent a compile-time
+// constant the index arithmetic folds and the short loops unroll (the general instance executes 34 K instructions
+// per thread and iteration, most of them divisions by run-time extents and 64-bit address arithmetic).
+constexpr CnnShape kLeNetShape = {{28, 1, 6, 16, 120, 84, 10, 0}, 16};
+
+// kFixed: kLeNetShape on a cluster of 8, rows and activations staged; otherwise everything is read from the launch.
+template <bool kFixed>
 __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) {
   extern __shared__ __align__(16) float smem[];
-  const int CL = (int)cluster_size(), rank = (int)cluster_rank();
+  const int CL = kFixed ? kMaxCl : (int)cluster_size(), rank = (int)cluster_rank();
   const int task = blockIdx.x / CL;
   const TaskDesc t = p.r.tasks[p.r.task_begin + task];
   if (!debug_task_ok(p.r, t)) return;   // debug checks only: rows and slots in range, else flag and skip (the whole cluster alike)
-  const CnnDims D = make_cnn_dims(p.shape);
-  const int B = (int)p.shape.batch;
+  constexpr CnnDims kFixedDims = make_cnn_dims(kLeNetShape);
+  const CnnDims D = kFixed ? kFixedDims : make_cnn_dims(p.shape);
+  const int B = kFixed ? (int)kLeNetShape.batch : (int)p.shape.batch;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   float* w = smem;                                     // the client's model, whole round, one copy per CTA
   int* idx = reinterpret_cast<int*>(smem + ((D.P + 3) & ~3));
@@ -135,13 +143,13 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
   float* Urow = p.r.U + (size_t)t.u_row * p.r.stride;
   // this CTA's samples of the minibatch, its row of gradient partials, its slice of the parameters
   const int per = (B + CL - 1) / CL, nact = (B + per - 1) / per;
-  const int b0 = min(B, rank * per), nb = min(B, b0 + per) - b0;
+  const int b0 = kFixed ? rank * per : min(B, rank * per), nb = kFixed ? per : min(B, b0 + per) - b0;   // kFixed: 16 = 8 x 2
   float* G = act + D.total + (size_t)rank * D.Ppad;
   const int slice = (D.P + CL - 1) / CL, k_lo = min(D.P, rank * slice), k_hi = min(D.P, k_lo + slice);
   // Where the launch found room, the CTA's minibatch rows and all its activations except the first convolution's
   // maps sit in shared memory behind the model (indexed by the sample's place in the minibatch all the same);
   // otherwise they stay in global scratch.
-  const bool rows_staged = p.stage_rows != 0, acts_staged = p.stage_acts != 0;
+  const bool rows_staged = kFixed || p.stage_rows != 0, acts_staged = kFixed || p.stage_acts != 0;
   float* xs = reinterpret_cast<float*>(ylab + B);
   float* sa = xs + (rows_staged ? per * rowlen : 0);
   auto place = [&](int per_sample, int global_off) -> float* {
@@ -516,7 +524,9 @@ cudaError_t launch_cnn_rounds(const CnnLaunch& p0, cudaStream_t s) {
   if (!smem) smem = cnn_smem_bytes_staged(p.shape, cl, false);
   p.stage_rows = smem != 0;
   if (!smem) smem = cnn_smem_bytes(p.shape);
-  cudaError_t e = cudaFuncSetAttribute(cnn_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  bool fixed = cl == kMaxCl && p.stage_acts && p.shape.batch == kLeNetShape.batch;
+  for (int i = 0; i < 7; ++i) fixed = fixed && p.shape.dims[i] == kLeNetShape.dims[i];
+  cudaError_t e = cudaFuncSetAttribute(fixed ? cnn_round_kernel<true> : cnn_round_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(p.r.n_tasks * cl, 1, 1);
@@ -530,7 +540,7 @@ cudaError_t launch_cnn_rounds(const CnnLaunch& p0, cudaStream_t s) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, cnn_round_kernel, p);
+  return fixed ? cudaLaunchKernelEx(&cfg, cnn_round_kernel<true>, p) : cudaLaunchKernelEx(&cfg, cnn_round_kernel<false>, p);
 }
 
 }  // namespace aet
