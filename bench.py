@@ -57,7 +57,7 @@ MIN_TIMED_S = 2.0           # short passes are repeated inside a step until the 
 # Set an entry to None when its kernel changes after the counters were taken.
 TRAFFIC_RATIO = {
     "cfg2": (20.505344 / 21.1008, "profiles/lr_block_kernel_cfg2.md"),
-    "cfg5": (48.25 / 51.94816, "profiles/lr_tc_kernel_cfg5_512clients.md"),
+    "cfg5": (48.44 / 51.94816, "profiles/lr_tc_kernel_cfg5_512clients.md"),
 }
 
 
