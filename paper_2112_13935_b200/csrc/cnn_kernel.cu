@@ -267,6 +267,23 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
     // This CTA's share of the gradient of a dense layer: warps `wfirst`, `wfirst + wstep`, ... of the CTA take the
     // input rows in turn (row K is the bias), lanes run across the outputs - no index arithmetic per parameter.
     auto dense_grad = [&](int wfirst, int wstep, const float* in, const float* dout, int K, int N, int oW, int ob) {
+      if (nb <= 4) {
+        // few samples per CTA: a lane keeps its column of dOut in registers and walks the rows
+        for (int j = lane; j < N; j += 32) {
+          float d[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) d[q] = q < nb ? dout[(size_t)(b0 + q) * N + j] : 0.f;
+          for (int i = wfirst; i < K; i += wstep) {
+            float g = 0.f;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              if (q < nb) g = fmaf(in[(size_t)(b0 + q) * K + i], d[q], g);
+            G[oW + i * N + j] = g;
+          }
+          if (wfirst == K % wstep) G[ob + j] = ((d[0] + d[1]) + d[2]) + d[3];   // the bias row, by the warp whose turn it would be
+        }
+        return;
+      }
       for (int i = wfirst; i <= K; i += wstep)
         for (int j = lane; j < N; j += 32) {
           float g = 0.f;
@@ -436,22 +453,34 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
 #pragma unroll
       for (int q = 0; q < kMaxCl; ++q)
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer_w[q]) : "r"((uint32_t)__cvta_generic_to_shared(w)), "r"((uint32_t)(q < CL ? q : 0)));
-      for (int k = k_lo + tid; k < k_hi; k += kCnnThreads) {
-        float part[kMaxCl];
+      // four parameters per thread and trip, so that 32 loads of partials and 4 of U are in flight at once
+      constexpr int kTrip = 4;
+      for (int kb = k_lo + tid; kb < k_hi; kb += kTrip * kCnnThreads) {
+        float part[kTrip][kMaxCl], uold[kTrip];
 #pragma unroll
-        for (int q = 0; q < kMaxCl; ++q) part[q] = q < nact ? G0[(size_t)q * D.Ppad + k] : 0.f;
-        float g = 0.f;
+        for (int r = 0; r < kTrip; ++r) {
+          const int k = kb + r * kCnnThreads;
 #pragma unroll
-        for (int q = 0; q < kMaxCl; ++q) g += part[q];
-        const bool bias = (k >= D.ob1 && k < D.oW2) || (k >= D.ob2 && k < D.oF1) || (k >= D.obF1 && k < D.oF2) ||
-                          (k >= D.obF2 && k < D.oF3) || k >= D.obF3;   // biases take no l2 term
-        const float wk = w[k];
-        const float gt = bias ? g : fmaf(lambda, wk, g);
-        const float wn = fmaf(-eta, gt, wk);
-        Urow[k] += gt;
+          for (int q = 0; q < kMaxCl; ++q) part[r][q] = (k < k_hi && q < nact) ? G0[(size_t)q * D.Ppad + k] : 0.f;
+          uold[r] = k < k_hi ? Urow[k] : 0.f;
+        }
 #pragma unroll
-        for (int q = 0; q < kMaxCl; ++q)
-          if (q < CL) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_w[q] + 4u * (uint32_t)k), "f"(wn) : "memory");
+        for (int r = 0; r < kTrip; ++r) {
+          const int k = kb + r * kCnnThreads;
+          if (k >= k_hi) break;
+          float g = 0.f;
+#pragma unroll
+          for (int q = 0; q < kMaxCl; ++q) g += part[r][q];
+          const bool bias = (k >= D.ob1 && k < D.oW2) || (k >= D.ob2 && k < D.oF1) || (k >= D.obF1 && k < D.oF2) ||
+                            (k >= D.obF2 && k < D.oF3) || k >= D.obF3;   // biases take no l2 term
+          const float wk = w[k];
+          const float gt = bias ? g : fmaf(lambda, wk, g);
+          const float wn = fmaf(-eta, gt, wk);
+          Urow[k] = uold[r] + gt;
+#pragma unroll
+          for (int q = 0; q < kMaxCl; ++q)
+            if (q < CL) asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(peer_w[q] + 4u * (uint32_t)k), "f"(wn) : "memory");
+        }
       }
     }
     cluster_sync();   // the new weights are in every CTA's copy
