@@ -252,22 +252,24 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       }
       return w;
     };
-    // W0 and W1 in work-row order (destination pieces in turn: contiguous stores, strided 16-byte loads); of a pair,
-    // each CTA the blocks it will own
-    for (size_t e4 = tid; e4 < (size_t)D0 * kH0 / 4 / NR; e4 += kSThreads) {
-      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 15), own = (int)(e4 >> 11);
-      const int half = own & 1, hh = NR == 1 ? (own >> 1) & 1 : rank, c = NR == 1 ? own >> 2 : own >> 1;
-      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + (e4 & 2047);
-      const size_t j = oW0 + (size_t)(c * kCh + r) * kH0 + hh * 128 + half * 64 + 4 * k;
+    // W0 and W1 into work-row order.  The walk is in the natural order (a warp takes 512 contiguous bytes of a row:
+    // whole lines of the snapshot, of the sums in flight and of U), the work row takes the scattered 16-byte stores;
+    // of a pair, each CTA the columns (W0) or rows (W1) it will own.
+    constexpr int kColQ = kH0 / 4 / NR;   // float4 columns of W0 a CTA owns
+    for (size_t e4 = tid; e4 < (size_t)D0 * kColQ; e4 += kSThreads) {
+      const int i = (int)(e4 / kColQ), q = (int)(e4 % kColQ) + (NR == 2 ? rank * kColQ : 0);   // row, float4 column
+      const int c = i >> 7, r = i & 127, hh = q >> 5, half = (q >> 4) & 1, k = q & 15;
+      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + ((size_t)k << 7) + r;
+      const size_t j = oW0 + (size_t)i * kH0 + 4 * q;
       const float4 w = start4(j);
       *reinterpret_cast<float4*>(work + oW0 + 4 * d4) = w;
       *reinterpret_cast<float4*>(Urow + j) = w;
     }
     for (size_t e4 = tid; e4 < (size_t)kH0 * kH1 / 4 / NR; e4 += kSThreads) {
-      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 7), own = (int)(e4 >> 10);
-      const int g32 = own & 3, tl = NR == 1 ? own >> 2 : rank;
-      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + (e4 & 1023);
-      const size_t j = oW1 + (size_t)(tl * 128 + r) * kH1 + g32 * 32 + 4 * k;
+      const int i = (int)(e4 / (kH1 / 4)) + (NR == 2 ? rank * 128 : 0), q = (int)(e4 % (kH1 / 4));
+      const int tl = i >> 7, r = i & 127, g32 = q >> 3, k = q & 7;
+      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + ((size_t)k << 7) + r;
+      const size_t j = oW1 + (size_t)i * kH1 + 4 * q;
       const float4 w = start4(j);
       *reinterpret_cast<float4*>(work + oW1 + 4 * d4) = w;
       *reinterpret_cast<float4*>(Urow + j) = w;
@@ -746,17 +748,18 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
       *reinterpret_cast<float4*>(Urow + j) = make_float4((a.x - w.x) * inv_eta, (a.y - w.y) * inv_eta, (a.z - w.z) * inv_eta, (a.w - w.w) * inv_eta);
       if (wend) *reinterpret_cast<float4*>(wend + j) = w;
     };
-    for (size_t e4 = tid; e4 < (size_t)D0 * kH0 / 4 / NR; e4 += kSThreads) {
-      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 15), own = (int)(e4 >> 11);
-      const int half = own & 1, hh = NR == 1 ? (own >> 1) & 1 : rank, c = NR == 1 ? own >> 2 : own >> 1;
-      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + (e4 & 2047);
-      finish4(oW0 + (size_t)(c * kCh + r) * kH0 + hh * 128 + half * 64 + 4 * k, *reinterpret_cast<const float4*>(work + oW0 + 4 * d4));
+    constexpr int kColQ = kH0 / 4 / NR;
+    for (size_t e4 = tid; e4 < (size_t)D0 * kColQ; e4 += kSThreads) {   // natural order, as at the start
+      const int i = (int)(e4 / kColQ), q = (int)(e4 % kColQ) + (NR == 2 ? rank * kColQ : 0);
+      const int c = i >> 7, r = i & 127, hh = q >> 5, half = (q >> 4) & 1, k = q & 15;
+      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + ((size_t)k << 7) + r;
+      finish4(oW0 + (size_t)i * kH0 + 4 * q, *reinterpret_cast<const float4*>(work + oW0 + 4 * d4));
     }
     for (size_t e4 = tid; e4 < (size_t)kH0 * kH1 / 4 / NR; e4 += kSThreads) {
-      const int r = (int)(e4 & 127), k = (int)((e4 >> 7) & 7), own = (int)(e4 >> 10);
-      const int g32 = own & 3, tl = NR == 1 ? own >> 2 : rank;
-      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + (e4 & 1023);
-      finish4(oW1 + (size_t)(tl * 128 + r) * kH1 + g32 * 32 + 4 * k, *reinterpret_cast<const float4*>(work + oW1 + 4 * d4));
+      const int i = (int)(e4 / (kH1 / 4)) + (NR == 2 ? rank * 128 : 0), q = (int)(e4 % (kH1 / 4));
+      const int tl = i >> 7, r = i & 127, g32 = q >> 3, k = q & 7;
+      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + ((size_t)k << 7) + r;
+      finish4(oW1 + (size_t)i * kH1 + 4 * q, *reinterpret_cast<const float4*>(work + oW1 + 4 * d4));
     }
     // the narrow parameters: identical in both CTAs of a pair except the first bias, of which each holds its half
     for (int j = tid; j < kH0 + kH1 + kH1 * C + C; j += kSThreads) {
