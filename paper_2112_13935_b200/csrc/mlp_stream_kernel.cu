@@ -243,37 +243,57 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
   // ---- start model: snapshot minus own update sums still in flight; rows of U of the wide layers keep w_start ----
   {
     const float* snap = p.r.snaps + (size_t)t.snap_slot * p.r.stride;
-    auto start4 = [&](size_t j) {   // four consecutive parameters from natural index j
-      float4 w = *reinterpret_cast<const float4*>(snap + j);
-      for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
-        const InflightRef ref = p.r.inflight[t.inflight_off + f];
-        const float4 u = *reinterpret_cast<const float4*>(p.r.U + (size_t)ref.row * p.r.stride + j);
-        w.x = fmaf(-ref.eta, u.x, w.x); w.y = fmaf(-ref.eta, u.y, w.y); w.z = fmaf(-ref.eta, u.z, w.z); w.w = fmaf(-ref.eta, u.w, w.w);
+    // Eight 16-byte pieces per thread and trip: all loads of a trip (snapshot, then each sum in flight) are issued
+    // before its first store, so that a thread has eight lines on their way instead of one load - store chain
+    // (the compiler cannot move a load above a store here: the arrays may alias for all it knows).
+    constexpr int kTrip = 8;
+    // `where(e4, j, d4)` maps the e4-th piece of this CTA's share to its natural float index j and its work-row piece d4
+    auto start_range = [&](size_t total, size_t o_layer, auto where) {
+      for (size_t base = tid; base < total; base += (size_t)kTrip * kSThreads) {
+        float4 w[kTrip];
+        size_t jj[kTrip], dd[kTrip];
+#pragma unroll
+        for (int q = 0; q < kTrip; ++q) {
+          const size_t e4 = base + (size_t)q * kSThreads;
+          where(e4 < total ? e4 : 0, jj[q], dd[q]);
+          w[q] = *reinterpret_cast<const float4*>(snap + jj[q]);
+        }
+        for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
+          const InflightRef ref = p.r.inflight[t.inflight_off + f];
+          const float* urow = p.r.U + (size_t)ref.row * p.r.stride;
+          float4 u[kTrip];
+#pragma unroll
+          for (int q = 0; q < kTrip; ++q) u[q] = *reinterpret_cast<const float4*>(urow + jj[q]);
+#pragma unroll
+          for (int q = 0; q < kTrip; ++q) {
+            w[q].x = fmaf(-ref.eta, u[q].x, w[q].x); w[q].y = fmaf(-ref.eta, u[q].y, w[q].y);
+            w[q].z = fmaf(-ref.eta, u[q].z, w[q].z); w[q].w = fmaf(-ref.eta, u[q].w, w[q].w);
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < kTrip; ++q)
+          if (base + (size_t)q * kSThreads < total) {
+            *reinterpret_cast<float4*>(work + o_layer + 4 * dd[q]) = w[q];
+            *reinterpret_cast<float4*>(Urow + jj[q]) = w[q];
+          }
       }
-      return w;
     };
     // W0 and W1 into work-row order.  The walk is in the natural order (a warp takes 512 contiguous bytes of a row:
     // whole lines of the snapshot, of the sums in flight and of U), the work row takes the scattered 16-byte stores;
     // of a pair, each CTA the columns (W0) or rows (W1) it will own.
     constexpr int kColQ = kH0 / 4 / NR;   // float4 columns of W0 a CTA owns
-    for (size_t e4 = tid; e4 < (size_t)D0 * kColQ; e4 += kSThreads) {
+    start_range((size_t)D0 * kColQ, oW0, [&](size_t e4, size_t& j, size_t& d4) {
       const int i = (int)(e4 / kColQ), q = (int)(e4 % kColQ) + (NR == 2 ? rank * kColQ : 0);   // row, float4 column
       const int c = i >> 7, r = i & 127, hh = q >> 5, half = (q >> 4) & 1, k = q & 15;
-      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + ((size_t)k << 7) + r;
-      const size_t j = oW0 + (size_t)i * kH0 + 4 * q;
-      const float4 w = start4(j);
-      *reinterpret_cast<float4*>(work + oW0 + 4 * d4) = w;
-      *reinterpret_cast<float4*>(Urow + j) = w;
-    }
-    for (size_t e4 = tid; e4 < (size_t)kH0 * kH1 / 4 / NR; e4 += kSThreads) {
+      d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + ((size_t)k << 7) + r;
+      j = oW0 + (size_t)i * kH0 + 4 * q;
+    });
+    start_range((size_t)kH0 * kH1 / 4 / NR, oW1, [&](size_t e4, size_t& j, size_t& d4) {
       const int i = (int)(e4 / (kH1 / 4)) + (NR == 2 ? rank * 128 : 0), q = (int)(e4 % (kH1 / 4));
       const int tl = i >> 7, r = i & 127, g32 = q >> 3, k = q & 7;
-      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + ((size_t)k << 7) + r;
-      const size_t j = oW1 + (size_t)i * kH1 + 4 * q;
-      const float4 w = start4(j);
-      *reinterpret_cast<float4*>(work + oW1 + 4 * d4) = w;
-      *reinterpret_cast<float4*>(Urow + j) = w;
-    }
+      d4 = ((size_t)(tl * 4 + g32) << 10) + ((size_t)k << 7) + r;
+      j = oW1 + (size_t)i * kH1 + 4 * q;
+    });
     // the narrow rest stays in shared memory for the round (in both CTAs of a pair)
     for (int j = tid; j < kH0 + kH1 + kH1 * C + C; j += kSThreads) {
       const size_t g = j < kH0 ? ob0 + j : (j < kH0 + kH1 ? ob1 + (j - kH0) : oW2 + (j - kH0 - kH1));
@@ -743,24 +763,41 @@ __global__ void __launch_bounds__(kSThreads, 1) mlp_stream_kernel(MlpLaunch p) {
   {
     const float inv_eta = 1.f / eta;
     float* wend = p.r.w_end ? p.r.w_end + (size_t)t.u_row * p.r.stride : nullptr;
-    auto finish4 = [&](size_t j, const float4 w) {   // U = (w_start - w_end) / eta for four consecutive parameters
-      const float4 a = *reinterpret_cast<const float4*>(Urow + j);
-      *reinterpret_cast<float4*>(Urow + j) = make_float4((a.x - w.x) * inv_eta, (a.y - w.y) * inv_eta, (a.z - w.z) * inv_eta, (a.w - w.w) * inv_eta);
-      if (wend) *reinterpret_cast<float4*>(wend + j) = w;
+    // U = (w_start - w_end) / eta, piece by piece, in the natural order and eight pieces per thread and trip as at the start
+    constexpr int kTrip = 8;
+    auto finish_range = [&](size_t total, size_t o_layer, auto where) {
+      for (size_t base = tid; base < total; base += (size_t)kTrip * kSThreads) {
+        float4 w[kTrip], a[kTrip];
+        size_t jj[kTrip], dd[kTrip];
+#pragma unroll
+        for (int q = 0; q < kTrip; ++q) {
+          const size_t e4 = base + (size_t)q * kSThreads;
+          where(e4 < total ? e4 : 0, jj[q], dd[q]);
+          w[q] = *reinterpret_cast<const float4*>(work + o_layer + 4 * dd[q]);
+          a[q] = *reinterpret_cast<const float4*>(Urow + jj[q]);
+        }
+#pragma unroll
+        for (int q = 0; q < kTrip; ++q)
+          if (base + (size_t)q * kSThreads < total) {
+            *reinterpret_cast<float4*>(Urow + jj[q]) = make_float4((a[q].x - w[q].x) * inv_eta, (a[q].y - w[q].y) * inv_eta,
+                                                                     (a[q].z - w[q].z) * inv_eta, (a[q].w - w[q].w) * inv_eta);
+            if (wend) *reinterpret_cast<float4*>(wend + jj[q]) = w[q];
+          }
+      }
     };
     constexpr int kColQ = kH0 / 4 / NR;
-    for (size_t e4 = tid; e4 < (size_t)D0 * kColQ; e4 += kSThreads) {   // natural order, as at the start
+    finish_range((size_t)D0 * kColQ, oW0, [&](size_t e4, size_t& j, size_t& d4) {
       const int i = (int)(e4 / kColQ), q = (int)(e4 % kColQ) + (NR == 2 ? rank * kColQ : 0);
       const int c = i >> 7, r = i & 127, hh = q >> 5, half = (q >> 4) & 1, k = q & 15;
-      const size_t d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + ((size_t)k << 7) + r;
-      finish4(oW0 + (size_t)i * kH0 + 4 * q, *reinterpret_cast<const float4*>(work + oW0 + 4 * d4));
-    }
-    for (size_t e4 = tid; e4 < (size_t)kH0 * kH1 / 4 / NR; e4 += kSThreads) {
+      d4 = ((size_t)((c * 2 + hh) * 2 + half) << 11) + ((size_t)k << 7) + r;
+      j = oW0 + (size_t)i * kH0 + 4 * q;
+    });
+    finish_range((size_t)kH0 * kH1 / 4 / NR, oW1, [&](size_t e4, size_t& j, size_t& d4) {
       const int i = (int)(e4 / (kH1 / 4)) + (NR == 2 ? rank * 128 : 0), q = (int)(e4 % (kH1 / 4));
       const int tl = i >> 7, r = i & 127, g32 = q >> 3, k = q & 7;
-      const size_t d4 = ((size_t)(tl * 4 + g32) << 10) + ((size_t)k << 7) + r;
-      finish4(oW1 + (size_t)i * kH1 + 4 * q, *reinterpret_cast<const float4*>(work + oW1 + 4 * d4));
-    }
+      d4 = ((size_t)(tl * 4 + g32) << 10) + ((size_t)k << 7) + r;
+      j = oW1 + (size_t)i * kH1 + 4 * q;
+    });
     // the narrow parameters: identical in both CTAs of a pair except the first bias, of which each holds its half
     for (int j = tid; j < kH0 + kH1 + kH1 * C + C; j += kSThreads) {
       const size_t g = j < kH0 ? ob0 + j : (j < kH0 + kH1 ? ob1 + (j - kH0) : oW2 + (j - kH0 - kH1));
