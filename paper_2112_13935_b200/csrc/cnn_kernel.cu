@@ -175,14 +175,30 @@ __global__ void __launch_bounds__(kCnnThreads, 1) cnn_round_kernel(CnnLaunch p) 
   // ---- start model: snapshot minus own update sums still in flight; U_i = 0 ----
   {
     const float* snap = p.r.snaps + (size_t)t.snap_slot * p.r.stride;
-    for (int k = tid; k < D.P; k += kCnnThreads) {
-      float v = snap[k];
+    // eight parameters per thread and trip, all loads of a trip before its first store (the stores to U could
+    // alias the loads for all the compiler knows, which would leave one load in flight per thread)
+    constexpr int kTrip = 8;
+    for (int kb = tid; kb < D.P; kb += kTrip * kCnnThreads) {
+      float v[kTrip];
+#pragma unroll
+      for (int q = 0; q < kTrip; ++q) v[q] = kb + q * kCnnThreads < D.P ? snap[kb + q * kCnnThreads] : 0.f;
       for (uint32_t f = 0; f < t.inflight_cnt; ++f) {
         const InflightRef ref = p.r.inflight[t.inflight_off + f];
-        v = fmaf(-ref.eta, p.r.U[(size_t)ref.row * p.r.stride + k], v);
+        const float* urow = p.r.U + (size_t)ref.row * p.r.stride;
+        float u[kTrip];
+#pragma unroll
+        for (int q = 0; q < kTrip; ++q) u[q] = kb + q * kCnnThreads < D.P ? urow[kb + q * kCnnThreads] : 0.f;
+#pragma unroll
+        for (int q = 0; q < kTrip; ++q) v[q] = fmaf(-ref.eta, u[q], v[q]);
       }
-      w[k] = v;
-      if (k >= k_lo && k < k_hi) Urow[k] = 0.f;
+#pragma unroll
+      for (int q = 0; q < kTrip; ++q) {
+        const int k = kb + q * kCnnThreads;
+        if (k < D.P) {
+          w[k] = v[q];
+          if (k >= k_lo && k < k_hi) Urow[k] = 0.f;
+        }
+      }
     }
   }
   __syncthreads();
