@@ -552,13 +552,12 @@ const char* cnn_check_shape(const CnnShape& s) {
 
 cudaError_t launch_cnn_rounds(const CnnLaunch& p0, cudaStream_t s) {
   if (p0.r.n_tasks == 0) return cudaSuccess;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, n = 0;
+  int sms = 0;   // asked of the current device at every launch: cheap, and right on any device of the process
+  {
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    sms = n;
   }
   // CTAs per round-task: as many as the minibatch has samples and the launch leaves SMs for
   uint32_t cl = kMaxCl;

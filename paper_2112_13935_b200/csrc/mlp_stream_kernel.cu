@@ -835,13 +835,12 @@ bool mlp_stream_eligible(const MlpShape& s) {
 
 cudaError_t launch_mlp_stream_rounds(const MlpLaunch& p, cudaStream_t s) {
   if (p.r.n_tasks == 0) return cudaSuccess;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, n = 0;
+  int sms = 0;   // asked of the current device at every launch: cheap, and right on any device of the process
+  {
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    sms = n;
   }
   // two SMs per round-task while the launch leaves that many free; a fuller launch runs one CTA per round-task
   const bool pair = 2 * (int)p.r.n_tasks <= sms;
