@@ -45,6 +45,17 @@ def test_conv_classifier_end_to_end_and_round_U(over):
     print("conv classifier per-round U errors: max %.1e" % max(errs))
 
 
+def test_conv_runs_are_bit_identical():
+    # clusters of 8 sum their partial gradients in rank order and push the new weights into every copy between
+    # two cluster barriers: nothing may depend on timing
+    cfg = workloads.get_config("cfg7", n_clients=6, n_rounds=3, data=dict(total=1200))
+    data, w0 = make(cfg)
+    a = run_gpu(cfg, data, w0)
+    b = run_gpu(cfg, data, w0)
+    assert a["w"].tobytes() == b["w"].tobytes() and a["blob"] == b["blob"]
+    assert all(u.tobytes() == v.tobytes() for u, v in zip(a["U"], b["U"]))
+
+
 def test_cfg7_full_size_against_the_checker():
     # 16 clients, LeNet shape on 60,000 28x28 images, minibatch 16, s_i = 32 i + 32 for 12 rounds: 39,936 samples
     cfg = workloads.get_config("cfg7")

@@ -116,6 +116,18 @@ def test_stream_kernel_one_cta_and_pair_instances_agree():
             check_round_U(cfg, data, s.h, e["client"], 0, w0, BF16_U_TOL, **BF16_FLIPS)
 
 
+def test_stream_kernel_runs_are_bit_identical():
+    # pairs of CTAs exchange activations and weights over distributed shared memory under cluster barriers:
+    # a missing barrier would show as run-to-run differences
+    cfg = workloads.get_config("cfg4", n_clients=24, n_rounds=3, dims=[512, 256, 128, 10], n_stragglers=2,
+                               data=dict(kind="iid", total=4800, dim=512))
+    data, w0 = make(cfg)
+    a = run_gpu(cfg, data, w0)
+    b = run_gpu(cfg, data, w0)
+    assert a["w"].tobytes() == b["w"].tobytes() and a["blob"] == b["blob"]
+    assert all(u.tobytes() == v.tobytes() for u, v in zip(a["U"], b["U"]))
+
+
 def test_bf16_shapes_with_fp32_operands_meet_the_fp32_bar():
     # the cut-down cfg4 of the bf16 test above, precision 0: every per-round update sum within 1e-5
     cfg = workloads.get_config("cfg4", precision=0, n_clients=4, n_rounds=3, dims=[3072, 64, 32, 10],
