@@ -221,8 +221,9 @@ aet_status aet_get_event_log(aet_handle* h, aet_event* out, size_t capacity,
 
 /* Update sum number `seq` of the most recent aet_run_rounds (host or device
  * pointer, n_params floats).  Needs AET_FLAG_KEEP_UPDATE_SUMS (AET_ERR_STATE
- * without it).  In the ring topology `seq` counts round-tasks in (trigger time,
- * node, round) order and the flag is not needed.  Synchronises `cuda_stream`. */
+ * without it: rows are recycled in both topologies).  In the ring topology
+ * `seq` counts round-tasks in (trigger time, node, round) order.  Synchronises
+ * `cuda_stream`. */
 aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_params,
                               void* cuda_stream);
 

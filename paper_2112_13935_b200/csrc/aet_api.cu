@@ -258,7 +258,7 @@ aet_status run_ring_rounds(aet_handle* h, uint32_t n_rounds, cudaStream_t s) {
     std::string err;
     if (!simulate_ring(h->cfg, n_rounds, st, h->delays, cp.sched, err)) return fail(h, AET_ERR_CONFIG, err);
     cp.after = st;
-    build_ring_plan(h->cfg, h->delays, cp.sched, cp.plan);
+    build_ring_plan(h->cfg, h->delays, cp.sched, (h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0, cp.plan);
     cp.valid = true;
   }
   const RingPlan& plan = cp.plan;
@@ -267,7 +267,7 @@ aet_status run_ring_rounds(aet_handle* h, uint32_t n_rounds, cudaStream_t s) {
 
   aet_status st_up = upload_clients(h, s);
   if (st_up != AET_OK) return st_up;
-  bool ok = h->U.reserve(T * h->stride) && h->d_tasks.reserve(T) && h->d_trig.reserve(T) &&
+  bool ok = h->U.reserve((size_t)plan.n_u_rows * h->stride) && h->d_tasks.reserve(T) && h->d_trig.reserve(T) &&
             h->d_ring_applies.reserve(plan.applies.size() + 1) && h->d_ring_ops.reserve(plan.ops.size() + 1);
   if (ok && !h->lr_fast) ok = h->act.reserve((size_t)plan.max_wave_tasks * h->act_floats());
   if (!ok) return fail(h, AET_ERR_NOMEM, "device allocation failed");
@@ -288,7 +288,7 @@ aet_status run_ring_rounds(aet_handle* h, uint32_t n_rounds, cudaStream_t s) {
   r.trig = h->d_trig.p; r.status = h->d_status.p; r.stride = h->stride; r.l2 = h->cfg.l2;
   r.debug_checks = (h->cfg.flags & AET_FLAG_DEBUG_CHECKS) ? 1u : 0u;
   r.step_by_step = (h->cfg.flags & AET_FLAG_STEPWISE_RECURRENCE) ? 1u : 0u;
-  r.n_u_rows = (uint32_t)T; r.n_snap = h->cfg.n_clients;
+  r.n_u_rows = plan.n_u_rows; r.n_snap = h->cfg.n_clients;
   RingApplyLaunch a{};
   a.applies = h->d_ring_applies.p; a.ops = h->d_ring_ops.p; a.U = h->U.p; a.node_w = h->node_w.p;
   a.status = h->d_status.p; a.stride = h->stride; a.n_params = h->P;
@@ -633,7 +633,7 @@ aet_status aet_get_update_sum(aet_handle* h, uint32_t seq, float* out, size_t n_
   if (!h || !out) return h ? fail(h, AET_ERR_ARG, "null argument") : AET_ERR_ARG;
   if (n_params != h->P) return fail(h, AET_ERR_ARG, "n_params does not match the model");
   if (seq >= h->last_n_events) return fail(h, AET_ERR_ARG, "seq is not an event of the most recent run");
-  if (h->cfg.topology == 0 && !(h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS))
+  if (!(h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS))
     return fail(h, AET_ERR_STATE, "update sums are recycled during a run unless the handle was created with AET_FLAG_KEEP_UPDATE_SUMS");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaMemcpyAsync(out, h->U.p + (size_t)seq * h->stride, (size_t)h->P * sizeof(float), cudaMemcpyDefault, s));

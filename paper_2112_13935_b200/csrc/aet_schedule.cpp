@@ -600,7 +600,7 @@ bool simulate_ring(const aet_config& c, uint32_t n_rounds, RingState& st, DelayC
 // started.  Before wave L the model of every node with a task in L takes, in this order, the
 // node's own previous sum (the net effect of that round's inner loop) and the sums that arrived
 // since its previous start; after the last wave every node takes what is still outstanding.
-void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingResult& r, RingPlan& plan) {
+void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingResult& r, bool keep_all, RingPlan& plan) {
   plan = RingPlan{};
   const uint32_t n = c.n_clients;
   const size_t T = r.tasks.size();
@@ -677,6 +677,40 @@ void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingRes
     plan.applies.push_back(a);
   }
   plan.apply_off[n_waves + 1] = (uint32_t)plan.applies.size();
+
+  // Rows of the update-sum array.  Up to here tasks and operations name a sum by its round-task.  A sum is read
+  // for the last time by the Receive step of some slot L (slot L runs before wave L; the slot after the last wave
+  // takes what is left), so its row can be written again by a round-task of wave L or later.  keep_all: one row
+  // per round-task, row = round-task (the caller wants to read the sums back).
+  std::vector<uint32_t> row_of(T);
+  if (keep_all) {
+    for (size_t k = 0; k < T; ++k) row_of[k] = (uint32_t)k;
+    plan.n_u_rows = (uint32_t)T;
+  } else {
+    std::vector<uint32_t> last_use(T, 0);
+    for (uint32_t L = 0; L <= n_waves; ++L)
+      for (uint32_t q = plan.apply_off[L]; q < plan.apply_off[L + 1]; ++q) {
+        const RingApplyDesc& a = plan.applies[q];
+        for (uint32_t o = 0; o < a.op_cnt; ++o) last_use[plan.ops[a.op_off + o].u_row] = L;   // slots ascend
+      }
+    std::vector<std::vector<uint32_t>> dies_at(n_waves + 1);
+    for (size_t k = 0; k < T; ++k) dies_at[std::max(last_use[k], level[k])].push_back((uint32_t)k);
+    std::vector<uint32_t> free_rows;
+    uint32_t n_rows = 0;
+    for (uint32_t L = 0; L < n_waves; ++L) {
+      // sums whose last reader is slot L or earlier: slot L has run when wave L is launched
+      for (uint32_t k : dies_at[L])
+        if (last_use[k] <= L && level[k] - 1 < L) free_rows.push_back(row_of[k]);
+      for (uint32_t q = plan.wave_off[L]; q < plan.wave_off[L + 1]; ++q) {
+        const uint32_t k = by_wave[q];
+        if (!free_rows.empty()) { row_of[k] = free_rows.back(); free_rows.pop_back(); }
+        else row_of[k] = n_rows++;
+      }
+    }
+    plan.n_u_rows = n_rows ? n_rows : 1;
+  }
+  for (TaskDesc& d : plan.tasks) d.u_row = row_of[d.u_row];
+  for (RingOp& o : plan.ops) o.u_row = row_of[o.u_row];
 }
 
 }  // namespace aet

@@ -108,14 +108,15 @@ bool simulate_ring(const aet_config& c, uint32_t n_rounds, RingState& st, DelayC
 struct RingOp { uint32_t u_row; float eta; };   // w_node -= eta * U[u_row]
 struct RingApplyDesc { uint32_t node, op_off, op_cnt, pad; };
 struct RingPlan {
-  std::vector<TaskDesc> tasks;          // sorted by wave; snap_slot = node, u_row = task index, no sums in flight
+  std::vector<TaskDesc> tasks;          // sorted by wave; snap_slot = node, u_row = its row of the update-sum array, no sums in flight
   std::vector<uint32_t> wave_off;
   // before wave L (and once more after the last wave): the nodes whose models move and their operations
   std::vector<RingApplyDesc> applies;   // grouped by wave: [apply_off[L], apply_off[L + 1])
   std::vector<uint32_t> apply_off;      // n_waves + 2 entries
   std::vector<RingOp> ops;
   uint32_t max_wave_tasks = 0;
+  uint32_t n_u_rows = 0;                // rows of the update-sum array the plan uses (rows are recycled unless keep_all)
 };
-void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingResult& r, RingPlan& plan);
+void build_ring_plan(const aet_config& c, const DelayCache& cache, const RingResult& r, bool keep_all, RingPlan& plan);
 
 }  // namespace aet

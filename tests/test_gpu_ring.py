@@ -12,6 +12,8 @@ pytestmark = pytest.mark.gpu
 
 
 def run_ring_gpu(cfg, data, w0, n_rounds=None, calls=None):
+    if not calls:   # the update sums are read back below: their rows must not be recycled
+        cfg = dict(cfg, flags=cfg.get("flags", 0) | api.FLAG_KEEP_UPDATE_SUMS)
     with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
         for r in (calls or [n_rounds]):
             s.run(r)
@@ -107,3 +109,24 @@ def test_the_papers_ring_experiment_setting_110_rounds():
         for k in (0, 250, 549):
             e = ref["tasks"][k]
             check_round_U(cfg, data, s.h, e["client"], e["round"], ref["w_start"][k])
+
+
+@pytest.mark.parametrize("name, over", [
+    ("cfg6", dict(n_rounds=30)),
+    ("cfg3", dict(n_clients=6, n_rounds=4, data=dict(total=1800))),
+])
+def test_ring_with_recycled_rows_equals_ring_with_kept_rows(name, over):
+    # without AET_FLAG_KEEP_UPDATE_SUMS a row of the update-sum array is written again once its last Receive has run
+    cfg = workloads.get_config(name, topology=1, **over)
+    data, w0 = make(cfg)
+    kept = run_ring_gpu(cfg, data, w0)                                   # sets the flag: one row per round-task
+    with api.Session(cfg, to_device(data), torch.from_numpy(w0).cuda()) as s:
+        s.run(cfg["n_rounds"])
+        blob, _ = s.log(raw=True)
+        W = [api.aet_get_node_model(s.h, c) for c in range(cfg["n_clients"])]
+        with pytest.raises(api.AetError) as e:
+            api.aet_get_update_sum(s.h, 0)
+        assert e.value.status == 3
+    assert blob == kept["blob"]
+    for c in range(cfg["n_clients"]):
+        assert W[c].tobytes() == kept["W"][c].tobytes()
