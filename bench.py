@@ -425,18 +425,19 @@ def main():
     w0_pin = torch.from_numpy(w0).pin_memory()
     out_pin = torch.empty(w0.size, dtype=torch.float32).pin_memory()
     h2d = sum(x.numel() * 4 + y.numel() * 4 for x, y in pinned) + w0.size * 4
-    d2h = w0.size * 4
+    d2h = w0.size * 4 + 32 * m["events"]          # the model, and per event the trigger and apply records the log call checks
     e2e_s = []
     for k in range(args.e2e_steps + 1 if args.e2e_steps > 0 else 0):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         h = api.aet_create(cfg)
+        api.aet_prepare_rounds(h, R)                   # the schedule and the launch plan, under the copies below
         api.aet_set_global_model(h, w0_pin)
         for c, (x, y) in enumerate(pinned):
             api.aet_load_client_data(h, c, x, y)
         api.aet_run_rounds(h, R)
         api.aet_get_global_model(h, out_pin)
-        ev, _ = api.aet_get_event_log(h)
+        ev, _ = api.aet_get_event_log(h, raw=True)     # the log with the library's cross-check of the device records
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
         api.aet_destroy(h)
@@ -483,7 +484,7 @@ def main():
                     "multi_gpu": "independent replicas, one seed per rank"},
             "clocks": m["clocks"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": len(e2e_s), "note": "one pass per e2e step: create, load from pinned host memory, run, model back"},
+                    "steps": len(e2e_s), "note": "one pass per e2e step: create, schedule on a library thread under the copies, load from pinned host memory, run, model and event log back"},
             "gpu_launches": m["launches_per_pass"] * m["n_pass"],
             "roofline": m["roof"],
             "cpu_baseline": cpu,

@@ -191,6 +191,17 @@ aet_status aet_load_client_data(aet_handle* h, uint32_t client, const void* x,
  * AET_ERR_CONFIG (batch does not divide s_i), AET_ERR_CUDA, AET_ERR_NOMEM. */
 aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream);
 
+/* Optional: start computing, on a host thread of the library, what the next
+ * aet_run_rounds(h, n_rounds) does on the host - the integer schedule of start,
+ * trigger and apply times (Section 3.3.2 delays; Algorithm 3, Synchronize) and
+ * the launch plan - so that it overlaps the caller's aet_load_client_data
+ * copies.  Returns at once.  The result is used only if the handle's state is
+ * the one it was computed for (otherwise aet_run_rounds computes its own); a
+ * schedule error is reported by aet_run_rounds, not here.  aet_run_rounds,
+ * aet_reset, aet_debug_run_client_round and aet_destroy wait for the thread.
+ * Errors: AET_ERR_ARG (null), AET_ERR_STATE (no thread could be started). */
+aet_status aet_prepare_rounds(aet_handle* h, uint32_t n_rounds);
+
 /* Copy the server's model out: the global model w the server keeps and
  * broadcasts (Section 1; Algorithm 3, Receive: w = w - eta_k U).  Host or device
  * pointer, n_params floats.  Synchronises `cuda_stream`.  Errors:

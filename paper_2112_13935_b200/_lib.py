@@ -58,6 +58,7 @@ PROTOTYPES = {
     "aet_reset": (C.c_int, [C.c_void_p, C.c_void_p]),
     "aet_set_global_model": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "aet_load_client_data": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]),
+    "aet_prepare_rounds": (C.c_int, [C.c_void_p, C.c_uint32]),
     "aet_run_rounds": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p]),
     "aet_get_global_model": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "aet_get_node_model": (C.c_int, [C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]),

@@ -99,6 +99,11 @@ def aet_run_rounds(h, n_rounds: int, stream=None):
     _check(h, _lib.load().aet_run_rounds(h, n_rounds, _stream(stream)))
 
 
+def aet_prepare_rounds(h, n_rounds: int):
+    """Start the host-side schedule and launch plan of the next aet_run_rounds(h, n_rounds) on a library thread."""
+    _check(h, _lib.load().aet_prepare_rounds(h, n_rounds))
+
+
 def aet_n_params(h) -> int:
     return int(_lib.load().aet_n_params(h))
 

@@ -7,6 +7,7 @@
 #include <chrono>
 #include <new>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include "../../include/aet.h"
@@ -106,6 +107,13 @@ struct aet_handle {
   DelayCache delays;
   CachedPlan cached;
   CachedRingPlan ring_cached;
+  // aet_prepare_rounds: schedule and launch plan of the next run computed by a host thread of its own, on copies
+  // of the scheduling state; aet_run_rounds takes the result over if it still fits.
+  std::thread prep_thread;
+  CachedPlan prep;
+  CachedRingPlan prep_ring;
+  DelayCache prep_delays;
+  bool prep_ok = false;
   std::vector<RingTask> last_ring_tasks;
   std::vector<aet_event> log;
   aet_summary total{};
@@ -242,11 +250,22 @@ aet_status launch_rounds(aet_handle* h, const RoundLaunch& r, cudaStream_t s) {
   return AET_OK;
 }
 
+// Waits for the thread aet_prepare_rounds started, if any.
+void join_prepare(aet_handle* h) {
+  if (h->prep_thread.joinable()) h->prep_thread.join();
+}
+
 // Peer-to-peer ring: waves of round-tasks (each from its node's own model), and before every wave
 // the Receive step of the nodes about to start; after the last wave every node takes what is left.
 aet_status run_ring_rounds(aet_handle* h, uint32_t n_rounds, cudaStream_t s) {
   auto t0 = std::chrono::steady_clock::now();
   CachedRingPlan& cp = h->ring_cached;
+  if (h->prep_ok && h->prep_ring.valid && h->prep_ring.rounds_before == h->rst.rounds_done && h->prep_ring.n_rounds == n_rounds &&
+      h->prep_ring.before.clock == h->rst.clock && h->prep_ring.before.H == h->rst.H) {
+    cp = std::move(h->prep_ring);   // prepared by aet_prepare_rounds for exactly this state
+    h->delays = std::move(h->prep_delays);
+  }
+  h->prep_ok = false;
   if (!(cp.valid && cp.rounds_before == h->rst.rounds_done && cp.n_rounds == n_rounds &&
         cp.before.clock == h->rst.clock && cp.before.H == h->rst.H)) {
     cp.valid = false;
@@ -392,6 +411,7 @@ aet_status aet_create(const aet_config* cfg, aet_handle** out) {
 
 aet_status aet_destroy(aet_handle* h) {
   if (!h) return AET_ERR_ARG;
+  join_prepare(h);
   cudaDeviceSynchronize();
   collect_timings(h);
   for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
@@ -409,6 +429,7 @@ aet_status aet_destroy(aet_handle* h) {
 
 aet_status aet_reset(aet_handle* h, void* cuda_stream) {
   if (!h) return AET_ERR_ARG;
+  join_prepare(h);
   cudaStream_t s = (cudaStream_t)cuda_stream;
   AET_CUDA(h, cudaMemcpyAsync(h->w_cur(), h->w0.p, h->stride * sizeof(float), cudaMemcpyDeviceToDevice, s));
   AET_CUDA(h, cudaMemsetAsync(h->d_H.p, 0, h->cfg.n_clients * sizeof(uint32_t), s));
@@ -510,6 +531,7 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   for (uint32_t c = 0; c < h->cfg.n_clients; ++c)
     if (!h->h_clients[c].x) return fail(h, AET_ERR_STATE, "client " + std::to_string(c) + " has no data");
   if (n_rounds == 0) return AET_OK;
+  join_prepare(h);
   collect_timings(h);
   h->stats = aet_stats{};
   if (h->cfg.topology == 1) return run_ring_rounds(h, n_rounds, s);
@@ -517,6 +539,12 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   // ---- a0: integer schedule and launch plan (cached for repeated runs) ----
   auto t0 = std::chrono::steady_clock::now();
   CachedPlan& cp = h->cached;
+  if (h->prep_ok && h->prep.valid && h->prep.rounds_before == h->st.rounds_done && h->prep.n_rounds == n_rounds &&
+      h->prep.before.clock == h->st.clock && h->prep.before.H == h->st.H) {
+    cp = std::move(h->prep);   // prepared by aet_prepare_rounds for exactly this state
+    h->delays = std::move(h->prep_delays);
+  }
+  h->prep_ok = false;
   if (!(cp.valid && cp.rounds_before == h->st.rounds_done && cp.n_rounds == n_rounds &&
         cp.before.clock == h->st.clock && cp.before.H == h->st.H)) {
     cp.valid = false;
@@ -600,6 +628,50 @@ aet_status aet_run_rounds(aet_handle* h, uint32_t n_rounds, void* cuda_stream) {
   h->total.samples_total += q.samples_total; h->total.messages_if_per_sample += q.messages_if_per_sample;
   h->total.messages_if_constant_b += q.messages_if_constant_b; h->total.t_end_ticks = q.t_end_ticks;
   h->st = cp.after;
+  return AET_OK;
+}
+
+aet_status aet_prepare_rounds(aet_handle* h, uint32_t n_rounds) {
+  if (!h) return AET_ERR_ARG;
+  join_prepare(h);
+  h->prep_ok = false;
+  if (n_rounds == 0) return AET_OK;
+  h->prep_delays = h->delays;   // the thread works on copies: nothing it touches is shared until it is joined
+  if (h->cfg.topology == 1) {
+    h->prep_ring = CachedRingPlan{};
+    h->prep_ring.before = h->rst;
+    h->prep_ring.rounds_before = h->rst.rounds_done;
+    h->prep_ring.n_rounds = n_rounds;
+  } else {
+    h->prep = CachedPlan{};
+    h->prep.before = h->st;
+    h->prep.rounds_before = h->st.rounds_done;
+    h->prep.n_rounds = n_rounds;
+  }
+  try {
+    h->prep_thread = std::thread([h, n_rounds]() {
+      std::string err;
+      const bool keep = (h->cfg.flags & AET_FLAG_KEEP_UPDATE_SUMS) != 0;
+      if (h->cfg.topology == 1) {
+        CachedRingPlan& cp = h->prep_ring;
+        RingState st = cp.before;
+        if (!simulate_ring(h->cfg, n_rounds, st, h->prep_delays, cp.sched, err)) return;   // aet_run_rounds will report it
+        cp.after = st;
+        build_ring_plan(h->cfg, h->prep_delays, cp.sched, keep, cp.plan);
+        cp.valid = true;
+      } else {
+        CachedPlan& cp = h->prep;
+        SchedState st = cp.before;
+        if (!simulate(h->cfg, n_rounds, st, h->prep_delays, cp.sched, err)) return;
+        cp.after = st;
+        build_plan(h->cfg, h->prep_delays, cp.sched.events, keep, cp.plan);
+        cp.valid = true;
+      }
+      h->prep_ok = true;
+    });
+  } catch (...) {
+    return fail(h, AET_ERR_STATE, "could not start the schedule thread");
+  }
   return AET_OK;
 }
 
@@ -697,6 +769,7 @@ aet_status aet_debug_run_client_round(aet_handle* h, uint32_t client, uint32_t r
   if (client >= h->cfg.n_clients) return fail(h, AET_ERR_ARG, "client index out of range");
   if (round < h->cfg.round_base) return fail(h, AET_ERR_ARG, "round is before round_base");
   if (!h->h_clients[client].x) return fail(h, AET_ERR_STATE, "client has no data");
+  join_prepare(h);
   ensure_split(h->cfg, round + 1, h->delays);
   const uint32_t s_i = node_sample_size(h->cfg, h->delays, client, round);
   if (s_i % h->cfg.batch || (s_i == 0 && !h->cfg.split_mode))

@@ -78,3 +78,35 @@ def test_debug_checks_change_nothing_on_good_input_and_flag_a_bad_label(name, ov
         assert api.aet_get_global_model(h).tobytes() == plain["w"].tobytes()
     finally:
         api.aet_destroy(h)
+
+
+@pytest.mark.parametrize("topology", [0, 1])
+def test_prepared_schedule_gives_the_same_run(topology):
+    # aet_prepare_rounds computes the schedule and the launch plan on a library thread under the data copies;
+    # the run that follows uses them if the state still fits, and computes its own otherwise
+    cfg = workloads.get_config("cfg1", topology=topology, n_clients=5, l2=0.0, data=dict(per_client=200))
+    data, w0 = make(cfg)
+
+    def run(prepare_for, rounds):
+        h = api.aet_create(cfg)
+        try:
+            if prepare_for:
+                api.aet_prepare_rounds(h, prepare_for)
+            api.aet_set_global_model(h, w0)
+            for c, (x, y) in enumerate(data):
+                api.aet_load_client_data(h, c, x, y)
+            for r in rounds:
+                api.aet_run_rounds(h, r)
+            blob, _ = api.aet_get_event_log(h, raw=True)
+            W = [api.aet_get_node_model(h, c) for c in range(5)] if topology else [api.aet_get_global_model(h)]
+        finally:
+            api.aet_destroy(h)
+        return blob, W
+
+    plain = run(0, [3, 2])
+    for prepared in (run(3, [3, 2]), run(4, [3, 2])):      # the plan that fits, and one for another run length
+        assert prepared[0] == plain[0]
+        assert all(a.tobytes() == b.tobytes() for a, b in zip(prepared[1], plain[1]))
+    h = api.aet_create(cfg)                                # a thread still running when the handle goes away is waited for
+    api.aet_prepare_rounds(h, 5)
+    api.aet_destroy(h)
